@@ -1,0 +1,176 @@
+"""numpy-facing wrapper around the CPU oracle (``patch_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: importable from ``tests/``, from the smoke check and from the
+benchmark's CPU-baseline legs.  The product package never imports this module, and this
+module never imports the product package's CUDA binding.
+
+All matrices are numpy ``uint16`` arrays of bf16 bit patterns, C-contiguous.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "patch_oracle.c")
+_LIB = os.path.join(_HERE, "libpatch_oracle.so")
+
+KIND_DENSE, KIND_SPARSE = 0, 1
+MAGIC = 0x48435450
+
+
+class Layout(ctypes.Structure):
+    _fields_ = [("magic", ctypes.c_uint32), ("version", ctypes.c_uint32),
+                ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("tile_n", ctypes.c_int32), ("tile_k", ctypes.c_int32),
+                ("n_dense", ctypes.c_int64), ("n_sparse", ctypes.c_int64),
+                ("table_off", ctypes.c_uint64), ("payload_off", ctypes.c_uint64),
+                ("payload_bytes", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64)]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2, OpenMP over outputs, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
+               "-Wall", "-Wextra", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def _flags(f):
+    return np.ascontiguousarray(f, dtype=np.uint8).reshape(-1)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise ValueError(f"oracle {what} failed with status {rc}")
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def mask(W, flags, tile_n=128, tile_k=128) -> np.ndarray:
+    """Hard mask M* (uint8, 1 = keep), Algorithm 1's merged tile / 2:4 mask."""
+    W = _u16(W)
+    N, K = W.shape
+    out = np.empty((N, K), np.uint8)
+    _check(lib().oracle_mask(_p(W), ctypes.c_int64(N), ctypes.c_int64(K), _p(_flags(flags)),
+                             tile_n, tile_k, _p(out)), "mask")
+    return out
+
+
+def prune(W, flags, tile_n=128, tile_k=128) -> np.ndarray:
+    """Pruned weight What = W (.) M* (bf16 bits; pruned entries are +0)."""
+    W = _u16(W)
+    N, K = W.shape
+    out = np.empty((N, K), np.uint16)
+    _check(lib().oracle_prune(_p(W), ctypes.c_int64(N), ctypes.c_int64(K), _p(_flags(flags)),
+                              tile_n, tile_k, _p(out)), "prune")
+    return out
+
+
+def packed_size(N, K, flags, tile_n=128, tile_k=128) -> Layout:
+    L = Layout()
+    _check(lib().oracle_packed_size(ctypes.c_int64(N), ctypes.c_int64(K), tile_n, tile_k,
+                                    _p(_flags(flags)), ctypes.byref(L)), "packed_size")
+    return L
+
+
+def pack(W, flags, tile_n=128, tile_k=128):
+    """Canonical packed blob (uint8 array) and its layout."""
+    W = _u16(W)
+    N, K = W.shape
+    L = packed_size(N, K, flags, tile_n, tile_k)
+    blob = np.empty(L.total_bytes, np.uint8)
+    _check(lib().oracle_pack(_p(W), _p(_flags(flags)), ctypes.byref(L), _p(blob),
+                             ctypes.c_uint64(blob.nbytes)), "pack")
+    return blob, L
+
+
+def unpack(blob) -> np.ndarray:
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    L = Layout.from_buffer_copy(blob[:ctypes.sizeof(Layout)].tobytes())
+    out = np.empty((L.N, L.K), np.uint16)
+    _check(lib().oracle_unpack(_p(blob), ctypes.c_uint64(blob.nbytes), _p(out)), "unpack")
+    return out
+
+
+def device_image(canon_blob) -> np.ndarray:
+    """Canonical blob -> device image (per-tile byte bijection; 128x128 tiles only)."""
+    canon_blob = np.ascontiguousarray(canon_blob, dtype=np.uint8)
+    out = np.zeros_like(canon_blob)
+    _check(lib().oracle_device_image(_p(canon_blob), ctypes.c_uint64(canon_blob.nbytes), _p(out)),
+           "device_image")
+    return out
+
+
+def gemm_f64(X, What, want_bf16=True):
+    """Y = X What^T, double accumulation -> (fp32 [M x N], bf16 bits [M x N] or None)."""
+    X, What = _u16(X), _u16(What)
+    M, K = X.shape
+    N, K2 = What.shape
+    assert K == K2
+    Y32 = np.empty((M, N), np.float32)
+    Y16 = np.empty((M, N), np.uint16) if want_bf16 else None
+    _check(lib().oracle_gemm_f64(_p(X), ctypes.c_int64(M), ctypes.c_int64(K), _p(What),
+                                 ctypes.c_int64(N), _p(Y32),
+                                 _p(Y16) if want_bf16 else ctypes.c_void_p(0)), "gemm_f64")
+    return Y32, Y16
+
+
+def gemm_f32(X, What) -> np.ndarray:
+    X, What = _u16(X), _u16(What)
+    M, K = X.shape
+    N, _ = What.shape
+    Y32 = np.empty((M, N), np.float32)
+    _check(lib().oracle_gemm_f32(_p(X), ctypes.c_int64(M), ctypes.c_int64(K), _p(What),
+                                 ctypes.c_int64(N), _p(Y32)), "gemm_f32")
+    return Y32
+
+
+def gemm_f64_rows(X, rows, What) -> np.ndarray:
+    """Rows ``rows`` of Y only (sampled parity at large M)."""
+    X, What = _u16(X), _u16(What)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    _, K = X.shape
+    N, _ = What.shape
+    Y32 = np.empty((len(rows), N), np.float32)
+    _check(lib().oracle_gemm_f64_rows(_p(X), ctypes.c_int64(K), _p(rows), ctypes.c_int64(len(rows)),
+                                      _p(What), ctypes.c_int64(N), _p(Y32)), "gemm_f64_rows")
+    return Y32
+
+
+def parity_metrics(Y_test_f32, Y_ref_f32):
+    """relF = |dY|_F / |Yref|_F and max|dY| / max|Yref| (the two tolerances of the benchmark spec)."""
+    d = Y_test_f32.astype(np.float64) - Y_ref_f32.astype(np.float64)
+    ref = Y_ref_f32.astype(np.float64)
+    nref = float(np.sqrt((ref * ref).sum()))
+    relF = float(np.sqrt((d * d).sum())) / nref if nref > 0 else float(np.abs(d).max(initial=0.0))
+    mref = float(np.abs(ref).max(initial=0.0))
+    maxrel = float(np.abs(d).max(initial=0.0)) / mref if mref > 0 else float(np.abs(d).max(initial=0.0))
+    return relF, maxrel

@@ -1,0 +1,398 @@
+/*
+ * CPU oracle for the tile-hybrid linear layer  Y = X * What^T  of PATCH.
+ *
+ * TEST INFRASTRUCTURE ONLY.  Plain, slow, obviously-correct C.  Nothing in the product path
+ * may call into this file; it shares no code, header or table with the CUDA library.
+ *
+ * What it computes, and the passage of the paper each step follows:
+ *   - hard mask  M* = M*_tile + (1 - M*_tile) (.) M*_2:4   (Algorithm 1, last three lines; Eq. 4
+ *     in its hard form).  M*_tile is 1 on tiles flagged dense; M*_2:4 keeps two of every four
+ *     consecutive elements along K (Preliminaries, "Learnable 2:4 Mask": six candidate patterns
+ *     per group of four).  The 2:4 mask itself is magnitude top-2 per group, the selection the
+ *     workloads fix; ties go to the lower index.
+ *   - pruned weight  What = W (.) M*  (Algorithm 1, "Final pruned weights"), done as a select so
+ *     that a pruned element is +0.
+ *   - compression of the mixed matrix into kept values + metadata, per tile (Appendix A:
+ *     "Matrix compression and metadata generation are determined by the chosen tile size");
+ *     two metadata bits per kept value, the cost that reproduces the compression-ratio column
+ *     of the 4-bit quantisation table.
+ *   - the linear layer itself, on the same bf16-rounded inputs, accumulated in double (and in
+ *     plain fp32 as a cross-check) in k order.
+ *
+ * Pins: every function here is pinned by tests that do not call it to produce their expected
+ * value (brute force over the six patterns, closed-form byte counts, numpy matmul, round trips,
+ * hand-written fixtures).  No function is "parity unpinned".
+ *
+ * Conventions: W is [N x K] row-major bf16 (uint16 bit patterns), N = out-features,
+ * K = in-features; X is [M x K]; Y is [M x N].  flags[tn*TK + tk]: 0 = dense, 1 = 2:4.
+ */
+#include <stdint.h>
+#include <stddef.h>
+#include <string.h>
+#include <stdlib.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_MAGIC   0x48435450u /* "PTCH" little-endian */
+#define ORACLE_VERSION 1u
+#define KIND_DENSE  0u
+#define KIND_SPARSE 1u
+
+typedef struct {
+    uint32_t magic, version;
+    int64_t  N, K;
+    int32_t  tile_n, tile_k;
+    int64_t  n_dense, n_sparse;
+    uint64_t table_off, payload_off, payload_bytes, total_bytes;
+} oracle_layout_t;
+
+/* ------------------------------------------------------------------------------------------- */
+/* bf16 helpers (exact widening; round-to-nearest-even narrowing)                               */
+
+static float bf16_to_f32(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+static uint16_t f32_to_bf16_rne(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u); /* NaN stays NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------------------------- */
+/* 2:4 selection inside one group of four: keep the two largest |w|; equal magnitudes are       */
+/* ordered by position, lower first.  Magnitude is the bf16 bit pattern without its sign bit,   */
+/* which orders finite values exactly like |w| (and +0 == -0).                                  */
+
+static void select_top2(const uint16_t w[4], int keep[4]) {
+    for (int j = 0; j < 4; ++j) {
+        uint32_t mj = w[j] & 0x7FFFu;
+        int rank = 0; /* how many elements come before j in (magnitude desc, index asc) order */
+        for (int l = 0; l < 4; ++l) {
+            uint32_t ml = w[l] & 0x7FFFu;
+            if (ml > mj || (ml == mj && l < j)) ++rank;
+        }
+        keep[j] = rank < 2;
+    }
+}
+
+static int check_shape(int64_t N, int64_t K, int tile_n, int tile_k) {
+    if (N <= 0 || K <= 0 || tile_n <= 0 || tile_k <= 0) return -2;
+    if (tile_k % 4 != 0) return -3;
+    if (N % tile_n != 0 || K % tile_k != 0) return -2;
+    return 0;
+}
+
+/* Hard mask M* as bytes (1 = keep).  Algorithm 1: M* = M*_tile + (1 - M*_tile) (.) M*_2:4. */
+int oracle_mask(const uint16_t* W, int64_t N, int64_t K, const uint8_t* flags,
+                int tile_n, int tile_k, uint8_t* mask) {
+    int rc = check_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    int64_t TK = K / tile_k;
+    for (int64_t t = 0; t < (N / tile_n) * TK; ++t)
+        if (flags[t] > 1) return -4;
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t g = 0; g < K / 4; ++g) {
+            int64_t k0 = 4 * g;
+            int m_tile = flags[(n / tile_n) * TK + k0 / tile_k] == KIND_DENSE; /* 1 = dense tile */
+            int keep[4];
+            select_top2(&W[n * K + k0], keep);
+            for (int j = 0; j < 4; ++j)
+                mask[n * K + k0 + j] = (uint8_t)(m_tile + (1 - m_tile) * keep[j]);
+        }
+    }
+    return 0;
+}
+
+/* What = W (.) M*  as a select: kept elements verbatim, pruned elements +0. */
+int oracle_prune(const uint16_t* W, int64_t N, int64_t K, const uint8_t* flags,
+                 int tile_n, int tile_k, uint16_t* What) {
+    uint8_t* mask = (uint8_t*)malloc((size_t)(N * K));
+    if (!mask) return -6;
+    int rc = oracle_mask(W, N, K, flags, tile_n, tile_k, mask);
+    if (rc == 0)
+        for (int64_t i = 0; i < N * K; ++i) What[i] = mask[i] ? W[i] : (uint16_t)0;
+    free(mask);
+    return rc;
+}
+
+/* ------------------------------------------------------------------------------------------- */
+static uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+/* Canonical packed blob:
+ *   [ header 256 B | table: 16 B per tile, padded to 1024 B | payloads ]
+ * Tile order t = tn*TK + tk.  Dense payload: tile_n rows x tile_k bf16, row-major.
+ * 2:4 payload: vals[tile_n][tile_k/2] bf16 (the two kept elements of each group, in position
+ * order; the block is padded to a multiple of 16 B) followed by meta[tile_n][words]
+ * little-endian uint32, words = ceil(tile_k/32); the nibble of group g sits at bits
+ * [4*(g%8), +4) of word g/8 and equals i0 | (i1 << 2) with i0 < i1 the kept positions.
+ * Payloads are aligned to 1024 B for 128x128 tiles, 16 B otherwise.
+ * Table entry: { u32 kind, u32 payload_off/16, u32 meta_off/16 (0xFFFFFFFF if dense), u32 0 },
+ * offsets from the start of the blob. */
+
+static uint64_t payload_align(int tile_n, int tile_k) {
+    return (tile_n == 128 && tile_k == 128) ? 1024u : 16u;
+}
+static uint64_t dense_bytes(int tile_n, int tile_k) { return (uint64_t)tile_n * tile_k * 2; }
+static uint64_t meta_words(int tile_k) { return (uint64_t)(tile_k + 31) / 32; }
+/* kept values of a 2:4 tile, padded to 16 B so that the metadata offset is expressible */
+static uint64_t vals_bytes(int tile_n, int tile_k) {
+    return round_up((uint64_t)tile_n * (tile_k / 2) * 2, 16);
+}
+static uint64_t sparse_bytes(int tile_n, int tile_k) {
+    return vals_bytes(tile_n, tile_k) + (uint64_t)tile_n * meta_words(tile_k) * 4;
+}
+
+int oracle_packed_size(int64_t N, int64_t K, int tile_n, int tile_k, const uint8_t* flags,
+                       oracle_layout_t* L) {
+    int rc = check_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    int64_t T = (N / tile_n) * (K / tile_k);
+    int64_t nd = 0, ns = 0;
+    uint64_t al = payload_align(tile_n, tile_k), bytes = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        if (flags[t] == KIND_DENSE) { ++nd; bytes += round_up(dense_bytes(tile_n, tile_k), al); }
+        else if (flags[t] == KIND_SPARSE) { ++ns; bytes += round_up(sparse_bytes(tile_n, tile_k), al); }
+        else return -4;
+    }
+    memset(L, 0, sizeof *L);
+    L->magic = ORACLE_MAGIC; L->version = ORACLE_VERSION;
+    L->N = N; L->K = K; L->tile_n = tile_n; L->tile_k = tile_k;
+    L->n_dense = nd; L->n_sparse = ns;
+    L->table_off = 256;
+    L->payload_off = round_up(256 + 16 * (uint64_t)T, 1024);
+    L->payload_bytes = bytes;
+    L->total_bytes = L->payload_off + bytes;
+    return 0;
+}
+
+static void write_header_and_table(const oracle_layout_t* L, const uint8_t* flags, uint8_t* blob) {
+    memset(blob, 0, (size_t)L->payload_off);
+    memcpy(blob, L, sizeof *L);
+    int64_t T = (L->N / L->tile_n) * (L->K / L->tile_k);
+    uint64_t al = payload_align(L->tile_n, L->tile_k), off = L->payload_off;
+    uint32_t* table = (uint32_t*)(blob + L->table_off);
+    for (int64_t t = 0; t < T; ++t) {
+        table[4 * t + 0] = flags[t];
+        table[4 * t + 1] = (uint32_t)(off / 16);
+        if (flags[t] == KIND_DENSE) {
+            table[4 * t + 2] = 0xFFFFFFFFu;
+            off += round_up(dense_bytes(L->tile_n, L->tile_k), al);
+        } else {
+            table[4 * t + 2] = (uint32_t)((off + vals_bytes(L->tile_n, L->tile_k)) / 16);
+            off += round_up(sparse_bytes(L->tile_n, L->tile_k), al);
+        }
+        table[4 * t + 3] = 0;
+    }
+}
+
+int oracle_pack(const uint16_t* W, const uint8_t* flags, const oracle_layout_t* L,
+                uint8_t* blob, uint64_t capacity) {
+    if (!W || !flags || !L || !blob) return -1;
+    if (L->magic != ORACLE_MAGIC || L->version != ORACLE_VERSION) return -7;
+    if (capacity < L->total_bytes) return -6;
+    int tn_ = L->tile_n, tk_ = L->tile_k;
+    int64_t N = L->N, K = L->K, TN = N / tn_, TK = K / tk_;
+    memset(blob, 0, (size_t)L->total_bytes);
+    write_header_and_table(L, flags, blob);
+    const uint32_t* table = (const uint32_t*)(blob + L->table_off);
+    for (int64_t tn = 0; tn < TN; ++tn)
+        for (int64_t tk = 0; tk < TK; ++tk) {
+            int64_t t = tn * TK + tk;
+            uint8_t* pay = blob + (uint64_t)table[4 * t + 1] * 16;
+            if (table[4 * t + 0] == KIND_DENSE) {
+                uint16_t* d = (uint16_t*)pay;
+                for (int r = 0; r < tn_; ++r)
+                    for (int c = 0; c < tk_; ++c)
+                        d[r * tk_ + c] = W[(tn * tn_ + r) * K + tk * tk_ + c];
+            } else {
+                uint16_t* vals = (uint16_t*)pay;
+                uint32_t* meta = (uint32_t*)(blob + (uint64_t)table[4 * t + 2] * 16);
+                int words = (int)meta_words(tk_);
+                for (int r = 0; r < tn_; ++r)
+                    for (int g = 0; g < tk_ / 4; ++g) {
+                        const uint16_t* w = &W[(tn * tn_ + r) * K + tk * tk_ + 4 * g];
+                        int keep[4], pos[2], cnt = 0;
+                        select_top2(w, keep);
+                        for (int j = 0; j < 4; ++j) if (keep[j]) pos[cnt++] = j;
+                        vals[r * (tk_ / 2) + 2 * g + 0] = w[pos[0]];
+                        vals[r * (tk_ / 2) + 2 * g + 1] = w[pos[1]];
+                        uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
+                        meta[r * words + g / 8] |= nib << (4 * (g % 8));
+                    }
+            }
+        }
+    return 0;
+}
+
+/* Inverse of oracle_pack: canonical blob -> What [N x K]. */
+int oracle_unpack(const uint8_t* blob, uint64_t blob_bytes, uint16_t* What) {
+    if (!blob || !What) return -1;
+    if (blob_bytes < sizeof(oracle_layout_t)) return -6;
+    oracle_layout_t L;
+    memcpy(&L, blob, sizeof L);
+    if (L.magic != ORACLE_MAGIC || L.version != ORACLE_VERSION) return -7;
+    if (blob_bytes < L.total_bytes) return -6;
+    int tn_ = L.tile_n, tk_ = L.tile_k;
+    int64_t K = L.K, TN = L.N / tn_, TK = K / tk_;
+    const uint32_t* table = (const uint32_t*)(blob + L.table_off);
+    for (int64_t tn = 0; tn < TN; ++tn)
+        for (int64_t tk = 0; tk < TK; ++tk) {
+            int64_t t = tn * TK + tk;
+            const uint8_t* pay = blob + (uint64_t)table[4 * t + 1] * 16;
+            if (table[4 * t + 0] == KIND_DENSE) {
+                const uint16_t* d = (const uint16_t*)pay;
+                for (int r = 0; r < tn_; ++r)
+                    for (int c = 0; c < tk_; ++c)
+                        What[(tn * tn_ + r) * K + tk * tk_ + c] = d[r * tk_ + c];
+            } else if (table[4 * t + 0] == KIND_SPARSE) {
+                const uint16_t* vals = (const uint16_t*)pay;
+                const uint32_t* meta = (const uint32_t*)(blob + (uint64_t)table[4 * t + 2] * 16);
+                int words = (int)meta_words(tk_);
+                for (int r = 0; r < tn_; ++r)
+                    for (int g = 0; g < tk_ / 4; ++g) {
+                        uint16_t* w = &What[(tn * tn_ + r) * K + tk * tk_ + 4 * g];
+                        uint32_t nib = (meta[r * words + g / 8] >> (4 * (g % 8))) & 0xFu;
+                        int i0 = (int)(nib & 3u), i1 = (int)(nib >> 2);
+                        if (i0 >= i1) return -7;
+                        w[0] = w[1] = w[2] = w[3] = 0;
+                        w[i0] = vals[r * (tk_ / 2) + 2 * g + 0];
+                        w[i1] = vals[r * (tk_ / 2) + 2 * g + 1];
+                    }
+            } else return -7;
+        }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------- */
+/* Device image (128x128 tiles only): a per-tile bijection of the canonical payload bytes.      */
+/* Header and table are identical to the canonical blob.                                        */
+/*                                                                                              */
+/* Values are stored as "swizzled K-major atoms" of 128 rows x 64 bf16 (16 384 B): row r, 16-B  */
+/* chunk c (8 elements) of the 128-B row lives at                                               */
+/*      (r / 8) * 1024 + (r % 8) * 128 + ((c ^ (r % 8)) * 16).                                  */
+/* A dense tile is two atoms (columns 0..63, then 64..127); a 2:4 tile is one atom holding its  */
+/* 64 kept values per row.                                                                      */
+/*                                                                                              */
+/* Metadata (2 048 B) is stored as 128 rows of four uint32.  Row L = 16*q + 8*h + i (i < 8),    */
+/* word j (the j-th run of 32 columns): low 16 bits = the four nibbles of tile row 16q+i for    */
+/* columns [32j + 16h, 32j + 16h + 16), high 16 bits = the same for tile row 16q+8+i.           */
+
+static uint64_t atom_offset(int r, int col) { /* col in [0,64): element column inside the atom */
+    int chunk = col / 8, within = col % 8;
+    return (uint64_t)(r / 8) * 1024 + (uint64_t)(r % 8) * 128 + (uint64_t)((chunk ^ (r % 8)) * 16)
+           + (uint64_t)within * 2;
+}
+
+int oracle_device_image(const uint8_t* canon, uint64_t blob_bytes, uint8_t* image) {
+    if (!canon || !image) return -1;
+    if (blob_bytes < sizeof(oracle_layout_t)) return -6;
+    oracle_layout_t L;
+    memcpy(&L, canon, sizeof L);
+    if (L.magic != ORACLE_MAGIC || L.version != ORACLE_VERSION) return -7;
+    if (L.tile_n != 128 || L.tile_k != 128) return -3;
+    if (blob_bytes < L.total_bytes) return -6;
+    memcpy(image, canon, (size_t)L.payload_off);
+    int64_t T = (L.N / 128) * (L.K / 128);
+    const uint32_t* table = (const uint32_t*)(canon + L.table_off);
+    for (int64_t t = 0; t < T; ++t) {
+        uint64_t off = (uint64_t)table[4 * t + 1] * 16;
+        if (table[4 * t + 0] == KIND_DENSE) {
+            const uint16_t* src = (const uint16_t*)(canon + off);
+            for (int r = 0; r < 128; ++r)
+                for (int c = 0; c < 128; ++c) {
+                    uint64_t o = (uint64_t)(c / 64) * 16384 + atom_offset(r, c % 64);
+                    memcpy(image + off + o, &src[r * 128 + c], 2);
+                }
+        } else {
+            const uint16_t* src = (const uint16_t*)(canon + off);
+            for (int r = 0; r < 128; ++r)
+                for (int c = 0; c < 64; ++c)
+                    memcpy(image + off + atom_offset(r, c), &src[r * 64 + c], 2);
+            uint64_t moff = (uint64_t)table[4 * t + 2] * 16;
+            const uint32_t* cm = (const uint32_t*)(canon + moff);
+            for (int Lr = 0; Lr < 128; ++Lr) {
+                int q = Lr / 16, h = (Lr / 8) % 2, i = Lr % 8;
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t lo = (cm[(16 * q + i) * 4 + j] >> (16 * h)) & 0xFFFFu;
+                    uint32_t hi = (cm[(16 * q + 8 + i) * 4 + j] >> (16 * h)) & 0xFFFFu;
+                    uint32_t word = lo | (hi << 16);
+                    memcpy(image + moff + (uint64_t)Lr * 16 + (uint64_t)j * 4, &word, 4);
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------- */
+/* The linear layer.  Y[m][n] = sum_k X[m][k] * What[n][k], k ascending.                        */
+
+/* double accumulation, rounded once to fp32 (Y32) and from that, RNE, to bf16 (Y16, optional) */
+int oracle_gemm_f64(const uint16_t* X, int64_t M, int64_t K, const uint16_t* What, int64_t N,
+                    float* Y32, uint16_t* Y16) {
+    if (!X || !What || !Y32) return -1;
+    if (M < 0 || K <= 0 || N <= 0) return -2;
+    int64_t MN = M * N;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < MN; ++i) {
+        int64_t m = i / N, n = i % N;
+        double acc = 0.0;
+        for (int64_t k = 0; k < K; ++k)
+            acc += (double)bf16_to_f32(X[m * K + k]) * (double)bf16_to_f32(What[n * K + k]);
+        float y = (float)acc;
+        Y32[i] = y;
+        if (Y16) Y16[i] = f32_to_bf16_rne(y);
+    }
+    return 0;
+}
+
+/* plain fp32 accumulation in k order: "an fp32 matmul on the same bf16-rounded inputs" */
+int oracle_gemm_f32(const uint16_t* X, int64_t M, int64_t K, const uint16_t* What, int64_t N,
+                    float* Y32) {
+    if (!X || !What || !Y32) return -1;
+    if (M < 0 || K <= 0 || N <= 0) return -2;
+    int64_t MN = M * N;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < MN; ++i) {
+        int64_t m = i / N, n = i % N;
+        volatile float acc = 0.0f; /* volatile: forbid reassociation / wider intermediates */
+        for (int64_t k = 0; k < K; ++k) {
+            float p = bf16_to_f32(X[m * K + k]) * bf16_to_f32(What[n * K + k]);
+            acc = acc + p;
+        }
+        Y32[i] = acc;
+    }
+    return 0;
+}
+
+/* Selected rows of Y only (for sampled parity at large M): rows[i] indexes X. */
+int oracle_gemm_f64_rows(const uint16_t* X, int64_t K, const int64_t* rows, int64_t n_rows,
+                         const uint16_t* What, int64_t N, float* Y32) {
+    if (!X || !What || !Y32 || !rows) return -1;
+    int64_t total = n_rows * N;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < total; ++i) {
+        int64_t m = rows[i / N], n = i % N;
+        double acc = 0.0;
+        for (int64_t k = 0; k < K; ++k)
+            acc += (double)bf16_to_f32(X[m * K + k]) * (double)bf16_to_f32(What[n * K + k]);
+        Y32[i] = (float)acc;
+    }
+    return 0;
+}
