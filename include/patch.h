@@ -1,0 +1,179 @@
+/*
+ * patch.h -- C ABI of the B200 (sm_100a) tile-hybrid linear layer  Y = X * What^T.
+ *
+ * The weight W [N x K] (N = out-features, K = in-features, row-major bf16) is cut into
+ * 128 x 128 tiles; a per-tile flag says whether the tile is stored dense or 2:4-sparse
+ * (two kept values of every four consecutive elements along K, plus two position bits per
+ * kept value).  This is the deployment format of PATCH (arXiv 2509.23410): the hard mask
+ * M* = M*_tile + (1 - M*_tile) (.) M*_2:4 of Algorithm 1 applied to W, compressed per tile
+ * ("Efficient deployment", Appendix A), and the matmul in which "tiles within a matrix
+ * [are] either dense or sparse" within one multiplication.
+ *
+ * General rules
+ *   - Every function returns a status (PATCH_OK = 0, errors negative).  Nothing throws,
+ *     prints or exits.  All argument validation happens on the host before any launch.
+ *   - Pointers named *_dev are device pointers, *_host are host pointers.  The library
+ *     allocates no device memory and keeps no global state; every buffer is the caller's.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
+ *     and return; patch_pack and patch_gemm_host are the exceptions noted below.
+ *   - Supported: tile_n = tile_k = 128, N % 128 == 0, K % 128 == 0, device pointers 16-byte
+ *     aligned, leading dimensions multiples of 8 elements.  Device must be sm_100
+ *     (PATCH_ERR_ARCH otherwise; there is no fallback path).
+ */
+#ifndef PATCH_B200_H_
+#define PATCH_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Tile kinds.  The flag is 1 - M*_tile of Algorithm 1 (the paper's tile mask is 1 = dense). */
+enum { PATCH_TILE_DENSE = 0, PATCH_TILE_SPARSE_2_4 = 1 };
+
+enum {
+    PATCH_OK = 0,
+    PATCH_ERR_NULL = -1,    /* a required pointer is NULL */
+    PATCH_ERR_SHAPE = -2,   /* N, K, M or a leading dimension is not supported */
+    PATCH_ERR_TILE = -3,    /* tile shape other than 128 x 128 */
+    PATCH_ERR_FLAG = -4,    /* a tile flag is neither DENSE nor SPARSE_2_4 */
+    PATCH_ERR_ALIGN = -5,   /* a device pointer or row pitch is not 16-byte aligned */
+    PATCH_ERR_SIZE = -6,    /* a buffer (packed blob, workspace) is too small */
+    PATCH_ERR_FORMAT = -7,  /* layout magic / version / offsets are inconsistent */
+    PATCH_ERR_ARCH = -8,    /* current device is not sm_100 */
+    PATCH_ERR_CUDA = -9,    /* a CUDA runtime call failed */
+    PATCH_ERR_TIMEOUT = -10 /* a bounded device-side wait expired (reported through status_dev) */
+};
+
+/* Kernel choice for patch_gemm_ex. */
+enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2 };
+
+/*
+ * Description of a packed blob.  Plain host struct, caller-owned, filled by patch_packed_size.
+ * The blob in device memory is position independent (offsets only):
+ *   [ header 256 B (a copy of this struct, zero padded)
+ *   | tile table: 16 B per tile in (tn, tk) row-major order, zero padded to a multiple of 1024 B
+ *   | payloads, each 1024-byte aligned: 32 768 B per dense tile, 18 432 B per 2:4 tile ]
+ * Table entry: { u32 kind, u32 payload_off / 16, u32 meta_off / 16 (0xFFFFFFFF if dense), u32 0 },
+ * offsets counted from the start of the blob.
+ *
+ * Payload bytes (the "device image"):
+ *   values are stored in 16 384-byte atoms of 128 rows x 64 bf16; inside an atom the 16-byte
+ *   chunk c (8 elements) of row r lives at (r/8)*1024 + (r%8)*128 + ((c ^ (r%8))*16), i.e. the
+ *   128-byte-swizzled K-major layout the tensor core reads from shared memory, so a linear
+ *   copy of the payload is ready to multiply.  A dense tile is two atoms (columns 0..63, then
+ *   64..127).  A 2:4 tile is one atom holding the 64 kept values of each row (in position
+ *   order), followed by 2 048 B of metadata: 128 rows x four u32; row L = 16q + 8h + i
+ *   (i < 8), word j: low 16 bits = the four 4-bit position codes (i0 | i1 << 2, i0 < i1) of
+ *   tile row 16q+i for columns [32j + 16h, 32j + 16h + 16), high 16 bits = the same for tile
+ *   row 16q+8+i.
+ */
+typedef struct patch_layout_t {
+    uint32_t magic;          /* 0x48435450 */
+    uint32_t version;        /* 1 */
+    int64_t  N, K;
+    int32_t  tile_n, tile_k;
+    int64_t  n_dense, n_sparse;
+    uint64_t table_off;      /* 256 */
+    uint64_t payload_off;    /* first payload byte */
+    uint64_t payload_bytes;  /* 32768 * n_dense + 18432 * n_sparse */
+    uint64_t total_bytes;    /* payload_off + payload_bytes = size of the blob */
+} patch_layout_t;
+
+/*
+ * Size and layout of the packed blob for a weight of N x K with the given tile flags.
+ * (Appendix A: compression "determined by the chosen tile size"; here fixed at 128 x 128.)
+ *   tile_flags_host  [N/128 x K/128] row-major bytes, PATCH_TILE_DENSE or PATCH_TILE_SPARSE_2_4
+ *   layout_out       filled on success
+ * Host only; touches no device.
+ */
+int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
+                      const uint8_t* tile_flags_host, patch_layout_t* layout_out);
+
+/*
+ * Compress W into the packed blob (the paper's `compress` step of the conversion pseudocode,
+ * Appendix A; mask semantics of Algorithm 1's last four lines).
+ * In every 2:4 tile, each group of four consecutive elements along K keeps its two largest
+ * magnitudes (equal magnitudes: lower index first; magnitude = bit pattern without sign);
+ * dense tiles are copied.  A weight that is already 2:4 inside those tiles is packed losslessly.
+ *   W_dev            bf16 [N x ldw], ldw >= K elements, ldw % 8 == 0
+ *   tile_flags_host  as for patch_packed_size; must be the flags `layout` was computed from
+ *   packed_dev       destination, packed_capacity >= layout->total_bytes, 1024-byte aligned
+ * Copies header and tile table host->device on `stream` (the host staging buffer is consumed
+ * before the call returns), then launches one kernel.  Every byte of the blob is written.
+ */
+int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* tile_flags_host,
+               const patch_layout_t* layout, void* packed_dev, size_t packed_capacity,
+               void* stream);
+
+/*
+ * Inverse of patch_pack: writes What = W (.) M* (pruned elements are +0) as bf16 [N x ldw].
+ */
+int patch_unpack(const patch_layout_t* layout, const void* packed_dev, void* What_dev,
+                 int64_t ldw, void* stream);
+
+/*
+ * Scratch memory patch_gemm needs for `M` tokens (may be 0 bytes).  The scratch holds fp32
+ * split-K partial sums and arrival counters of the small-M schedules ("alternative kernel
+ * execution schemes such as split-K parallelism", Appendix A).
+ */
+int patch_gemm_workspace_size(const patch_layout_t* layout, int64_t M, size_t* bytes_out);
+
+/*
+ * Zero a workspace once after allocating it (the arrival counters must start at zero; every
+ * successful patch_gemm leaves them zero again).
+ */
+int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
+ * Y = X * What^T with fp32 accumulation and bf16 (round-to-nearest-even) output: the hybrid
+ * dense / 2:4 tile matmul of Appendix A.  One kernel launch; no host synchronisation, no
+ * allocation, no host<->device copy.
+ *   X_dev   bf16 [M x ldx], ldx >= K, ldx % 8 == 0
+ *   Y_dev   bf16 [M x ldy], ldy >= N, ldy % 8 == 0
+ *   workspace_dev / workspace_bytes   at least patch_gemm_workspace_size(layout, M) bytes,
+ *           256-byte aligned, initialised once with patch_workspace_init; may be NULL if 0
+ *   status_dev   optional device int, must be zero before the call; receives
+ *           PATCH_ERR_TIMEOUT if a bounded device-side wait expired (the kernel then stops
+ *           early and Y is undefined).  NULL = not reported.
+ * M == 0 returns PATCH_OK without launching.  Calls sharing a workspace must be ordered on
+ * one stream.
+ */
+int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
+               const patch_layout_t* layout, const void* packed_dev,
+               void* Y_dev, int64_t ldy,
+               void* workspace_dev, size_t workspace_bytes, int* status_dev, void* stream);
+
+/* patch_gemm with an explicit kernel choice (benchmarks and tests).
+ *   PATCH_VARIANT_GEMV  CUDA-core decode kernel, M <= 8 only (PATCH_ERR_SHAPE otherwise)
+ *   PATCH_VARIANT_MMA   tcgen05 tensor-core kernel, any M */
+int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
+                  const patch_layout_t* layout, const void* packed_dev,
+                  void* Y_dev, int64_t ldy,
+                  void* workspace_dev, size_t workspace_bytes, int* status_dev, void* stream,
+                  int variant);
+
+/*
+ * End-to-end form with HOST activations and results: copies X host->device into
+ * X_stage_dev, runs patch_gemm, copies Y device->host and synchronises `stream`.
+ *   X_host  bf16 [M x K] contiguous; Y_host bf16 [M x N] contiguous (pinned memory advised)
+ *   X_stage_dev / Y_stage_dev   device staging buffers of M*K and M*N bf16
+ * The packed weight stays resident on the device.
+ */
+int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* layout,
+                    const void* packed_dev, void* Y_host,
+                    void* X_stage_dev, void* Y_stage_dev,
+                    void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Human-readable text for a status code (static storage). */
+const char* patch_strerror(int status);
+
+/* Library version (1). */
+int patch_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PATCH_B200_H_ */

@@ -1,0 +1,167 @@
+"""Thin ctypes binding over the C ABI declared in ``include/patch.h``.
+
+Argument marshalling only: every step of the path (mask selection, packing, the matmul, its
+split-K reduction and the bf16 epilogue) runs in the CUDA library.  There is no CPU fallback:
+if ``libpatch_b200.so`` is missing this module raises on first use.
+
+Tensors are torch CUDA tensors used purely as device buffers (``data_ptr()``); weights,
+activations and results are ``torch.bfloat16``; packed blobs and workspaces are ``torch.uint8``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpatch_b200.so")
+
+TILE_DENSE, TILE_SPARSE_2_4 = 0, 1
+VARIANT_AUTO, VARIANT_GEMV, VARIANT_MMA = 0, 1, 2
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
+ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
+
+EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
+           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_host",
+           "patch_strerror", "patch_version"]
+
+
+class Layout(ctypes.Structure):
+    """Mirror of ``patch_layout_t``."""
+    _fields_ = [("magic", ctypes.c_uint32), ("version", ctypes.c_uint32),
+                ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("tile_n", ctypes.c_int32), ("tile_k", ctypes.c_int32),
+                ("n_dense", ctypes.c_int64), ("n_sparse", ctypes.c_int64),
+                ("table_off", ctypes.c_uint64), ("payload_off", ctypes.c_uint64),
+                ("payload_bytes", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64)]
+
+
+class PatchError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2509_23410_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
+        L.patch_packed_size.argtypes = [i64, i64, ctypes.c_int, ctypes.c_int, vp, ctypes.POINTER(Layout)]
+        L.patch_pack.argtypes = [vp, i64, vp, ctypes.POINTER(Layout), vp, sz, vp]
+        L.patch_unpack.argtypes = [ctypes.POINTER(Layout), vp, vp, i64, vp]
+        L.patch_gemm_workspace_size.argtypes = [ctypes.POINTER(Layout), i64, ctypes.POINTER(sz)]
+        L.patch_workspace_init.argtypes = [vp, sz, vp]
+        L.patch_gemm.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, sz, vp, vp]
+        L.patch_gemm_ex.argtypes = L.patch_gemm.argtypes + [ctypes.c_int]
+        L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
+        L.patch_strerror.argtypes = [ctypes.c_int]
+        L.patch_strerror.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name != "patch_strerror":
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().patch_strerror(status).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise PatchError(status, where)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else ctypes.c_void_p(0)
+
+
+def _stream(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _flags_buf(flags):
+    import numpy as np
+    f = np.ascontiguousarray(flags, dtype=np.uint8).reshape(-1)
+    return f, ctypes.c_void_p(f.ctypes.data)
+
+
+def patch_packed_size(N: int, K: int, flags, tile_n: int = 128, tile_k: int = 128) -> Layout:
+    L = Layout()
+    f, fp = _flags_buf(flags)
+    _check(lib().patch_packed_size(N, K, tile_n, tile_k, fp, ctypes.byref(L)), "patch_packed_size")
+    return L
+
+
+def patch_pack(W, flags, layout: Layout | None = None, out=None, stream=None):
+    """Pack a bf16 CUDA weight [N x K]; returns (packed uint8 tensor, layout)."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    N, K = W.shape
+    if layout is None:
+        layout = patch_packed_size(N, K, flags)
+    if out is None:
+        out = torch.empty(layout.total_bytes, dtype=torch.uint8, device=W.device)
+    f, fp = _flags_buf(flags)
+    _check(lib().patch_pack(_ptr(W), W.stride(0), fp, ctypes.byref(layout), _ptr(out), out.numel(),
+                            _stream(stream)), "patch_pack")
+    return out, layout
+
+
+def patch_unpack(layout: Layout, packed, out=None, stream=None):
+    import torch
+    if out is None:
+        out = torch.empty((layout.N, layout.K), dtype=torch.bfloat16, device=packed.device)
+    _check(lib().patch_unpack(ctypes.byref(layout), _ptr(packed), _ptr(out), out.stride(0), _stream(stream)),
+           "patch_unpack")
+    return out
+
+
+def patch_gemm_workspace_size(layout: Layout, M: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().patch_gemm_workspace_size(ctypes.byref(layout), M, ctypes.byref(n)), "patch_gemm_workspace_size")
+    return int(n.value)
+
+
+def patch_workspace_init(workspace, stream=None):
+    if workspace is not None and workspace.numel():
+        _check(lib().patch_workspace_init(_ptr(workspace), workspace.numel(), _stream(stream)), "patch_workspace_init")
+
+
+def patch_gemm(X, layout: Layout, packed, Y=None, workspace=None, status=None, stream=None,
+               variant: int = VARIANT_AUTO):
+    """Y = X @ What^T.  X bf16 [M x K] (row stride >= K), returns Y bf16 [M x N]."""
+    import torch
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and (X.shape[0] == 0 or X.stride(1) == 1)
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, layout.N), dtype=torch.bfloat16, device=X.device)
+    ws_bytes = workspace.numel() if workspace is not None else 0
+    _check(lib().patch_gemm_ex(_ptr(X), X.stride(0) if M else layout.K, M, ctypes.byref(layout), _ptr(packed),
+                               _ptr(Y), Y.stride(0) if M else layout.N, _ptr(workspace), ws_bytes,
+                               _ptr(status), _stream(stream), variant), "patch_gemm")
+    return Y
+
+
+def patch_gemm_host(X_host, layout: Layout, packed, Y_host, X_stage, Y_stage, workspace=None, stream=None):
+    """End-to-end call with host (pinned) X and Y; synchronises the stream."""
+    M = X_host.shape[0]
+    ws_bytes = workspace.numel() if workspace is not None else 0
+    _check(lib().patch_gemm_host(_ptr(X_host), M, ctypes.byref(layout), _ptr(packed), _ptr(Y_host),
+                                 _ptr(X_stage), _ptr(Y_stage), _ptr(workspace), ws_bytes, _stream(stream)),
+           "patch_gemm_host")
+    return Y_host
+
+
+def patch_version() -> int:
+    return int(lib().patch_version())

@@ -1,0 +1,105 @@
+// C-ABI entry points of the matmul: argument validation and kernel choice.
+#include "patch_internal.cuh"
+
+using namespace patch;
+
+static int check_gemm_args(const void* X, int64_t ldx, int64_t M, const patch_layout_t* L, const void* packed,
+                           const void* Y, int64_t ldy) {
+    if (!L) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (M < 0) return PATCH_ERR_SHAPE;
+    if (M == 0) return PATCH_OK;
+    if (!X || !packed || !Y) return PATCH_ERR_NULL;
+    if (ldx < L->K || ldy < L->N || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(Y) || (reinterpret_cast<uintptr_t>(packed) & 1023u)) return PATCH_ERR_ALIGN;
+    return PATCH_OK;
+}
+
+extern "C" int patch_gemm_workspace_size(const patch_layout_t* L, int64_t M, size_t* bytes_out) {
+    if (!L || !bytes_out) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (M < 0) return PATCH_ERR_SHAPE;
+    *bytes_out = mma_workspace_bytes(L, M);
+    return PATCH_OK;
+}
+
+extern "C" int patch_workspace_init(void* workspace_dev, size_t bytes, void* stream) {
+    if (bytes == 0) return PATCH_OK;
+    if (!workspace_dev) return PATCH_ERR_NULL;
+    return cudaMemsetAsync(workspace_dev, 0, bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,
+                             const void* packed_dev, void* Y_dev, int64_t ldy, void* workspace_dev,
+                             size_t workspace_bytes, int* status_dev, void* stream, int variant) {
+    int rc = check_gemm_args(X_dev, ldx, M, L, packed_dev, Y_dev, ldy);
+    if (rc) return rc;
+    if (M == 0) return PATCH_OK;
+    if (variant != PATCH_VARIANT_AUTO && variant != PATCH_VARIANT_GEMV && variant != PATCH_VARIANT_MMA)
+        return PATCH_ERR_SHAPE;
+    if (variant == PATCH_VARIANT_GEMV && M > 4) return PATCH_ERR_SHAPE;
+    const size_t need = mma_workspace_bytes(L, M);
+    if (need > 0) {
+        if (!workspace_dev) return PATCH_ERR_NULL;
+        if (workspace_bytes < need) return PATCH_ERR_SIZE;
+        if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return PATCH_ERR_ALIGN;
+    }
+    rc = check_device();
+    if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(X_dev);
+    __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(Y_dev);
+    const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
+    if (variant == PATCH_VARIANT_AUTO) variant = M <= 2 ? PATCH_VARIANT_GEMV : PATCH_VARIANT_MMA;
+    if (variant == PATCH_VARIANT_GEMV) return launch_gemv(X, ldx, int(M), L, packed, Y, ldy, status_dev, s);
+    return launch_mma(X, ldx, M, L, packed, Y, ldy, workspace_dev, workspace_bytes, status_dev, s);
+}
+
+extern "C" int patch_gemm(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,
+                          const void* packed_dev, void* Y_dev, int64_t ldy, void* workspace_dev,
+                          size_t workspace_bytes, int* status_dev, void* stream) {
+    return patch_gemm_ex(X_dev, ldx, M, L, packed_dev, Y_dev, ldy, workspace_dev, workspace_bytes, status_dev,
+                         stream, PATCH_VARIANT_AUTO);
+}
+
+extern "C" int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* L, const void* packed_dev,
+                               void* Y_host, void* X_stage_dev, void* Y_stage_dev, void* workspace_dev,
+                               size_t workspace_bytes, void* stream) {
+    if (!L) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (M < 0) return PATCH_ERR_SHAPE;
+    if (M == 0) return PATCH_OK;
+    if (!X_host || !Y_host || !X_stage_dev || !Y_stage_dev) return PATCH_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(X_stage_dev, X_host, size_t(M) * L->K * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return PATCH_ERR_CUDA;
+    rc = patch_gemm(X_stage_dev, L->K, M, L, packed_dev, Y_stage_dev, L->N, workspace_dev, workspace_bytes,
+                    nullptr, stream);
+    if (rc) return rc;
+    if (cudaMemcpyAsync(Y_host, Y_stage_dev, size_t(M) * L->N * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return PATCH_ERR_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" const char* patch_strerror(int status) {
+    switch (status) {
+        case PATCH_OK: return "ok";
+        case PATCH_ERR_NULL: return "a required pointer is NULL";
+        case PATCH_ERR_SHAPE: return "unsupported shape or leading dimension";
+        case PATCH_ERR_TILE: return "tile shape must be 128 x 128";
+        case PATCH_ERR_FLAG: return "tile flag is neither dense nor 2:4";
+        case PATCH_ERR_ALIGN: return "pointer or pitch is not sufficiently aligned";
+        case PATCH_ERR_SIZE: return "buffer too small";
+        case PATCH_ERR_FORMAT: return "inconsistent packed layout";
+        case PATCH_ERR_ARCH: return "device is not sm_100";
+        case PATCH_ERR_CUDA: return "CUDA runtime error";
+        case PATCH_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int patch_version(void) { return 1; }

@@ -1,0 +1,239 @@
+// patch_packed_size / patch_pack / patch_unpack: the per-tile compression of the hybrid weight.
+//
+// Semantics follow the last lines of Algorithm 1 of the paper (hard mask
+// M* = M*_tile + (1 - M*_tile) (.) M*_2:4, What = W (.) M*) with magnitude top-2 selection per
+// group of four along K, and Appendix A's "compress" step (values + metadata per tile).
+// Both kernels are pure data movement plus integer compares, bound by HBM bandwidth:
+// per element of W they read 2 B and write 2 B (dense tile) or 1.125 B (2:4 tile).
+#include <vector>
+#include <cstring>
+#include "patch_internal.cuh"
+
+namespace patch {
+
+int validate_layout(const patch_layout_t* L) {
+    if (!L) return PATCH_ERR_NULL;
+    if (L->magic != kMagic || L->version != kVersion) return PATCH_ERR_FORMAT;
+    if (L->tile_n != kTile || L->tile_k != kTile) return PATCH_ERR_TILE;
+    if (L->N <= 0 || L->K <= 0 || L->N % kTile || L->K % kTile) return PATCH_ERR_SHAPE;
+    if (L->n_dense < 0 || L->n_sparse < 0) return PATCH_ERR_FORMAT;
+    uint64_t T = uint64_t(L->N / kTile) * uint64_t(L->K / kTile);
+    if (uint64_t(L->n_dense) + uint64_t(L->n_sparse) != T) return PATCH_ERR_FORMAT;
+    if (L->table_off != kHeaderBytes) return PATCH_ERR_FORMAT;
+    uint64_t pay = (kHeaderBytes + 16 * T + 1023) / 1024 * 1024;
+    if (L->payload_off != pay) return PATCH_ERR_FORMAT;
+    if (L->payload_bytes != uint64_t(kDenseBytes) * L->n_dense + uint64_t(kSparseBytes) * L->n_sparse)
+        return PATCH_ERR_FORMAT;
+    if (L->total_bytes != L->payload_off + L->payload_bytes) return PATCH_ERR_FORMAT;
+    if (L->total_bytes / 16 > 0xFFFFFFF0ull) return PATCH_ERR_SHAPE;  // offsets are stored as u32 * 16
+    return PATCH_OK;
+}
+
+int check_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PATCH_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return PATCH_ERR_CUDA;
+    return major == 10 ? PATCH_OK : PATCH_ERR_ARCH;
+}
+
+// ---------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Keep the two largest magnitudes of four bf16 values (ties: lower index first).
+// Returns the 4-bit position code i0 | (i1 << 2), i0 < i1, and the two kept bit patterns.
+__device__ __forceinline__ uint32_t top2_of_4(const uint32_t w[4], uint32_t& v0, uint32_t& v1) {
+    // distinct sort keys: magnitude in the high bits, reversed index in the low two bits
+    uint32_t key[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) key[j] = ((w[j] & 0x7FFFu) << 2) | uint32_t(3 - j);
+    bool keep[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        int before = 0;  // number of elements ordered before j
+#pragma unroll
+        for (int l = 0; l < 4; ++l) before += key[l] > key[j];
+        keep[j] = before < 2;
+    }
+    // exactly two are kept: the first kept index is at most 2, the second at least 1
+    const uint32_t i0 = keep[0] ? 0u : (keep[1] ? 1u : 2u);
+    const uint32_t i1 = keep[3] ? 3u : (keep[2] ? 2u : 1u);
+    v0 = keep[0] ? w[0] : (keep[1] ? w[1] : w[2]);
+    v1 = keep[3] ? w[3] : (keep[2] ? w[2] : w[1]);
+    return i0 | (i1 << 2);
+}
+
+// One CTA per tile.  W is read with 16-byte loads, the payload is written with 16-byte stores.
+__global__ void __launch_bounds__(256)
+pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob,
+            uint64_t table_off) {
+    const int t = blockIdx.x;
+    const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+    const int tn = t / TK, tk = t - tn * TK;
+    const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
+    uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
+    if (d.kind == PATCH_TILE_DENSE) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 4, c = idx & 15u;
+            const uint4 v = ld_stream(wt + int64_t(r) * ldw + c * 8);
+            *reinterpret_cast<uint4*>(pay + (c >> 3) * kAtomBytes + atom_chunk_offset(r, c & 7u)) = v;
+        }
+    } else {
+        uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            // 16 consecutive elements of one row: four groups -> 8 kept values + 16 metadata bits
+            const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 3, u = idx & 7u;
+            const uint16_t* src = wt + int64_t(r) * ldw + u * 16;
+            const uint4 a = ld_stream(src), b = ld_stream(src + 8);
+            const uint32_t in[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            uint32_t out[4], code = 0;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const uint32_t w[4] = {in[2 * g] & 0xFFFFu, in[2 * g] >> 16,
+                                       in[2 * g + 1] & 0xFFFFu, in[2 * g + 1] >> 16};
+                uint32_t v0, v1;
+                code |= top2_of_4(w, v0, v1) << (4 * g);
+                out[g] = v0 | (v1 << 16);
+            }
+            *reinterpret_cast<uint4*>(pay + atom_chunk_offset(r, u)) = make_uint4(out[0], out[1], out[2], out[3]);
+            // metadata row L = 16q + 8h + i, word j, low half for tile rows 16q+i, high for 16q+8+i
+            const uint32_t L = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
+            *reinterpret_cast<uint16_t*>(meta + L * 16 + j * 4 + hi * 2) = uint16_t(code);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+unpack_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
+              uint16_t* __restrict__ What, int64_t ldw) {
+    const int t = blockIdx.x;
+    const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+    const int tn = t / TK, tk = t - tn * TK;
+    uint16_t* wt = What + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
+    const uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
+    if (d.kind == PATCH_TILE_DENSE) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 4, c = idx & 15u;
+            const uint4 v = *reinterpret_cast<const uint4*>(pay + (c >> 3) * kAtomBytes + atom_chunk_offset(r, c & 7u));
+            *reinterpret_cast<uint4*>(wt + int64_t(r) * ldw + c * 8) = v;
+        }
+    } else {
+        const uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 3, u = idx & 7u;
+            const uint4 v = *reinterpret_cast<const uint4*>(pay + atom_chunk_offset(r, u));
+            const uint32_t L = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
+            const uint32_t code = *reinterpret_cast<const uint16_t*>(meta + L * 16 + j * 4 + hi * 2);
+            const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+            uint32_t out[8];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const uint32_t nib = (code >> (4 * g)) & 0xFu, i0 = nib & 3u, i1 = nib >> 2;
+                uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int j2 = 0; j2 < 4; ++j2) {
+                    if (uint32_t(j2) == i0) w[j2] = in[g] & 0xFFFFu;
+                    if (uint32_t(j2) == i1) w[j2] = in[g] >> 16;
+                }
+                out[2 * g] = w[0] | (w[1] << 16);
+                out[2 * g + 1] = w[2] | (w[3] << 16);
+            }
+            uint16_t* dst = wt + int64_t(r) * ldw + u * 16;
+            *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+            *reinterpret_cast<uint4*>(dst + 8) = make_uint4(out[4], out[5], out[6], out[7]);
+        }
+    }
+}
+
+}  // namespace patch
+
+using namespace patch;
+
+extern "C" int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
+                                 const uint8_t* flags, patch_layout_t* out) {
+    if (!flags || !out) return PATCH_ERR_NULL;
+    if (tile_n != kTile || tile_k != kTile) return PATCH_ERR_TILE;
+    if (N <= 0 || K <= 0 || N % kTile || K % kTile) return PATCH_ERR_SHAPE;
+    const int64_t T = (N / kTile) * (K / kTile);
+    int64_t nd = 0, ns = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        if (flags[t] == PATCH_TILE_DENSE) ++nd;
+        else if (flags[t] == PATCH_TILE_SPARSE_2_4) ++ns;
+        else return PATCH_ERR_FLAG;
+    }
+    patch_layout_t L;
+    std::memset(&L, 0, sizeof L);
+    L.magic = kMagic; L.version = kVersion;
+    L.N = N; L.K = K; L.tile_n = kTile; L.tile_k = kTile;
+    L.n_dense = nd; L.n_sparse = ns;
+    L.table_off = kHeaderBytes;
+    L.payload_off = (kHeaderBytes + 16 * uint64_t(T) + 1023) / 1024 * 1024;
+    L.payload_bytes = uint64_t(kDenseBytes) * nd + uint64_t(kSparseBytes) * ns;
+    L.total_bytes = L.payload_off + L.payload_bytes;
+    if (L.total_bytes / 16 > 0xFFFFFFF0ull) return PATCH_ERR_SHAPE;
+    *out = L;
+    return PATCH_OK;
+}
+
+extern "C" int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* flags,
+                          const patch_layout_t* L, void* packed_dev, size_t capacity, void* stream) {
+    if (!W_dev || !flags || !L || !packed_dev) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (ldw < L->K || ldw % 8) return PATCH_ERR_SHAPE;
+    if (!aligned16(W_dev) || (reinterpret_cast<uintptr_t>(packed_dev) & 1023u)) return PATCH_ERR_ALIGN;
+    if (capacity < L->total_bytes) return PATCH_ERR_SIZE;
+    const int64_t TK = L->K / kTile, T = (L->N / kTile) * TK;
+    // header + tile table, built on the host from the flags
+    std::vector<uint8_t> head(L->payload_off, 0);
+    std::memcpy(head.data(), L, sizeof *L);
+    TileDesc* table = reinterpret_cast<TileDesc*>(head.data() + L->table_off);
+    uint64_t off = L->payload_off;
+    int64_t nd = 0, ns = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        if (flags[t] == PATCH_TILE_DENSE) {
+            table[t] = TileDesc{PATCH_TILE_DENSE, uint32_t(off / 16), 0xFFFFFFFFu, 0};
+            off += kDenseBytes; ++nd;
+        } else if (flags[t] == PATCH_TILE_SPARSE_2_4) {
+            table[t] = TileDesc{PATCH_TILE_SPARSE_2_4, uint32_t(off / 16), uint32_t((off + kAtomBytes) / 16), 0};
+            off += kSparseBytes; ++ns;
+        } else return PATCH_ERR_FLAG;
+    }
+    if (nd != L->n_dense || ns != L->n_sparse) return PATCH_ERR_FORMAT;  // flags do not match the layout
+    rc = check_device();
+    if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // pageable source: the runtime stages it before returning, so `head` may die at scope exit
+    if (cudaMemcpyAsync(packed_dev, head.data(), head.size(), cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return PATCH_ERR_CUDA;
+    pack_kernel<<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                            static_cast<uint8_t*>(packed_dev), L->table_off);
+    return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_unpack(const patch_layout_t* L, const void* packed_dev, void* What_dev,
+                            int64_t ldw, void* stream) {
+    if (!L || !packed_dev || !What_dev) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (ldw < L->K || ldw % 8) return PATCH_ERR_SHAPE;
+    if (!aligned16(What_dev) || !aligned16(packed_dev)) return PATCH_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    const int64_t TK = L->K / kTile, T = (L->N / kTile) * TK;
+    unpack_kernel<<<unsigned(T), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(packed_dev), L->table_off, int(TK),
+        static_cast<uint16_t*>(What_dev), ldw);
+    return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}

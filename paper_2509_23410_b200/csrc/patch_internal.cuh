@@ -1,0 +1,51 @@
+// Internal definitions shared by the library's translation units (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/patch.h"
+
+namespace patch {
+
+constexpr uint32_t kMagic = 0x48435450u;
+constexpr uint32_t kVersion = 1u;
+constexpr int kTile = 128;
+constexpr uint32_t kDenseBytes = 32768u;    // two 16 KB atoms
+constexpr uint32_t kSparseBytes = 18432u;   // one 16 KB atom + 2 KB metadata
+constexpr uint32_t kAtomBytes = 16384u;
+constexpr uint32_t kMetaBytes = 2048u;
+constexpr uint32_t kHeaderBytes = 256u;
+
+// One entry of the tile table inside the packed blob.
+struct TileDesc {
+    uint32_t kind;          // PATCH_TILE_DENSE / PATCH_TILE_SPARSE_2_4
+    uint32_t payload_off16; // byte offset / 16 from the start of the blob
+    uint32_t meta_off16;    // byte offset / 16 of the metadata block, 0xFFFFFFFF if dense
+    uint32_t reserved;
+};
+static_assert(sizeof(TileDesc) == 16, "tile table entry is 16 bytes");
+
+// Byte offset of 16-byte chunk `c` (0..7) of row `r` (0..127) inside a 128-byte-swizzled
+// K-major atom of 128 rows x 128 bytes.
+__host__ __device__ inline uint32_t atom_chunk_offset(uint32_t r, uint32_t c) {
+    return (r >> 3) * 1024u + (r & 7u) * 128u + ((c ^ (r & 7u)) << 4);
+}
+
+// Host-side checks of a layout struct handed in by the caller.
+int validate_layout(const patch_layout_t* L);
+
+// Status of the current device: PATCH_OK if it is sm_100, PATCH_ERR_ARCH / PATCH_ERR_CUDA otherwise.
+int check_device();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Kernel launchers implemented in the .cu files; all return a PATCH_* status.
+int launch_gemv(const __nv_bfloat16* X, int64_t ldx, int M, const patch_layout_t* L,
+                const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev,
+                cudaStream_t stream);
+int launch_mma(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
+               const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace,
+               size_t workspace_bytes, int* status_dev, cudaStream_t stream);
+size_t mma_workspace_bytes(const patch_layout_t* L, int64_t M);
+
+}  // namespace patch

@@ -1,0 +1,95 @@
+"""Host-side checks of the C ABI: the library loads without a GPU, exports every symbol the
+header declares, and rejects bad arguments before touching a device."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2509_23410_b200 import build
+    build.build()
+    from paper_2509_23410_b200 import binding as b
+    return b
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "patch.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(patch_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(binding):
+    names = declared_functions()
+    assert "patch_gemm" in names and "patch_pack" in names and len(names) >= 9
+    L = binding.lib()
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_layout_struct_matches_header(binding):
+    assert ctypes.sizeof(binding.Layout) == 80
+    assert binding.patch_version() == 1
+
+
+def test_packed_size_and_validation(binding, oracle):
+    flags = np.array([[0, 1, 1], [1, 0, 0]], np.uint8)
+    L = binding.patch_packed_size(256, 384, flags)
+    Lo = oracle.packed_size(256, 384, flags)
+    for f, _ in binding.Layout._fields_:
+        assert getattr(L, f) == getattr(Lo, f), f
+    assert L.payload_bytes == 3 * 32768 + 3 * 18432
+    with pytest.raises(binding.PatchError) as e:
+        binding.patch_packed_size(256, 384, np.full((2, 3), 2, np.uint8))
+    assert e.value.status == binding.ERR_FLAG
+    with pytest.raises(binding.PatchError) as e:
+        binding.patch_packed_size(250, 384, flags)
+    assert e.value.status == binding.ERR_SHAPE
+    with pytest.raises(binding.PatchError) as e:
+        binding.patch_packed_size(256, 384, flags, 64, 128)
+    assert e.value.status == binding.ERR_TILE
+
+
+def test_gemm_rejects_bad_arguments_on_host(binding):
+    lib = binding.lib()
+    flags = np.zeros((1, 1), np.uint8)
+    L = binding.patch_packed_size(128, 128, flags)
+    null = ctypes.c_void_p(0)
+    fake = ctypes.c_void_p(1024 * 1024)   # never dereferenced: validation fails first
+    args = lambda X, ldx, M, Lp, P, Y, ldy: (X, ldx, M, Lp, P, Y, ldy, null, 0, null, null)
+    assert lib.patch_gemm(*args(null, 128, 4, ctypes.byref(L), fake, fake, 128)) == binding.ERR_NULL
+    assert lib.patch_gemm(*args(fake, 64, 4, ctypes.byref(L), fake, fake, 128)) == binding.ERR_SHAPE
+    assert lib.patch_gemm(*args(fake, 128, 4, ctypes.byref(L), fake, fake, 100)) == binding.ERR_SHAPE
+    assert lib.patch_gemm(*args(ctypes.c_void_p(1024 * 1024 + 2), 128, 4, ctypes.byref(L), fake, fake, 128)) == binding.ERR_ALIGN
+    assert lib.patch_gemm(*args(fake, 128, -1, ctypes.byref(L), fake, fake, 128)) == binding.ERR_SHAPE
+    assert lib.patch_gemm(*args(null, 128, 0, ctypes.byref(L), null, null, 128)) == binding.OK   # M = 0: no launch
+    bad = binding.Layout.from_buffer_copy(bytes(L))
+    bad.magic = 0
+    assert lib.patch_gemm(*args(fake, 128, 4, ctypes.byref(bad), fake, fake, 128)) == binding.ERR_FORMAT
+    bad = binding.Layout.from_buffer_copy(bytes(L))
+    bad.payload_bytes += 1024
+    assert lib.patch_gemm(*args(fake, 128, 4, ctypes.byref(bad), fake, fake, 128)) == binding.ERR_FORMAT
+    bad = binding.Layout.from_buffer_copy(bytes(L))
+    bad.tile_k = 64
+    assert lib.patch_gemm(*args(fake, 128, 4, ctypes.byref(bad), fake, fake, 128)) == binding.ERR_TILE
+    assert lib.patch_gemm_ex(*args(fake, 128, 9, ctypes.byref(L), fake, fake, 128), binding.VARIANT_GEMV) == binding.ERR_SHAPE
+    assert lib.patch_pack(null, 128, null, ctypes.byref(L), fake, 1 << 20, null) == binding.ERR_NULL
+    f = np.zeros(1, np.uint8)
+    assert lib.patch_pack(fake, 128, ctypes.c_void_p(f.ctypes.data), ctypes.byref(L), fake, 10, null) == binding.ERR_SIZE
+    assert b"timed out" in lib.patch_strerror(binding.ERR_TIMEOUT)
+
+
+def test_product_package_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2509_23410_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, fn)).read()
+                assert "import oracle" not in text and "from oracle" not in text, fn
+                assert "patch_oracle" not in text, fn
