@@ -1,0 +1,444 @@
+#!/usr/bin/env python
+"""Benchmark of the tile-hybrid linear layer (hybrid dense / 2:4 tile GEMM) on B200.
+
+One step = one pass of the hot path over one batch of synthetic input: every GEMM of the
+workload's case list, launched back to back from one CUDA graph (the paper times generation
+through CUDA graphs as well).  Default workload: the LLaMA-2-7B-shaped decode linears
+(3 weight shapes x 2:4-tile fraction in {0, .35, .7, 1} x M in {1, 16} = 24 GEMMs over 12
+packed matrices, ~0.66 GB of packed weights per pass, so every weight read comes from HBM).
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_23410_b200 import inputs  # noqa: E402
+
+HBM_SPEC_GBS = 8000.0            # roofline constants of the task definition
+DENSE_SPEC_TFLOPS = 2250.0
+SPARSE_SPEC_TFLOPS = 4500.0
+L2_BYTES = 126e6
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def workload_cases(name: str):
+    if name == "decode":
+        cases = inputs.decode_cases()
+        # all M=1 GEMMs first, then all M=16: a matrix is re-read only after ~0.66 GB of other weights
+        return sorted(cases, key=lambda c: c["M"])
+    if name == "prefill":
+        return sorted(inputs.prefill_cases(), key=lambda c: c["M"])
+    if name == "13b":
+        return sorted(inputs.llama13b_cases(), key=lambda c: c["M"])
+    if name == "single":
+        return [inputs.single_gemm_case()]
+    raise SystemExit(f"unknown workload {name}")
+
+
+def case_costs(case, layout):
+    """Algorithmic bytes and flops of one GEMM (realised tile counts, not expected ones)."""
+    M, N, K = case["M"], case["N"], case["K"]
+    T = (N // 128) * (K // 128)
+    nbytes = layout.payload_bytes + 16 * T + M * K * 2 + M * N * 2
+    f_dense = 2.0 * M * 16384 * layout.n_dense
+    f_sparse = 2.0 * M * 16384 * layout.n_sparse
+    return dict(bytes=float(nbytes), flops=f_dense + f_sparse, f_dense=f_dense, f_sparse=f_sparse)
+
+
+def roofline_seconds(cost, hbm_gbs, dense_tf, sparse_tf):
+    t_mem = cost["bytes"] / (hbm_gbs * 1e9)
+    t_tc = cost["f_dense"] / (dense_tf * 1e12) + cost["f_sparse"] / (sparse_tf * 1e12)
+    return max(t_mem, t_tc), ("hbm" if t_mem >= t_tc else "tensor")
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks sampler
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.samples = []
+        self.proc = None
+        self.index = index
+        self.marks = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.12)
+        self.proc.terminate()
+        rows = [s for t, s in self.samples if t0 - 0.05 <= t <= t1 + 0.1] or [s for _, s in self.samples[-3:]]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+
+
+def oracle_sample(cases, budget_s):
+    """Time the oracle GEMM on the leading cases of the step until ~budget_s of CPU work."""
+    import oracle
+    oracle.build()
+    done, flops, secs = [], 0.0, 0.0
+    for case in cases:
+        W, flags, X = inputs.make_case_inputs(case)
+        What = oracle.prune(W, flags)
+        t = time.perf_counter()
+        oracle.gemm_f64(X, What, want_bf16=True)
+        dt = time.perf_counter() - t
+        secs += dt
+        flops += 2.0 * case["M"] * case["N"] * case["K"]
+        done.append(case["name"])
+        if secs >= budget_s:
+            break
+    return dict(value=flops / secs / 1e12, unit="TFLOP/s", cores=oracle.num_threads(), kind="oracle",
+                sample=f"oracle GEMM (double accumulation) on the first {len(done)} GEMMs of the step "
+                       f"({done[0]} .. {done[-1]}), {secs:.1f} s of CPU time"), secs
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    cases = workload_cases(args.workload)
+    # bounded sample per step: the two GEMMs (M = 1 and 16) on the first 4096 x 4096 matrix with mixed tiles
+    sample = [c for c in cases if c["N"] == 4096 and c["K"] == 4096 and 0 < c["p"] < 1][:1]
+    sample += [c for c in cases if c["N"] == 4096 and c["K"] == 4096 and 0 < c["p"] < 1 and c["M"] != sample[0]["M"]][:1]
+    prepared = []
+    for c in sample:
+        W, flags, X = inputs.make_case_inputs(c)
+        prepared.append((X, oracle.prune(W, flags), 2.0 * c["M"] * c["N"] * c["K"]))
+    steps = min(args.steps, 50)
+    for _ in range(min(args.warmup, 3)):
+        for X, What, _ in prepared:
+            oracle.gemm_f64(X, What)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        for X, What, _ in prepared:
+            oracle.gemm_f64(X, What)
+    dt = time.perf_counter() - t0
+    flops = sum(f for _, _, f in prepared) * steps
+    value = flops / dt / 1e12
+    names = ", ".join(c["name"] for c in sample)
+    cpu = dict(value=value, unit="TFLOP/s", cores=oracle.num_threads(), kind="oracle",
+               sample=f"{steps} steps of the oracle GEMM on {names}")
+    print(json.dumps({
+        "impl": "reference", "metric": "hybrid_tile_gemm_effective_tflops", "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 3), "ms_per_step": dt / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": names},
+        "cpu_baseline": cpu,
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------------------------
+# our arm
+
+
+def run_ours(args):
+    import torch
+    from paper_2509_23410_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()
+    peaks = measured_peaks()
+
+    def to_dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    cases = workload_cases(args.workload)
+    # ---- setup (untimed): weights, packing, activations; replicas: every rank holds the whole workload
+    mats = {}
+    pack_bytes, pack_secs = 0.0, 0.0
+    for c in cases:
+        key = (c["N"], c["K"], c["stream"])
+        if key in mats:
+            continue
+        W = to_dev(inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]))
+        flags = inputs.tile_flags(c["N"], c["K"], c["p"], inputs.MASTER_SEED, *c["stream"])
+        layout = B.patch_packed_size(c["N"], c["K"], flags)
+        packed = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
+        B.patch_pack(W, flags, layout=layout, out=packed)          # warm
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.patch_pack(W, flags, layout=layout, out=packed)
+        e1.record()
+        torch.cuda.synchronize()
+        pack_secs += e0.elapsed_time(e1) * 1e-3
+        pack_bytes += c["N"] * c["K"] * 2 + layout.total_bytes
+        mats[key] = (layout, packed)
+        del W
+    jobs = []
+    for c in cases:
+        layout, packed = mats[(c["N"], c["K"], c["stream"])]
+        X = to_dev(inputs.activation(c["M"], c["K"], inputs.MASTER_SEED, *c["stream"], c["M"]))
+        Y = torch.empty((c["M"], c["N"]), dtype=torch.bfloat16, device=dev)
+        ws = torch.zeros(max(B.patch_gemm_workspace_size(layout, c["M"]), 256), dtype=torch.uint8, device=dev)
+        jobs.append(dict(case=c, layout=layout, packed=packed, X=X, Y=Y, ws=ws, cost=case_costs(c, layout)))
+    weight_bytes = sum(m[0].total_bytes for m in mats.values())
+
+    # weights are packed once, before any step; in this workload no GEMM reads another GEMM's output
+    launch_flags = B.WEIGHTS_STATIC | (B.INPUT_STATIC if args.launch == "independent" else 0)
+
+    def launch_all(js):
+        for j in js:
+            B.patch_gemm(j["X"], j["layout"], j["packed"], Y=j["Y"], workspace=j["ws"],
+                         variant=args.variant | launch_flags)
+
+    def make_graph(js):
+        launch_all(js)                      # first call sets kernel attributes; must precede capture
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            launch_all(js)
+        return g
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def time_graph(g, reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / reps
+
+    step_graph = make_graph(jobs)
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step_graph.replay()
+    barrier()
+    t_wall0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step_graph.replay()
+    e1.record()
+    barrier()
+    secs = e0.elapsed_time(e1) * 1e-3
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([secs], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        secs = float(t.item())
+    step_s = secs / args.steps
+    step_flops = sum(j["cost"]["flops"] for j in jobs)
+    value = world * step_flops / step_s / 1e12
+
+    # ---- dominant kernel: the launches that take the largest share of the step, timed on their own
+    groups = {}
+    for j in jobs:
+        groups.setdefault(j["case"]["M"], []).append(j)
+    dom = None
+    for M, js in groups.items():
+        g = make_graph(js)
+        for _ in range(3):
+            g.replay()
+        t = time_graph(g, max(10, args.steps // 10))
+        if dom is None or t > dom[1]:
+            dom = (M, t, js)
+    dM, dt, djs = dom
+    kernel_name = B_kernel_name(dM)
+    bound = roofline_seconds(djs[0]["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)[1]
+    per_launch = dt / len(djs)
+    if bound == "hbm":
+        alg = sum(j["cost"]["bytes"] for j in djs) / len(djs)
+        achieved, peak, unit = alg / per_launch / 1e9, peaks["hbm_gbs"], "GB/s"
+    else:
+        alg = sum(j["cost"]["flops"] for j in djs) / len(djs)
+        # mixed dense / sparse contraction: the peak is the flop-weighted mix (sparse tiles at twice the dense rate)
+        fd = sum(j["cost"]["f_dense"] for j in djs)
+        fs = sum(j["cost"]["f_sparse"] for j in djs)
+        achieved, unit = alg / per_launch / 1e12, "TFLOP/s"
+        peak = (fd + fs) / (fd / peaks["bf16_tflops_sustained"] + fs / (2 * peaks["bf16_tflops_sustained"]))
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    roof = dict(bound=bound, achieved=achieved, peak=peak, unit=unit, frac=achieved / peak,
+                traffic=load_traffic(kernel_name), kernel=kernel_name, launches_timed=len(djs),
+                us_per_launch=per_launch * 1e6, peak_source=peaks["source"],
+                algorithmic_per_launch=alg)
+    spec_t = sum(roofline_seconds(j["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)[0] for j in jobs)
+    meas_t = sum(roofline_seconds(j["cost"], peaks["hbm_gbs"], peaks["bf16_tflops_sustained"],
+                                  2 * peaks["bf16_tflops_sustained"])[0] for j in jobs)
+
+    # ---- end to end through the host-buffer entry point (H2D of X and D2H of Y inside the timed region)
+    for j in jobs:
+        j["Xh"] = j["X"].cpu().pin_memory()
+        j["Yh"] = torch.empty(j["Y"].shape, dtype=torch.bfloat16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 200))
+
+    def e2e_step():
+        for j in jobs:
+            B.patch_gemm_host(j["Xh"], j["layout"], j["packed"], j["Yh"], j["X"], j["Y"], j["ws"])
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    h2d = sum(j["X"].numel() * 2 for j in jobs)
+    d2h = sum(j["Y"].numel() * 2 for j in jobs)
+
+    # ---- per-case table (each GEMM on rotating copies of its packed weight so reads come from HBM)
+    table = []
+    if args.detail and rank == 0:
+        for j in jobs:
+            blob = j["packed"]
+            n_copies = int(min(max(3 * L2_BYTES // blob.numel() + 1, 2), 24))
+            copies = [blob.clone() for _ in range(n_copies)]
+            js = [dict(j, packed=cp) for cp in copies]
+            g = make_graph(js)
+            for _ in range(3):
+                g.replay()
+            t = time_graph(g, 10) / n_copies
+            rs, b = roofline_seconds(j["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)
+            rm, _ = roofline_seconds(j["cost"], peaks["hbm_gbs"], peaks["bf16_tflops_sustained"],
+                                     2 * peaks["bf16_tflops_sustained"])
+            table.append(dict(name=j["case"]["name"], us=round(t * 1e6, 2),
+                              eff_tflops=round(j["cost"]["flops"] / t / 1e12, 2), bound=b,
+                              frac_spec=round(rs / t, 3), frac_measured=round(rm / t, 3),
+                              f_sparse=round(j["layout"].n_sparse / (j["layout"].n_sparse + j["layout"].n_dense), 3)))
+            del copies, js, g
+
+    if rank != 0:
+        return
+    cpu, _ = oracle_sample(cases, args.cpu_budget) if world == 1 else (None, 0)
+    out = {
+        "metric": "hybrid_tile_gemm_effective_tflops", "value": value, "unit": "TFLOP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"llama2-7b {args.workload} linears" if args.workload != "13b" else "llama2-13b linears",
+                   "gemms_per_step": len(jobs), "tile": "128x128",
+                   "packed_weight_bytes": weight_bytes,
+                   "l2": "inputs larger than L2: each step streams all packed matrices once per M",
+                   "multi_gpu": "replicas only" if world > 1 else "single gpu", "cuda_graph": True,
+                   "launch": args.launch},
+        "us_per_gemm": step_s / len(jobs) * 1e6,
+        "frac_of_roofline_spec": spec_t / step_s, "frac_of_roofline_measured": meas_t / step_s,
+        "roofline": roof,
+        "e2e": {"value": world * step_flops / e2e_s / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3},
+        "gpu_launches": args.steps * len(jobs),
+        "clocks": clocks,
+        "pack": {"gbs": pack_bytes / pack_secs / 1e9, "frac_of_measured_hbm": pack_bytes / pack_secs / 1e9 / peaks["hbm_gbs"]},
+    }
+    if cpu is not None:
+        out["cpu_baseline"] = cpu
+    if table:
+        out["cases"] = table
+    print(json.dumps(out))
+
+
+def B_kernel_name(M):
+    return "gemv_kernel" if M <= 2 else "mma_kernel"
+
+
+def load_traffic(kernel):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as fh:
+            return json.load(fh).get(kernel)
+    except (OSError, ValueError):
+        return None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single"])
+    ap.add_argument("--launch", default="dependent", choices=["dependent", "independent"],
+                    help="dependent: every GEMM waits for the previous one before reading X; independent: "
+                         "the caller promises X is not produced by the preceding kernel")
+    ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 decode GEMV (M <= 4), 2 tensor-core kernel")
+    ap.add_argument("--detail", action="store_true", help="add the per-GEMM table (us, TFLOP/s, roofline fraction)")
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -47,8 +47,18 @@ enum {
     PATCH_ERR_TIMEOUT = -10 /* a bounded device-side wait expired (reported through status_dev) */
 };
 
-/* Kernel choice for patch_gemm_ex. */
+/* Kernel choice for patch_gemm_ex (low bits), optionally OR-ed with PATCH_GEMM_WEIGHTS_STATIC. */
 enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2 };
+/* Promise that the packed weight was NOT written by the operation that precedes this call in
+ * the stream (the serving case: weights are packed once, offline).  The kernel is launched with
+ * programmatic dependent launch either way; with this flag it also requests its first weight
+ * tiles before the previous kernel has finished.  Activations and outputs always wait. */
+enum { PATCH_GEMM_WEIGHTS_STATIC = 0x100 };
+/* Promise (only honoured together with PATCH_GEMM_WEIGHTS_STATIC) that X was NOT written by the
+ * operation that precedes this call in the stream (e.g. the k projection after the q projection,
+ * which read the same X).  Activations are then fetched without waiting for the previous
+ * kernel; writes to Y and to the workspace still wait for it. */
+enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
 
 /*
  * Description of a packed blob.  Plain host struct, caller-owned, filled by patch_packed_size.
@@ -146,9 +156,10 @@ int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
                void* Y_dev, int64_t ldy,
                void* workspace_dev, size_t workspace_bytes, int* status_dev, void* stream);
 
-/* patch_gemm with an explicit kernel choice (benchmarks and tests).
- *   PATCH_VARIANT_GEMV  CUDA-core decode kernel, M <= 8 only (PATCH_ERR_SHAPE otherwise)
- *   PATCH_VARIANT_MMA   tcgen05 tensor-core kernel, any M */
+/* patch_gemm with an explicit kernel choice and options.
+ *   PATCH_VARIANT_GEMV  CUDA-core decode kernel, M <= 4 only (PATCH_ERR_SHAPE otherwise)
+ *   PATCH_VARIANT_MMA   tcgen05 tensor-core kernel, any M
+ *   | PATCH_GEMM_WEIGHTS_STATIC  see above */
 int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
                   const patch_layout_t* layout, const void* packed_dev,
                   void* Y_dev, int64_t ldy,

@@ -17,6 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libpatch_b200.so")
 
 TILE_DENSE, TILE_SPARSE_2_4 = 0, 1
 VARIANT_AUTO, VARIANT_GEMV, VARIANT_MMA = 0, 1, 2
+WEIGHTS_STATIC = 0x100   # OR into `variant`: the packed weight is not produced by the preceding kernel
+INPUT_STATIC = 0x200     # OR into `variant`: X is not produced by the preceding kernel
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10

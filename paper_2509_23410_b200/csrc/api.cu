@@ -21,7 +21,7 @@ extern "C" int patch_gemm_workspace_size(const patch_layout_t* L, int64_t M, siz
     int rc = validate_layout(L);
     if (rc) return rc;
     if (M < 0) return PATCH_ERR_SHAPE;
-    *bytes_out = mma_workspace_bytes(L, M);
+    *bytes_out = decode_workspace_bytes(L, M);
     return PATCH_OK;
 }
 
@@ -38,10 +38,13 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     int rc = check_gemm_args(X_dev, ldx, M, L, packed_dev, Y_dev, ldy);
     if (rc) return rc;
     if (M == 0) return PATCH_OK;
+    const bool wstatic = (variant & PATCH_GEMM_WEIGHTS_STATIC) != 0;
+    const bool xstatic = (variant & PATCH_GEMM_INPUT_STATIC) != 0;
+    variant &= ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC);
     if (variant != PATCH_VARIANT_AUTO && variant != PATCH_VARIANT_GEMV && variant != PATCH_VARIANT_MMA)
         return PATCH_ERR_SHAPE;
     if (variant == PATCH_VARIANT_GEMV && M > 4) return PATCH_ERR_SHAPE;
-    const size_t need = mma_workspace_bytes(L, M);
+    const size_t need = decode_workspace_bytes(L, M);
     if (need > 0) {
         if (!workspace_dev) return PATCH_ERR_NULL;
         if (workspace_bytes < need) return PATCH_ERR_SIZE;
@@ -53,9 +56,9 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(X_dev);
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(Y_dev);
     const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
-    if (variant == PATCH_VARIANT_AUTO) variant = M <= 2 ? PATCH_VARIANT_GEMV : PATCH_VARIANT_MMA;
     if (variant == PATCH_VARIANT_GEMV) return launch_gemv(X, ldx, int(M), L, packed, Y, ldy, status_dev, s);
-    return launch_mma(X, ldx, M, L, packed, Y, ldy, workspace_dev, workspace_bytes, status_dev, s);
+    if (M <= 64) return launch_decode(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s, wstatic, xstatic);
+    return launch_prefill(X, ldx, M, L, packed, Y, ldy, status_dev, s);
 }
 
 extern "C" int patch_gemm(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,

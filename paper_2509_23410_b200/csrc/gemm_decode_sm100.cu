@@ -1,0 +1,465 @@
+// Small-M (decode) schedule of the hybrid dense / 2:4 tile matmul on the sm_100a tensor cores.
+//
+// The paper names decode as "the primary bottleneck" of generation and split-K as the schedule
+// its inspector picks there (Appendix A).  At M <= 64 tokens the layer is bound by the bytes of
+// the packed weight, so the whole design serves one purpose: keep HBM busy.
+//
+//   * Work = the T = TN x TK weight tiles in (tn, tk) order.  One CTA per SM; CTA c streams the
+//     contiguous run of tiles whose payload starts in the c-th 1/G of the payload bytes (a
+//     byte-balanced split-K: a 2:4 tile costs 9/16 of a dense one).  The run boundaries are
+//     found by a two-level warp-parallel search over the tile table.
+//   * Per tile the MMA warp issues eight dense tcgen05.mma or four tcgen05.mma.sp (metadata
+//     copied to TMEM) into an fp32 TMEM accumulator [128 out-features x N_TOK tokens]; weights
+//     are the A operand, tokens ride the MMA N dimension (16/32/64).
+//   * A run covers at most one partial row-block at each end.  Partial sums go to the caller's
+//     workspace; a 64-bit counter per row-block collects {tiles, contributors, first
+//     contributor}.  The CTA that completes the tile count sums the partials in ascending K
+//     order (deterministic) and writes bf16.  Two TMEM accumulators let this epilogue overlap
+//     the next row-block's MMAs.
+//   * The kernel uses half an SM's shared memory and is launched with programmatic dependent
+//     launch: the next GEMM's CTAs become resident while this one streams, fetch their first
+//     weight tiles, and wait for this grid only where they touch X, Y or the workspace.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports
+// PATCH_ERR_TIMEOUT through status_dev, drains its copies in flight, frees TMEM and returns.
+#include "sm100_ptx.cuh"
+
+namespace patch {
+
+constexpr int kMaxDecodeCtas = 192;      // workspace is sized for this many CTAs
+
+template <int N_TOK, int STAGES>
+struct DecodeConfig {
+    static constexpr uint32_t kXAtomBytes = N_TOK * 128;           // N_TOK rows x 64 bf16
+    static constexpr uint32_t kXBytes = 2 * kXAtomBytes;           // 128 columns of K
+    static constexpr uint32_t kStageBytes = kDenseBytes + kXBytes;
+    static constexpr uint32_t kBarrierOffset = STAGES * kStageBytes;
+    static constexpr uint32_t kSmemBytes = kBarrierOffset + 256 + 1024;  // + barriers + alignment slack
+    static constexpr uint32_t kTmemNeeded = 2 * N_TOK + 4 * STAGES;      // two accumulators + metadata
+    static constexpr uint32_t kTmemCols = kTmemNeeded <= 32 ? 32 : kTmemNeeded <= 64 ? 64 : kTmemNeeded <= 128 ? 128
+                                          : kTmemNeeded <= 256 ? 256 : 512;
+    static_assert(N_TOK % 16 == 0 && N_TOK >= 16 && N_TOK <= 64, "decode schedule: MMA N in {16, 32, 48, 64}");
+    static_assert(STAGES >= 2 && STAGES <= 8, "2..8 pipeline stages");
+};
+
+// Number of table entries base[i * stride] (i < n) that are < target, over a whole warp.
+__device__ __forceinline__ int warp_count_below(const uint32_t* base, int64_t stride_words, int n, uint32_t target,
+                                                int lane) {
+    int cnt = 0;
+    for (int i = lane; i < n; i += 32) cnt += __ldg(base + int64_t(i) * stride_words) < target;
+    return __reduce_add_sync(0xFFFFFFFFu, cnt);
+}
+
+// First tile whose payload offset (in 16-byte units) is >= target.  Offsets increase with the
+// tile index, so: find the last row-block starting below target, then count inside it.
+__device__ __forceinline__ int first_tile_at_or_after(const TileDesc* table, int TN, int TK, uint32_t target, int lane) {
+    const uint32_t* off = &table[0].payload_off16;
+    const int nb = warp_count_below(off, int64_t(TK) * 4, TN, target, lane);
+    if (nb == 0) return 0;
+    const int jb = nb - 1;
+    return jb * TK + warp_count_below(off + int64_t(jb) * TK * 4, 4, TK, target, lane);
+}
+
+__device__ __forceinline__ unsigned long long atom_add_acq_rel_gpu(unsigned long long* p, unsigned long long v) {
+    unsigned long long old;
+    asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], %2;" : "=l"(old) : "l"(p), "l"(v) : "memory");
+    return old;
+}
+
+// Barrier over the 128 epilogue threads that also ANDs a predicate.
+__device__ __forceinline__ bool epilogue_all(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"(uint32_t(pred)) : "memory");
+    return r != 0;
+}
+
+// L2 load that the compiler keeps in program order, so that a batch of them is issued back to
+// back before the first result is consumed.
+__device__ __forceinline__ uint4 ld_cg_issue(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Last contributor of a row-block: sum the partial tiles in ascending K order (contributor
+// order), 16 tokens at a time, and write bf16.  `info` = {tiles:16, contributors:16, first
+// contributor's slot + 1 : 32}; later contributors are the following CTAs' first slots.
+// Loads are unconditional (indices clamped) so that eight contributors are in flight together.
+template <int N_TOK>
+__device__ __forceinline__ void reduce_row_block(const float* __restrict__ partials, unsigned long long info,
+                                                 uint32_t row, int M, __nv_bfloat16* ycol, int64_t ldy) {
+    const int n_contrib = int((info >> 16) & 0xFFFFu);
+    const int first_slot = int(info >> 32) - 1;
+    const int c_lo = first_slot >> 1;
+#pragma unroll 1
+    for (int c0 = 0; c0 < M; c0 += 16) {
+        float a[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] = 0.f;
+#pragma unroll 1
+        for (int j0 = 0; j0 < n_contrib; j0 += 8) {
+            uint4 q[8][4];
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+                const int j = j0 + jj < n_contrib ? j0 + jj : n_contrib - 1;
+                const int s = j == 0 ? first_slot : 2 * (c_lo + j);
+                const uint4* src = reinterpret_cast<const uint4*>(partials + (int64_t(s) * kTile + row) * N_TOK + c0);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) q[jj][i] = ld_cg_issue(src + i);
+            }
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+                if (j0 + jj < n_contrib) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        a[4 * i + 0] += __uint_as_float(q[jj][i].x);
+                        a[4 * i + 1] += __uint_as_float(q[jj][i].y);
+                        a[4 * i + 2] += __uint_as_float(q[jj][i].z);
+                        a[4 * i + 3] += __uint_as_float(q[jj][i].w);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (c0 + i < M) ycol[int64_t(c0 + i) * ldy] = __float2bfloat16_rn(a[i]);
+    }
+}
+
+// XSTATIC: the caller promises that X was not written by the operation preceding this launch
+//          in the stream, so activations may be fetched before the grid dependency resolves.
+// Weight tiles are always fetched early only if WSTATIC (same promise about the packed blob).
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC>
+__global__ void __launch_bounds__(192)
+decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
+              uint32_t pay0_16, uint32_t pay_total_16, int TN, int TK, int M,
+              __nv_bfloat16* __restrict__ Y, int64_t ldy,
+              unsigned long long* __restrict__ counters, float* __restrict__ partials, int* status_dev) {
+    using Cfg = DecodeConfig<N_TOK, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const uint32_t bar_full = smem_base + Cfg::kBarrierOffset;    // 8 x 8 B
+    const uint32_t bar_empty = bar_full + 64;                     // 8 x 8 B
+    const uint32_t bar_acc_full = bar_empty + 64;                 // 2 x 8 B
+    const uint32_t bar_acc_empty = bar_acc_full + 16;             // 2 x 8 B
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + Cfg::kBarrierOffset + 160);
+    uint32_t* tmem_slot = misc;                                   // [0]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 1);
+    volatile int* range = reinterpret_cast<volatile int*>(misc + 2);          // [2], [3]: t0, t1
+    volatile uint32_t* stage_kind = misc + 4;                                 // [4 .. 4+STAGES)
+    volatile unsigned long long* red_info = reinterpret_cast<volatile unsigned long long*>(misc + 12);  // 8-B aligned
+
+    grid_launch_dependents();   // the next kernel in the stream may become resident now
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int c = blockIdx.x, G = gridDim.x;
+    if (warp == 0) PATCH_TRACE_AT(0);
+    const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off);
+
+    if (warp == 0) {
+        if constexpr (!WSTATIC) grid_dependency_wait();
+        // byte-balanced run of tiles for this CTA
+        const uint32_t lo = pay0_16 + uint32_t(uint64_t(c) * pay_total_16 / G);
+        const uint32_t hi = pay0_16 + uint32_t(uint64_t(c + 1) * pay_total_16 / G);
+        const int t0 = first_tile_at_or_after(table, TN, TK, lo, lane);
+        const int t1 = (c + 1 == G) ? TN * TK : first_tile_at_or_after(table, TN, TK, hi, lane);
+        if (lane == 0) { range[0] = t0; range[1] = t1; }
+    }
+    if (threadIdx.x == 64) {       // a thread outside warp 0, whose lanes are busy with the search
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_acc_full + 8 * i, 1);
+            mbar_init(bar_acc_empty + 8 * i, 4);     // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_map(&tmap_x);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int t0 = range[0], t1 = range[1], n_tiles = t1 - t0;
+    if (warp == 0) PATCH_TRACE_AT(1);
+    const uint32_t tmem_meta = tmem_base + 2 * N_TOK;    // 4 columns per stage; accumulators at 0 and N_TOK
+
+    if (warp == 0) {
+        // ---------------- producer: streams tiles t0 .. t1-1 through the stage ring ----------------
+        const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
+        TileDesc mine = TileDesc{0, 0, 0, 0};
+        int issued = 0;
+        bool ok = true;
+        // Weight tiles of the first STAGES steps may be requested before the grid dependency is
+        // resolved (WSTATIC); their activations follow once it is (unless XSTATIC).
+        const int n_early = (WSTATIC && !XSTATIC) ? (n_tiles < STAGES ? n_tiles : STAGES) : 0;
+        for (int i = 0; i < n_tiles && ok; ++i) {
+            if ((i & 31) == 0 && i + lane < n_tiles) mine = table[t0 + i + lane];   // 32 descriptors per load
+            const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
+            const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
+            if (lane == 0) {
+                const int stage = i % STAGES;
+                const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
+                const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
+                const uint32_t full = bar_full + 8 * stage;
+                if (i >= n_early)
+                    ok = mbar_wait(bar_empty + 8 * stage, (uint32_t(i / STAGES) & 1u) ^ 1u, abort_flag, status_dev);
+                if (ok) {
+                    stage_kind[stage] = kind;
+                    mbar_expect_tx(full, wbytes + Cfg::kXBytes);
+                    tma_bulk_load(sW, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
+                    if (i == 0) PATCH_TRACE_AT(2);
+                    if (i < n_early) {
+                        if (i + 1 == n_early) {
+                            grid_dependency_wait();
+                            for (int j = 0; j < n_early; ++j) {
+                                const uint32_t sX = smem_base + j * Cfg::kStageBytes + kDenseBytes;
+                                const int k = ((t0 + j) % TK) * kTile;
+                                tma_tile_load(sX, &tmap_x, k, 0, bar_full + 8 * j, pol_x);
+                                tma_tile_load(sX + Cfg::kXAtomBytes, &tmap_x, k + 64, 0, bar_full + 8 * j, pol_x);
+                            }
+                        }
+                    } else {
+                        const uint32_t sX = sW + kDenseBytes;
+                        const int k = ((t0 + i) % TK) * kTile;
+                        tma_tile_load(sX, &tmap_x, k, 0, full, pol_x);
+                        tma_tile_load(sX + Cfg::kXAtomBytes, &tmap_x, k + 64, 0, full, pol_x);
+                    }
+                    issued = i + 1;
+                }
+            }
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+        }
+        if (lane == 0 && *abort_flag) {
+            // drain: wait (bounded) until the copies this thread started have landed
+            const uint64_t tstart = global_timer_ns();
+            for (int j = issued > STAGES ? issued - STAGES : 0; j < issued; ++j) {
+                const uint32_t bar = bar_full + 8 * (j % STAGES), parity = uint32_t(j / STAGES) & 1u;
+                while (!mbar_try_wait(bar, parity) && global_timer_ns() - tstart < kDrainLimitNs) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            int seg = 0, tk = t0 % TK;
+            bool first = true, ok = true;
+            for (int i = 0; i < n_tiles && ok; ++i) {
+                const int stage = i % STAGES;
+                if (first)   // the accumulator of segment `seg` must have been drained by the epilogue
+                    ok = mbar_wait(bar_acc_empty + 8 * (seg & 1), (uint32_t(seg >> 1) & 1u) ^ 1u, abort_flag, status_dev);
+                if (ok) ok = mbar_wait(bar_full + 8 * stage, uint32_t(i / STAGES) & 1u, abort_flag, status_dev);
+                if (!ok) break;
+                if (i == 0) PATCH_TRACE_AT(3);
+                tc_fence_after();
+                const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
+                issue_tile_mma<N_TOK>(stage_kind[stage], sW, sW + kDenseBytes, Cfg::kXAtomBytes,
+                                      tmem_base + uint32_t(seg & 1) * N_TOK, tmem_meta + 4 * stage, first);
+                mma_commit(bar_empty + 8 * stage);            // frees the stage once these MMAs have read it
+                const bool last = (tk == TK - 1) || (i == n_tiles - 1);
+                if (last) { mma_commit(bar_acc_full + 8 * (seg & 1)); ++seg; }
+                first = last;
+                tk = (tk == TK - 1) ? 0 : tk + 1;
+            }
+            PATCH_TRACE_AT(4);
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue: warps 2..5, TMEM lane quadrant = warp % 4 ----------------
+        const uint32_t quad = warp & 3u, row = quad * 32 + lane;   // out-feature inside the row-block
+        const int et = threadIdx.x - 64;                           // 0..127
+        bool waited = false, ok = true;
+        int seg = 0;
+        // A run has at most two partial row-blocks: its first segment (k = 0) and its last (k = 1).
+        // Thread 32k updates the counter of partial k; the result is looked at only after every
+        // segment of the run is out, so the two updates and the second segment's writes overlap.
+        int part_tn[2] = {-1, -1};
+        unsigned long long seen = 0ull;
+        for (int ts = t0; ts < t1 && ok; ++seg) {
+            const int tn = ts / TK;
+            const int te = (tn + 1) * TK < t1 ? (tn + 1) * TK : t1;
+            const int ntiles = te - ts;
+            ok = mbar_wait(bar_acc_full + 8 * (seg & 1), uint32_t(seg >> 1) & 1u, abort_flag, status_dev);
+            ok = epilogue_all(ok);      // same decision in all 128 threads: they share barriers below
+            if (!ok) break;
+            tc_fence_after();
+            if (seg == 0 && warp == 2) PATCH_TRACE_AT(5);
+            if (!waited) {              // Y and the workspace may be in use by the previous kernel until here
+                grid_dependency_wait();
+                waited = true;
+                if (warp == 2) PATCH_TRACE_AT(8);
+            }
+            const uint32_t acc = tmem_base + uint32_t(seg & 1) * N_TOK + ((quad * 32u) << 16);
+            if (ntiles == TK) {
+                // whole row-block in this run: finish it here
+                __nv_bfloat16* ycol = Y + int64_t(tn) * kTile + row;
+#pragma unroll 1
+                for (int c0 = 0; c0 < M; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(acc + uint32_t(c0), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c0 + j < M) ycol[int64_t(c0 + j) * ldy] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (seg & 1));
+            } else {
+                // partial row-block: write fp32 partial sums ([slot][row][token]), then count in
+                const int k = seg == 0 ? 0 : 1;
+                float* slot = partials + (int64_t(2 * c + k) * kTile + row) * N_TOK;
+#pragma unroll 1
+                for (int c0 = 0; c0 < M; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(acc + uint32_t(c0), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4)
+                        __stcg(reinterpret_cast<uint4*>(slot + c0 + j), make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (seg & 1));
+                asm volatile("bar.sync 1, 128;" ::: "memory");      // all 128 epilogue threads have written
+                if (warp == 2) PATCH_TRACE_AT(k == 0 ? 9 : 12);
+                part_tn[k] = tn;
+                if (et == 32 * k) {
+                    // {tiles : 16, contributors : 16, (first contributor's slot + 1) : 32}
+                    unsigned long long add = (unsigned long long)ntiles | (1ull << 16);
+                    if (ts == tn * TK) add |= (unsigned long long)(2 * c + k + 1) << 32;
+                    // release: publishes the partial sums written before the barrier;
+                    // acquire: the last contributor then sees every other contributor's
+                    seen = atom_add_acq_rel_gpu(&counters[tn], add) + add;
+                }
+            }
+            ts = te;
+        }
+        if (ok && (part_tn[0] >= 0 || part_tn[1] >= 0)) {
+            if (et == 0 || et == 32) {
+                const int k = et >> 5;
+                const bool is_last = part_tn[k] >= 0 && int(seen & 0xFFFFu) == TK;
+                if (is_last) counters[part_tn[k]] = 0;             // ready for the next launch
+                red_info[k] = is_last ? seen : 0ull;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (warp == 2) PATCH_TRACE_AT(10);
+#pragma unroll 1
+            for (int k = 0; k < 2; ++k) {
+                const unsigned long long info = red_info[k];
+                if (info != 0ull) {     // this CTA completed row-block part_tn[k]: sum its partials
+                    reduce_row_block<N_TOK>(partials, info, row, M, Y + int64_t(part_tn[k]) * kTile + row, ldy);
+                    if (warp == 2) PATCH_TRACE_AT(k == 0 ? 11 : 14);
+                }
+            }
+        }
+        if (warp == 2) PATCH_TRACE_AT(6);
+    }
+
+    grid_dependency_wait();     // completion of this grid implies completion of its predecessors
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    if (warp == 0) PATCH_TRACE_AT(7);
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+
+static int decode_n_tok(int64_t M) { return M <= 16 ? 16 : M <= 32 ? 32 : 64; }
+
+static size_t counters_bytes(const patch_layout_t* L) {
+    return (size_t(L->N / kTile) * 8 + 255) / 256 * 256;
+}
+
+size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M) {
+    if (M > 64) return 0;
+    return counters_bytes(L) + size_t(2) * kMaxDecodeCtas * decode_n_tok(M) * kTile * sizeof(float);
+}
+
+static int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        return v;
+    }();
+    return n;
+}
+
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC>
+static int launch_decode_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
+                           __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream) {
+    using Cfg = DecodeConfig<N_TOK, STAGES>;
+    auto kern = decode_kernel<N_TOK, STAGES, WSTATIC, XSTATIC>;
+    static bool configured = false;   // per-process attribute, idempotent
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+            return PATCH_ERR_CUDA;
+        configured = true;
+    }
+    const int TN = int(L->N / kTile), TK = int(L->K / kTile);
+    if (TK > 65535) return PATCH_ERR_SHAPE;
+    int G = sm_count();
+    if (G <= 0) return PATCH_ERR_CUDA;
+    if (G > kMaxDecodeCtas) G = kMaxDecodeCtas;
+    // every CTA's byte range must be longer than the largest tile so that no run is empty
+    // (the reduction assumes the contributors of a row-block are consecutive CTAs)
+    const uint64_t by_bytes = L->payload_bytes / (2 * kDenseBytes);
+    if (uint64_t(G) > by_bytes) G = by_bytes ? int(by_bytes) : 1;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(G, 1, 1);
+    cfg.blockDim = dim3(192, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    unsigned long long* counters = static_cast<unsigned long long*>(workspace);
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + counters_bytes(L));
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, packed, uint64_t(L->table_off),
+                                       uint32_t(L->payload_off / 16), uint32_t(L->payload_bytes / 16), TN, TK, M, Y,
+                                       ldy, counters, partials, status_dev);
+    return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+template <int N_TOK, int STAGES>
+static int launch_decode_f(bool wstatic, bool xstatic, const CUtensorMap& map, const patch_layout_t* L,
+                           const uint8_t* packed, int M, __nv_bfloat16* Y, int64_t ldy, void* workspace,
+                           int* status_dev, cudaStream_t stream) {
+    if (wstatic && xstatic) return launch_decode_t<N_TOK, STAGES, true, true>(map, L, packed, M, Y, ldy, workspace, status_dev, stream);
+    if (wstatic) return launch_decode_t<N_TOK, STAGES, true, false>(map, L, packed, M, Y, ldy, workspace, status_dev, stream);
+    // X may only be fetched early if the weight may be as well (the flag alone changes nothing)
+    return launch_decode_t<N_TOK, STAGES, false, false>(map, L, packed, M, Y, ldy, workspace, status_dev, stream);
+}
+
+int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
+                  __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream,
+                  bool wstatic, bool xstatic) {
+    const int n_tok = decode_n_tok(M);
+    CUtensorMap map;
+    int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
+    if (rc) return rc;
+    switch (n_tok) {
+        case 16:
+            // Measured: when consecutive kernels stream concurrently (X static) a shallower ring keeps
+            // the loaded memory latency, and with it the reduction tail, shorter; a kernel that must
+            // wait for its predecessor before touching X does better with three stages of prefetch.
+            if (wstatic && xstatic)
+                return launch_decode_f<16, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+            return launch_decode_f<16, 3>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+        case 32: return launch_decode_f<32, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+        default: return launch_decode_f<64, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+    }
+}
+
+}  // namespace patch

@@ -50,6 +50,10 @@ gemv_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int M,
             const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
             __nv_bfloat16* __restrict__ Y, int64_t ldy) {
     cg::cluster_group cluster = cg::this_cluster();
+    // programmatic dependent launch: let the next kernel start its prologue, then wait until the
+    // previous kernel's results (X, and the last readers of Y) are complete
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int S = gridDim.x, s = blockIdx.x, tn = blockIdx.y;
     const int tk0 = int(int64_t(s) * TK / S), tk1 = int(int64_t(s + 1) * TK / S);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -167,13 +171,15 @@ static int launch_gemv_t(const __nv_bfloat16* X, int64_t ldx, int M, const patch
     cfg.blockDim = dim3(256, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = S;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_kernel<M_MAX>, X, ldx, M, packed,
                                        uint64_t(L->table_off), TK, Y, ldy);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;

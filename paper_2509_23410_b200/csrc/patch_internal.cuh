@@ -40,12 +40,16 @@ int check_device();
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Kernel launchers implemented in the .cu files; all return a PATCH_* status.
+// `wstatic` / `xstatic`: the packed weight / X was not written by the operation preceding this
+// launch in the stream.
 int launch_gemv(const __nv_bfloat16* X, int64_t ldx, int M, const patch_layout_t* L,
                 const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev,
                 cudaStream_t stream);
-int launch_mma(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
-               const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace,
-               size_t workspace_bytes, int* status_dev, cudaStream_t stream);
-size_t mma_workspace_bytes(const patch_layout_t* L, int64_t M);
+int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
+                  const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev,
+                  cudaStream_t stream, bool wstatic, bool xstatic);
+int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
+                   const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M);
 
 }  // namespace patch

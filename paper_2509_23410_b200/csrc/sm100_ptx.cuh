@@ -1,0 +1,197 @@
+// Inline-PTX wrappers for sm_100a: mbarriers, TMA (bulk and tensor copies), tcgen05 (TMEM
+// allocation, MMA, sparse MMA, copies, loads), programmatic dependent launch.
+#pragma once
+#include <cuda.h>
+#include <stdint.h>
+#include "patch_internal.cuh"
+
+namespace patch {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
+constexpr uint64_t kDrainLimitNs = 2000000ull;    // 2 ms for copies already in flight
+
+// Bounded wait.  Returns false if the wait was given up (own timeout, or another role of this
+// CTA raised the abort flag).  On timeout the flag is raised and the status word is set.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status_dev) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// L2 eviction policies for streamed-once (weights) and reused (activations) data.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+// 1-D bulk copy global -> shared, completion counted on an mbarrier.
+__device__ __forceinline__ void tma_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                              uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+// 2-D tiled copy global -> shared through a tensor map.
+__device__ __forceinline__ void tma_tile_load(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                              uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], dense bf16, fp32 accumulate
+__device__ __forceinline__ void mma_dense(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// same with A stored 2:4-compressed and its position metadata in TMEM
+__device__ __forceinline__ void mma_sparse(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t e_tmem,
+                                           uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrive on an mbarrier once all previously issued tcgen05 operations of this thread completed
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// shared memory (128 rows x 16 bytes) -> TMEM (128 lanes x 4 columns)
+__device__ __forceinline__ void tmem_copy_128x128b(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns -> 16 registers per thread (thread = lane)
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// programmatic dependent launch: allow the next kernel to start / wait for the previous one
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, K-major operand in 128-byte-swizzled atoms
+// (8 rows x 128 B = 1024 B per row group): start address, stride between row groups, sm_100
+// descriptor version, swizzle mode.
+__device__ __forceinline__ uint64_t desc_kmajor_sw128(uint32_t saddr) {
+    return uint64_t((saddr & 0x3FFFFu) >> 4) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) |
+           (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+// Unswizzled 128 rows x 16 B block (8-row groups of 128 B): source of the metadata copy.
+__device__ __forceinline__ uint64_t desc_rows16(uint32_t saddr) {
+    return uint64_t((saddr & 0x3FFFFu) >> 4) | (uint64_t(128 >> 4) << 16) | (uint64_t(128 >> 4) << 32) |
+           (uint64_t(1) << 46);
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n_tok.
+__host__ __device__ constexpr uint32_t instr_desc(int n_tok, bool sparse) {
+    return (sparse ? (1u << 2) : 0u) | (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n_tok >> 3) << 17) |
+           (uint32_t(128 >> 4) << 24);
+}
+
+// Issues the MMAs of one 128 x 128 weight tile held in shared memory at sW (payload image)
+// against the activation tile at sX (two K-halves of x_atom_bytes each).
+//   dense: eight tcgen05.mma, K = 16 each (32 B of every operand row per step)
+//   2:4  : metadata block -> TMEM columns e_tmem..e_tmem+3, then four tcgen05.mma.sp, K = 32 each
+//          (32 B of A, 64 B of B per row); metadata column ks is addressed as the even column
+//          in the TMEM address plus the column's parity in the descriptor's selector field.
+template <int N_TOK>
+__device__ __forceinline__ void issue_tile_mma(uint32_t kind, uint32_t sW, uint32_t sX, uint32_t x_atom_bytes,
+                                               uint32_t acc_tmem, uint32_t e_tmem, bool first) {
+    constexpr uint32_t idesc_d = instr_desc(N_TOK, false), idesc_s = instr_desc(N_TOK, true);
+    const uint64_t dA = desc_kmajor_sw128(sW), dB = desc_kmajor_sw128(sX);
+    if (kind == PATCH_TILE_DENSE) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t a = dA + uint64_t(((ks >> 2) * kAtomBytes + (ks & 3) * 32) >> 4);
+            const uint64_t b = dB + uint64_t(((ks >> 2) * x_atom_bytes + (ks & 3) * 32) >> 4);
+            mma_dense(acc_tmem, a, b, idesc_d, !(first && ks == 0));
+        }
+    } else {
+        tmem_copy_128x128b(e_tmem, desc_rows16(sW + kAtomBytes));
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t a = dA + uint64_t((ks * 32) >> 4);
+            const uint64_t b = dB + uint64_t(((ks >> 1) * x_atom_bytes + (ks & 1) * 64) >> 4);
+            mma_sparse(acc_tmem, a, b, e_tmem + (ks & 2), idesc_s | uint32_t(ks & 1), !(first && ks == 0));
+        }
+    }
+}
+
+// Host: tensor map over X [M x ldx] bf16 with a box of 64 columns (128 B) x n_tok rows,
+// 128-byte swizzle, zero fill outside the matrix.
+int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok);
+
+#ifdef PATCH_TRACE
+// Debug build only: status_dev is reinterpreted as a buffer of 16 timestamps (ns) per CTA.
+#define PATCH_TRACE_AT(slot) do { if ((threadIdx.x & 31) == 0) reinterpret_cast<unsigned long long*>(status_dev)[(blockIdx.y * gridDim.x + blockIdx.x) * 16 + (slot)] = global_timer_ns(); } while (0)
+#else
+#define PATCH_TRACE_AT(slot) do {} while (0)
+#endif
+
+}  // namespace patch

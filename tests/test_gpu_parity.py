@@ -1,0 +1,292 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Packing is compared bit for bit; GEMM outputs within the stated tolerance
+(relative Frobenius error <= 2e-3 and max |dY| <= 1e-2 * max |Yref|)."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from paper_2509_23410_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+REL_F_TOL = 2e-3
+MAX_TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("no CUDA device: GPU tests must run on a B200")
+    from paper_2509_23410_b200 import binding
+    binding.lib()   # raises if the CUDA library is missing -- there is no fallback
+    return torch, binding
+
+
+def to_dev(torch, bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def to_bits(t):
+    import torch
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+f32 = inputs.bf16_bits_to_f32
+
+
+def check_parity(oracle, Y_bits, Y32, what=""):
+    relF, maxrel = oracle.parity_metrics(f32(Y_bits), Y32)
+    assert relF <= REL_F_TOL and maxrel <= MAX_TOL, f"{what}: relF={relF:.3e} maxrel={maxrel:.3e}"
+    return relF, maxrel
+
+
+def run_gemm(gpu, X_bits, layout, packed, variant):
+    torch, B = gpu
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(max(B.patch_gemm_workspace_size(layout, X_bits.shape[0]), 1), dtype=torch.uint8, device="cuda")
+    Y = B.patch_gemm(to_dev(torch, X_bits), layout, packed, workspace=ws, status=status, variant=variant)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device-side wait timed out"
+    return to_bits(Y)
+
+
+# ---------------------------------------------------------------------------------------------
+# packing: bit exact, image and round trip
+
+
+@pytest.mark.parametrize("N,K,p", [(128, 128, 0.0), (128, 128, 1.0), (256, 384, 0.5), (1024, 1024, 0.5),
+                                   (640, 256, 0.35), (4096, 4096, 0.7)])
+def test_pack_bit_exact(gpu, oracle, N, K, p):
+    torch, B = gpu
+    W = inputs.weight(N, K, 11, "pack", N, K)
+    W[::13, ::7] = 0          # exact zeros and ties
+    W[5::17, 3::4] = W[5::17, 2::4]
+    flags = inputs.tile_flags(N, K, p, 11, "pack", N, K)
+    canon, Lo = oracle.pack(W, flags)
+    image = oracle.device_image(canon)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    torch.cuda.synchronize()
+    assert (L.n_dense, L.n_sparse, L.total_bytes) == (Lo.n_dense, Lo.n_sparse, Lo.total_bytes)
+    got = packed.cpu().numpy()
+    assert got.shape == image.shape and (got == image).all()
+    What = oracle.prune(W, flags)
+    assert (to_bits(B.patch_unpack(L, packed)) == What).all()
+    # packing the pruned weight again reproduces the blob (idempotence through the GPU path)
+    packed2, _ = B.patch_pack(B.patch_unpack(L, packed), flags)
+    assert torch.equal(packed, packed2)
+
+
+def test_pack_with_row_pitch(gpu, oracle):
+    torch, B = gpu
+    N, K, ld = 256, 256, 320
+    W = inputs.weight(N, K, 12, "pitch")
+    flags = np.array([[1, 0], [0, 1]], np.uint8)
+    big = torch.zeros((N, ld), dtype=torch.bfloat16, device="cuda")
+    big[:, :K] = to_dev(torch, W)
+    packed, L = B.patch_pack(big[:, :K], flags)
+    image = oracle.device_image(oracle.pack(W, flags)[0])
+    assert (packed.cpu().numpy() == image).all()
+    out = torch.zeros((N, ld), dtype=torch.bfloat16, device="cuda")
+    B.patch_unpack(L, packed, out=out[:, :K])
+    assert (to_bits(out[:, :K]) == oracle.prune(W, flags)).all()
+    assert (to_bits(out[:, K:]) == 0).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# identity probe: X = I makes every output a single product, so Y[m][n] == What[n][m] exactly
+
+
+@pytest.mark.parametrize("variant", ["gemv", "mma"])
+@pytest.mark.parametrize("p", [0.0, 1.0, 0.5])
+def test_identity_probe(gpu, oracle, variant, p):
+    torch, B = gpu
+    N, K = 256, 384
+    # weights whose value encodes (row, column): a wrong permutation shows as exact mismatches
+    r, c = np.meshgrid(np.arange(N), np.arange(K), indexing="ij")
+    Wf = ((1.0 + (c % 128) / 128.0) * np.where(r % 2 == 0, 1.0, -1.0) * (1 + (r % 128) // 16)).astype(np.float32)
+    W = inputs.f32_to_bf16_bits(Wf)
+    W ^= inputs.weight(N, K, 13, "ident") & 0x0003    # break exact ties differently per element
+    flags = inputs.tile_flags(N, K, p, 13, "ident")
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    if variant == "mma":
+        X = np.zeros((K, K), np.uint16)
+        X[np.arange(K), np.arange(K)] = 0x3F80
+        Y = run_gemm(gpu, X, L, packed, B.VARIANT_MMA)
+        assert (f32(Y) == f32(What).T).all()
+    else:
+        for k0 in (0, 1, 2, 3, 127, 128, 255, 383):   # one-hot rows through the decode kernel
+            X = np.zeros((2, K), np.uint16)
+            X[0, k0] = 0x3F80
+            X[1, (k0 + 77) % K] = 0x4000               # 2.0
+            Y = run_gemm(gpu, X, L, packed, B.VARIANT_GEMV)
+            assert (f32(Y[0]) == f32(What[:, k0])).all()
+            assert (f32(Y[1]) == 2.0 * f32(What[:, (k0 + 77) % K])).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# GEMM parity at sizes spanning several tiles and ragged token counts
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4])
+@pytest.mark.parametrize("N,K,p", [(384, 640, 0.5), (128, 128, 1.0), (1024, 1024, 0.5)])
+def test_gemv_parity(gpu, oracle, M, N, K, p):
+    torch, B = gpu
+    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=p, stream=("gemv", N, K)), 21, M)
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y = run_gemm(gpu, X, L, packed, B.VARIANT_GEMV)
+    Y32, _ = oracle.gemm_f64(X, What)
+    check_parity(oracle, Y, Y32, f"gemv M={M}")
+
+
+@pytest.mark.parametrize("M", [1, 5, 16, 17, 32, 33, 64, 65, 100, 128, 129, 256, 300, 513])
+@pytest.mark.parametrize("N,K,p", [(384, 640, 0.5), (256, 1152, 0.0), (256, 1152, 1.0)])
+def test_mma_parity(gpu, oracle, M, N, K, p):
+    torch, B = gpu
+    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=p, stream=("mma", N, K)), 22, M)
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y = run_gemm(gpu, X, L, packed, B.VARIANT_MMA)
+    Y32, Y16 = oracle.gemm_f64(X, What)
+    check_parity(oracle, Y, Y32, f"mma M={M}")
+    assert (Y == Y16).mean() > 0.99      # fp32 accumulation: almost every output rounds identically
+
+
+def test_single_gemm_config(gpu, oracle):
+    """X [16 x 1024], W [1024 x 1024], Bernoulli(0.5) tiles: all three call forms agree."""
+    torch, B = gpu
+    case = inputs.single_gemm_case()
+    W, flags, X = inputs.make_case_inputs(case)
+    What = oracle.prune(W, flags)
+    assert 0 < flags.sum() < flags.size
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y32, _ = oracle.gemm_f64(X, What)
+    for variant in (B.VARIANT_AUTO, B.VARIANT_MMA, B.VARIANT_MMA | B.WEIGHTS_STATIC, B.VARIANT_AUTO | B.WEIGHTS_STATIC):
+        check_parity(oracle, run_gemm(gpu, X, L, packed, variant), Y32, "single")
+    # strided X and Y (row pitch > row length)
+    Xd = torch.zeros((16, 1024 + 64), dtype=torch.bfloat16, device="cuda")
+    Xd[:, :1024] = to_dev(torch, X)
+    Yd = torch.full((16, 1024 + 8), 7.0, dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(B.patch_gemm_workspace_size(L, 16), dtype=torch.uint8, device="cuda")
+    B.patch_gemm(Xd[:, :1024], L, packed, Y=Yd[:, :1024], workspace=ws)
+    torch.cuda.synchronize()
+    check_parity(oracle, to_bits(Yd[:, :1024]), Y32, "strided")
+    assert (Yd[:, 1024:] == 7.0).all()
+
+
+def test_linearity_and_zero(gpu, oracle):
+    torch, B = gpu
+    W, flags, X = inputs.make_case_inputs(dict(N=256, K=512, p=0.5, stream=("lin",)), 23, 16)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    for variant, Xv in ((B.VARIANT_MMA, X), (B.VARIANT_GEMV, X[:3])):
+        Y1 = run_gemm(gpu, Xv, L, packed, variant)
+        X2 = inputs.f32_to_bf16_bits(2.0 * f32(Xv))
+        Y2 = run_gemm(gpu, X2, L, packed, variant)
+        assert (f32(Y2) == 2.0 * f32(Y1)).all()          # power-of-two scaling is exact
+        Y0 = run_gemm(gpu, np.zeros_like(Xv), L, packed, variant)
+        assert (f32(Y0) == 0).all()
+        assert (run_gemm(gpu, Xv, L, packed, variant) == Y1).all()   # deterministic
+
+
+def test_m_zero_and_errors(gpu):
+    torch, B = gpu
+    flags = np.zeros((1, 1), np.uint8)
+    W = torch.zeros((128, 128), dtype=torch.bfloat16, device="cuda")
+    packed, L = B.patch_pack(W, flags)
+    Y = B.patch_gemm(torch.zeros((0, 128), dtype=torch.bfloat16, device="cuda"), L, packed)   # M = 0: nothing runs
+    assert Y.shape == (0, 128)
+    with pytest.raises(B.PatchError) as e:
+        B.patch_gemm(torch.zeros((5, 128), dtype=torch.bfloat16, device="cuda"), L, packed, variant=B.VARIANT_GEMV)
+    assert e.value.status == B.ERR_SHAPE
+    with pytest.raises(B.PatchError) as e:
+        B.patch_pack(W, np.ones((1, 1), np.uint8), layout=L)      # flags disagree with the layout
+    assert e.value.status == B.ERR_FORMAT
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.PatchError) as e:
+        B.patch_pack(W, flags, out=small)
+    assert e.value.status == B.ERR_SIZE
+
+
+def test_host_buffer_entry_point(gpu, oracle):
+    torch, B = gpu
+    W, flags, X = inputs.make_case_inputs(dict(N=512, K=384, p=0.5, stream=("host",)), 24, 16)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Xh = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Yh = torch.empty((16, 512), dtype=torch.bfloat16).pin_memory()
+    Xs = torch.empty((16, 384), dtype=torch.bfloat16, device="cuda")
+    Ys = torch.empty((16, 512), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(B.patch_gemm_workspace_size(L, 16), dtype=torch.uint8, device="cuda")
+    B.patch_gemm_host(Xh, L, packed, Yh, Xs, Ys, workspace=ws)
+    Y32, _ = oracle.gemm_f64(X, oracle.prune(W, flags))
+    check_parity(oracle, Yh.view(torch.int16).numpy().view(np.uint16), Y32, "host entry point")
+
+
+# ---------------------------------------------------------------------------------------------
+# full-size shapes in the launch configuration the benchmark times
+
+
+@pytest.mark.parametrize("shape", ["attn_qkvo", "mlp_gate_up", "mlp_down"])
+@pytest.mark.parametrize("p", [0.35, 1.0])
+def test_decode_shapes_full_output(gpu, oracle, shape, p):
+    torch, B = gpu
+    N, K = inputs.LLAMA2_7B_SHAPES[shape]
+    case = dict(N=N, K=K, p=p, stream=("decode", shape, p))
+    W = inputs.weight(N, K, inputs.MASTER_SEED, *case["stream"])
+    flags = inputs.tile_flags(N, K, p, inputs.MASTER_SEED, *case["stream"])
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    assert (to_bits(B.patch_unpack(L, packed)) == What).all()
+    for M in (1, 16):
+        X = inputs.activation(M, K, inputs.MASTER_SEED, *case["stream"], M)
+        Y32, _ = oracle.gemm_f64(X, What)
+        check_parity(oracle, run_gemm(gpu, X, L, packed, B.VARIANT_AUTO), Y32, f"{shape} M={M} auto")
+        check_parity(oracle, run_gemm(gpu, X, L, packed, B.VARIANT_MMA | B.WEIGHTS_STATIC), Y32, f"{shape} M={M} mma")
+    X = inputs.activation(1, K, inputs.MASTER_SEED, *case["stream"], 1)
+    check_parity(oracle, run_gemm(gpu, X, L, packed, B.VARIANT_GEMV), oracle.gemm_f64(X, What)[0], "gemv")
+
+
+@pytest.mark.parametrize("N,K,M,p", [(4096, 4096, 2048, 0.5), (11008, 4096, 512, 0.5), (4096, 11008, 4096, 1.0),
+                                     (5120, 13824, 64, 0.6), (13824, 5120, 8, 0.3)])
+def test_prefill_shapes_sampled(gpu, oracle, N, K, M, p):
+    """Large M: compare 64 random token rows over all N, plus the four corner tiles' rows."""
+    torch, B = gpu
+    stream = ("prefill", N, K, p)
+    W = inputs.weight(N, K, inputs.MASTER_SEED, *stream)
+    flags = inputs.tile_flags(N, K, p, inputs.MASTER_SEED, *stream)
+    X = inputs.activation(M, K, inputs.MASTER_SEED, *stream, M)
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO)
+    rng = inputs.generator(inputs.MASTER_SEED, "rows", N, K, M)
+    rows = np.unique(np.concatenate([rng.integers(0, M, 60), [0, M - 1, min(M - 1, 127), min(M - 1, 128)]]))
+    Y32 = oracle.gemm_f64_rows(X, rows, What)
+    check_parity(oracle, Y[rows], Y32, f"sampled rows N={N} K={K} M={M}")
+    # property that holds at any size: doubling X doubles every output exactly
+    Y2 = run_gemm(gpu, inputs.f32_to_bf16_bits(2.0 * f32(X)), L, packed, B.VARIANT_AUTO)
+    assert (f32(Y2) == 2.0 * f32(Y)).all()
+
+
+def test_back_to_back_launches_are_ordered(gpu, oracle):
+    """A chain of dependent GEMMs on one stream (each launched with programmatic dependent
+    launch): Y of one call is X of the next, so early starts must still see finished inputs."""
+    torch, B = gpu
+    N = K = 512
+    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=0.5, stream=("chain",)), 25, 16)
+    W = inputs.f32_to_bf16_bits(f32(W) * 2.0)      # keep magnitudes from collapsing along the chain
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    torch.cuda.synchronize()
+    bufs = [to_dev(torch, X)] + [torch.empty((16, N), dtype=torch.bfloat16, device="cuda") for _ in range(6)]
+    ws = torch.zeros(B.patch_gemm_workspace_size(L, 16), dtype=torch.uint8, device="cuda")
+    for i in range(6):
+        B.patch_gemm(bufs[i], L, packed, Y=bufs[i + 1], workspace=ws, variant=B.VARIANT_MMA | B.WEIGHTS_STATIC)
+    torch.cuda.synchronize()
+    ref = X
+    for i in range(6):
+        Y32, Y16 = oracle.gemm_f64(ref, What)
+        got = to_bits(bufs[i + 1])
+        check_parity(oracle, got, Y32, f"chain step {i}")
+        ref = got                                   # feed the GPU's own bf16 output forward
