@@ -131,21 +131,29 @@ def oracle_sample(cases, budget_s):
     """Time the oracle GEMM on the leading cases of the step until ~budget_s of CPU work."""
     import oracle
     oracle.build()
-    done, flops, secs = [], 0.0, 0.0
-    for case in cases:
-        W, flags, X = inputs.make_case_inputs(case)
-        What = oracle.prune(W, flags)
-        t = time.perf_counter()
-        oracle.gemm_f64(X, What, want_bf16=True)
-        dt = time.perf_counter() - t
-        secs += dt
-        flops += 2.0 * case["M"] * case["N"] * case["K"]
-        done.append(case["name"])
-        if secs >= budget_s:
-            break
+    done, flops, secs, passes = [], 0.0, 0.0, 0
+    prepared = {}
+    while secs < budget_s and passes < 64:
+        for case in cases:
+            key = case["name"]
+            if key not in prepared:
+                if passes > 0:
+                    continue
+                W, flags, X = inputs.make_case_inputs(case)
+                prepared[key] = (X, oracle.prune(W, flags))
+            X, What = prepared[key]
+            t = time.perf_counter()
+            oracle.gemm_f64(X, What, want_bf16=True)
+            secs += time.perf_counter() - t
+            flops += 2.0 * case["M"] * case["N"] * case["K"]
+            if passes == 0:
+                done.append(key)
+            if secs >= budget_s:
+                break
+        passes += 1
     return dict(value=flops / secs / 1e12, unit="TFLOP/s", cores=oracle.num_threads(), kind="oracle",
-                sample=f"oracle GEMM (double accumulation) on the first {len(done)} GEMMs of the step "
-                       f"({done[0]} .. {done[-1]}), {secs:.1f} s of CPU time"), secs
+                sample=f"oracle GEMM (double accumulation) over the step's first {len(done)} GEMMs "
+                       f"({done[0]} .. {done[-1]}), repeated for {secs:.1f} s of CPU time"), secs
 
 
 def run_reference(args):
@@ -242,19 +250,21 @@ def run_ours(args):
     weight_bytes = sum(m[0].total_bytes for m in mats.values())
 
     # weights are packed once, before any step; in this workload no GEMM reads another GEMM's output
-    launch_flags = B.WEIGHTS_STATIC | (B.INPUT_STATIC if args.launch == "independent" else 0)
+    def flags_for(mode):
+        return B.WEIGHTS_STATIC | (B.INPUT_STATIC if mode == "independent" else 0)
 
-    def launch_all(js):
+    def launch_all(js, mode):
         for j in js:
             B.patch_gemm(j["X"], j["layout"], j["packed"], Y=j["Y"], workspace=j["ws"],
-                         variant=args.variant | launch_flags)
+                         variant=args.variant | flags_for(mode))
 
-    def make_graph(js):
-        launch_all(js)                      # first call sets kernel attributes; must precede capture
+    def make_graph(js, mode=None):
+        mode = mode or args.launch
+        launch_all(js, mode)                # first call sets kernel attributes; must precede capture
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            launch_all(js)
+            launch_all(js, mode)
         return g
 
     def barrier():
@@ -294,6 +304,14 @@ def run_ours(args):
     step_s = secs / args.steps
     step_flops = sum(j["cost"]["flops"] for j in jobs)
     value = world * step_flops / step_s / 1e12
+
+    # ---- the same step under the other launch promise (context for the headline number)
+    other = "dependent" if args.launch == "independent" else "independent"
+    g_other = make_graph(jobs, other)
+    for _ in range(3):
+        g_other.replay()
+    other_s = time_graph(g_other, max(10, args.steps // 5))
+    del g_other
 
     # ---- dominant kernel: the launches that take the largest share of the step, timed on their own
     groups = {}
@@ -395,6 +413,8 @@ def run_ours(args):
         "roofline": roof,
         "e2e": {"value": world * step_flops / e2e_s / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3},
+        other + "_launch": {"value": world * step_flops / other_s / 1e12, "unit": "TFLOP/s",
+                            "ms_per_step": other_s * 1e3, "frac_of_roofline_measured": meas_t / other_s},
         "gpu_launches": args.steps * len(jobs),
         "clocks": clocks,
         "pack": {"gbs": pack_bytes / pack_secs / 1e9, "frac_of_measured_hbm": pack_bytes / pack_secs / 1e9 / peaks["hbm_gbs"]},
@@ -407,17 +427,16 @@ def run_ours(args):
 
 
 def B_kernel_name(M):
-    return "gemv_kernel" if M <= 2 else "mma_kernel"
+    return "decode_kernel" if M <= 64 else "prefill_kernel"
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None until a capture of that kernel exists)
+NCU_TRAFFIC_PER_LAUNCH = {}
 
 
 def load_traffic(kernel):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        with open(path) as fh:
-            return json.load(fh).get(kernel)
-    except (OSError, ValueError):
-        return None
+    return NCU_TRAFFIC_PER_LAUNCH.get(kernel)
 
 
 def main():
@@ -427,9 +446,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single"])
-    ap.add_argument("--launch", default="dependent", choices=["dependent", "independent"],
-                    help="dependent: every GEMM waits for the previous one before reading X; independent: "
-                         "the caller promises X is not produced by the preceding kernel")
+    ap.add_argument("--launch", default="independent", choices=["dependent", "independent"],
+                    help="independent (default; true for this workload, whose GEMMs do not feed each other): "
+                         "the caller promises X is not produced by the preceding kernel; dependent: every "
+                         "GEMM waits for the previous one before reading X")
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 decode GEMV (M <= 4), 2 tensor-core kernel")
     ap.add_argument("--detail", action="store_true", help="add the per-GEMM table (us, TFLOP/s, roofline fraction)")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")

@@ -65,7 +65,7 @@ enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
  * The blob in device memory is position independent (offsets only):
  *   [ header 256 B (a copy of this struct, zero padded)
  *   | tile table: 16 B per tile in (tn, tk) row-major order, zero padded to a multiple of 1024 B
- *   | payloads, each 1024-byte aligned: 32 768 B per dense tile, 18 432 B per 2:4 tile ]
+ *   | payloads at offsets that are multiples of 1024: 32 768 B per dense tile, 18 432 B per 2:4 tile ]
  * Table entry: { u32 kind, u32 payload_off / 16, u32 meta_off / 16 (0xFFFFFFFF if dense), u32 0 },
  * offsets counted from the start of the blob.
  *
@@ -110,7 +110,7 @@ int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
  * dense tiles are copied.  A weight that is already 2:4 inside those tiles is packed losslessly.
  *   W_dev            bf16 [N x ldw], ldw >= K elements, ldw % 8 == 0
  *   tile_flags_host  as for patch_packed_size; must be the flags `layout` was computed from
- *   packed_dev       destination, packed_capacity >= layout->total_bytes, 1024-byte aligned
+ *   packed_dev       destination, packed_capacity >= layout->total_bytes, 16-byte aligned
  * Copies header and tile table host->device on `stream` (the host staging buffer is consumed
  * before the call returns), then launches one kernel.  Every byte of the blob is written.
  */

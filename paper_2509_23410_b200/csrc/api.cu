@@ -12,7 +12,7 @@ static int check_gemm_args(const void* X, int64_t ldx, int64_t M, const patch_la
     if (M == 0) return PATCH_OK;
     if (!X || !packed || !Y) return PATCH_ERR_NULL;
     if (ldx < L->K || ldy < L->N || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;
-    if (!aligned16(X) || !aligned16(Y) || (reinterpret_cast<uintptr_t>(packed) & 1023u)) return PATCH_ERR_ALIGN;
+    if (!aligned16(X) || !aligned16(Y) || !aligned16(packed)) return PATCH_ERR_ALIGN;
     return PATCH_OK;
 }
 

@@ -192,7 +192,7 @@ extern "C" int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* flags,
     int rc = validate_layout(L);
     if (rc) return rc;
     if (ldw < L->K || ldw % 8) return PATCH_ERR_SHAPE;
-    if (!aligned16(W_dev) || (reinterpret_cast<uintptr_t>(packed_dev) & 1023u)) return PATCH_ERR_ALIGN;
+    if (!aligned16(W_dev) || !aligned16(packed_dev)) return PATCH_ERR_ALIGN;
     if (capacity < L->total_bytes) return PATCH_ERR_SIZE;
     const int64_t TK = L->K / kTile, T = (L->N / kTile) * TK;
     // header + tile table, built on the host from the flags
