@@ -178,6 +178,33 @@ int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* layout,
                     void* X_stage_dev, void* Y_stage_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/*
+ * patch_gemm for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this is a convenience of this library.)
+ *
+ * Some callers of a GEMM run where cudaMalloc is off limits: inside a framework's capture or
+ * replay phase, under a memory pool that must not be disturbed, in a plug-in that is handed
+ * pointers and a stream and nothing else, or late in a process whose memory is fully committed.
+ * They cannot provide the workspace patch_gemm needs for its split-K partial sums.  This entry
+ * point keeps that scratch in a fixed array inside the library image instead (about 3.2 MB,
+ * held on every GPU that loads the library until the process exits) and calls no cudaMalloc,
+ * cudaFree or any allocating routine.
+ *
+ *   Arguments as for patch_gemm, without workspace and status.  Result and rounding are those
+ *   of patch_gemm (same kernel, same summation order).
+ *   Limits: M <= 16 tokens and N <= 131072; beyond them the call returns PATCH_ERR_SIZE and
+ *   launches nothing (use patch_gemm with a caller-owned workspace instead).
+ *   The first call on each device looks up the array's device address; make that first call
+ *   with the device current and before any stream capture.  Every call enqueues a small memset
+ *   of the arrival counters followed by the kernel.
+ *   All calls on a device share the one array, which keeps the last call's contents: calls that
+ *   may overlap on the GPU (different streams) race with each other -- issue them on one stream
+ *   or order them with events.
+ */
+int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M,
+                       const patch_layout_t* layout, const void* packed_dev,
+                       void* Y_dev, int64_t ldy, void* stream);
+
 /* Human-readable text for a status code (static storage). */
 const char* patch_strerror(int status);
 

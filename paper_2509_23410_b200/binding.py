@@ -24,7 +24,7 @@ ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
-           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_host",
+           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_host", "patch_gemm_noalloc",
            "patch_strerror", "patch_version"]
 
 
@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.patch_gemm.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, sz, vp, vp]
         L.patch_gemm_ex.argtypes = L.patch_gemm.argtypes + [ctypes.c_int]
         L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
+        L.patch_gemm_noalloc.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp]
         L.patch_strerror.argtypes = [ctypes.c_int]
         L.patch_strerror.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -163,6 +164,17 @@ def patch_gemm_host(X_host, layout: Layout, packed, Y_host, X_stage, Y_stage, wo
                                  _ptr(X_stage), _ptr(Y_stage), _ptr(workspace), ws_bytes, _stream(stream)),
            "patch_gemm_host")
     return Y_host
+
+
+def patch_gemm_noalloc(X, layout: Layout, packed, Y, stream=None):
+    """Y = X @ What^T for callers that may not allocate: the library's own fixed scratch array is used.
+
+    The caller passes every buffer, Y included; nothing is allocated here either.  M <= 16.
+    """
+    M = X.shape[0]
+    _check(lib().patch_gemm_noalloc(_ptr(X), X.stride(0) if M else layout.K, M, ctypes.byref(layout), _ptr(packed),
+                                    _ptr(Y), Y.stride(0) if M else layout.N, _stream(stream)), "patch_gemm_noalloc")
+    return Y
 
 
 def patch_version() -> int:

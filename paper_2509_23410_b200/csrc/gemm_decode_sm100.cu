@@ -463,3 +463,53 @@ int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_la
 }
 
 }  // namespace patch
+
+// ---------------------------------------------------------------------------------------------
+// Entry point that brings its own scratch memory (see include/patch.h: patch_gemm_noalloc).
+
+namespace {
+
+constexpr int kNoAllocMaxTokens = 16;         // decode only
+constexpr int kNoAllocMaxRowBlocks = 1024;    // N <= 131072
+constexpr size_t kNoAllocCounterBytes = size_t(kNoAllocMaxRowBlocks) * 8;
+constexpr size_t kNoAllocScratchBytes =
+    kNoAllocCounterBytes + size_t(2) * patch::kMaxDecodeCtas * kNoAllocMaxTokens * patch::kTile * sizeof(float);
+
+// Lives in the library image: every GPU that loads the library holds these ~3.2 MB until exit.
+// In host code this name is only a handle; the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices];             // device address of the array, per device, once known
+
+}  // namespace
+
+extern "C" int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,
+                                  const void* packed_dev, void* Y_dev, int64_t ldy, void* stream) {
+    using namespace patch;
+    if (!L) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (M < 0) return PATCH_ERR_SHAPE;
+    if (M == 0) return PATCH_OK;
+    if (M > kNoAllocMaxTokens || L->N / kTile > kNoAllocMaxRowBlocks) return PATCH_ERR_SIZE;
+    if (!X_dev || !packed_dev || !Y_dev) return PATCH_ERR_NULL;
+    if (ldx < L->K || ldy < L->N || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;
+    if (!aligned16(X_dev) || !aligned16(Y_dev) || !aligned16(packed_dev)) return PATCH_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PATCH_ERR_CUDA;
+    if (!g_noalloc_ptr[dev]) {
+        // set-up, once per device, with that device current
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return PATCH_ERR_CUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    void* scratch = g_noalloc_ptr[dev];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the arrival counters must start at zero; the array keeps whatever the last call left
+    if (cudaMemsetAsync(scratch, 0, kNoAllocCounterBytes, s) != cudaSuccess) return PATCH_ERR_CUDA;
+    return launch_decode(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
+                         static_cast<__nv_bfloat16*>(Y_dev), ldy, scratch, nullptr, s, false, false);
+}
