@@ -342,7 +342,7 @@ def run_ours(args):
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1)
     roof = dict(bound=bound, achieved=achieved, peak=peak, unit=unit, frac=achieved / peak,
-                traffic=load_traffic(kernel_name), kernel=kernel_name, launches_timed=len(djs),
+                traffic=load_traffic(kernel_name, alg) if bound == "hbm" else None, kernel=kernel_name, launches_timed=len(djs),
                 us_per_launch=per_launch * 1e6, peak_source=peaks["source"],
                 algorithmic_per_launch=alg)
     spec_t = sum(roofline_seconds(j["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)[0] for j in jobs)
@@ -430,13 +430,15 @@ def B_kernel_name(M):
     return "decode_kernel" if M <= 64 else "prefill_kernel"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (None until a capture of that kernel exists)
-NCU_TRAFFIC_PER_LAUNCH = {}
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes per launch, from the ncu
+# captures summarised in profiles/decode_kernel_llama7b_decode.md (three launches: 1.035, 1.029, 1.008).
+# Traffic grows in proportion to the payload, so the ratio scales to any launch of the kernel.
+NCU_TRAFFIC_RATIO = {"decode_kernel": 1.03}
 
 
-def load_traffic(kernel):
-    return NCU_TRAFFIC_PER_LAUNCH.get(kernel)
+def load_traffic(kernel, algorithmic):
+    r = NCU_TRAFFIC_RATIO.get(kernel)
+    return None if r is None else r * algorithmic
 
 
 def main():
