@@ -2,15 +2,20 @@
 //
 // Computes Y^T[N x M] = What[N x K] * X^T[K x M]: the packed weight is the MMA "A" operand
 // (the only operand tcgen05.mma.sp accepts in compressed form), out-features ride the 128 TMEM
-// lanes, tokens ride the MMA N dimension.  One CTA per (row-block tn, token tile of N_TOK): it
-// walks all TK weight tiles of its row-block and issues, per tile, eight dense tcgen05.mma or
-// four tcgen05.mma.sp into one fp32 TMEM accumulator -- the paper's mixed execution "within a
-// single matrix multiplication" (Appendix A).
+// lanes, tokens ride the MMA N dimension.  An output tile is (row-block tn) x (n_tok tokens); its
+// mainloop walks the TK weight tiles of the row-block and issues, per tile, eight dense
+// tcgen05.mma or four tcgen05.mma.sp into one fp32 TMEM accumulator -- the paper's mixed
+// execution "within a single matrix multiplication" (Appendix A).
+//
+// Persistent kernel: one CTA per SM loops over output tiles (tile index = mt * TN + tn, so CTAs
+// running side by side share an X tile in L2 and stream different row-blocks).  Two TMEM
+// accumulators: the epilogue of one output tile (tcgen05.ld, bf16, transposed store) overlaps the
+// mainloop of the next.  n_tok (a multiple of 16, at most 240) is chosen per problem so that the
+// number of output tiles fills whole waves of SMs.
 //
 // Warp roles (192 threads): warp 0 streams tiles with TMA (one linear bulk copy per weight
 // tile, whose payload is already in the swizzled shared-memory layout, and two tensor copies
-// for the activations); warp 1 owns TMEM and issues the MMAs; warps 2..5 read the accumulator
-// back (tcgen05.ld), convert to bf16 and store the transposed result.
+// for the activations); warp 1 owns TMEM and issues the MMAs; warps 2..5 are the epilogue.
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports
 // PATCH_ERR_TIMEOUT through status_dev, drains its copies in flight, frees TMEM and returns.
@@ -18,34 +23,32 @@
 
 namespace patch {
 
-template <int N_TOK, int STAGES>
+constexpr int kPrefillMaxTok = 240;      // two accumulators + metadata must fit 512 TMEM columns
+constexpr int kPrefillStages = 2;
+
 struct PrefillConfig {
-    static constexpr uint32_t kXAtomBytes = N_TOK * 128;           // N_TOK rows x 64 bf16
-    static constexpr uint32_t kXBytes = 2 * kXAtomBytes;           // 128 columns of K
-    static constexpr uint32_t kStageBytes = kDenseBytes + kXBytes;
-    static constexpr uint32_t kBarrierOffset = STAGES * kStageBytes;
+    static constexpr uint32_t kXBytesMax = kPrefillMaxTok * 256;   // n_tok rows x 128 columns of K
+    static constexpr uint32_t kStageBytes = kDenseBytes + kXBytesMax;
+    static constexpr uint32_t kBarrierOffset = kPrefillStages * kStageBytes;
     static constexpr uint32_t kSmemBytes = kBarrierOffset + 256 + 1024;  // + barriers + alignment slack
-    static constexpr uint32_t kTmemNeeded = N_TOK + 4 * STAGES;
-    static constexpr uint32_t kTmemCols = kTmemNeeded <= 32 ? 32 : kTmemNeeded <= 64 ? 64 : kTmemNeeded <= 128 ? 128
-                                          : kTmemNeeded <= 256 ? 256 : 512;
-    static_assert(N_TOK % 16 == 0 && N_TOK >= 16 && N_TOK <= 256, "MMA N must be a multiple of 16 in [16, 256]");
-    static_assert(kTmemNeeded <= 512, "accumulator + metadata exceed TMEM");
-    static_assert(STAGES <= 8, "barrier block holds at most 8 stages");
+    static constexpr uint32_t kTmemCols = 512;
+    static constexpr uint32_t kAcc1Col = 256, kMetaCol = 240;      // acc0 [0,240) meta [240,248) acc1 [256,496)
 };
 
-template <int N_TOK, int STAGES>
 __global__ void __launch_bounds__(192)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
-               int TK, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
-    using Cfg = PrefillConfig<N_TOK, STAGES>;
+               int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
+    using Cfg = PrefillConfig;
+    constexpr int STAGES = kPrefillStages;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
 
     const uint32_t bar_full = smem_base + Cfg::kBarrierOffset;    // 8 x 8 B
     const uint32_t bar_empty = bar_full + 64;                     // 8 x 8 B
-    const uint32_t bar_acc = bar_empty + 64;                      // 8 B
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Cfg::kBarrierOffset + 144);
+    const uint32_t bar_acc_full = bar_empty + 64;                 // 2 x 8 B
+    const uint32_t bar_acc_empty = bar_acc_full + 16;             // 2 x 8 B
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Cfg::kBarrierOffset + 160);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile uint32_t* stage_kind = reinterpret_cast<volatile uint32_t*>(tmem_slot + 2);  // STAGES words
 
@@ -53,15 +56,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
     grid_dependency_wait();     // X, the packed weight and Y may belong to the previous kernel until here
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tn = blockIdx.x, m0 = blockIdx.y * N_TOK;
-    const int n_tiles = TK;
+    if (warp == 0) PATCH_TRACE_AT(0);
+    const int MT = (M + n_tok - 1) / n_tok;
+    const int n_out = TN * MT;                                    // output tiles, index = mt * TN + tn
+    const uint32_t x_atom_bytes = uint32_t(n_tok) * 128u;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) {
             mbar_init(bar_full + 8 * i, 1);
             mbar_init(bar_empty + 8 * i, 1);
         }
-        mbar_init(bar_acc, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_acc_full + 8 * i, 1);
+            mbar_init(bar_acc_empty + 8 * i, 4);     // one arrival per epilogue warp
+        }
         *abort_flag = 0;
         mbar_init_fence();
         tma_prefetch_map(&tmap_x);
@@ -71,36 +79,39 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_acc = tmem_base;                 // columns [0, N_TOK)
-    const uint32_t tmem_meta = tmem_base + N_TOK;        // 4 columns per stage
+    if (warp == 0) PATCH_TRACE_AT(1);
 
     if (warp == 0) {
         // ---------------- producer ----------------
-        const uint64_t pol_w = l2_policy_evict_last(), pol_x = l2_policy_evict_last();
-        const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off) + int64_t(tn) * TK;
-        TileDesc mine = TileDesc{0, 0, 0, 0};
-        int issued = 0;
+        const uint64_t pol = l2_policy_evict_last();     // weights and activations are both re-read from L2
+        const TileDesc* table0 = reinterpret_cast<const TileDesc*>(blob + table_off);
+        int issued = 0;      // stage-ring position, continues across output tiles
         bool ok = true;
-        for (int i = 0; i < n_tiles && ok; ++i) {
-            if ((i & 31) == 0 && i + lane < n_tiles) mine = table[i + lane];   // 32 descriptors per warp load
-            const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
-            const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
-            if (lane == 0) {
-                const int stage = i % STAGES;
-                ok = mbar_wait(bar_empty + 8 * stage, (uint32_t(i / STAGES) & 1u) ^ 1u, abort_flag, status_dev);
-                if (ok) {
-                    const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
-                    const uint32_t sW = smem_base + stage * Cfg::kStageBytes, sX = sW + kDenseBytes;
-                    const uint32_t full = bar_full + 8 * stage;
-                    stage_kind[stage] = kind;
-                    mbar_expect_tx(full, wbytes + Cfg::kXBytes);
-                    tma_bulk_load(sW, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
-                    tma_tile_load(sX, &tmap_x, i * kTile, m0, full, pol_x);
-                    tma_tile_load(sX + Cfg::kXAtomBytes, &tmap_x, i * kTile + 64, m0, full, pol_x);
-                    issued = i + 1;
+        for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x) {
+            const int tn = t % TN, m0 = (t / TN) * n_tok;
+            const TileDesc* table = table0 + int64_t(tn) * TK;
+            TileDesc mine = TileDesc{0, 0, 0, 0};
+            for (int i = 0; i < TK && ok; ++i) {
+                if ((i & 31) == 0 && i + lane < TK) mine = table[i + lane];   // 32 descriptors per warp load
+                const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
+                const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
+                if (lane == 0) {
+                    const int stage = issued % STAGES;
+                    ok = mbar_wait(bar_empty + 8 * stage, (uint32_t(issued / STAGES) & 1u) ^ 1u, abort_flag, status_dev);
+                    if (ok) {
+                        const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
+                        const uint32_t sW = smem_base + stage * Cfg::kStageBytes, sX = sW + kDenseBytes;
+                        const uint32_t full = bar_full + 8 * stage;
+                        stage_kind[stage] = kind;
+                        mbar_expect_tx(full, wbytes + 2 * x_atom_bytes);
+                        tma_bulk_load(sW, blob + uint64_t(off16) * 16, wbytes, full, pol);
+                        tma_tile_load(sX, &tmap_x, i * kTile, m0, full, pol);
+                        tma_tile_load(sX + x_atom_bytes, &tmap_x, i * kTile + 64, m0, full, pol);
+                        ++issued;
+                    }
                 }
+                ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             }
-            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
         }
         if (lane == 0 && *abort_flag) {
             // drain: wait (bounded) until the copies this thread started have landed
@@ -114,42 +125,61 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             bool ok = true;
-            for (int i = 0; i < n_tiles && ok; ++i) {
-                const int stage = i % STAGES;
-                ok = mbar_wait(bar_full + 8 * stage, uint32_t(i / STAGES) & 1u, abort_flag, status_dev);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
-                issue_tile_mma<N_TOK>(stage_kind[stage], sW, sW + kDenseBytes, Cfg::kXAtomBytes, tmem_acc,
-                                      tmem_meta + 4 * stage, i == 0);
-                mma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
+            int step = 0, j = 0;      // stage-ring position; local output-tile counter
+            for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x, ++j) {
+                const uint32_t acc = tmem_base + (j & 1 ? Cfg::kAcc1Col : 0u);
+                // the epilogue must have drained this accumulator (two tiles ago)
+                ok = mbar_wait(bar_acc_empty + 8 * (j & 1), (uint32_t(j >> 1) & 1u) ^ 1u, abort_flag, status_dev);
+                for (int i = 0; i < TK && ok; ++i, ++step) {
+                    const int stage = step % STAGES;
+                    ok = mbar_wait(bar_full + 8 * stage, uint32_t(step / STAGES) & 1u, abort_flag, status_dev);
+                    if (!ok) break;
+                    if (step == 0) PATCH_TRACE_AT(2);
+                    tc_fence_after();
+                    const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
+                    issue_tile_mma_n(stage_kind[stage], sW, sW + kDenseBytes, x_atom_bytes, acc,
+                                     tmem_base + Cfg::kMetaCol + 4 * stage, i == 0, uint32_t(n_tok));
+                    mma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
+                }
+                if (ok) mma_commit(bar_acc_full + 8 * (j & 1));      // accumulator complete
             }
-            mma_commit(bar_acc);                     // accumulator complete
+            PATCH_TRACE_AT(3);
         }
         __syncwarp();
     } else {
         // ---------------- epilogue: warps 2..5, TMEM lane quadrant = warp % 4 ----------------
         const uint32_t quad = warp & 3u, row = quad * 32 + lane;   // out-feature inside the row-block
-        const bool ok = mbar_wait(bar_acc, 0, abort_flag, status_dev);
-        tc_fence_after();
-        const int valid = M - m0 < N_TOK ? M - m0 : N_TOK;          // tokens of this tile that exist
-        if (ok) {
+        bool ok = true;
+        int j = 0;
+        for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x, ++j) {
+            const int tn = t % TN, m0 = (t / TN) * n_tok;
+            ok = mbar_wait(bar_acc_full + 8 * (j & 1), uint32_t(j >> 1) & 1u, abort_flag, status_dev);
+            if (!ok) break;
+            tc_fence_after();
+            if (j == 0 && warp == 2) PATCH_TRACE_AT(4);
+            const uint32_t acc = tmem_base + (j & 1 ? Cfg::kAcc1Col : 0u) + ((quad * 32u) << 16);
+            const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
 #pragma unroll 1
             for (int c0 = 0; c0 < valid; c0 += 16) {
                 uint32_t v[16];
-                tmem_ld16(tmem_acc + ((quad * 32u) << 16) + uint32_t(c0), v);
+                tmem_ld16(acc + uint32_t(c0), v);
                 tmem_ld_wait();
                 __nv_bfloat16* y = Y + int64_t(m0 + c0) * ldy + int64_t(tn) * kTile + row;
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (c0 + j < valid) y[int64_t(j) * ldy] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                for (int q = 0; q < 16; ++q)
+                    if (c0 + q < valid) y[int64_t(q) * ldy] = __float2bfloat16_rn(__uint_as_float(v[q]));
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (j & 1));
         }
+        if (warp == 2) PATCH_TRACE_AT(5);
     }
 
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    if (warp == 0) PATCH_TRACE_AT(6);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -184,43 +214,79 @@ int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int
     return r == CUDA_SUCCESS ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
-template <int N_TOK, int STAGES>
-static int launch_prefill_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M,
-                            __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
-    using Cfg = PrefillConfig<N_TOK, STAGES>;
-    auto kern = prefill_kernel<N_TOK, STAGES>;
-    static bool configured = false;   // per-process attribute, idempotent
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
-            return PATCH_ERR_CUDA;
-        configured = true;
+static int sm_count_prefill() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        return v;
+    }();
+    return n;
+}
+
+int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
+                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+
+// Schedule choice: token-tile width n (a multiple of 16 in [128, 240]) and one or two row-blocks
+// per CTA, by a small cost model -- waves of output tiles over the SMs times the time of one tile,
+// which is the slower of the tensor pipe (0.55 us per 128 x 128 x 256 step at full clocks) and
+// what one SM pulls from L2 (measured: ~105 GB/s with two whole-tile stages, ~120 GB/s with the
+// two-ring pipeline), plus a per-tile prologue/epilogue cost.
+struct PrefillPlan { int n_tok; bool two_row_blocks; };
+
+static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms) {
+    PrefillPlan best = {240, false};
+    double best_cost = 1e300;
+    const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : 240, n_lo = M <= 128 ? n_hi : 128;
+    for (int n = n_hi; n >= n_lo; n -= 16) {
+        const int64_t MT = (M + n - 1) / n;
+        for (int two = 0; two < 2; ++two) {
+            const int64_t tiles = int64_t(two ? (TN + 1) / 2 : TN) * MT;
+            const int64_t waves = (tiles + sms - 1) / sms;
+            const double mma_ns = (two ? 1100.0 : 550.0) * n / 256.0;
+            const double load_ns = two ? (65536.0 + n * 256.0) / 120.0 : (32768.0 + n * 256.0) / 105.0;
+            const double tile_ns = TK * (mma_ns > load_ns ? mma_ns : load_ns) + (two ? 10000.0 : 6000.0);
+            const double cost = double(waves) * tile_ns;
+            if (cost < best_cost) { best_cost = cost; best = {n, two != 0}; }
+        }
     }
-    const int TN = int(L->N / kTile), TK = int(L->K / kTile);
-    const int64_t MT = (M + N_TOK - 1) / N_TOK;
-    if (MT > 65535) return PATCH_ERR_SHAPE;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    cfg.gridDim = dim3(TN, unsigned(MT), 1);
-    cfg.blockDim = dim3(192, 1, 1);
-    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
-    cfg.stream = stream;
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, packed, uint64_t(L->table_off), TK, int(M), Y, ldy, status_dev);
-    return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+    return best;
 }
 
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                    __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
     if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
-    const int n_tok = M <= 128 ? 128 : 256;
+    const int sms = sm_count_prefill();
+    if (sms <= 0) return PATCH_ERR_CUDA;
+    const int TN = int(L->N / kTile), TK = int(L->K / kTile);
+    const PrefillPlan plan = plan_prefill(M, TN, TK, sms);
+    const int n_tok = plan.n_tok;
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
-    if (n_tok == 128) return launch_prefill_t<128, 3>(map, L, packed, M, Y, ldy, status_dev, stream);
-    return launch_prefill_t<256, 2>(map, L, packed, M, Y, ldy, status_dev, stream);
+    if (plan.two_row_blocks) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream);
+    static bool configured = false;   // per-process attribute, idempotent
+    if (!configured) {
+        if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PrefillConfig::kSmemBytes) != cudaSuccess)
+            return PATCH_ERR_CUDA;
+        configured = true;
+    }
+    const int64_t n_out = int64_t(TN) * ((M + n_tok - 1) / n_tok);
+    if (n_out > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(unsigned(n_out < sms ? n_out : sms), 1, 1);
+    cfg.blockDim = dim3(192, 1, 1);
+    cfg.dynamicSmemBytes = PrefillConfig::kSmemBytes;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
+                                       Y, ldy, status_dev);
+    return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
 }  // namespace patch

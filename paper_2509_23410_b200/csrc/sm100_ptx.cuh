@@ -183,6 +183,30 @@ __device__ __forceinline__ void issue_tile_mma(uint32_t kind, uint32_t sW, uint3
     }
 }
 
+// Same with the token count of the MMA (its N dimension) chosen at run time.
+__device__ __forceinline__ void issue_tile_mma_n(uint32_t kind, uint32_t sW, uint32_t sX, uint32_t x_atom_bytes,
+                                                 uint32_t acc_tmem, uint32_t e_tmem, bool first, uint32_t n_tok) {
+    const uint32_t idesc_d = instr_desc(0, false) | ((n_tok >> 3) << 17);
+    const uint32_t idesc_s = idesc_d | (1u << 2);
+    const uint64_t dA = desc_kmajor_sw128(sW), dB = desc_kmajor_sw128(sX);
+    if (kind == PATCH_TILE_DENSE) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t a = dA + uint64_t(((ks >> 2) * kAtomBytes + (ks & 3) * 32) >> 4);
+            const uint64_t b = dB + uint64_t(((ks >> 2) * x_atom_bytes + (ks & 3) * 32) >> 4);
+            mma_dense(acc_tmem, a, b, idesc_d, !(first && ks == 0));
+        }
+    } else {
+        tmem_copy_128x128b(e_tmem, desc_rows16(sW + kAtomBytes));
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t a = dA + uint64_t((ks * 32) >> 4);
+            const uint64_t b = dB + uint64_t(((ks >> 1) * x_atom_bytes + (ks & 1) * 64) >> 4);
+            mma_sparse(acc_tmem, a, b, e_tmem + (ks & 2), idesc_s | uint32_t(ks & 1), !(first && ks == 0));
+        }
+    }
+}
+
 // Host: tensor map over X [M x ldx] bf16 with a box of 64 columns (128 B) x n_tok rows,
 // 128-byte swizzle, zero fill outside the matrix.
 int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok);
