@@ -427,7 +427,7 @@ def run_ours(args):
 
 
 def B_kernel_name(M):
-    return "decode_kernel" if M <= 64 else "prefill_kernel"
+    return "decode_kernel" if M <= 64 else "prefill2_kernel (two row-blocks per CTA) or prefill_kernel, chosen per shape"
 
 
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes per launch, from the ncu

@@ -33,13 +33,14 @@ constexpr uint32_t kASlotBytes = kSparseBytes;                 // 18 432
 constexpr uint32_t kBSlotBytes = kMaxTok * 128;                // 30 720
 constexpr uint32_t kBOffset = NA * kASlotBytes;
 constexpr uint32_t kBarrierOffset = kBOffset + NB * kBSlotBytes;
-constexpr uint32_t kSmemBytes = kBarrierOffset + 512 + 1024;   // + barriers/misc + alignment slack
+constexpr uint32_t kStageOffset = kBarrierOffset + 512;         // 8 epilogue warps x 1 KB transpose staging
+constexpr uint32_t kSmemBytes = kStageOffset + 8 * 1024 + 1024; // + alignment slack
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAcc1Col = 256;                              // acc0 [0,240)  acc1 [256,496)
 // metadata: 4 TMEM columns per A slot, in the gaps [240,256) and [496,512)
 __device__ __forceinline__ uint32_t meta_col(int slot) { return slot < 4 ? 240u + 4u * slot : 496u + 4u * (slot - 4); }
-// what an A slot holds
-constexpr uint32_t kHalf0 = 0, kHalf1 = 1, kSparse = 2;
+// what an A slot holds: 0 / 1 = first / second K-half of a dense tile, 2 = a whole 2:4 tile
+constexpr uint32_t kSparse = 2;
 }  // namespace p2
 
 __global__ void __launch_bounds__(320)
@@ -235,7 +236,7 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
         __syncwarp();
     } else {
         // ---------------- epilogue: warps 2..9; lane quadrant = warp % 4, column half = (warp - 2) / 4 ----
-        const uint32_t quad = warp & 3u, row = quad * 32 + lane;
+        const uint32_t quad = warp & 3u;
         const int half = (warp - 2) >> 2;
         bool ok = true;
         int j = 0;
@@ -245,6 +246,9 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             ok = mbar_wait(bar_acc_full, uint32_t(j) & 1u, abort_flag, status_dev);
             if (!ok) break;
             tc_fence_after();
+#ifdef PATCH_TRACE
+            const long long te0 = clock64();
+#endif
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             const int chunks = (valid + 15) / 16, c_begin = half == 0 ? 0 : (chunks + 1) / 2,
                       c_end = half == 0 ? (chunks + 1) / 2 : chunks;
@@ -252,21 +256,23 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             for (int rb = 0; rb < 2; ++rb) {
                 if (rb == 1 && !has1) break;
                 const uint32_t acc = tmem_base + (rb ? kAcc1Col : 0u) + ((quad * 32u) << 16);
+                __nv_bfloat16* ytile = Y + int64_t(m0) * ldy + int64_t(tn0 + rb) * kTile + quad * 32;
 #pragma unroll 1
                 for (int ch = c_begin; ch < c_end; ++ch) {
                     const int c0 = ch * 16;
                     uint32_t v[16];
                     tmem_ld16(acc + uint32_t(c0), v);
                     tmem_ld_wait();
-                    __nv_bfloat16* y = Y + int64_t(m0 + c0) * ldy + int64_t(tn0 + rb) * kTile + row;
-#pragma unroll
-                    for (int q = 0; q < 16; ++q)
-                        if (c0 + q < valid) y[int64_t(q) * ldy] = __float2bfloat16_rn(__uint_as_float(v[q]));
+                    store_fragment_transposed(v, smem + kStageOffset + (warp - 2) * 1024, lane, ytile + int64_t(c0) * ldy, ldy,
+                                              valid - c0);
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty);
+#ifdef PATCH_TRACE
+            if (warp == 2 && lane == 0) reinterpret_cast<unsigned long long*>(status_dev)[blockIdx.x * 16 + 5] += clock64() - te0;
+#endif
         }
     }
 

@@ -30,7 +30,8 @@ struct PrefillConfig {
     static constexpr uint32_t kXBytesMax = kPrefillMaxTok * 256;   // n_tok rows x 128 columns of K
     static constexpr uint32_t kStageBytes = kDenseBytes + kXBytesMax;
     static constexpr uint32_t kBarrierOffset = kPrefillStages * kStageBytes;
-    static constexpr uint32_t kSmemBytes = kBarrierOffset + 256 + 1024;  // + barriers + alignment slack
+    static constexpr uint32_t kStageOffset = kBarrierOffset + 256;       // 4 epilogue warps x 1 KB transpose staging
+    static constexpr uint32_t kSmemBytes = kStageOffset + 4 * 1024 + 1024;   // + alignment slack
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kAcc1Col = 256, kMetaCol = 240;      // acc0 [0,240) meta [240,248) acc1 [256,496)
 };
@@ -148,7 +149,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
         __syncwarp();
     } else {
         // ---------------- epilogue: warps 2..5, TMEM lane quadrant = warp % 4 ----------------
-        const uint32_t quad = warp & 3u, row = quad * 32 + lane;   // out-feature inside the row-block
+        const uint32_t quad = warp & 3u;     // this warp's 32 out-features inside the row-block
         bool ok = true;
         int j = 0;
         for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x, ++j) {
@@ -159,15 +160,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
             if (j == 0 && warp == 2) PATCH_TRACE_AT(4);
             const uint32_t acc = tmem_base + (j & 1 ? Cfg::kAcc1Col : 0u) + ((quad * 32u) << 16);
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
+            __nv_bfloat16* ytile = Y + int64_t(m0) * ldy + int64_t(tn) * kTile + quad * 32;
 #pragma unroll 1
             for (int c0 = 0; c0 < valid; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(acc + uint32_t(c0), v);
                 tmem_ld_wait();
-                __nv_bfloat16* y = Y + int64_t(m0 + c0) * ldy + int64_t(tn) * kTile + row;
-#pragma unroll
-                for (int q = 0; q < 16; ++q)
-                    if (c0 + q < valid) y[int64_t(q) * ldy] = __float2bfloat16_rn(__uint_as_float(v[q]));
+                store_fragment_transposed(v, smem + Cfg::kStageOffset + (warp - 2) * 1024, lane, ytile + int64_t(c0) * ldy, ldy,
+                                          valid - c0);
             }
             tc_fence_before();
             __syncwarp();

@@ -207,6 +207,26 @@ __device__ __forceinline__ void issue_tile_mma_n(uint32_t kind, uint32_t sW, uin
     }
 }
 
+// Epilogue helper.  A warp holds a 32-row x 16-token fp32 fragment (thread = out-feature row,
+// v[j] = token j) and Y is [token][out-feature]: storing straight from registers would be sixteen
+// 2-byte stores per thread.  The fragment is converted to bf16, transposed through 1 KB of this
+// warp's shared memory and written as two 16-byte vectors per thread (64 contiguous bytes per token).
+//   stage   this warp's 1 KB staging buffer      y   &Y[first token of the fragment][first row of the warp]
+__device__ __forceinline__ void store_fragment_transposed(const uint32_t (&v)[16], uint8_t* stage, int lane,
+                                                          __nv_bfloat16* y, int64_t ldy, int n_valid) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+        *reinterpret_cast<__nv_bfloat16*>(stage + j * 64 + lane * 2) = __float2bfloat16_rn(__uint_as_float(v[j]));
+    __syncwarp();
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+        const int tok = p * 8 + (lane >> 2), chunk = lane & 3;
+        const uint4 q = *reinterpret_cast<const uint4*>(stage + tok * 64 + chunk * 16);
+        if (tok < n_valid) *reinterpret_cast<uint4*>(y + int64_t(tok) * ldy + chunk * 8) = q;
+    }
+    __syncwarp();
+}
+
 // Host: tensor map over X [M x ldx] bf16 with a box of 64 columns (128 B) x n_tok rows,
 // 128-byte swizzle, zero fill outside the matrix.
 int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok);
