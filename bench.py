@@ -43,7 +43,7 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-def workload_cases(name: str):
+def workload_cases(name: str, stack_m: int = 1):
     if name == "decode":
         cases = inputs.decode_cases()
         # all M=1 GEMMs first, then all M=16: a matrix is re-read only after ~0.66 GB of other weights
@@ -54,6 +54,9 @@ def workload_cases(name: str):
         return sorted(inputs.llama13b_cases(), key=lambda c: c["M"])
     if name == "single":
         return [inputs.single_gemm_case()]
+    if name == "stack":
+        # 32 blocks x (q,k,v,o,gate,up,down) = 224 matrices, per-matrix 2:4-tile fraction ~ U[0,1]
+        return [dict(c, M=stack_m) for c in inputs.stack_cases()]
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -218,7 +221,7 @@ def run_ours(args):
     def to_dev(bits):
         return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
 
-    cases = workload_cases(args.workload)
+    cases = workload_cases(args.workload, args.stack_m)
     # ---- setup (untimed): weights, packing, activations; replicas: every rank holds the whole workload
     mats = {}
     pack_bytes, pack_secs = 0.0, 0.0
@@ -226,7 +229,13 @@ def run_ours(args):
         key = (c["N"], c["K"], c["stream"])
         if key in mats:
             continue
-        W = to_dev(inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]))
+        if args.workload == "stack":
+            # 6.5 G weights: drawn on the device (torch Philox, seeded per matrix) instead of on the host
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(inputs.MASTER_SEED * 1000 + len(mats))
+            W = torch.empty((c["N"], c["K"]), dtype=torch.bfloat16, device=dev).normal_(0.0, 0.02, generator=gen)
+        else:
+            W = to_dev(inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]))
         flags = inputs.tile_flags(c["N"], c["K"], c["p"], inputs.MASTER_SEED, *c["stream"])
         layout = B.patch_packed_size(c["N"], c["K"], flags)
         packed = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
@@ -240,12 +249,21 @@ def run_ours(args):
         pack_bytes += c["N"] * c["K"] * 2 + layout.total_bytes
         mats[key] = (layout, packed)
         del W
-    jobs = []
+    jobs, stack_x, shared_ws = [], {}, {}
     for c in cases:
         layout, packed = mats[(c["N"], c["K"], c["stream"])]
-        X = to_dev(inputs.activation(c["M"], c["K"], inputs.MASTER_SEED, *c["stream"], c["M"]))
+        xkey = (c["M"], c["K"]) if args.workload == "stack" else None
+        if xkey is not None and xkey in stack_x:
+            X = stack_x[xkey]                # the stack shares one activation per (M, K); outputs are not chained
+        else:
+            X = to_dev(inputs.activation(c["M"], c["K"], inputs.MASTER_SEED, *c["stream"], c["M"]))
+            if xkey is not None:
+                stack_x[xkey] = X
         Y = torch.empty((c["M"], c["N"]), dtype=torch.bfloat16, device=dev)
-        ws = torch.zeros(max(B.patch_gemm_workspace_size(layout, c["M"]), 256), dtype=torch.uint8, device=dev)
+        wkey = (c["M"], c["N"])
+        if wkey not in shared_ws:            # GEMMs on one stream are ordered, so they may share a workspace
+            shared_ws[wkey] = torch.zeros(max(B.patch_gemm_workspace_size(layout, c["M"]), 256), dtype=torch.uint8, device=dev)
+        ws = shared_ws[wkey]
         jobs.append(dict(case=c, layout=layout, packed=packed, X=X, Y=Y, ws=ws, cost=case_costs(c, layout)))
     weight_bytes = sum(m[0].total_bytes for m in mats.values())
 
@@ -402,7 +420,8 @@ def run_ours(args):
         "metric": "hybrid_tile_gemm_effective_tflops", "value": value, "unit": "TFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_s * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"llama2-7b {args.workload} linears" if args.workload != "13b" else "llama2-13b linears",
+        "config": {"workload": {"13b": "llama2-13b linears", "stack": f"llama2-7b full linear stack, M={args.stack_m}",
+                                "single": "single 1024x1024 GEMM"}.get(args.workload, f"llama2-7b {args.workload} linears"),
                    "gemms_per_step": len(jobs), "tile": "128x128",
                    "packed_weight_bytes": weight_bytes,
                    "l2": "inputs larger than L2: each step streams all packed matrices once per M",
@@ -447,7 +466,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack"])
+    ap.add_argument("--stack-m", type=int, default=1, help="tokens per GEMM of the 224-GEMM stack workload")
     ap.add_argument("--launch", default="independent", choices=["dependent", "independent"],
                     help="independent (default; true for this workload, whose GEMMs do not feed each other): "
                          "the caller promises X is not produced by the preceding kernel; dependent: every "

@@ -13,9 +13,10 @@
 //     are the A operand, tokens ride the MMA N dimension (16/32/64).
 //   * A run covers at most one partial row-block at each end.  Partial sums go to the caller's
 //     workspace; a 64-bit counter per row-block collects {tiles, contributors, first
-//     contributor}.  The CTA that completes the tile count sums the partials in ascending K
-//     order (deterministic) and writes bf16.  Two TMEM accumulators let this epilogue overlap
-//     the next row-block's MMAs.
+//     contributor}.  Partials are summed in ascending K order (deterministic) and written as
+//     bf16: for up to 16 tokens by the CTA that completes the tile count; for 32 or 64 tokens
+//     every contributor waits for the count and finishes a share of the rows.  Two TMEM
+//     accumulators let this epilogue overlap the next row-block's MMAs.
 //   * The kernel uses half an SM's shared memory and is launched with programmatic dependent
 //     launch: the next GEMM's CTAs become resident while this one streams, fetch their first
 //     weight tiles, and wait for this grid only where they touch X, Y or the workspace.
@@ -86,13 +87,14 @@ __device__ __forceinline__ uint4 ld_cg_issue(const uint4* p) {
 
 // Last contributor of a row-block: sum the partial tiles in ascending K order (contributor
 // order), 16 tokens at a time, and write bf16.  `info` = {tiles:16, contributors:16, first
-// contributor's slot + 1 : 32}; later contributors are the following CTAs' first slots.
+// contributor's slot + 1 : 16, finished readers : 16}; later contributors are the following
+// CTAs' first slots.
 // Loads are unconditional (indices clamped) so that eight contributors are in flight together.
 template <int N_TOK>
 __device__ __forceinline__ void reduce_row_block(const float* __restrict__ partials, unsigned long long info,
                                                  uint32_t row, int M, __nv_bfloat16* ycol, int64_t ldy) {
     const int n_contrib = int((info >> 16) & 0xFFFFu);
-    const int first_slot = int(info >> 32) - 1;
+    const int first_slot = int((info >> 32) & 0xFFFFu) - 1;
     const int c_lo = first_slot >> 1;
 #pragma unroll 1
     for (int c0 = 0; c0 < M; c0 += 16) {
@@ -126,6 +128,57 @@ __device__ __forceinline__ void reduce_row_block(const float* __restrict__ parti
 #pragma unroll
         for (int i = 0; i < 16; ++i)
             if (c0 + i < M) ycol[int64_t(c0 + i) * ldy] = __float2bfloat16_rn(a[i]);
+    }
+}
+
+__device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Every contributor of a row-block finishes rows [r0, r1) of it: thread `et` (0..127) takes
+// (row, 16-token chunk) items, sums the n_contrib partial tiles in ascending K order and writes bf16.
+template <int N_TOK>
+__device__ __forceinline__ void reduce_row_share(const float* __restrict__ partials, int first_slot, int n_contrib,
+                                                 int r0, int r1, int M, __nv_bfloat16* ytile, int64_t ldy, int et) {
+    constexpr int CH = N_TOK / 16;
+    const int c_lo = first_slot >> 1;
+    const int items = (r1 - r0) * CH;
+#pragma unroll 1
+    for (int it = et; it < items; it += 128) {
+        const int row = r0 + it / CH, c0 = (it % CH) * 16;
+        if (c0 >= M) continue;
+        float a[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] = 0.f;
+#pragma unroll 1
+        for (int j0 = 0; j0 < n_contrib; j0 += 8) {
+            uint4 q[8][4];
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+                const int j = j0 + jj < n_contrib ? j0 + jj : n_contrib - 1;
+                const int s = j == 0 ? first_slot : 2 * (c_lo + j);
+                const uint4* src = reinterpret_cast<const uint4*>(partials + (int64_t(s) * kTile + row) * N_TOK + c0);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) q[jj][i] = ld_cg_issue(src + i);
+            }
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+                if (j0 + jj < n_contrib) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        a[4 * i + 0] += __uint_as_float(q[jj][i].x);
+                        a[4 * i + 1] += __uint_as_float(q[jj][i].y);
+                        a[4 * i + 2] += __uint_as_float(q[jj][i].z);
+                        a[4 * i + 3] += __uint_as_float(q[jj][i].w);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (c0 + i < M) ytile[int64_t(c0 + i) * ldy + row] = __float2bfloat16_rn(a[i]);
     }
 }
 
@@ -332,7 +385,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                 if (warp == 2) PATCH_TRACE_AT(k == 0 ? 9 : 12);
                 part_tn[k] = tn;
                 if (et == 32 * k) {
-                    // {tiles : 16, contributors : 16, (first contributor's slot + 1) : 32}
+                    // {tiles : 16, contributors : 16, first contributor's slot + 1 : 16, finished readers : 16}
                     unsigned long long add = (unsigned long long)ntiles | (1ull << 16);
                     if (ts == tn * TK) add |= (unsigned long long)(2 * c + k + 1) << 32;
                     // release: publishes the partial sums written before the barrier;
@@ -342,21 +395,62 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
             }
             ts = te;
         }
-        if (ok && (part_tn[0] >= 0 || part_tn[1] >= 0)) {
-            if (et == 0 || et == 32) {
-                const int k = et >> 5;
-                const bool is_last = part_tn[k] >= 0 && int(seen & 0xFFFFu) == TK;
-                if (is_last) counters[part_tn[k]] = 0;             // ready for the next launch
-                red_info[k] = is_last ? seen : 0ull;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (warp == 2) PATCH_TRACE_AT(10);
+        if constexpr (N_TOK <= 16) {
+            // small partial tiles: the contributor that completed the tile count finishes the row-block
+            if (ok && (part_tn[0] >= 0 || part_tn[1] >= 0)) {
+                if (et == 0 || et == 32) {
+                    const int k = et >> 5;
+                    const bool is_last = part_tn[k] >= 0 && int(seen & 0xFFFFu) == TK;
+                    if (is_last) counters[part_tn[k]] = 0;             // ready for the next launch
+                    red_info[k] = is_last ? seen : 0ull;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (warp == 2) PATCH_TRACE_AT(10);
 #pragma unroll 1
-            for (int k = 0; k < 2; ++k) {
+                for (int k = 0; k < 2; ++k) {
+                    const unsigned long long info = red_info[k];
+                    if (info != 0ull) {     // this CTA completed row-block part_tn[k]: sum its partials
+                        reduce_row_block<N_TOK>(partials, info, row, M, Y + int64_t(part_tn[k]) * kTile + row, ldy);
+                        if (warp == 2) PATCH_TRACE_AT(k == 0 ? 11 : 14);
+                    }
+                }
+            }
+        } else {
+            // large partial tiles (32 or 64 tokens): every contributor finishes a share of the rows.  All
+            // partials of this CTA are already published above, so waiting here cannot form a cycle.
+#pragma unroll 1
+            for (int k = 0; k < 2 && ok; ++k) {
+                if (part_tn[k] < 0) continue;
+                unsigned long long* ctr = &counters[part_tn[k]];
+                if (et == 32 * k) {
+                    unsigned long long cur = seen;
+                    const uint64_t tstart = global_timer_ns();
+                    while (int(cur & 0xFFFFu) != TK) {                 // bounded wait for the other contributors
+                        cur = ld_acquire_gpu(ctr);
+                        if (*abort_flag || global_timer_ns() - tstart > kWaitLimitNs) {
+                            *abort_flag = 1;
+                            if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                            cur = 0ull;
+                            break;
+                        }
+                    }
+                    red_info[k] = cur;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
                 const unsigned long long info = red_info[k];
-                if (info != 0ull) {     // this CTA completed row-block part_tn[k]: sum its partials
-                    reduce_row_block<N_TOK>(partials, info, row, M, Y + int64_t(part_tn[k]) * kTile + row, ldy);
-                    if (warp == 2) PATCH_TRACE_AT(k == 0 ? 11 : 14);
+                ok = info != 0ull;
+                if (ok) {
+                    const int n_contrib = int((info >> 16) & 0xFFFFu);
+                    const int first_slot = int((info >> 32) & 0xFFFFu) - 1;
+                    const int mine = (2 * c + k == first_slot) ? 0 : c - (first_slot >> 1);   // position in K order
+                    reduce_row_share<N_TOK>(partials, first_slot, n_contrib, kTile * mine / n_contrib,
+                                            kTile * (mine + 1) / n_contrib, M, Y + int64_t(part_tn[k]) * kTile, ldy, et);
+                    asm volatile("bar.sync 1, 128;" ::: "memory");     // every thread has read its partials
+                    if (et == 32 * k) {
+                        // count finished readers in bits 48..63; the last one clears the counter for the next launch
+                        const unsigned long long old = atomicAdd(ctr, 1ull << 48);
+                        if (int(old >> 48) + 1 == n_contrib) *ctr = 0ull;
+                    }
                 }
             }
         }
