@@ -203,7 +203,7 @@ def run_reference(args):
 
 def run_ours(args):
     import torch
-    from paper_2509_23410_b200 import binding as B
+    from paper_2509_23410_b200 import binding as B, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -314,11 +314,7 @@ def run_ours(args):
     e1.record()
     barrier()
     secs = e0.elapsed_time(e1) * 1e-3
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([secs], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        secs = float(t.item())
+    secs = replicas.max_over_ranks(secs, dev)
     step_s = secs / args.steps
     step_flops = sum(j["cost"]["flops"] for j in jobs)
     value = world * step_flops / step_s / 1e12
@@ -384,11 +380,7 @@ def run_ours(args):
         e2e_step()
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = replicas.max_over_ranks(e2e_s, dev)
     h2d = sum(j["X"].numel() * 2 for j in jobs)
     d2h = sum(j["Y"].numel() * 2 for j in jobs)
 
