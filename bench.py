@@ -191,7 +191,7 @@ def run_reference(args):
         "impl": "reference", "metric": "hybrid_tile_gemm_effective_tflops", "value": value, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 3), "ms_per_step": dt / steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "sample": names},
+        "config": {"workload": workload_label(args), "sample": names},
         "cpu_baseline": cpu,
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -412,8 +412,7 @@ def run_ours(args):
         "metric": "hybrid_tile_gemm_effective_tflops", "value": value, "unit": "TFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_s * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": {"13b": "llama2-13b linears", "stack": f"llama2-7b full linear stack, M={args.stack_m}",
-                                "single": "single 1024x1024 GEMM"}.get(args.workload, f"llama2-7b {args.workload} linears"),
+        "config": {"workload": workload_label(args),
                    "gemms_per_step": len(jobs), "tile": "128x128",
                    "packed_weight_bytes": weight_bytes,
                    "l2": "inputs larger than L2: each step streams all packed matrices once per M",
@@ -435,6 +434,11 @@ def run_ours(args):
     if table:
         out["cases"] = table
     print(json.dumps(out))
+
+
+def workload_label(args):
+    return {"13b": "llama2-13b linears", "stack": f"llama2-7b full linear stack, M={args.stack_m}",
+            "single": "single 1024x1024 GEMM"}.get(args.workload, f"llama2-7b {args.workload} linears")
 
 
 def B_kernel_name(M):
