@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(128) rate_kernel(int mode, int n_tok, int iter
             }
         }
         mma_commit(smem_u32(&bar));
-        while (!mbar_try_wait(smem_u32(&bar), 0)) {}
+        for (long long spin = 0; spin < (1ll << 26) && !mbar_try_wait(smem_u32(&bar), 0); ++spin) {}   // bounded
         t1 = clock64();
         out[blockIdx.x] = t1 - t0;
     }
