@@ -132,8 +132,9 @@ int patch_unpack(const patch_layout_t* layout, const void* packed_dev, void* Wha
 int patch_gemm_workspace_size(const patch_layout_t* layout, int64_t M, size_t* bytes_out);
 
 /*
- * Zero a workspace once after allocating it (the arrival counters must start at zero; every
- * successful patch_gemm leaves them zero again).
+ * Zero a workspace once after allocating it (arrival counters and partial-sum flags must start at
+ * zero; every successful patch_gemm leaves them zero again).  Zero it again after a call that
+ * reported PATCH_ERR_TIMEOUT.
  */
 int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream);
 
@@ -195,8 +196,8 @@ int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* layout,
  *   Limits: M <= 16 tokens and N <= 131072; beyond them the call returns PATCH_ERR_SIZE and
  *   launches nothing (use patch_gemm with a caller-owned workspace instead).
  *   The first call on each device looks up the array's device address; make that first call
- *   with the device current and before any stream capture.  Every call enqueues a small memset
- *   of the arrival counters followed by the kernel.
+ *   with the device current and before any stream capture.  Every call enqueues a memset of
+ *   the scratch array (it must start empty) followed by the kernel.
  *   All calls on a device share the one array, which keeps the last call's contents: calls that
  *   may overlap on the GPU (different streams) race with each other -- issue them on one stream
  *   or order them with events.

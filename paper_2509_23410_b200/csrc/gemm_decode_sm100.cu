@@ -11,12 +11,15 @@
 //   * Per tile the MMA warp issues eight dense tcgen05.mma or four tcgen05.mma.sp (metadata
 //     copied to TMEM) into an fp32 TMEM accumulator [128 out-features x N_TOK tokens]; weights
 //     are the A operand, tokens ride the MMA N dimension (16/32/64).
-//   * A run covers at most one partial row-block at each end.  Partial sums go to the caller's
-//     workspace; a 64-bit counter per row-block collects {tiles, contributors, first
-//     contributor}.  Partials are summed in ascending K order (deterministic) and written as
-//     bf16: for up to 16 tokens by the CTA that completes the tile count; for 32 or 64 tokens
-//     every contributor waits for the count and finishes a share of the rows.  Two TMEM
-//     accumulators let this epilogue overlap the next row-block's MMAs.
+//   * A run covers at most one partial row-block at each end; partial sums go through the
+//     caller's workspace and are added in ascending K order (deterministic) before the single
+//     bf16 rounding.  Up to 16 tokens: the partial-sum words double as flags (0 = empty); the CTA
+//     that owns a row-block's first tile finishes it by polling the following CTAs' words (their
+//     number follows from inverting the byte partition), then empties them -- one memory round
+//     trip between the last MMA and the result.  32 or 64 tokens (partial tiles of 16-32 KB): a
+//     64-bit counter per row-block collects {tiles, contributors, first contributor}; every
+//     contributor waits for the count and finishes a share of the rows.  Two TMEM accumulators
+//     let the epilogue of one row-block overlap the next row-block's MMAs.
 //   * The kernel uses half an SM's shared memory and is launched with programmatic dependent
 //     launch: the next GEMM's CTAs become resident while this one streams, fetch their first
 //     weight tiles, and wait for this grid only where they touch X, Y or the workspace.
@@ -85,51 +88,19 @@ __device__ __forceinline__ uint4 ld_cg_issue(const uint4* p) {
     return v;
 }
 
-// Last contributor of a row-block: sum the partial tiles in ascending K order (contributor
-// order), 16 tokens at a time, and write bf16.  `info` = {tiles:16, contributors:16, first
-// contributor's slot + 1 : 16, finished readers : 16}; later contributors are the following
-// CTAs' first slots.
-// Loads are unconditional (indices clamped) so that eight contributors are in flight together.
-template <int N_TOK>
-__device__ __forceinline__ void reduce_row_block(const float* __restrict__ partials, unsigned long long info,
-                                                 uint32_t row, int M, __nv_bfloat16* ycol, int64_t ldy) {
-    const int n_contrib = int((info >> 16) & 0xFFFFu);
-    const int first_slot = int((info >> 32) & 0xFFFFu) - 1;
-    const int c_lo = first_slot >> 1;
-#pragma unroll 1
-    for (int c0 = 0; c0 < M; c0 += 16) {
-        float a[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) a[i] = 0.f;
-#pragma unroll 1
-        for (int j0 = 0; j0 < n_contrib; j0 += 8) {
-            uint4 q[8][4];
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
-                const int j = j0 + jj < n_contrib ? j0 + jj : n_contrib - 1;
-                const int s = j == 0 ? first_slot : 2 * (c_lo + j);
-                const uint4* src = reinterpret_cast<const uint4*>(partials + (int64_t(s) * kTile + row) * N_TOK + c0);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) q[jj][i] = ld_cg_issue(src + i);
-            }
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
-                if (j0 + jj < n_contrib) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        a[4 * i + 0] += __uint_as_float(q[jj][i].x);
-                        a[4 * i + 1] += __uint_as_float(q[jj][i].y);
-                        a[4 * i + 2] += __uint_as_float(q[jj][i].z);
-                        a[4 * i + 3] += __uint_as_float(q[jj][i].w);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-            if (c0 + i < M) ycol[int64_t(c0 + i) * ldy] = __float2bfloat16_rn(a[i]);
-    }
+// 16-byte vector accesses at GPU scope that bypass L1.  A vector access is four 32-bit accesses,
+// each single-copy atomic, which is all the flagged-partials protocol needs: every 32-bit word is
+// either still empty (0) or the complete partial sum.
+__device__ __forceinline__ void st_relaxed_gpu_v4(uint32_t* p, uint4 v) {
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ uint4 ld_relaxed_gpu_v4(const uint32_t* p) {
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// A partial sum of +0 would look like an empty word; -0 adds to the same result.
+__device__ __forceinline__ uint32_t nonempty(uint32_t bits) { return bits == 0u ? 0x80000000u : bits; }
 
 __device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long long* p) {
     unsigned long long v;
@@ -221,7 +192,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
         const uint32_t hi = pay0_16 + uint32_t(uint64_t(c + 1) * pay_total_16 / G);
         const int t0 = first_tile_at_or_after(table, TN, TK, lo, lane);
         const int t1 = (c + 1 == G) ? TN * TK : first_tile_at_or_after(table, TN, TK, hi, lane);
-        if (lane == 0) { range[0] = t0; range[1] = t1; }
+        int n_others = -1;
+        if constexpr (N_TOK == 16) {
+            // Flagged-partials protocol: if this run ends inside a row-block whose first tile it
+            // owns, this CTA finishes that row-block.  The other contributors are the next CTAs, up
+            // to the owner of the row-block's last tile (inverse of the byte partition above).
+            const int tn_b = (t1 - 1) / TK;
+            if (t1 > t0 && t1 < (tn_b + 1) * TK && t0 <= tn_b * TK) {
+                const uint32_t d = table[(tn_b + 1) * TK - 1].payload_off16 - pay0_16;
+                const int c_last = int(((uint64_t(d) + 1) * uint64_t(G) - 1) / pay_total_16);
+                n_others = c_last - c;
+            }
+        }
+        if (lane == 0) { range[0] = t0; range[1] = t1; misc[16] = uint32_t(n_others); }
     }
     if (threadIdx.x == 64) {       // a thread outside warp 0, whose lanes are busy with the search
         for (int i = 0; i < STAGES; ++i) {
@@ -365,6 +348,81 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (seg & 1));
+            } else if constexpr (N_TOK == 16) {
+                // Partial row-block, flagged-partials protocol.  A slot is [CTA][row][16 tokens] fp32 whose
+                // words double as flags: 0 = not written yet (+0 is stored as -0).  The finishing CTA polls
+                // the words themselves, so no fence, counter or second round trip separates writer and reader.
+                uint32_t* words = reinterpret_cast<uint32_t*>(partials);
+                uint32_t v[16];
+                tmem_ld16(acc, v);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (seg & 1));
+                if (seg == 0 && t0 > tn * TK) {
+                    // the run starts inside this row-block: hand the partial to the CTA that owns its first tile
+                    uint32_t* mine = words + (int64_t(c) * kTile + row) * 16;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4)
+                        st_relaxed_gpu_v4(mine + j, make_uint4(nonempty(v[j]), nonempty(v[j + 1]), nonempty(v[j + 2]),
+                                                               nonempty(v[j + 3])));
+                    if (warp == 2) PATCH_TRACE_AT(9);
+                } else {
+                    // this run owns the row-block's first tile and ends inside it: add the following CTAs'
+                    // partials in ascending K order, four contributors in flight at a time
+                    const int n_others = int(misc[16]);
+                    float a[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) a[j] = __uint_as_float(v[j]);
+#pragma unroll 1
+                    for (int j0 = 0; j0 < n_others && ok; j0 += 4) {
+                        uint4 w[4][4];
+                        const uint64_t tstart = global_timer_ns();
+                        for (bool all = false; !all;) {
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj) {
+                                const int cj = c + 1 + (j0 + jj < n_others ? j0 + jj : n_others - 1);
+                                const uint32_t* src = words + (int64_t(cj) * kTile + row) * 16;
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) w[jj][q] = ld_relaxed_gpu_v4(src + 4 * q);
+                            }
+                            all = true;
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    all = all && w[jj][q].x != 0u && w[jj][q].y != 0u && w[jj][q].z != 0u && w[jj][q].w != 0u;
+                            if (!all && (*abort_flag || global_timer_ns() - tstart > kWaitLimitNs)) {
+                                *abort_flag = 1;
+                                if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                                ok = false;
+                                break;
+                            }
+                        }
+                        if (!ok) break;
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj) {
+                            if (j0 + jj < n_others) {
+                                uint32_t* src = words + (int64_t(c + 1 + j0 + jj) * kTile + row) * 16;
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    a[4 * q + 0] += __uint_as_float(w[jj][q].x);
+                                    a[4 * q + 1] += __uint_as_float(w[jj][q].y);
+                                    a[4 * q + 2] += __uint_as_float(w[jj][q].z);
+                                    a[4 * q + 3] += __uint_as_float(w[jj][q].w);
+                                    st_relaxed_gpu_v4(src + 4 * q, make_uint4(0, 0, 0, 0));   // empty again for the next launch
+                                }
+                            }
+                        }
+                    }
+                    if (ok) {
+                        __nv_bfloat16* ycol = Y + int64_t(tn) * kTile + row;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (j < M) ycol[int64_t(j) * ldy] = __float2bfloat16_rn(a[j]);
+                    }
+                    if (warp == 2) PATCH_TRACE_AT(14);
+                }
             } else {
                 // partial row-block: write fp32 partial sums ([slot][row][token]), then count in
                 const int k = seg == 0 ? 0 : 1;
@@ -395,27 +453,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
             }
             ts = te;
         }
-        if constexpr (N_TOK <= 16) {
-            // small partial tiles: the contributor that completed the tile count finishes the row-block
-            if (ok && (part_tn[0] >= 0 || part_tn[1] >= 0)) {
-                if (et == 0 || et == 32) {
-                    const int k = et >> 5;
-                    const bool is_last = part_tn[k] >= 0 && int(seen & 0xFFFFu) == TK;
-                    if (is_last) counters[part_tn[k]] = 0;             // ready for the next launch
-                    red_info[k] = is_last ? seen : 0ull;
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (warp == 2) PATCH_TRACE_AT(10);
-#pragma unroll 1
-                for (int k = 0; k < 2; ++k) {
-                    const unsigned long long info = red_info[k];
-                    if (info != 0ull) {     // this CTA completed row-block part_tn[k]: sum its partials
-                        reduce_row_block<N_TOK>(partials, info, row, M, Y + int64_t(part_tn[k]) * kTile + row, ldy);
-                        if (warp == 2) PATCH_TRACE_AT(k == 0 ? 11 : 14);
-                    }
-                }
-            }
-        } else {
+        if constexpr (N_TOK > 16) {
             // large partial tiles (32 or 64 tokens): every contributor finishes a share of the rows.  All
             // partials of this CTA are already published above, so waiting here cannot form a cycle.
 #pragma unroll 1
@@ -602,8 +640,8 @@ extern "C" int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M, con
     }
     void* scratch = g_noalloc_ptr[dev];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // the arrival counters must start at zero; the array keeps whatever the last call left
-    if (cudaMemsetAsync(scratch, 0, kNoAllocCounterBytes, s) != cudaSuccess) return PATCH_ERR_CUDA;
+    // counters and partial-sum flags must start at zero; the array keeps whatever the last call left
+    if (cudaMemsetAsync(scratch, 0, kNoAllocScratchBytes, s) != cudaSuccess) return PATCH_ERR_CUDA;
     return launch_decode(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
                          static_cast<__nv_bfloat16*>(Y_dev), ldy, scratch, nullptr, s, false, false);
 }
