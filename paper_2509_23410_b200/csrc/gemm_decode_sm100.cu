@@ -369,18 +369,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                     if (warp == 2) PATCH_TRACE_AT(9);
                 } else {
                     // this run owns the row-block's first tile and ends inside it: add the following CTAs'
-                    // partials in ascending K order, four contributors in flight at a time
+                    // partials in ascending K order, five contributors in flight at a time
+                    constexpr int kBatch = 5;     // covers the usual 148 / TN + 1 contributors in one round trip
                     const int n_others = int(misc[16]);
                     float a[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) a[j] = __uint_as_float(v[j]);
 #pragma unroll 1
-                    for (int j0 = 0; j0 < n_others && ok; j0 += 4) {
-                        uint4 w[4][4];
+                    for (int j0 = 0; j0 < n_others && ok; j0 += kBatch) {
+                        uint4 w[kBatch][4];
                         const uint64_t tstart = global_timer_ns();
                         for (bool all = false; !all;) {
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj) {
+                            for (int jj = 0; jj < kBatch; ++jj) {
                                 const int cj = c + 1 + (j0 + jj < n_others ? j0 + jj : n_others - 1);
                                 const uint32_t* src = words + (int64_t(cj) * kTile + row) * 16;
 #pragma unroll
@@ -388,7 +389,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                             }
                             all = true;
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj)
+                            for (int jj = 0; jj < kBatch; ++jj)
 #pragma unroll
                                 for (int q = 0; q < 4; ++q)
                                     all = all && w[jj][q].x != 0u && w[jj][q].y != 0u && w[jj][q].z != 0u && w[jj][q].w != 0u;
@@ -401,7 +402,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                         }
                         if (!ok) break;
 #pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) {
+                        for (int jj = 0; jj < kBatch; ++jj) {
                             if (j0 + jj < n_others) {
                                 uint32_t* src = words + (int64_t(c + 1 + j0 + jj) * kTile + row) * 16;
 #pragma unroll
