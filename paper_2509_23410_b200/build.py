@@ -28,6 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("PATCH_NVCC_FLAGS", "").split()     # tuning experiments, e.g. -DNAME=value
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
     return LIB

@@ -31,6 +31,9 @@
 namespace patch {
 
 constexpr int kMaxDecodeCtas = 192;      // workspace is sized for this many CTAs
+#ifndef PATCH_XSTATIC_STAGES
+#define PATCH_XSTATIC_STAGES 3           // ring depth when consecutive kernels stream concurrently (2 measured 2 % slower)
+#endif
 
 template <int N_TOK, int STAGES>
 struct DecodeConfig {
@@ -584,11 +587,8 @@ int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_la
     if (rc) return rc;
     switch (n_tok) {
         case 16:
-            // Measured: when consecutive kernels stream concurrently (X static) a shallower ring keeps
-            // the loaded memory latency, and with it the reduction tail, shorter; a kernel that must
-            // wait for its predecessor before touching X does better with three stages of prefetch.
             if (wstatic && xstatic)
-                return launch_decode_f<16, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+                return launch_decode_f<16, PATCH_XSTATIC_STAGES>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
             return launch_decode_f<16, 3>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
         case 32: return launch_decode_f<32, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
         default: return launch_decode_f<64, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
