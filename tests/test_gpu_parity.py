@@ -290,3 +290,67 @@ def test_back_to_back_launches_are_ordered(gpu, oracle):
         got = to_bits(bufs[i + 1])
         check_parity(oracle, got, Y32, f"chain step {i}")
         ref = got                                   # feed the GPU's own bf16 output forward
+
+
+# ---------------------------------------------------------------------------------------------
+# the benchmark's workloads, case by case, in the launch configuration bench.py times
+# (WEIGHTS_STATIC | INPUT_STATIC, automatic kernel choice); large M: sampled token rows
+
+
+def _check_case(gpu, oracle, W, flags, X, what, n_rows=16):
+    torch, B = gpu
+    M = X.shape[0]
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
+    if M <= 64:
+        Y32, _ = oracle.gemm_f64(X, What)
+        check_parity(oracle, Y, Y32, what)
+    else:
+        rng = inputs.generator(inputs.MASTER_SEED, "rows", what)
+        rows = np.unique(np.concatenate([rng.integers(0, M, n_rows), [0, M - 1, 239, 240, M // 2]]))
+        check_parity(oracle, Y[rows], oracle.gemm_f64_rows(X, rows, What), what)
+    return packed, L
+
+
+_PREFILL = [(s, p) for s in inputs.LLAMA2_7B_SHAPES for p in (0.0, 0.5, 1.0)]
+
+
+@pytest.mark.parametrize("shape,p", _PREFILL)
+def test_prefill_workload_cases(gpu, oracle, shape, p):
+    N, K = inputs.LLAMA2_7B_SHAPES[shape]
+    stream = ("prefill", shape, p)
+    W = inputs.weight(N, K, inputs.MASTER_SEED, *stream)
+    flags = inputs.tile_flags(N, K, p, inputs.MASTER_SEED, *stream)
+    for M in (512, 2048, 4096):
+        X = inputs.activation(M, K, inputs.MASTER_SEED, *stream, M)
+        _check_case(gpu, oracle, W, flags, X, f"7b.{shape}.p{p}.M{M}")
+
+
+@pytest.mark.parametrize("shape", list(inputs.LLAMA2_13B_SHAPES))
+def test_13b_workload_cases(gpu, oracle, shape):
+    cases = [c for c in inputs.llama13b_cases() if c["stream"][1] == shape]
+    N, K, p = cases[0]["N"], cases[0]["K"], cases[0]["p"]
+    W = inputs.weight(N, K, inputs.MASTER_SEED, *cases[0]["stream"])
+    flags = inputs.tile_flags(N, K, p, inputs.MASTER_SEED, *cases[0]["stream"])
+    assert 0 < flags.mean() < 1
+    for c in cases:                                   # M in {1, 8, 64, 512, 4096}
+        X = inputs.activation(c["M"], K, inputs.MASTER_SEED, *c["stream"], c["M"])
+        _check_case(gpu, oracle, W, flags, X, c["name"])
+
+
+def test_stack_workload_sample(gpu, oracle):
+    """Four matrices of the 224-matrix stack (per-matrix tile fraction ~ U[0,1]) at M = 1 and M = 2048,
+    with weights drawn on the device as the benchmark does and copied back for the oracle."""
+    torch, B = gpu
+    cases = inputs.stack_cases()
+    for idx in (0, 5, 118, 223):
+        c = cases[idx]
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(inputs.MASTER_SEED * 1000 + idx)
+        Wd = torch.empty((c["N"], c["K"]), dtype=torch.bfloat16, device="cuda").normal_(0.0, 0.02, generator=gen)
+        W = to_bits(Wd)
+        flags = inputs.tile_flags(c["N"], c["K"], c["p"], inputs.MASTER_SEED, *c["stream"])
+        for M in (1, 2048):
+            X = inputs.activation(M, c["K"], inputs.MASTER_SEED, *c["stream"], M)
+            _check_case(gpu, oracle, W, flags, X, f"{c['name']}.M{M}", n_rows=8)
