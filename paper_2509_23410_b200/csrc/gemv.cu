@@ -44,6 +44,84 @@ __device__ __forceinline__ float dot_group(uint32_t v, uint32_t x01, uint32_t x2
     return fmaf(bf_hi(v), bf_hi(xp), acc);
 }
 
+// One tile's worth of this lane's operands: 4 payload rows x one 16-byte chunk per K-half (dense: 8
+// loads, 2:4: 4 loads + 4 metadata half-words), and the matching activations.
+template <int M_MAX>
+struct TileRegs {
+    uint4 w[8];
+    uint32_t code[4];
+    uint4 x[2][M_MAX];     // dense: columns 64h + 8c .. +8 for h = 0, 1; 2:4: columns 16c .. 16c+15 as two vectors
+    uint32_t kind;
+};
+
+template <int M_MAX>
+__device__ __forceinline__ void load_tile(TileRegs<M_MAX>& t, const TileDesc& d, const uint8_t* __restrict__ blob,
+                                          const __nv_bfloat16* __restrict__ X, int64_t ldx, int M, int tk,
+                                          uint32_t row0, uint32_t c) {
+    const uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    t.kind = d.kind;
+    if (d.kind == PATCH_TILE_DENSE) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int p = 0; p < 4; ++p)
+                t.w[4 * h + p] = ldg_stream(pay + h * kAtomBytes + atom_chunk_offset(row0 + 32u * p, c));
+#pragma unroll
+            for (int m = 0; m < M_MAX; ++m)
+                t.x[h][m] = m < M ? __ldg(reinterpret_cast<const uint4*>(X + int64_t(m) * ldx + int64_t(tk) * kTile + 64 * h + 8 * c))
+                                  : zero4;
+        }
+    } else {
+        const uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const uint32_t r = row0 + 32u * p;
+            t.w[p] = ldg_stream(pay + atom_chunk_offset(r, c));
+            // metadata row L = 16q + 8h + i, word j; chunk c covers columns [16c, 16c+16): j = c/2, h = c%2
+            const uint32_t L = (r & ~15u) + 8u * (c & 1u) + (r & 7u);
+            t.code[p] = __ldg(reinterpret_cast<const uint16_t*>(meta + L * 16 + (c >> 1) * 4 + ((r >> 3) & 1u) * 2));
+        }
+#pragma unroll
+        for (int m = 0; m < M_MAX; ++m) {
+            const uint4* px = reinterpret_cast<const uint4*>(X + int64_t(m) * ldx + int64_t(tk) * kTile + 16 * c);
+            t.x[0][m] = m < M ? __ldg(px) : zero4;
+            t.x[1][m] = m < M ? __ldg(px + 1) : zero4;
+        }
+    }
+}
+
+template <int M_MAX>
+__device__ __forceinline__ void fma_tile(const TileRegs<M_MAX>& t, float (&acc)[4][M_MAX]) {
+    if (t.kind == PATCH_TILE_DENSE) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int p = 0; p < 4; ++p)
+#pragma unroll
+                for (int m = 0; m < M_MAX; ++m) acc[p][m] = dot8(t.w[4 * h + p], t.x[h][m], acc[p][m]);
+    } else {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            uint32_t sel[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const uint32_t nib = (t.code[p] >> (4 * g)) & 0xFu, i0 = nib & 3u, i1 = nib >> 2;
+                sel[g] = (i0 * 0x22u + 0x10u) | ((i1 * 0x22u + 0x10u) << 8);
+            }
+#pragma unroll
+            for (int m = 0; m < M_MAX; ++m) {
+                float a = acc[p][m];
+                a = dot_group(t.w[p].x, t.x[0][m].x, t.x[0][m].y, sel[0], a);
+                a = dot_group(t.w[p].y, t.x[0][m].z, t.x[0][m].w, sel[1], a);
+                a = dot_group(t.w[p].z, t.x[1][m].x, t.x[1][m].y, sel[2], a);
+                a = dot_group(t.w[p].w, t.x[1][m].z, t.x[1][m].w, sel[3], a);
+                acc[p][m] = a;
+            }
+        }
+    }
+}
+
 template <int M_MAX>
 __global__ void __launch_bounds__(256)
 gemv_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int M,
@@ -61,6 +139,7 @@ gemv_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int M,
     const uint32_t row0 = 4u * warp + (lane >> 3);
 
     __shared__ float part[M_MAX][kTile];     // this CTA's K-slice partial sums
+    __shared__ TileDesc descs[256];          // tile descriptors of the slice, staged 256 at a time
 
     float acc[4][M_MAX];
 #pragma unroll
@@ -69,65 +148,18 @@ gemv_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int M,
         for (int m = 0; m < M_MAX; ++m) acc[p][m] = 0.f;
 
     const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off) + int64_t(tn) * TK;
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-
-    for (int tk = tk0; tk < tk1; ++tk) {
-        const TileDesc d = table[tk];
-        const uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
-        if (d.kind == PATCH_TILE_DENSE) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint4 w[4];
-#pragma unroll
-                for (int p = 0; p < 4; ++p)
-                    w[p] = ldg_stream(pay + h * kAtomBytes + atom_chunk_offset(row0 + 32u * p, c));
-                uint4 x[M_MAX];
-#pragma unroll
-                for (int m = 0; m < M_MAX; ++m)
-                    x[m] = m < M ? __ldg(reinterpret_cast<const uint4*>(X + int64_t(m) * ldx + int64_t(tk) * kTile + 64 * h + 8 * c))
-                                 : zero4;
-#pragma unroll
-                for (int p = 0; p < 4; ++p)
-#pragma unroll
-                    for (int m = 0; m < M_MAX; ++m) acc[p][m] = dot8(w[p], x[m], acc[p][m]);
-            }
-        } else {
-            const uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
-            uint4 w[4];
-            uint32_t code[4];
-#pragma unroll
-            for (int p = 0; p < 4; ++p) {
-                const uint32_t r = row0 + 32u * p;
-                w[p] = ldg_stream(pay + atom_chunk_offset(r, c));
-                // metadata row L = 16q + 8h + i, word j; chunk c covers columns [16c, 16c+16): j = c/2, h = c%2
-                const uint32_t L = (r & ~15u) + 8u * (c & 1u) + (r & 7u);
-                code[p] = __ldg(reinterpret_cast<const uint16_t*>(meta + L * 16 + (c >> 1) * 4 + ((r >> 3) & 1u) * 2));
-            }
-            uint4 xa[M_MAX], xb[M_MAX];   // 16 activations per token: columns 16c .. 16c+15
-#pragma unroll
-            for (int m = 0; m < M_MAX; ++m) {
-                const uint4* px = reinterpret_cast<const uint4*>(X + int64_t(m) * ldx + int64_t(tk) * kTile + 16 * c);
-                xa[m] = m < M ? __ldg(px) : zero4;
-                xb[m] = m < M ? __ldg(px + 1) : zero4;
-            }
-#pragma unroll
-            for (int p = 0; p < 4; ++p) {
-                uint32_t sel[4];
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const uint32_t nib = (code[p] >> (4 * g)) & 0xFu, i0 = nib & 3u, i1 = nib >> 2;
-                    sel[g] = (i0 * 0x22u + 0x10u) | ((i1 * 0x22u + 0x10u) << 8);
-                }
-#pragma unroll
-                for (int m = 0; m < M_MAX; ++m) {
-                    float a = acc[p][m];
-                    a = dot_group(w[p].x, xa[m].x, xa[m].y, sel[0], a);
-                    a = dot_group(w[p].y, xa[m].z, xa[m].w, sel[1], a);
-                    a = dot_group(w[p].z, xb[m].x, xb[m].y, sel[2], a);
-                    a = dot_group(w[p].w, xb[m].z, xb[m].w, sel[3], a);
-                    acc[p][m] = a;
-                }
-            }
+    // Register double buffer: the loads of tile i+1 are in flight while tile i is multiplied.
+    TileRegs<M_MAX> cur, nxt;
+    for (int base = tk0; base < tk1; base += 256) {
+        const int n = tk1 - base < 256 ? tk1 - base : 256;
+        __syncthreads();
+        if (int(threadIdx.x) < n) descs[threadIdx.x] = table[base + threadIdx.x];
+        __syncthreads();
+        load_tile<M_MAX>(cur, descs[0], blob, X, ldx, M, base, row0, c);
+        for (int i = 0; i < n; ++i) {
+            if (i + 1 < n) load_tile<M_MAX>(nxt, descs[i + 1], blob, X, ldx, M, base + i + 1, row0, c);
+            fma_tile<M_MAX>(cur, acc);
+            if (i + 1 < n) cur = nxt;
         }
     }
 
