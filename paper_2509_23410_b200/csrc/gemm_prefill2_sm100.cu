@@ -98,9 +98,14 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             const bool has1 = tn0 + 1 < TN;
             // lanes 0..15 hold the next 16 descriptors of row-block tn0, lanes 16..31 those of tn0+1
             const TileDesc* table = table0 + int64_t(tn0 + (lane >> 4 && has1 ? 1 : 0)) * TK;
-            TileDesc mine = TileDesc{0, 0, 0, 0};
+            // fetched one batch of 16 ahead, so that the table read is never waited for inside the K loop
+            TileDesc mine = TileDesc{0, 0, 0, 0}, next = TileDesc{0, 0, 0, 0};
+            if ((lane & 15) < TK) next = table[lane & 15];
             for (int k = 0; k < TK && ok; ++k) {
-                if ((k & 15) == 0 && k + (lane & 15) < TK) mine = table[k + (lane & 15)];
+                if ((k & 15) == 0) {
+                    mine = next;
+                    if (k + 16 + (lane & 15) < TK) next = table[k + 16 + (lane & 15)];
+                }
                 uint32_t kind[2], off16[2];
                 kind[0] = __shfl_sync(0xFFFFFFFFu, mine.kind, k & 15);
                 off16[0] = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, k & 15);

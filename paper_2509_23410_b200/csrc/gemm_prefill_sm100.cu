@@ -19,6 +19,7 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports
 // PATCH_ERR_TIMEOUT through status_dev, drains its copies in flight, frees TMEM and returns.
+#include <cstdlib>
 #include "sm100_ptx.cuh"
 
 namespace patch {
@@ -227,27 +228,39 @@ static int sm_count_prefill() {
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
                     int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
 
+// Testing / tuning aid: PATCH_PREFILL_SCHEDULE=1|2 in the environment pins the schedule (one or two
+// row-blocks per CTA); anything else lets the cost model choose.
+static int forced_schedule() {
+    static int v = [] {
+        const char* e = getenv("PATCH_PREFILL_SCHEDULE");
+        return (e && e[0] >= '1' && e[0] <= '2' && e[1] == 0) ? e[0] - '0' : 0;
+    }();
+    return v;
+}
+
 // Schedule choice: token-tile width n (a multiple of 16 in [128, 240]) and one or two row-blocks
 // per CTA, by a small cost model -- waves of output tiles over the SMs times the time of one tile,
 // which is the slower of the tensor pipe (0.55 us per 128 x 128 x 256 step at full clocks) and
 // what one SM pulls from L2 (measured: ~105 GB/s with two whole-tile stages, ~120 GB/s with the
 // two-ring pipeline), plus a per-tile prologue/epilogue cost.
-struct PrefillPlan { int n_tok; bool two_row_blocks; };
+struct PrefillPlan { int n_tok; int schedule; };   // schedule: row-blocks per CTA (1 or 2)
 
 static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms) {
-    PrefillPlan best = {240, false};
+    PrefillPlan best = {240, 1};
     double best_cost = 1e300;
     const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : 240, n_lo = M <= 128 ? n_hi : 128;
+    const int forced = forced_schedule();
     for (int n = n_hi; n >= n_lo; n -= 16) {
         const int64_t MT = (M + n - 1) / n;
-        for (int two = 0; two < 2; ++two) {
-            const int64_t tiles = int64_t(two ? (TN + 1) / 2 : TN) * MT;
+        for (int sched = 1; sched <= 2; ++sched) {
+            if (forced && sched != forced) continue;
+            const int64_t tiles = int64_t(sched == 1 ? TN : (TN + 1) / 2) * MT;
             const int64_t waves = (tiles + sms - 1) / sms;
-            const double mma_ns = (two ? 1100.0 : 550.0) * n / 256.0;
-            const double load_ns = two ? (65536.0 + n * 256.0) / 120.0 : (32768.0 + n * 256.0) / 105.0;
-            const double tile_ns = TK * (mma_ns > load_ns ? mma_ns : load_ns) + (two ? 10000.0 : 6000.0);
+            const double mma_ns = (sched == 1 ? 550.0 : 1100.0) * n / 256.0;
+            const double load_ns = sched == 1 ? (32768.0 + n * 256.0) / 105.0 : (65536.0 + n * 256.0) / 120.0;
+            const double tile_ns = TK * (mma_ns > load_ns ? mma_ns : load_ns) + (sched == 1 ? 6000.0 : 10000.0);
             const double cost = double(waves) * tile_ns;
-            if (cost < best_cost) { best_cost = cost; best = {n, two != 0}; }
+            if (cost < best_cost) { best_cost = cost; best = {n, sched}; }
         }
     }
     return best;
@@ -264,7 +277,7 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
-    if (plan.two_row_blocks) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream);
+    if (plan.schedule == 2) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream);
     static bool configured = false;   // per-process attribute, idempotent
     if (!configured) {
         if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
