@@ -25,23 +25,25 @@
 namespace patch {
 
 constexpr int kPrefillMaxTok = 240;      // two accumulators + metadata must fit 512 TMEM columns
-constexpr int kPrefillStages = 2;
 
+// A stage holds a whole weight tile (32 KB reserved) and the n_tok x 128 activation tile; the ring
+// takes as many stages as fit: 2 at n_tok = 240 (92 KB each), 3 up to n_tok = 160, 4 at n_tok <= 80.
 struct PrefillConfig {
-    static constexpr uint32_t kXBytesMax = kPrefillMaxTok * 256;   // n_tok rows x 128 columns of K
-    static constexpr uint32_t kStageBytes = kDenseBytes + kXBytesMax;
-    static constexpr uint32_t kBarrierOffset = kPrefillStages * kStageBytes;
+    static constexpr uint32_t kRingBytes = 216 * 1024;
+    static constexpr int kMaxStages = 8;
+    static constexpr uint32_t kBarrierOffset = kRingBytes;
     static constexpr uint32_t kStageOffset = kBarrierOffset + 256;       // 4 epilogue warps x 1 KB transpose staging
     static constexpr uint32_t kSmemBytes = kStageOffset + 4 * 1024 + 1024;   // + alignment slack
     static constexpr uint32_t kTmemCols = 512;
-    static constexpr uint32_t kAcc1Col = 256, kMetaCol = 240;      // acc0 [0,240) meta [240,248) acc1 [256,496)
+    static constexpr uint32_t kAcc1Col = 256, kMetaCol = 240;      // acc0 [0,240) acc1 [256,496); metadata, 4 columns per stage: [240,256) then [496,512)
 };
 
 __global__ void __launch_bounds__(192)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
     using Cfg = PrefillConfig;
-    constexpr int STAGES = kPrefillStages;
+    const uint32_t stage_bytes = kDenseBytes + uint32_t(n_tok) * 256u;
+    const int STAGES = int(Cfg::kRingBytes / stage_bytes) < Cfg::kMaxStages ? int(Cfg::kRingBytes / stage_bytes) : Cfg::kMaxStages;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -52,7 +54,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
     const uint32_t bar_acc_empty = bar_acc_full + 16;             // 2 x 8 B
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Cfg::kBarrierOffset + 160);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile uint32_t* stage_kind = reinterpret_cast<volatile uint32_t*>(tmem_slot + 2);  // STAGES words
+    volatile uint32_t* stage_kind = reinterpret_cast<volatile uint32_t*>(tmem_slot + 2);  // kMaxStages words
 
     grid_launch_dependents();
     grid_dependency_wait();     // X, the packed weight and Y may belong to the previous kernel until here
@@ -102,7 +104,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
                     ok = mbar_wait(bar_empty + 8 * stage, (uint32_t(issued / STAGES) & 1u) ^ 1u, abort_flag, status_dev);
                     if (ok) {
                         const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
-                        const uint32_t sW = smem_base + stage * Cfg::kStageBytes, sX = sW + kDenseBytes;
+                        const uint32_t sW = smem_base + stage * stage_bytes, sX = sW + kDenseBytes;
                         const uint32_t full = bar_full + 8 * stage;
                         stage_kind[stage] = kind;
                         mbar_expect_tx(full, wbytes + 2 * x_atom_bytes);
@@ -138,9 +140,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
                     if (!ok) break;
                     if (step == 0) PATCH_TRACE_AT(2);
                     tc_fence_after();
-                    const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
+                    const uint32_t sW = smem_base + stage * stage_bytes;
                     issue_tile_mma_n(stage_kind[stage], sW, sW + kDenseBytes, x_atom_bytes, acc,
-                                     tmem_base + Cfg::kMetaCol + 4 * stage, i == 0, uint32_t(n_tok));
+                                     tmem_base + (stage < 4 ? Cfg::kMetaCol + 4 * stage : 496 + 4 * (stage - 4)), i == 0, uint32_t(n_tok));
                     mma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
                 }
                 if (ok) mma_commit(bar_acc_full + 8 * (j & 1));      // accumulator complete
@@ -241,8 +243,9 @@ static int forced_schedule() {
 // Schedule choice: token-tile width n (a multiple of 16 in [128, 240]) and one or two row-blocks
 // per CTA, by a small cost model -- waves of output tiles over the SMs times the time of one tile,
 // which is the slower of the tensor pipe (0.55 us per 128 x 128 x 256 step at full clocks) and
-// what one SM pulls from L2 (measured: ~105 GB/s with two whole-tile stages, ~120 GB/s with the
-// two-ring pipeline), plus a per-tile prologue/epilogue cost.
+// what one SM pulls from L2 (measured: a step's copies land ~1.75 us after they are issued, so
+// the one-row-block ring sustains one step per 1.75 us / stages; ~120 GB/s with the two-ring
+// pipeline), plus a per-tile prologue/epilogue cost.
 struct PrefillPlan { int n_tok; int schedule; };   // schedule: row-blocks per CTA (1 or 2)
 
 static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms) {
@@ -257,9 +260,16 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms) {
             const int64_t tiles = int64_t(sched == 1 ? TN : (TN + 1) / 2) * MT;
             const int64_t waves = (tiles + sms - 1) / sms;
             const double mma_ns = (sched == 1 ? 550.0 : 1100.0) * n / 256.0;
-            const double load_ns = sched == 1 ? (32768.0 + n * 256.0) / 105.0 : (65536.0 + n * 256.0) / 120.0;
+            // one row-block: the ring holds `stages` whole steps and a step's copies take ~1.75 us to land
+            const double stage_bytes = 32768.0 + n * 256.0;
+            const int stages = int(PrefillConfig::kRingBytes / stage_bytes) < PrefillConfig::kMaxStages
+                                   ? int(PrefillConfig::kRingBytes / stage_bytes) : PrefillConfig::kMaxStages;
+            const double load1_ns = 1750.0 / stages > stage_bytes / 150.0 ? 1750.0 / stages : stage_bytes / 150.0;
+            // two row-blocks: the rings hold ~1.5 steps, which bounds a step at ~1.2 us whatever its size
+            const double load2_ns = (65536.0 + n * 256.0) / 120.0 > 1200.0 ? (65536.0 + n * 256.0) / 120.0 : 1200.0;
+            const double load_ns = sched == 1 ? load1_ns : load2_ns;
             const double tile_ns = TK * (mma_ns > load_ns ? mma_ns : load_ns) + (sched == 1 ? 6000.0 : 10000.0);
-            const double cost = double(waves) * tile_ns;
+            const double cost = double(waves) * tile_ns + n;      // at equal time, the narrower tile (less padding)
             if (cost < best_cost) { best_cost = cost; best = {n, sched}; }
         }
     }
