@@ -57,6 +57,9 @@ def workload_cases(name: str, stack_m: int = 1):
     if name == "stack":
         # 32 blocks x (q,k,v,o,gate,up,down) = 224 matrices, per-matrix 2:4-tile fraction ~ U[0,1]
         return [dict(c, M=stack_m) for c in inputs.stack_cases()]
+    if name == "stack-fused":
+        # the same weights with q/k/v and gate/up stored as one matrix each: 128 GEMMs
+        return [dict(c, M=stack_m) for c in inputs.stack_fused_cases()]
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -229,14 +232,14 @@ def run_ours(args):
         key = (c["N"], c["K"], c["stream"])
         if key in mats:
             continue
-        if args.workload == "stack":
+        if args.workload.startswith("stack"):
             # 6.5 G weights: drawn on the device (torch Philox, seeded per matrix) instead of on the host
             gen = torch.Generator(device=dev)
             gen.manual_seed(inputs.MASTER_SEED * 1000 + len(mats))
             W = torch.empty((c["N"], c["K"]), dtype=torch.bfloat16, device=dev).normal_(0.0, 0.02, generator=gen)
         else:
             W = to_dev(inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]))
-        flags = inputs.tile_flags(c["N"], c["K"], c["p"], inputs.MASTER_SEED, *c["stream"])
+        flags = inputs.case_flags(c)
         layout = B.patch_packed_size(c["N"], c["K"], flags)
         packed = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
         B.patch_pack(W, flags, layout=layout, out=packed)          # warm
@@ -252,7 +255,7 @@ def run_ours(args):
     jobs, stack_x, shared_ws = [], {}, {}
     for c in cases:
         layout, packed = mats[(c["N"], c["K"], c["stream"])]
-        xkey = (c["M"], c["K"]) if args.workload == "stack" else None
+        xkey = (c["M"], c["K"]) if args.workload.startswith("stack") else None
         if xkey is not None and xkey in stack_x:
             X = stack_x[xkey]                # the stack shares one activation per (M, K); outputs are not chained
         else:
@@ -438,6 +441,7 @@ def run_ours(args):
 
 def workload_label(args):
     return {"13b": "llama2-13b linears", "stack": f"llama2-7b full linear stack, M={args.stack_m}",
+            "stack-fused": f"llama2-7b full linear stack with q/k/v and gate/up stacked, M={args.stack_m}",
             "single": "single 1024x1024 GEMM"}.get(args.workload, f"llama2-7b {args.workload} linears")
 
 
@@ -462,7 +466,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused"])
     ap.add_argument("--stack-m", type=int, default=1, help="tokens per GEMM of the 224-GEMM stack workload")
     ap.add_argument("--launch", default="independent", choices=["dependent", "independent"],
                     help="independent (default; true for this workload, whose GEMMs do not feed each other): "

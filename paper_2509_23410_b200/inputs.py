@@ -157,11 +157,35 @@ def stack_cases(seed: int = MASTER_SEED, n_blocks: int = 32):
     return out
 
 
+def stack_fused_cases(seed: int = MASTER_SEED, n_blocks: int = 32):
+    """The same stack with the linears that share an input stored as one matrix each: q/k/v stacked along N
+    (12288 x 4096) and gate/up stacked (22016 x 4096); 4 GEMMs per block instead of 7.  Every part keeps
+    the 2:4-tile fraction and the flag stream of its own matrix in ``stack_cases``."""
+    groups = [("qkv", ("q", "k", "v")), ("o", ("o",)), ("gate_up", ("gate", "up")), ("down", ("down",))]
+    shapes = {role: (N, K) for role, N, K in LLAMA2_7B_BLOCK}
+    out = []
+    for b in range(n_blocks):
+        for name, roles in groups:
+            K = shapes[roles[0]][1]
+            parts = [dict(N=shapes[r][0], p=fraction(0.0, 1.0, seed, "stack", b, r), stream=("stack", b, r)) for r in roles]
+            N = sum(q["N"] for q in parts)
+            p = sum(q["p"] * q["N"] for q in parts) / N
+            out.append(dict(name=f"stack.{b}.{name}", N=N, K=K, p=p, stream=("stack", b, name), parts=parts))
+    return out
+
+
+def case_flags(case: dict, seed: int = MASTER_SEED) -> np.ndarray:
+    """Tile flags of a case; a case made of stacked matrices concatenates its parts' flags along N."""
+    if "parts" in case:
+        return np.concatenate([tile_flags(q["N"], case["K"], q["p"], seed, *q["stream"]) for q in case["parts"]], axis=0)
+    return tile_flags(case["N"], case["K"], case["p"], seed, *case["stream"])
+
+
 def make_case_inputs(case: dict, seed: int = MASTER_SEED, M: int | None = None):
     """(W bits [N x K], flags [TN x TK], X bits [M x K]) for a case dict from the lists above."""
     N, K = case["N"], case["K"]
     M = case.get("M") if M is None else M
     W = weight(N, K, seed, *case["stream"])
-    flags = tile_flags(N, K, case["p"], seed, *case["stream"])
+    flags = case_flags(case, seed)
     X = activation(M, K, seed, *case["stream"], M)
     return W, flags, X

@@ -93,3 +93,16 @@ def test_product_package_does_not_import_the_oracle():
                 text = open(os.path.join(dirpath, fn)).read()
                 assert "import oracle" not in text and "from oracle" not in text, fn
                 assert "patch_oracle" not in text, fn
+
+
+def test_stacked_case_flags_concatenate_parts():
+    """Input recipe of the stacked-matrix workload: flags of q/k/v (gate/up) stacked along N."""
+    import numpy as np
+    from paper_2509_23410_b200 import inputs
+    plain = {c["name"]: c for c in inputs.stack_cases(n_blocks=1)}
+    fused = inputs.stack_fused_cases(n_blocks=1)
+    assert [c["N"] for c in fused] == [12288, 4096, 22016, 4096] and len(fused) == 4
+    qkv = inputs.case_flags(fused[0])
+    parts = [inputs.tile_flags(4096, 4096, plain[f"stack.0.{r}"]["p"], inputs.MASTER_SEED, "stack", 0, r) for r in "qkv"]
+    assert np.array_equal(qkv, np.concatenate(parts, axis=0))
+    assert abs(fused[0]["p"] - sum(plain[f"stack.0.{r}"]["p"] for r in "qkv") / 3) < 1e-12

@@ -354,3 +354,26 @@ def test_stack_workload_sample(gpu, oracle):
         for M in (1, 2048):
             X = inputs.activation(M, c["K"], inputs.MASTER_SEED, *c["stream"], M)
             _check_case(gpu, oracle, W, flags, X, f"{c['name']}.M{M}", n_rows=8)
+
+
+def test_stacked_matrices_sample(gpu, oracle):
+    """q/k/v and gate/up stored as one matrix each (N = 12288, 22016): the stacked flags are the parts'
+    flags, and the GEMM over the stacked weight is checked at M = 1 (whole output) and M = 2048 (sampled rows)."""
+    torch, B = gpu
+    cases = inputs.stack_fused_cases(n_blocks=2)
+    for idx in (0, 6):                                  # block 0 qkv, block 1 gate_up
+        c = cases[idx]
+        flags = inputs.case_flags(c)
+        assert flags.shape == (c["N"] // 128, c["K"] // 128)
+        row = 0
+        for part in c["parts"]:                         # every part keeps its own matrix's flags
+            ref = inputs.tile_flags(part["N"], c["K"], part["p"], inputs.MASTER_SEED, *part["stream"])
+            assert np.array_equal(flags[row:row + part["N"] // 128], ref)
+            row += part["N"] // 128
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(inputs.MASTER_SEED * 1000 + idx)
+        Wd = torch.empty((c["N"], c["K"]), dtype=torch.bfloat16, device="cuda").normal_(0.0, 0.02, generator=gen)
+        W = to_bits(Wd)
+        for M in (1, 2048):
+            X = inputs.activation(M, c["K"], inputs.MASTER_SEED, *c["stream"], M)
+            _check_case(gpu, oracle, W, flags, X, f"{c['name']}.M{M}", n_rows=8)
