@@ -113,8 +113,10 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long
 
 // Every contributor of a row-block finishes rows [r0, r1) of it: thread `et` (0..127) takes
 // (row, 16-token chunk) items, sums the n_contrib partial tiles in ascending K order and writes bf16.
+// Each partial word is read by exactly one thread, which stores zero back: the workspace is left as
+// the next call (of any M, whose flagged words share this memory) expects it.
 template <int N_TOK>
-__device__ __forceinline__ void reduce_row_share(const float* __restrict__ partials, int first_slot, int n_contrib,
+__device__ __forceinline__ void reduce_row_share(float* __restrict__ partials, int first_slot, int n_contrib,
                                                  int r0, int r1, int M, __nv_bfloat16* ytile, int64_t ldy, int et) {
     constexpr int CH = N_TOK / 16;
     const int c_lo = first_slot >> 1;
@@ -140,12 +142,16 @@ __device__ __forceinline__ void reduce_row_share(const float* __restrict__ parti
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
                 if (j0 + jj < n_contrib) {
+                    const int j = j0 + jj;
+                    const int s = j == 0 ? first_slot : 2 * (c_lo + j);
+                    uint4* src = reinterpret_cast<uint4*>(partials + (int64_t(s) * kTile + row) * N_TOK + c0);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         a[4 * i + 0] += __uint_as_float(q[jj][i].x);
                         a[4 * i + 1] += __uint_as_float(q[jj][i].y);
                         a[4 * i + 2] += __uint_as_float(q[jj][i].z);
                         a[4 * i + 3] += __uint_as_float(q[jj][i].w);
+                        __stcg(src + i, make_uint4(0u, 0u, 0u, 0u));
                     }
                 }
             }

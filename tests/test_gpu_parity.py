@@ -377,3 +377,54 @@ def test_stacked_matrices_sample(gpu, oracle):
         for M in (1, 2048):
             X = inputs.activation(M, c["K"], inputs.MASTER_SEED, *c["stream"], M)
             _check_case(gpu, oracle, W, flags, X, f"{c['name']}.M{M}", n_rows=8)
+
+
+def test_workspace_is_shared_across_token_counts(gpu, oracle):
+    """One workspace, zeroed once, serves calls of every M <= 64 in any order: each call leaves it
+    all zero (the 32/64-token schedule's partial sums share memory with the 16-token schedule's flags)."""
+    torch, B = gpu
+    N, K = 1792, 1280
+    W, flags, _ = inputs.make_case_inputs(dict(N=N, K=K, p=0.4, stream=("ws", N, K)), 31, 1)
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    ws = torch.zeros(B.patch_gemm_workspace_size(L, 64), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for M in (48, 8, 64, 16, 33, 1, 17, 5):
+        X = inputs.activation(M, K, 31, "ws", M)
+        for variant in (B.VARIANT_AUTO, B.VARIANT_MMA | B.WEIGHTS_STATIC | B.INPUT_STATIC):
+            Y = B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws, status=status, variant=variant)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            assert int(ws.count_nonzero()) == 0, f"workspace not clean after M={M}"
+            check_parity(oracle, to_bits(Y), oracle.gemm_f64(X, What)[0], f"shared workspace M={M}")
+
+
+def test_random_shapes_and_pitches(gpu, oracle):
+    """Seeded random (N, K, M, tile fraction, row pitches of X and Y): every schedule, ragged token counts,
+    outputs beyond column N untouched."""
+    torch, B = gpu
+    rng = inputs.generator(inputs.MASTER_SEED, "fuzz")
+    Ms = [1, 3, 4, 15, 16, 17, 33, 63, 64, 65, 100, 128, 129, 239, 240, 241, 300]
+    for it in range(24):
+        TN, TK = int(rng.integers(1, 14)), int(rng.integers(1, 14))
+        N, K, M = 128 * TN, 128 * TK, Ms[int(rng.integers(0, len(Ms)))]
+        p = [0.0, 1.0, 0.5, float(rng.random())][int(rng.integers(0, 4))]
+        padx, pady = int(rng.choice([0, 8, 200])), int(rng.choice([0, 8, 200]))
+        W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=p, stream=("fuzz", it)), inputs.MASTER_SEED, M)
+        What = oracle.prune(W, flags)
+        Y32 = oracle.gemm_f64(X, What)[0]
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        Xfull = torch.zeros((M, K + padx), dtype=torch.bfloat16, device="cuda")
+        Xfull[:, :K] = to_dev(torch, X)
+        Yfull = torch.full((M, N + pady), 7.0, dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        variants = [B.VARIANT_AUTO, B.VARIANT_MMA | B.WEIGHTS_STATIC | B.INPUT_STATIC] + ([B.VARIANT_GEMV] if M <= 4 else [])
+        for variant in variants:
+            Yfull.fill_(7.0)
+            B.patch_gemm(Xfull[:, :K], L, packed, Y=Yfull[:, :N], workspace=ws, status=status, variant=variant)
+            torch.cuda.synchronize()
+            what = f"N={N} K={K} M={M} p={p:.2f} pitches +{padx}/+{pady} variant={variant:#x}"
+            assert int(status.item()) == 0, what
+            assert pady == 0 or bool((Yfull[:, N:] == 7.0).all()), what + ": wrote past column N"
+            check_parity(oracle, to_bits(Yfull[:, :N]), Y32, what)
