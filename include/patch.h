@@ -134,7 +134,8 @@ int patch_gemm_workspace_size(const patch_layout_t* layout, int64_t M, size_t* b
 /*
  * Zero a workspace once after allocating it (arrival counters and partial-sum flags must start at
  * zero; every successful patch_gemm leaves them zero again).  Zero it again after a call that
- * reported PATCH_ERR_TIMEOUT.
+ * reported PATCH_ERR_TIMEOUT.  A workspace of patch_gemm_workspace_size(layout, 64) bytes serves
+ * calls of every M in any order, and calls on different layouts with N <= 131072 may share it.
  */
 int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream);
 

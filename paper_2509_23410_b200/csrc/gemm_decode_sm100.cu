@@ -113,10 +113,8 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long
 
 // Every contributor of a row-block finishes rows [r0, r1) of it: thread `et` (0..127) takes
 // (row, 16-token chunk) items, sums the n_contrib partial tiles in ascending K order and writes bf16.
-// Each partial word is read by exactly one thread, which stores zero back: the workspace is left as
-// the next call (of any M, whose flagged words share this memory) expects it.
 template <int N_TOK>
-__device__ __forceinline__ void reduce_row_share(float* __restrict__ partials, int first_slot, int n_contrib,
+__device__ __forceinline__ void reduce_row_share(const float* __restrict__ partials, int first_slot, int n_contrib,
                                                  int r0, int r1, int M, __nv_bfloat16* ytile, int64_t ldy, int et) {
     constexpr int CH = N_TOK / 16;
     const int c_lo = first_slot >> 1;
@@ -142,16 +140,12 @@ __device__ __forceinline__ void reduce_row_share(float* __restrict__ partials, i
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
                 if (j0 + jj < n_contrib) {
-                    const int j = j0 + jj;
-                    const int s = j == 0 ? first_slot : 2 * (c_lo + j);
-                    uint4* src = reinterpret_cast<uint4*>(partials + (int64_t(s) * kTile + row) * N_TOK + c0);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         a[4 * i + 0] += __uint_as_float(q[jj][i].x);
                         a[4 * i + 1] += __uint_as_float(q[jj][i].y);
                         a[4 * i + 2] += __uint_as_float(q[jj][i].z);
                         a[4 * i + 3] += __uint_as_float(q[jj][i].w);
-                        __stcg(src + i, make_uint4(0u, 0u, 0u, 0u));
                     }
                 }
             }
@@ -517,13 +511,21 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
 
 static int decode_n_tok(int64_t M) { return M <= 16 ? 16 : M <= 32 ? 32 : 64; }
 
+// Workspace layout: [arrival counters | flagged partial sums of the 16-token schedule | partial tiles of the
+// 32/64-token schedule].  The flagged words must be zero between calls (the schedule that uses them leaves
+// them so); the partial tiles need not be (they are written before they are read and are never taken for
+// flags), so the two regions are disjoint.  The counter region is 8 KB for every N <= 131072, which makes
+// the offsets the same for all such layouts: one workspace, zeroed once, serves any mix of them and of M.
 static size_t counters_bytes(const patch_layout_t* L) {
-    return (size_t(L->N / kTile) * 8 + 255) / 256 * 256;
+    const size_t need = (size_t(L->N / kTile) * 8 + 255) / 256 * 256;
+    return need > 8192 ? need : 8192;
 }
+constexpr size_t kFlaggedBytes = size_t(2) * kMaxDecodeCtas * 16 * kTile * sizeof(float);
 
 size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M) {
     if (M > 64) return 0;
-    return counters_bytes(L) + size_t(2) * kMaxDecodeCtas * decode_n_tok(M) * kTile * sizeof(float);
+    const int n_tok = decode_n_tok(M);
+    return counters_bytes(L) + kFlaggedBytes + (n_tok > 16 ? size_t(2) * kMaxDecodeCtas * n_tok * kTile * sizeof(float) : 0);
 }
 
 static int sm_count() {
@@ -567,7 +569,7 @@ static int launch_decode_t(const CUtensorMap& map, const patch_layout_t* L, cons
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     unsigned long long* counters = static_cast<unsigned long long*>(workspace);
-    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + counters_bytes(L));
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + counters_bytes(L) + (N_TOK > 16 ? kFlaggedBytes : 0));
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, packed, uint64_t(L->table_off),
                                        uint32_t(L->payload_off / 16), uint32_t(L->payload_bytes / 16), TN, TK, M, Y,
                                        ldy, counters, partials, status_dev);

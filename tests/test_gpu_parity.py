@@ -379,24 +379,28 @@ def test_stacked_matrices_sample(gpu, oracle):
             _check_case(gpu, oracle, W, flags, X, f"{c['name']}.M{M}", n_rows=8)
 
 
-def test_workspace_is_shared_across_token_counts(gpu, oracle):
-    """One workspace, zeroed once, serves calls of every M <= 64 in any order: each call leaves it
-    all zero (the 32/64-token schedule's partial sums share memory with the 16-token schedule's flags)."""
+def test_workspace_is_shared_across_token_counts_and_layouts(gpu, oracle):
+    """One workspace, zeroed once, serves calls of every M <= 64 on two layouts of different N in any
+    order: the 32/64-token schedule's partial tiles never reach the 16-token schedule's flag words."""
     torch, B = gpu
-    N, K = 1792, 1280
-    W, flags, _ = inputs.make_case_inputs(dict(N=N, K=K, p=0.4, stream=("ws", N, K)), 31, 1)
-    What = oracle.prune(W, flags)
-    packed, L = B.patch_pack(to_dev(torch, W), flags)
-    ws = torch.zeros(B.patch_gemm_workspace_size(L, 64), dtype=torch.uint8, device="cuda")
+    mats = []
+    for N, K in ((1792, 1280), (4224, 768)):
+        W, flags, _ = inputs.make_case_inputs(dict(N=N, K=K, p=0.4, stream=("ws", N, K)), 31, 1)
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        mats.append((N, K, oracle.prune(W, flags), packed, L))
+    ws = torch.zeros(max(B.patch_gemm_workspace_size(m[4], 64) for m in mats), dtype=torch.uint8, device="cuda")
+    flagged_end = B.patch_gemm_workspace_size(mats[0][4], 16)     # counters + flag words: same offsets for both
+    assert flagged_end == B.patch_gemm_workspace_size(mats[1][4], 16)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    for M in (48, 8, 64, 16, 33, 1, 17, 5):
-        X = inputs.activation(M, K, 31, "ws", M)
+    for i, M in enumerate((48, 8, 64, 16, 33, 1, 17, 5, 64, 2)):
+        N, K, What, packed, L = mats[i % 2]
+        X = inputs.activation(M, K, 31, "ws", M, i)
         for variant in (B.VARIANT_AUTO, B.VARIANT_MMA | B.WEIGHTS_STATIC | B.INPUT_STATIC):
             Y = B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws, status=status, variant=variant)
             torch.cuda.synchronize()
             assert int(status.item()) == 0
-            assert int(ws.count_nonzero()) == 0, f"workspace not clean after M={M}"
-            check_parity(oracle, to_bits(Y), oracle.gemm_f64(X, What)[0], f"shared workspace M={M}")
+            assert int(ws[:flagged_end].count_nonzero()) == 0, f"counters / flag words not clean after M={M}"
+            check_parity(oracle, to_bits(Y), oracle.gemm_f64(X, What)[0], f"shared workspace N={N} M={M}")
 
 
 def test_random_shapes_and_pitches(gpu, oracle):
