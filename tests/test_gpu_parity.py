@@ -78,6 +78,27 @@ def test_pack_bit_exact(gpu, oracle, N, K, p):
     assert torch.equal(packed, packed2)
 
 
+@pytest.mark.parametrize("few_values", [False, True])
+def test_pack_arbitrary_bit_patterns(gpu, oracle, few_values):
+    """The kept pair is decided on the integer key bits & 0x7FFF with ties to the lower index, whatever the
+    bits mean: arbitrary 16-bit patterns (NaN, Inf, +-0, subnormals), and a handful of values so that most
+    groups tie."""
+    torch, B = gpu
+    N, K = 512, 640
+    rng = inputs.generator(inputs.MASTER_SEED, "bits", few_values)
+    if few_values:
+        pool = np.array([0x0000, 0x8000, 0x3C00, 0xBC00, 0x3C01, 0x7F80, 0xFF80, 0x7FC1, 0x0001, 0x8001], np.uint16)
+        W = pool[rng.integers(0, len(pool), (N, K))]
+    else:
+        W = rng.integers(0, 65536, (N, K)).astype(np.uint16)
+    flags = inputs.tile_flags(N, K, 0.7, inputs.MASTER_SEED, "bits", few_values)
+    image = oracle.device_image(oracle.pack(W, flags)[0])
+    Wd = torch.from_numpy(W.view(np.int16)).cuda().view(torch.bfloat16)
+    packed, L = B.patch_pack(Wd, flags)
+    assert (packed.cpu().numpy() == image).all()
+    assert (to_bits(B.patch_unpack(L, packed)) == oracle.prune(W, flags)).all()
+
+
 def test_pack_with_row_pitch(gpu, oracle):
     torch, B = gpu
     N, K, ld = 256, 256, 320
