@@ -290,18 +290,20 @@ def test_prefill_shapes_sampled(gpu, oracle, N, K, M, p):
     assert (f32(Y2) == 2.0 * f32(Y)).all()
 
 
-def test_back_to_back_launches_are_ordered(gpu, oracle):
+@pytest.mark.parametrize("M", [16, 48, 96, 300])
+def test_back_to_back_launches_are_ordered(gpu, oracle, M):
     """A chain of dependent GEMMs on one stream (each launched with programmatic dependent
-    launch): Y of one call is X of the next, so early starts must still see finished inputs."""
+    launch): Y of one call is X of the next, so early starts must still see finished inputs.
+    M = 16 / 48: the two small-M schedules; 96 / 300: the one- and two-row-block prefill kernels."""
     torch, B = gpu
     N = K = 512
-    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=0.5, stream=("chain",)), 25, 16)
+    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=0.5, stream=("chain",)), 25, M)
     W = inputs.f32_to_bf16_bits(f32(W) * 2.0)      # keep magnitudes from collapsing along the chain
     What = oracle.prune(W, flags)
     packed, L = B.patch_pack(to_dev(torch, W), flags)
     torch.cuda.synchronize()
-    bufs = [to_dev(torch, X)] + [torch.empty((16, N), dtype=torch.bfloat16, device="cuda") for _ in range(6)]
-    ws = torch.zeros(B.patch_gemm_workspace_size(L, 16), dtype=torch.uint8, device="cuda")
+    bufs = [to_dev(torch, X)] + [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(6)]
+    ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
     for i in range(6):
         B.patch_gemm(bufs[i], L, packed, Y=bufs[i + 1], workspace=ws, variant=B.VARIANT_MMA | B.WEIGHTS_STATIC)
     torch.cuda.synchronize()
