@@ -165,6 +165,23 @@ def gemm_f64_rows(X, rows, What) -> np.ndarray:
     return Y32
 
 
+def swiglu(Y_gu, block: int = 128) -> np.ndarray:
+    """Gated product of the MLP's gate and up projections (the "up, gate and down matrices of the MLP"
+    of the paper's per-layer allocation study; in the LLaMA models it measures, the MLP is
+    down(silu(gate x) * up x)), for a weight that stacks the two matrices with their row-blocks
+    interleaved: columns [2*block*j, 2*block*j + block) of ``Y_gu`` are gate outputs, the next
+    ``block`` columns the matching up outputs.  out[m, block*j + r] = silu(g) * u with
+    silu(x) = x / (1 + exp(-x)), evaluated in double on the GEMM result, returned as fp32."""
+    Y = np.asarray(Y_gu)
+    M, N = Y.shape
+    assert N % (2 * block) == 0
+    y = Y.astype(np.float64).reshape(M, N // (2 * block), 2, block)
+    g, u = y[:, :, 0, :], y[:, :, 1, :]
+    with np.errstate(over="ignore"):
+        out = g / (1.0 + np.exp(-g)) * u
+    return out.reshape(M, N // 2).astype(np.float32)
+
+
 def parity_metrics(Y_test_f32, Y_ref_f32):
     """relF = |dY|_F / |Yref|_F and max|dY| / max|Yref| (the two tolerances of the benchmark spec)."""
     d = Y_test_f32.astype(np.float64) - Y_ref_f32.astype(np.float64)

@@ -373,3 +373,36 @@ def test_rejects_bad_arguments(oracle):
         oracle.packed_size(100, 128, np.zeros(1, np.uint8))
     with pytest.raises(ValueError):
         oracle.packed_size(128, 128, np.zeros(1, np.uint8), 128, 6)
+
+
+def test_swiglu_against_library_sigmoid_and_closed_forms(oracle):
+    """silu(x) u with x sigmoid(x) from scipy (a different evaluation), the odd-part identity
+    silu(x) - silu(-x) = x, a value with a closed form, and the gate/up pairing of the interleaved layout."""
+    from scipy.special import expit
+    rng = np.random.default_rng(7)
+    M, blocks, b = 5, 3, 128
+    Y = (rng.standard_normal((M, 2 * b * blocks)) * 4).astype(np.float32)
+    Y[0, 0], Y[0, b] = np.float32(np.log(3.0)), np.float32(2.0)       # silu(ln 3) = 0.75 ln 3
+    Y[1, 1], Y[1, b + 1] = np.float32(0.0), np.float32(123.0)          # silu(0) = 0
+    Y[2, 2], Y[2, b + 2] = np.float32(-200.0), np.float32(1.0)         # exp overflows: the limit is -0
+    out = oracle.swiglu(Y)
+    assert out.shape == (M, b * blocks) and out.dtype == np.float32
+    y = Y.astype(np.float64).reshape(M, blocks, 2, b)
+    ref = (y[:, :, 0] * expit(y[:, :, 0]) * y[:, :, 1]).reshape(M, b * blocks)
+    assert np.allclose(out, ref, rtol=1e-6, atol=1e-30)
+    assert abs(out[0, 0] - 0.75 * np.log(3.0) * 2.0) < 1e-6
+    assert out[1, 1] == 0.0 and out[2, 2] == 0.0
+    # pairing: column block j of the output takes gate block 2j and up block 2j + 1, element by element
+    G = np.zeros((1, 2 * b * blocks), np.float32)
+    for j in range(blocks):
+        G[0, 2 * b * j:2 * b * j + b] = 50.0                            # silu(50) = 50 to fp32 precision
+        G[0, 2 * b * j + b:2 * b * (j + 1)] = np.arange(b) + 1000.0 * j
+    got = oracle.swiglu(G)
+    want = np.concatenate([50.0 * (np.arange(b) + 1000.0 * j) for j in range(blocks)])
+    assert np.allclose(got[0], want, rtol=1e-6)
+    # odd part of silu is x / 2 + x / 2: silu(x) - silu(-x) = x
+    x = np.linspace(-30, 30, 2 * b).astype(np.float32)
+    one = np.ones_like(x)
+    pos = oracle.swiglu(np.stack([x[:b], one[:b], x[b:], one[b:]]).reshape(1, -1))
+    neg = oracle.swiglu(np.stack([-x[:b], one[:b], -x[b:], one[b:]]).reshape(1, -1))
+    assert np.allclose(pos - neg, x.reshape(1, -1), atol=1e-5)
