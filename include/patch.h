@@ -169,6 +169,25 @@ int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
                   int variant);
 
 /*
+ * Gated product of the MLP's gate and up projections in one launch (a first step of the
+ * block-level fusion that follows the per-matrix matmul; the paper studies the "up, gate, and
+ * down matrices of the MLP" separately, and in the LLaMA models it measures the MLP computes
+ * down(silu(gate x) * up x)):
+ *     Y[m][128 j + r] = silu(G[m][128 j + r]) * U[m][128 j + r],   silu(x) = x / (1 + exp(-x)),
+ * where G = X Wgate^T and U = X Wup^T come from ONE packed weight that stacks the two matrices
+ * with their 128-row blocks interleaved: row-block 2j of the packed matrix is row-block j of
+ * Wgate, row-block 2j + 1 is row-block j of Wup (each keeps its own tile flags).  fp32
+ * accumulation, the product evaluated in fp32 on the accumulators, one bf16 rounding.
+ *   layout->N  must be a multiple of 256; Y_dev is bf16 [M x ldy], ldy >= N / 2, ldy % 8 == 0.
+ * Other arguments and error behaviour as patch_gemm; no workspace.  Any M is accepted, but the
+ * schedule is the large-M one (for M <= 64, patch_gemm on the same packed weight followed by
+ * the caller's own activation streams the weights faster).
+ */
+int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M,
+                     const patch_layout_t* layout, const void* packed_dev,
+                     void* Y_dev, int64_t ldy, int* status_dev, void* stream);
+
+/*
  * End-to-end form with HOST activations and results: copies X host->device into
  * X_stage_dev, runs patch_gemm, copies Y device->host and synchronises `stream`.
  *   X_host  bf16 [M x K] contiguous; Y_host bf16 [M x N] contiguous (pinned memory advised)

@@ -24,7 +24,8 @@ ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
-           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_host", "patch_gemm_noalloc",
+           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_host",
+           "patch_gemm_noalloc",
            "patch_strerror", "patch_version"]
 
 
@@ -63,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.patch_workspace_init.argtypes = [vp, sz, vp]
         L.patch_gemm.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, sz, vp, vp]
         L.patch_gemm_ex.argtypes = L.patch_gemm.argtypes + [ctypes.c_int]
+        L.patch_gemm_gated.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, vp]
         L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
         L.patch_gemm_noalloc.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp]
         L.patch_strerror.argtypes = [ctypes.c_int]
@@ -153,6 +155,31 @@ def patch_gemm(X, layout: Layout, packed, Y=None, workspace=None, status=None, s
     _check(lib().patch_gemm_ex(_ptr(X), X.stride(0) if M else layout.K, M, ctypes.byref(layout), _ptr(packed),
                                _ptr(Y), Y.stride(0) if M else layout.N, _ptr(workspace), ws_bytes,
                                _ptr(status), _stream(stream), variant), "patch_gemm")
+    return Y
+
+
+def interleave_row_blocks(A, B_, block: int = 128):
+    """Stack two [N x ...] arrays (torch or numpy) so that 128-row blocks alternate: A block 0, B block 0,
+    A block 1, ...  With ``block=1`` the same for per-tile flag arrays.  Data movement only."""
+    n = A.shape[0]
+    assert A.shape == B_.shape and n % block == 0
+    tail = tuple(A.shape[1:])
+    if hasattr(A, "cpu"):
+        import torch
+        return torch.stack((A.reshape(n // block, block, *tail), B_.reshape(n // block, block, *tail)), dim=1).reshape(2 * n, *tail)
+    import numpy as np
+    return np.stack((A.reshape(n // block, block, *tail), B_.reshape(n // block, block, *tail)), axis=1).reshape(2 * n, *tail)
+
+
+def patch_gemm_gated(X, layout: Layout, packed, Y=None, status=None, stream=None):
+    """Y [M x N/2] = silu(X Wgate^T) * (X Wup^T) for a packed weight with interleaved gate/up row-blocks."""
+    import torch
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, layout.N // 2), dtype=torch.bfloat16, device=X.device)
+    _check(lib().patch_gemm_gated(_ptr(X), X.stride(0) if M else layout.K, M, ctypes.byref(layout), _ptr(packed),
+                                  _ptr(Y), Y.stride(0) if M else layout.N // 2, _ptr(status), _stream(stream)),
+           "patch_gemm_gated")
     return Y
 
 

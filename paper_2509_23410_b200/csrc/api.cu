@@ -68,6 +68,23 @@ extern "C" int patch_gemm(const void* X_dev, int64_t ldx, int64_t M, const patch
                          stream, PATCH_VARIANT_AUTO);
 }
 
+extern "C" int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,
+                                const void* packed_dev, void* Y_dev, int64_t ldy, int* status_dev, void* stream) {
+    if (!L) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (L->N % (2 * kTile)) return PATCH_ERR_SHAPE;      // whole (gate, up) pairs of row-blocks
+    if (M < 0) return PATCH_ERR_SHAPE;
+    if (M == 0) return PATCH_OK;
+    if (!X_dev || !packed_dev || !Y_dev) return PATCH_ERR_NULL;
+    if (ldx < L->K || ldy < L->N / 2 || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;
+    if (!aligned16(X_dev) || !aligned16(Y_dev) || !aligned16(packed_dev)) return PATCH_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    return launch_prefill_gated(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
+                                static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* L, const void* packed_dev,
                                void* Y_host, void* X_stage_dev, void* Y_stage_dev, void* workspace_dev,
                                size_t workspace_bytes, void* stream) {

@@ -45,7 +45,8 @@ constexpr uint32_t kSparse = 2;
 
 __global__ void __launch_bounds__(320)
 prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
-                int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
+                int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev,
+                int gated) {
     using namespace p2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -257,8 +258,29 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             const int chunks = (valid + 15) / 16, c_begin = half == 0 ? 0 : (chunks + 1) / 2,
                       c_end = half == 0 ? (chunks + 1) / 2 : chunks;
+            if (gated) {
+                // the pair is (gate row-block, up row-block) of the same 128 outputs: Y = silu(gate) * up,
+                // one output row-block per pair
+                const uint32_t acc_g = tmem_base + ((quad * 32u) << 16), acc_u = acc_g + kAcc1Col;
+                __nv_bfloat16* ytile = Y + int64_t(m0) * ldy + int64_t(tn0 >> 1) * kTile + quad * 32;
 #pragma unroll 1
-            for (int rb = 0; rb < 2; ++rb) {
+                for (int ch = c_begin; ch < c_end; ++ch) {
+                    const int c0 = ch * 16;
+                    uint32_t g[16], u[16];
+                    tmem_ld16(acc_g + uint32_t(c0), g);
+                    tmem_ld16(acc_u + uint32_t(c0), u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        const float x = __uint_as_float(g[q]);
+                        g[q] = __float_as_uint(__fdividef(x, 1.0f + __expf(-x)) * __uint_as_float(u[q]));   // 2 MUFU ops, ~2 ulp
+                    }
+                    store_fragment_transposed(g, smem + kStageOffset + (warp - 2) * 1024, lane, ytile + int64_t(c0) * ldy, ldy,
+                                              valid - c0);
+                }
+            }
+#pragma unroll 1
+            for (int rb = 0; rb < 2 && !gated; ++rb) {
                 if (rb == 1 && !has1) break;
                 const uint32_t acc = tmem_base + (rb ? kAcc1Col : 0u) + ((quad * 32u) << 16);
                 __nv_bfloat16* ytile = Y + int64_t(m0) * ldy + int64_t(tn0 + rb) * kTile + quad * 32;
@@ -287,7 +309,7 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
 }
 
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
-                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated) {
     static bool configured = false;   // per-process attribute, idempotent
     if (!configured) {
         if (cudaFuncSetAttribute(prefill2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p2::kSmemBytes) != cudaSuccess)
@@ -308,7 +330,7 @@ int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, prefill2_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
-                                       Y, ldy, status_dev);
+                                       Y, ldy, status_dev, gated ? 1 : 0);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

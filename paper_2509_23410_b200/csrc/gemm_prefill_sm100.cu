@@ -228,7 +228,7 @@ static int sm_count_prefill() {
 }
 
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
-                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated);
 
 // Testing / tuning aid: PATCH_PREFILL_SCHEDULE=1|2 in the environment pins the schedule (one or two
 // row-blocks per CTA); anything else lets the cost model choose.
@@ -248,7 +248,7 @@ static int forced_schedule() {
 // pipeline), plus a per-tile prologue/epilogue cost.
 struct PrefillPlan { int n_tok; int schedule; };   // schedule: row-blocks per CTA (1 or 2)
 
-static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms) {
+static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row_blocks_only = false) {
     PrefillPlan best = {240, 1};
     double best_cost = 1e300;
     const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : 240, n_lo = M <= 128 ? n_hi : 128;
@@ -256,7 +256,7 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms) {
     for (int n = n_hi; n >= n_lo; n -= 16) {
         const int64_t MT = (M + n - 1) / n;
         for (int sched = 1; sched <= 2; ++sched) {
-            if (forced && sched != forced) continue;
+            if (two_row_blocks_only ? sched != 2 : (forced && sched != forced)) continue;
             const int64_t tiles = int64_t(sched == 1 ? TN : (TN + 1) / 2) * MT;
             const int64_t waves = (tiles + sms - 1) / sms;
             const double mma_ns = (sched == 1 ? 550.0 : 1100.0) * n / 256.0;
@@ -287,7 +287,7 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
-    if (plan.schedule == 2) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream);
+    if (plan.schedule == 2) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream, false);
     static bool configured = false;   // per-process attribute, idempotent
     if (!configured) {
         if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -310,6 +310,21 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
                                        Y, ldy, status_dev);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+// Gated product of a stacked gate/up weight whose row-blocks alternate (gate j, up j): always the
+// two-row-block kernel, whose CTA holds both accumulators of an output row-block.
+int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
+                         __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+    if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
+    const int sms = sm_count_prefill();
+    if (sms <= 0) return PATCH_ERR_CUDA;
+    const int TN = int(L->N / kTile), TK = int(L->K / kTile);
+    const PrefillPlan plan = plan_prefill(M, TN, TK, sms, true);
+    CUtensorMap map;
+    int rc = make_x_tensor_map(&map, X, ldx, M, L->K, plan.n_tok);
+    if (rc) return rc;
+    return launch_prefill2(map, L, packed, M, plan.n_tok, sms, Y, ldy, status_dev, stream, true);
 }
 
 }  // namespace patch

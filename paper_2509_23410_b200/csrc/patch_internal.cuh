@@ -50,6 +50,8 @@ int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_la
                   cudaStream_t stream, bool wstatic, bool xstatic);
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                    const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
+                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
 size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M);
 
 }  // namespace patch

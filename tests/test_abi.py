@@ -106,3 +106,21 @@ def test_stacked_case_flags_concatenate_parts():
     parts = [inputs.tile_flags(4096, 4096, plain[f"stack.0.{r}"]["p"], inputs.MASTER_SEED, "stack", 0, r) for r in "qkv"]
     assert np.array_equal(qkv, np.concatenate(parts, axis=0))
     assert abs(fused[0]["p"] - sum(plain[f"stack.0.{r}"]["p"] for r in "qkv") / 3) < 1e-12
+
+
+def test_gated_entry_validates_on_the_host():
+    """patch_gemm_gated: argument errors are reported before any launch (no GPU here)."""
+    import ctypes
+    import numpy as np
+    from paper_2509_23410_b200 import binding as B
+    lib = B.lib()
+    ok = B.patch_packed_size(512, 256, np.zeros((4, 2), np.uint8))
+    odd = B.patch_packed_size(384, 256, np.zeros((3, 2), np.uint8))
+    buf = ctypes.create_string_buffer(64)
+    p = ctypes.cast(buf, ctypes.c_void_p)
+    assert lib.patch_gemm_gated(p, 256, 4, ctypes.byref(odd), p, p, 192, None, None) == B.ERR_SHAPE   # N % 256
+    assert lib.patch_gemm_gated(None, 256, 4, ctypes.byref(ok), p, p, 256, None, None) == B.ERR_NULL
+    assert lib.patch_gemm_gated(p, 128, 4, ctypes.byref(ok), p, p, 256, None, None) == B.ERR_SHAPE    # ldx < K
+    assert lib.patch_gemm_gated(p, 256, 4, ctypes.byref(ok), p, p, 248, None, None) == B.ERR_SHAPE    # ldy < N / 2
+    assert lib.patch_gemm_gated(p, 256, 0, ctypes.byref(ok), p, p, 256, None, None) == 0                 # M = 0
+    assert lib.patch_gemm_gated(p, 256, -1, ctypes.byref(ok), p, p, 256, None, None) == B.ERR_SHAPE

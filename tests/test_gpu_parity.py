@@ -455,3 +455,52 @@ def test_random_shapes_and_pitches(gpu, oracle):
             assert int(status.item()) == 0, what
             assert pady == 0 or bool((Yfull[:, N:] == 7.0).all()), what + ": wrote past column N"
             check_parity(oracle, to_bits(Yfull[:, :N]), Y32, what)
+
+
+# ---------------------------------------------------------------------------------------------
+# gated gate/up product (stacked weight with interleaved row-blocks)
+
+
+def _gated_case(gpu, oracle, Nh, K, M, pg, pu, rows=None):
+    torch, B = gpu
+    Wg = inputs.weight(Nh, K, inputs.MASTER_SEED, "gated", "g", Nh, K)
+    Wu = inputs.weight(Nh, K, inputs.MASTER_SEED, "gated", "u", Nh, K)
+    Wg = inputs.f32_to_bf16_bits(f32(Wg) * 40.0)      # gate pre-activations of order 1: both tails of silu matter
+    fg = inputs.tile_flags(Nh, K, pg, inputs.MASTER_SEED, "gated", "g", Nh, K)
+    fu = inputs.tile_flags(Nh, K, pu, inputs.MASTER_SEED, "gated", "u", Nh, K)
+    W = B.interleave_row_blocks(Wg, Wu)
+    flags = B.interleave_row_blocks(fg, fu, block=1)
+    X = inputs.activation(M, K, inputs.MASTER_SEED, "gated", M)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = B.patch_gemm_gated(to_dev(torch, X), L, packed, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and tuple(Y.shape) == (M, Nh)
+    What = oracle.prune(W, flags)
+    if rows is None:
+        ref = oracle.swiglu(oracle.gemm_f64(X, What)[0])
+        check_parity(oracle, to_bits(Y), ref, f"gated Nh={Nh} K={K} M={M}")
+    else:
+        ref = oracle.swiglu(oracle.gemm_f64_rows(X, rows, What))
+        check_parity(oracle, to_bits(Y)[rows], ref, f"gated Nh={Nh} K={K} M={M} (sampled rows)")
+
+
+@pytest.mark.parametrize("M", [1, 16, 100, 300, 513])
+@pytest.mark.parametrize("pg,pu", [(0.0, 0.0), (1.0, 1.0), (0.3, 0.8)])
+def test_gated_product_parity(gpu, oracle, M, pg, pu):
+    _gated_case(gpu, oracle, 1024, 768, M, pg, pu)
+
+
+def test_gated_product_llama_mlp_shape(gpu, oracle):
+    M = 2048
+    rows = np.array([0, 1, 239, 240, 1023, 1024, 2047])
+    _gated_case(gpu, oracle, 11008, 4096, M, 0.6, 0.9, rows=rows)
+
+
+def test_gated_product_rejects_bad_shapes(gpu):
+    torch, B = gpu
+    W = inputs.weight(384, 256, 3, "gated-bad")                   # three row-blocks: no whole pairs
+    packed, L = B.patch_pack(to_dev(torch, W), np.zeros((3, 2), np.uint8))
+    X = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.PatchError):
+        B.patch_gemm_gated(X, L, packed)
