@@ -251,7 +251,7 @@ struct PrefillPlan { int n_tok; int schedule; };   // schedule: row-blocks per C
 static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row_blocks_only = false) {
     PrefillPlan best = {240, 1};
     double best_cost = 1e300;
-    const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : 240, n_lo = M <= 128 ? n_hi : 128;
+    const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : kPrefillMaxTok, n_lo = M <= 128 ? n_hi : 128;
     const int forced = forced_schedule();
     for (int n = n_hi; n >= n_lo; n -= 16) {
         const int64_t MT = (M + n - 1) / n;
