@@ -179,13 +179,20 @@ int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
  * Wgate, row-block 2j + 1 is row-block j of Wup (each keeps its own tile flags).  fp32
  * accumulation, the product evaluated in fp32 on the accumulators, one bf16 rounding.
  *   layout->N  must be a multiple of 256; Y_dev is bf16 [M x ldy], ldy >= N / 2, ldy % 8 == 0.
- * Other arguments and error behaviour as patch_gemm; no workspace.  Any M is accepted, but the
- * schedule is the large-M one (for M <= 64, patch_gemm on the same packed weight followed by
- * the caller's own activation streams the weights faster).
+ *   workspace_dev / workspace_bytes   optional.  With M <= 16 and at least
+ *           patch_gemm_gated_workspace_size(layout, M) bytes (256-byte aligned, zeroed once with
+ *           patch_workspace_init, left zero by every call, shareable with patch_gemm calls) the
+ *           small-M stream-K schedule is used: the finisher of a gate row-block publishes its
+ *           fp32 values, the finisher of the matching up row-block multiplies.  Otherwise (or for
+ *           larger M) the large-M schedule runs, whose CTA holds both accumulators.
+ *   flags   0 or PATCH_GEMM_WEIGHTS_STATIC [| PATCH_GEMM_INPUT_STATIC], as for patch_gemm_ex.
+ * Other arguments and error behaviour as patch_gemm.
  */
+int patch_gemm_gated_workspace_size(const patch_layout_t* layout, int64_t M, size_t* bytes_out);
 int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M,
                      const patch_layout_t* layout, const void* packed_dev,
-                     void* Y_dev, int64_t ldy, int* status_dev, void* stream);
+                     void* Y_dev, int64_t ldy,
+                     void* workspace_dev, size_t workspace_bytes, int* status_dev, void* stream, int flags);
 
 /*
  * End-to-end form with HOST activations and results: copies X host->device into

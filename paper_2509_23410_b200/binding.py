@@ -24,7 +24,7 @@ ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
-           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_host",
+           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host",
            "patch_gemm_noalloc",
            "patch_strerror", "patch_version"]
 
@@ -64,7 +64,8 @@ def lib() -> ctypes.CDLL:
         L.patch_workspace_init.argtypes = [vp, sz, vp]
         L.patch_gemm.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, sz, vp, vp]
         L.patch_gemm_ex.argtypes = L.patch_gemm.argtypes + [ctypes.c_int]
-        L.patch_gemm_gated.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, vp]
+        L.patch_gemm_gated.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp, sz, vp, vp, ctypes.c_int]
+        L.patch_gemm_gated_workspace_size.argtypes = [ctypes.POINTER(Layout), i64, ctypes.POINTER(sz)]
         L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
         L.patch_gemm_noalloc.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp]
         L.patch_strerror.argtypes = [ctypes.c_int]
@@ -171,14 +172,22 @@ def interleave_row_blocks(A, B_, block: int = 128):
     return np.stack((A.reshape(n // block, block, *tail), B_.reshape(n // block, block, *tail)), axis=1).reshape(2 * n, *tail)
 
 
-def patch_gemm_gated(X, layout: Layout, packed, Y=None, status=None, stream=None):
+def patch_gemm_gated_workspace_size(layout: Layout, M: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().patch_gemm_gated_workspace_size(ctypes.byref(layout), M, ctypes.byref(n)), "patch_gemm_gated_workspace_size")
+    return int(n.value)
+
+
+def patch_gemm_gated(X, layout: Layout, packed, Y=None, workspace=None, status=None, stream=None, flags: int = 0):
     """Y [M x N/2] = silu(X Wgate^T) * (X Wup^T) for a packed weight with interleaved gate/up row-blocks."""
     import torch
     M = X.shape[0]
     if Y is None:
         Y = torch.empty((M, layout.N // 2), dtype=torch.bfloat16, device=X.device)
+    ws_bytes = workspace.numel() if workspace is not None else 0
     _check(lib().patch_gemm_gated(_ptr(X), X.stride(0) if M else layout.K, M, ctypes.byref(layout), _ptr(packed),
-                                  _ptr(Y), Y.stride(0) if M else layout.N // 2, _ptr(status), _stream(stream)),
+                                  _ptr(Y), Y.stride(0) if M else layout.N // 2, _ptr(workspace), ws_bytes,
+                                  _ptr(status), _stream(stream), flags),
            "patch_gemm_gated")
     return Y
 

@@ -68,21 +68,40 @@ extern "C" int patch_gemm(const void* X_dev, int64_t ldx, int64_t M, const patch
                          stream, PATCH_VARIANT_AUTO);
 }
 
+extern "C" int patch_gemm_gated_workspace_size(const patch_layout_t* L, int64_t M, size_t* bytes_out) {
+    if (!L || !bytes_out) return PATCH_ERR_NULL;
+    int rc = validate_layout(L);
+    if (rc) return rc;
+    if (L->N % (2 * kTile) || M < 0) return PATCH_ERR_SHAPE;
+    *bytes_out = decode_gated_workspace_bytes(L, M);
+    return PATCH_OK;
+}
+
 extern "C" int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,
-                                const void* packed_dev, void* Y_dev, int64_t ldy, int* status_dev, void* stream) {
+                                const void* packed_dev, void* Y_dev, int64_t ldy, void* workspace_dev,
+                                size_t workspace_bytes, int* status_dev, void* stream, int flags) {
     if (!L) return PATCH_ERR_NULL;
     int rc = validate_layout(L);
     if (rc) return rc;
     if (L->N % (2 * kTile)) return PATCH_ERR_SHAPE;      // whole (gate, up) pairs of row-blocks
     if (M < 0) return PATCH_ERR_SHAPE;
+    if (flags & ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC)) return PATCH_ERR_SHAPE;
     if (M == 0) return PATCH_OK;
     if (!X_dev || !packed_dev || !Y_dev) return PATCH_ERR_NULL;
     if (ldx < L->K || ldy < L->N / 2 || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;
     if (!aligned16(X_dev) || !aligned16(Y_dev) || !aligned16(packed_dev)) return PATCH_ERR_ALIGN;
     rc = check_device();
     if (rc) return rc;
-    return launch_prefill_gated(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
-                                static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, static_cast<cudaStream_t>(stream));
+    const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(X_dev);
+    __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(Y_dev);
+    const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // small M with a workspace: the stream-K schedule; otherwise the two-row-block schedule, which needs none
+    const size_t need = decode_gated_workspace_bytes(L, M);
+    if (need > 0 && workspace_dev && workspace_bytes >= need && !(reinterpret_cast<uintptr_t>(workspace_dev) & 255u))
+        return launch_decode_gated(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s,
+                                   (flags & PATCH_GEMM_WEIGHTS_STATIC) != 0, (flags & PATCH_GEMM_INPUT_STATIC) != 0);
+    return launch_prefill_gated(X, ldx, M, L, packed, Y, ldy, status_dev, s);
 }
 
 extern "C" int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* L, const void* packed_dev,

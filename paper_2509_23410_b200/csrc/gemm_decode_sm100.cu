@@ -111,6 +111,49 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long
     return v;
 }
 
+// Gated mode (stacked gate/up weight, row-blocks interleaved): what the finisher of a row-block does with its 16
+// finished fp32 values of one out-feature row.  An even row-block is a gate: its values are published as flagged
+// words (0 = not there yet; +0 is stored as -0).  An odd row-block is the matching up projection: its finisher
+// fetches the gate values (bounded poll), empties the words again and writes silu(gate) * up.  The gate's
+// finisher waits for nothing here, and partial sums are always written before anything is polled, so the waits
+// cannot form a cycle.
+__device__ __forceinline__ bool finish_gated_row(const float (&a)[16], int tn, int row, int M, __nv_bfloat16* Y, int64_t ldy,
+                                                 uint32_t* gate_words, volatile int* abort_flag, int* status_dev) {
+    uint32_t* slot = gate_words + (int64_t(tn >> 1) * kTile + row) * 16;
+    if ((tn & 1) == 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            st_relaxed_gpu_v4(slot + 4 * q, make_uint4(nonempty(__float_as_uint(a[4 * q])), nonempty(__float_as_uint(a[4 * q + 1])),
+                                                      nonempty(__float_as_uint(a[4 * q + 2])), nonempty(__float_as_uint(a[4 * q + 3]))));
+        return true;
+    }
+    uint4 w[4];
+    const uint64_t tstart = global_timer_ns();
+    for (bool all = false; !all;) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) w[q] = ld_relaxed_gpu_v4(slot + 4 * q);
+        all = true;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) all = all && w[q].x != 0u && w[q].y != 0u && w[q].z != 0u && w[q].w != 0u;
+        if (!all && (*abort_flag || global_timer_ns() - tstart > kWaitLimitNs)) {
+            *abort_flag = 1;
+            if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+            return false;
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) st_relaxed_gpu_v4(slot + 4 * q, make_uint4(0, 0, 0, 0));   // empty again for the next launch
+    const uint32_t g[16] = {w[0].x, w[0].y, w[0].z, w[0].w, w[1].x, w[1].y, w[1].z, w[1].w,
+                            w[2].x, w[2].y, w[2].z, w[2].w, w[3].x, w[3].y, w[3].z, w[3].w};
+    __nv_bfloat16* ycol = Y + int64_t(tn >> 1) * kTile + row;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float x = __uint_as_float(g[j]);
+        if (j < M) ycol[int64_t(j) * ldy] = __float2bfloat16_rn(__fdividef(x, 1.0f + __expf(-x)) * a[j]);
+    }
+    return true;
+}
+
 // Every contributor of a row-block finishes rows [r0, r1) of it: thread `et` (0..127) takes
 // (row, 16-token chunk) items, sums the n_contrib partial tiles in ascending K order and writes bf16.
 template <int N_TOK>
@@ -159,12 +202,15 @@ __device__ __forceinline__ void reduce_row_share(const float* __restrict__ parti
 // XSTATIC: the caller promises that X was not written by the operation preceding this launch
 //          in the stream, so activations may be fetched before the grid dependency resolves.
 // Weight tiles are always fetched early only if WSTATIC (same promise about the packed blob).
-template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC>
+// GATED:   silu(gate) * up epilogue on a stacked gate/up weight (see finish_gated_row); 16-token schedule only.
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
 __global__ void __launch_bounds__(192)
 decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
               uint32_t pay0_16, uint32_t pay_total_16, int TN, int TK, int M,
               __nv_bfloat16* __restrict__ Y, int64_t ldy,
-              unsigned long long* __restrict__ counters, float* __restrict__ partials, int* status_dev) {
+              unsigned long long* __restrict__ counters, float* __restrict__ partials, int* status_dev,
+              uint32_t* __restrict__ gate_words) {
+    static_assert(!GATED || N_TOK == 16, "the gated epilogue exists for the 16-token schedule");
     using Cfg = DecodeConfig<N_TOK, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -336,7 +382,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                 if (warp == 2) PATCH_TRACE_AT(8);
             }
             const uint32_t acc = tmem_base + uint32_t(seg & 1) * N_TOK + ((quad * 32u) << 16);
-            if (ntiles == TK) {
+            if (GATED && ntiles == TK) {
+                // whole row-block in this run: its values are final
+                uint32_t v[16];
+                tmem_ld16(acc, v);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (seg & 1));
+                float a[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) a[j] = __uint_as_float(v[j]);
+                ok = finish_gated_row(a, tn, row, M, Y, ldy, gate_words, abort_flag, status_dev);
+            } else if (ntiles == TK) {
                 // whole row-block in this run: finish it here
                 __nv_bfloat16* ycol = Y + int64_t(tn) * kTile + row;
 #pragma unroll 1
@@ -419,7 +477,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                             }
                         }
                     }
-                    if (ok) {
+                    if (ok && GATED) {
+                        ok = finish_gated_row(a, tn, row, M, Y, ldy, gate_words, abort_flag, status_dev);
+                    } else if (ok) {
                         __nv_bfloat16* ycol = Y + int64_t(tn) * kTile + row;
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
@@ -522,6 +582,16 @@ static size_t counters_bytes(const patch_layout_t* L) {
 }
 constexpr size_t kFlaggedBytes = size_t(2) * kMaxDecodeCtas * 16 * kTile * sizeof(float);
 
+// Gated mode: one slot of [128 rows][16 tokens] flag words per (gate, up) pair of row-blocks, past everything
+// the plain schedules use of the same workspace (their partial tiles are not kept zero).
+static size_t gate_words_offset(const patch_layout_t* L) {
+    return counters_bytes(L) + kFlaggedBytes + size_t(2) * kMaxDecodeCtas * 64 * kTile * sizeof(float);
+}
+size_t decode_gated_workspace_bytes(const patch_layout_t* L, int64_t M) {
+    if (M > 16) return 0;
+    return gate_words_offset(L) + size_t(L->N / (2 * kTile)) * kTile * 16 * sizeof(float);
+}
+
 size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M) {
     if (M > 64) return 0;
     const int n_tok = decode_n_tok(M);
@@ -538,11 +608,11 @@ static int sm_count() {
     return n;
 }
 
-template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC>
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
 static int launch_decode_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
                            __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream) {
     using Cfg = DecodeConfig<N_TOK, STAGES>;
-    auto kern = decode_kernel<N_TOK, STAGES, WSTATIC, XSTATIC>;
+    auto kern = decode_kernel<N_TOK, STAGES, WSTATIC, XSTATIC, GATED>;
     static bool configured = false;   // per-process attribute, idempotent
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
@@ -570,9 +640,10 @@ static int launch_decode_t(const CUtensorMap& map, const patch_layout_t* L, cons
     cfg.numAttrs = 1;
     unsigned long long* counters = static_cast<unsigned long long*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + counters_bytes(L) + (N_TOK > 16 ? kFlaggedBytes : 0));
+    uint32_t* gate_words = GATED ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(workspace) + gate_words_offset(L)) : nullptr;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, packed, uint64_t(L->table_off),
                                        uint32_t(L->payload_off / 16), uint32_t(L->payload_bytes / 16), TN, TK, M, Y,
-                                       ldy, counters, partials, status_dev);
+                                       ldy, counters, partials, status_dev, gate_words);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
@@ -601,6 +672,19 @@ int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_la
         case 32: return launch_decode_f<32, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
         default: return launch_decode_f<64, 2>(wstatic, xstatic, map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
     }
+}
+
+// silu(gate) * up on a stacked gate/up weight with interleaved row-blocks, M <= 16: Y is [M x N / 2].
+int launch_decode_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
+                        __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream,
+                        bool wstatic, bool xstatic) {
+    CUtensorMap map;
+    int rc = make_x_tensor_map(&map, X, ldx, M, L->K, 16);
+    if (rc) return rc;
+    if (wstatic && xstatic)
+        return launch_decode_t<16, PATCH_XSTATIC_STAGES, true, true, true>(map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+    if (wstatic) return launch_decode_t<16, 3, true, false, true>(map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
+    return launch_decode_t<16, 3, false, false, true>(map, L, packed, int(M), Y, ldy, workspace, status_dev, stream);
 }
 
 }  // namespace patch

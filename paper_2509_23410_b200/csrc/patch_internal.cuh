@@ -53,5 +53,9 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
 int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                          const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
 size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M);
+int launch_decode_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
+                        const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev,
+                        cudaStream_t stream, bool wstatic, bool xstatic);
+size_t decode_gated_workspace_bytes(const patch_layout_t* L, int64_t M);   // 0 if the gated decode schedule does not apply
 
 }  // namespace patch

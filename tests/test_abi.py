@@ -118,9 +118,17 @@ def test_gated_entry_validates_on_the_host():
     odd = B.patch_packed_size(384, 256, np.zeros((3, 2), np.uint8))
     buf = ctypes.create_string_buffer(64)
     p = ctypes.cast(buf, ctypes.c_void_p)
-    assert lib.patch_gemm_gated(p, 256, 4, ctypes.byref(odd), p, p, 192, None, None) == B.ERR_SHAPE   # N % 256
-    assert lib.patch_gemm_gated(None, 256, 4, ctypes.byref(ok), p, p, 256, None, None) == B.ERR_NULL
-    assert lib.patch_gemm_gated(p, 128, 4, ctypes.byref(ok), p, p, 256, None, None) == B.ERR_SHAPE    # ldx < K
-    assert lib.patch_gemm_gated(p, 256, 4, ctypes.byref(ok), p, p, 248, None, None) == B.ERR_SHAPE    # ldy < N / 2
-    assert lib.patch_gemm_gated(p, 256, 0, ctypes.byref(ok), p, p, 256, None, None) == 0                 # M = 0
-    assert lib.patch_gemm_gated(p, 256, -1, ctypes.byref(ok), p, p, 256, None, None) == B.ERR_SHAPE
+
+    def call(X, ldx, M, L, Y, ldy, flags=0):
+        return lib.patch_gemm_gated(X, ldx, M, ctypes.byref(L), p, Y, ldy, None, 0, None, None, flags)
+
+    assert call(p, 256, 4, odd, p, 192) == B.ERR_SHAPE      # N % 256
+    assert call(None, 256, 4, ok, p, 256) == B.ERR_NULL
+    assert call(p, 128, 4, ok, p, 256) == B.ERR_SHAPE       # ldx < K
+    assert call(p, 256, 4, ok, p, 248) == B.ERR_SHAPE       # ldy < N / 2
+    assert call(p, 256, 0, ok, p, 256) == 0                 # M = 0
+    assert call(p, 256, -1, ok, p, 256) == B.ERR_SHAPE
+    assert call(p, 256, 4, ok, p, 256, flags=1) == B.ERR_SHAPE      # only the two *_STATIC flags
+    # workspace of the small-M schedule: past everything patch_gemm uses of a shared buffer, one slot per pair
+    assert B.patch_gemm_gated_workspace_size(ok, 16) == B.patch_gemm_workspace_size(ok, 64) + 2 * 128 * 16 * 4
+    assert B.patch_gemm_gated_workspace_size(ok, 17) == 0

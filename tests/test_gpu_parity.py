@@ -461,7 +461,7 @@ def test_random_shapes_and_pitches(gpu, oracle):
 # gated gate/up product (stacked weight with interleaved row-blocks)
 
 
-def _gated_case(gpu, oracle, Nh, K, M, pg, pu, rows=None):
+def _gated_case(gpu, oracle, Nh, K, M, pg, pu, rows=None, ws=None, flags_arg=0):
     torch, B = gpu
     Wg = inputs.weight(Nh, K, inputs.MASTER_SEED, "gated", "g", Nh, K)
     Wu = inputs.weight(Nh, K, inputs.MASTER_SEED, "gated", "u", Nh, K)
@@ -473,9 +473,13 @@ def _gated_case(gpu, oracle, Nh, K, M, pg, pu, rows=None):
     X = inputs.activation(M, K, inputs.MASTER_SEED, "gated", M)
     packed, L = B.patch_pack(to_dev(torch, W), flags)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    Y = B.patch_gemm_gated(to_dev(torch, X), L, packed, status=status)
+    if ws == "own":
+        ws = torch.zeros(max(B.patch_gemm_gated_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+    Y = B.patch_gemm_gated(to_dev(torch, X), L, packed, workspace=ws, status=status, flags=flags_arg)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and tuple(Y.shape) == (M, Nh)
+    if ws is not None:
+        assert int(ws.count_nonzero()) == 0, "gate words not left empty"
     What = oracle.prune(W, flags)
     if rows is None:
         ref = oracle.swiglu(oracle.gemm_f64(X, What)[0])
@@ -504,3 +508,48 @@ def test_gated_product_rejects_bad_shapes(gpu):
     X = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(B.PatchError):
         B.patch_gemm_gated(X, L, packed)
+
+
+@pytest.mark.parametrize("M", [1, 5, 16])
+@pytest.mark.parametrize("shape", [(1024, 768), (1408, 4096), (11008, 4096)])
+def test_gated_product_small_m_schedule(gpu, oracle, M, shape):
+    """M <= 16 with a workspace: the stream-K schedule, where the gate and up row-blocks of a pair are
+    usually finished by different CTAs; every launch-flag combination."""
+    torch, B = gpu
+    Nh, K = shape
+    for flags_arg in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC):
+        _gated_case(gpu, oracle, Nh, K, M, 0.3, 0.8, ws="own", flags_arg=flags_arg)
+
+
+def test_gated_and_plain_calls_share_a_workspace(gpu, oracle):
+    """The gate words live past everything patch_gemm uses of a workspace: plain calls of any M <= 64
+    and gated calls may alternate on one buffer."""
+    torch, B = gpu
+    Nh, K = 1024, 768
+    Wp = inputs.weight(2 * Nh, K, inputs.MASTER_SEED, "gated", "plain")
+    fp = inputs.tile_flags(2 * Nh, K, 0.5, inputs.MASTER_SEED, "gated", "plain")
+    packed_p, Lp = B.patch_pack(to_dev(torch, Wp), fp)
+    What_p = oracle.prune(Wp, fp)
+    ws = torch.zeros(B.patch_gemm_gated_workspace_size(Lp, 16), dtype=torch.uint8, device="cuda")
+    assert ws.numel() >= B.patch_gemm_workspace_size(Lp, 64)
+    for M in (48, 8, 64, 3):
+        X = inputs.activation(M, K, inputs.MASTER_SEED, "gated", "plain", M)
+        Y = B.patch_gemm(to_dev(torch, X), Lp, packed_p, workspace=ws)
+        torch.cuda.synchronize()
+        check_parity(oracle, to_bits(Y), oracle.gemm_f64(X, What_p)[0], f"plain M={M} on the shared workspace")
+        ws_gate = ws[B.patch_gemm_workspace_size(Lp, 64):]
+        assert int(ws_gate.count_nonzero()) == 0
+        for Mg in (16, 2):
+            Wg = inputs.weight(Nh, K, inputs.MASTER_SEED, "gated", "g", Nh, K)
+            Wu = inputs.weight(Nh, K, inputs.MASTER_SEED, "gated", "u", Nh, K)
+            fg = inputs.tile_flags(Nh, K, 0.3, inputs.MASTER_SEED, "gated", "g", Nh, K)
+            fu = inputs.tile_flags(Nh, K, 0.8, inputs.MASTER_SEED, "gated", "u", Nh, K)
+            W = B.interleave_row_blocks(inputs.f32_to_bf16_bits(f32(Wg) * 40.0), Wu)
+            flags = B.interleave_row_blocks(fg, fu, block=1)
+            packed, L = B.patch_pack(to_dev(torch, W), flags)
+            Xg = inputs.activation(Mg, K, inputs.MASTER_SEED, "gated", Mg)
+            Yg = B.patch_gemm_gated(to_dev(torch, Xg), L, packed, workspace=ws)
+            torch.cuda.synchronize()
+            ref = oracle.swiglu(oracle.gemm_f64(Xg, oracle.prune(W, flags))[0])
+            check_parity(oracle, to_bits(Yg), ref, f"gated M={Mg} after plain M={M}")
+            assert int(ws_gate.count_nonzero()) == 0
