@@ -67,6 +67,32 @@ __device__ __forceinline__ int first_tile_at_or_after(const TileDesc* table, int
     return jb * TK + warp_count_below(off + int64_t(jb) * TK * 4, 4, TK, target, lane);
 }
 
+// t0 / t1 = first tile at or after `lo` / `hi` (as above), and the offset of the last tile of t1's row-block
+// (t1 lies strictly inside that row-block whenever the caller needs it).
+__device__ __forceinline__ void find_run(const TileDesc* table, int TN, int TK, uint32_t lo, uint32_t hi, int lane,
+                                         int& t0, int& t1, uint32_t& off_last) {
+    const uint32_t* off = &table[0].payload_off16;
+    int c0 = 0, c1 = 0;
+    for (int i = lane; i < TN; i += 32) {
+        const uint32_t v = __ldg(off + int64_t(i) * TK * 4);
+        c0 += v < lo;
+        c1 += v < hi;
+    }
+    const int nb0 = __reduce_add_sync(0xFFFFFFFFu, c0), nb1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+    const int jb0 = nb0 ? nb0 - 1 : 0, jb1 = nb1 ? nb1 - 1 : 0;
+    const uint32_t* row0 = off + int64_t(jb0) * TK * 4;
+    const uint32_t* row1 = off + int64_t(jb1) * TK * 4;
+    int d0 = 0, d1 = 0;
+    for (int i = lane; i < TK; i += 32) {
+        const uint32_t a = __ldg(row0 + i * 4), b = __ldg(row1 + i * 4);
+        d0 += a < lo;
+        d1 += b < hi;
+    }
+    off_last = __ldg(row1 + (TK - 1) * 4);
+    t0 = nb0 ? jb0 * TK + __reduce_add_sync(0xFFFFFFFFu, d0) : 0;
+    t1 = nb1 ? jb1 * TK + __reduce_add_sync(0xFFFFFFFFu, d1) : 0;
+}
+
 __device__ __forceinline__ unsigned long long atom_add_acq_rel_gpu(unsigned long long* p, unsigned long long v) {
     unsigned long long old;
     asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], %2;" : "=l"(old) : "l"(p), "l"(v) : "memory");
@@ -239,8 +265,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
         // byte-balanced run of tiles for this CTA
         const uint32_t lo = pay0_16 + uint32_t(uint64_t(c) * pay_total_16 / G);
         const uint32_t hi = pay0_16 + uint32_t(uint64_t(c + 1) * pay_total_16 / G);
-        const int t0 = first_tile_at_or_after(table, TN, TK, lo, lane);
-        const int t1 = (c + 1 == G) ? TN * TK : first_tile_at_or_after(table, TN, TK, hi, lane);
+        // Both ends of the run in two round trips to the table instead of five dependent ones: the row-block
+        // starts serve both searches, the two in-row-block searches and the look-up below are independent.
+        int t0, t1;
+        uint32_t off_last;      // payload offset of the last tile of the row-block in which the run ends
+        find_run(table, TN, TK, lo, hi, lane, t0, t1, off_last);
+        if (c + 1 == G) t1 = TN * TK;
         int n_others = -1;
         if constexpr (N_TOK == 16) {
             // Flagged-partials protocol: if this run ends inside a row-block whose first tile it
@@ -248,7 +278,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
             // to the owner of the row-block's last tile (inverse of the byte partition above).
             const int tn_b = (t1 - 1) / TK;
             if (t1 > t0 && t1 < (tn_b + 1) * TK && t0 <= tn_b * TK) {
-                const uint32_t d = table[(tn_b + 1) * TK - 1].payload_off16 - pay0_16;
+                const uint32_t d = off_last - pay0_16;
                 const int c_last = int(((uint64_t(d) + 1) * uint64_t(G) - 1) / pay_total_16);
                 n_others = c_last - c;
             }
