@@ -14,6 +14,8 @@
  *     prints or exits.  All argument validation happens on the host before any launch.
  *   - Pointers named *_dev are device pointers, *_host are host pointers.  The library
  *     allocates no device memory and keeps no global state; every buffer is the caller's.
+ *   - Entry points may be called from several host threads (on different streams or devices);
+ *     calls that share a workspace must be ordered on one stream.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
  *     and return; patch_pack and patch_gemm_host are the exceptions noted below.
  *   - Supported: tile_n = tile_k = 128, N % 128 == 0, K % 128 == 0, device pointers 16-byte
