@@ -17,7 +17,7 @@
  *   - Entry points may be called from several host threads (on different streams or devices);
  *     calls that share a workspace must be ordered on one stream.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
- *     and return; patch_pack and patch_gemm_host are the exceptions noted below.
+ *     and return; patch_pack, patch_gemm_host and patch_gemm_host_batch are the exceptions noted below.
  *   - Supported: tile_n = tile_k = 128, N % 128 == 0, K % 128 == 0, device pointers 16-byte
  *     aligned, leading dimensions multiples of 8 elements.  Device must be sm_100
  *     (PATCH_ERR_ARCH otherwise; there is no fallback path).
@@ -207,6 +207,27 @@ int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* layout,
                     const void* packed_dev, void* Y_host,
                     void* X_stage_dev, void* Y_stage_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
+ * The same for a whole step of GEMMs with ONE synchronisation: all activations are copied to
+ * the device first, then all GEMMs are launched back to back, then all results are copied
+ * back, then `stream` is synchronised.  Because every copy of an X precedes every launch, the
+ * launches carry PATCH_GEMM_INPUT_STATIC whenever `weights_static` is non-zero (the caller's
+ * promise that no packed weight is written on this stream meanwhile).  Jobs are independent:
+ * no job's X_stage_dev, Y_stage_dev or Y_host may alias another's; jobs may share a workspace.
+ */
+typedef struct {
+    const void* X_host;             /* bf16 [M x K] contiguous */
+    int64_t M;
+    const patch_layout_t* layout;
+    const void* packed_dev;
+    void* Y_host;                   /* bf16 [M x N] contiguous */
+    void* X_stage_dev;              /* M*K bf16 */
+    void* Y_stage_dev;              /* M*N bf16 */
+    void* workspace_dev;
+    size_t workspace_bytes;
+} patch_host_job_t;
+int patch_gemm_host_batch(const patch_host_job_t* jobs, int n_jobs, int weights_static, void* stream);
 
 /*
  * patch_gemm for callers that cannot allocate device memory.  (The paper has no counterpart;

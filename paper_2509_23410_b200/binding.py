@@ -24,7 +24,7 @@ ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
-           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host",
+           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch",
            "patch_gemm_noalloc",
            "patch_strerror", "patch_version"]
 
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.patch_gemm_gated_workspace_size.argtypes = [ctypes.POINTER(Layout), i64, ctypes.POINTER(sz)]
         L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
         L.patch_gemm_noalloc.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp]
+        L.patch_gemm_host_batch.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp]
         L.patch_strerror.argtypes = [ctypes.c_int]
         L.patch_strerror.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -200,6 +201,31 @@ def patch_gemm_host(X_host, layout: Layout, packed, Y_host, X_stage, Y_stage, wo
                                  _ptr(X_stage), _ptr(Y_stage), _ptr(workspace), ws_bytes, _stream(stream)),
            "patch_gemm_host")
     return Y_host
+
+
+class HostJob(ctypes.Structure):
+    """Mirror of ``patch_host_job_t``."""
+    _fields_ = [("X_host", ctypes.c_void_p), ("M", ctypes.c_int64), ("layout", ctypes.POINTER(Layout)),
+                ("packed_dev", ctypes.c_void_p), ("Y_host", ctypes.c_void_p), ("X_stage_dev", ctypes.c_void_p),
+                ("Y_stage_dev", ctypes.c_void_p), ("workspace_dev", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
+def make_host_batch(jobs):
+    """Marshal a list of dicts (Xh, layout, packed, Yh, X, Y, ws) once; the arrays must outlive the result."""
+    arr = (HostJob * len(jobs))()
+    for a, j in zip(arr, jobs):
+        a.X_host, a.M, a.layout = j["Xh"].data_ptr(), j["Xh"].shape[0], ctypes.pointer(j["layout"])
+        a.packed_dev, a.Y_host = j["packed"].data_ptr(), j["Yh"].data_ptr()
+        a.X_stage_dev, a.Y_stage_dev = j["X"].data_ptr(), j["Y"].data_ptr()
+        ws = j.get("ws")
+        a.workspace_dev, a.workspace_bytes = (ws.data_ptr(), ws.numel()) if ws is not None else (None, 0)
+    return arr
+
+
+def patch_gemm_host_batch(batch, weights_static: bool = False, stream=None):
+    """One step of GEMMs with host X / Y: all copies in, all launches, all copies out, one synchronisation."""
+    _check(lib().patch_gemm_host_batch(batch, len(batch), 1 if weights_static else 0, _stream(stream)),
+           "patch_gemm_host_batch")
 
 
 def patch_gemm_noalloc(X, layout: Layout, packed, Y, stream=None):

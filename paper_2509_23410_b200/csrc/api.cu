@@ -124,6 +124,40 @@ extern "C" int patch_gemm_host(const void* X_host, int64_t M, const patch_layout
     return cudaStreamSynchronize(s) == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
+extern "C" int patch_gemm_host_batch(const patch_host_job_t* jobs, int n_jobs, int weights_static, void* stream) {
+    if (n_jobs < 0) return PATCH_ERR_SHAPE;
+    if (n_jobs == 0) return PATCH_OK;
+    if (!jobs) return PATCH_ERR_NULL;
+    for (int i = 0; i < n_jobs; ++i) {      // everything is checked before anything is enqueued
+        const patch_host_job_t& j = jobs[i];
+        if (!j.layout) return PATCH_ERR_NULL;
+        int rc = validate_layout(j.layout);
+        if (rc) return rc;
+        if (j.M < 0) return PATCH_ERR_SHAPE;
+        if (j.M > 0 && (!j.X_host || !j.Y_host || !j.X_stage_dev || !j.Y_stage_dev || !j.packed_dev)) return PATCH_ERR_NULL;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n_jobs; ++i) {
+        const patch_host_job_t& j = jobs[i];
+        if (j.M && cudaMemcpyAsync(j.X_stage_dev, j.X_host, size_t(j.M) * j.layout->K * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return PATCH_ERR_CUDA;
+    }
+    // with two or more jobs the operation before any launch is another launch or the copy of a different X
+    const int flags = weights_static ? (PATCH_GEMM_WEIGHTS_STATIC | (n_jobs >= 2 ? PATCH_GEMM_INPUT_STATIC : 0)) : 0;
+    for (int i = 0; i < n_jobs; ++i) {
+        const patch_host_job_t& j = jobs[i];
+        int rc = patch_gemm_ex(j.X_stage_dev, j.layout->K, j.M, j.layout, j.packed_dev, j.Y_stage_dev, j.layout->N,
+                               j.workspace_dev, j.workspace_bytes, nullptr, stream, PATCH_VARIANT_AUTO | flags);
+        if (rc) return rc;
+    }
+    for (int i = 0; i < n_jobs; ++i) {
+        const patch_host_job_t& j = jobs[i];
+        if (j.M && cudaMemcpyAsync(j.Y_host, j.Y_stage_dev, size_t(j.M) * j.layout->N * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return PATCH_ERR_CUDA;
+    }
+    return cudaStreamSynchronize(s) == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
 extern "C" const char* patch_strerror(int status) {
     switch (status) {
         case PATCH_OK: return "ok";

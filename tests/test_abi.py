@@ -132,3 +132,23 @@ def test_gated_entry_validates_on_the_host():
     # workspace of the small-M schedule: past everything patch_gemm uses of a shared buffer, one slot per pair
     assert B.patch_gemm_gated_workspace_size(ok, 16) == B.patch_gemm_workspace_size(ok, 64) + 2 * 128 * 16 * 4
     assert B.patch_gemm_gated_workspace_size(ok, 17) == 0
+
+
+def test_host_batch_validates_before_enqueueing():
+    """patch_gemm_host_batch: an empty batch is a no-op, bad jobs are rejected on the host (no GPU here)."""
+    import ctypes
+    import numpy as np
+    from paper_2509_23410_b200 import binding as B
+    lib = B.lib()
+    assert lib.patch_gemm_host_batch(None, 0, 0, None) == 0
+    assert lib.patch_gemm_host_batch(None, 2, 0, None) == B.ERR_NULL
+    assert lib.patch_gemm_host_batch(None, -1, 0, None) == B.ERR_SHAPE
+    L = B.patch_packed_size(256, 256, np.zeros((2, 2), np.uint8))
+    jobs = (B.HostJob * 2)()
+    for j in jobs:
+        j.M, j.layout = 4, ctypes.pointer(L)          # every pointer NULL
+    assert lib.patch_gemm_host_batch(jobs, 2, 1, None) == B.ERR_NULL
+    jobs[1].M = -3
+    assert lib.patch_gemm_host_batch(jobs, 2, 1, None) == B.ERR_NULL      # job 0 is checked first
+    jobs[0].M = 0
+    assert lib.patch_gemm_host_batch(jobs, 2, 1, None) == B.ERR_SHAPE

@@ -553,3 +553,25 @@ def test_gated_and_plain_calls_share_a_workspace(gpu, oracle):
             ref = oracle.swiglu(oracle.gemm_f64(Xg, oracle.prune(W, flags))[0])
             check_parity(oracle, to_bits(Yg), ref, f"gated M={Mg} after plain M={M}")
             assert int(ws_gate.count_nonzero()) == 0
+
+
+def test_host_batch_entry_point(gpu, oracle):
+    """patch_gemm_host_batch: a step of GEMMs of mixed sizes with pinned host X / Y, one synchronisation."""
+    torch, B = gpu
+    jobs, refs = [], []
+    for i, (N, K, M, p) in enumerate([(1024, 768, 1, 0.5), (1792, 1280, 16, 0.3), (512, 2048, 48, 1.0), (768, 512, 300, 0.0)]):
+        W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=p, stream=("batch", i)), 51, M)
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        Xh = torch.from_numpy(np.ascontiguousarray(X).view(np.int16)).view(torch.bfloat16).pin_memory()
+        Yh = torch.zeros((M, N), dtype=torch.bfloat16).pin_memory()
+        ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+        jobs.append(dict(Xh=Xh, layout=L, packed=packed, Yh=Yh, X=torch.empty((M, K), dtype=torch.bfloat16, device="cuda"),
+                         Y=torch.empty((M, N), dtype=torch.bfloat16, device="cuda"), ws=ws))
+        refs.append(oracle.gemm_f64(X, oracle.prune(W, flags))[0])
+    batch = B.make_host_batch(jobs)
+    for weights_static in (False, True):
+        for j in jobs:
+            j["Yh"].zero_()
+        B.patch_gemm_host_batch(batch, weights_static=weights_static)      # returns after the stream is synchronised
+        for j, ref in zip(jobs, refs):
+            check_parity(oracle, j["Yh"].view(torch.int16).numpy().view(np.uint16), ref, "host batch")
