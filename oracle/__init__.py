@@ -35,7 +35,7 @@ def build(force: bool = False) -> str:
     """Compile the oracle with gcc (plain -O2, OpenMP over outputs, no fast-math)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
-               "-Wall", "-Wextra", "-o", _LIB, _SRC]
+               "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -48,6 +48,9 @@ def lib():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.oracle_num_threads.restype = ctypes.c_int
+        _lib.oracle_uniform.restype = ctypes.c_double
+        _lib.oracle_gumbel.restype = ctypes.c_double
+        _lib.oracle_regularizers.restype = ctypes.c_double
     return _lib
 
 
@@ -109,6 +112,19 @@ def pack(W, flags, tile_n=128, tile_k=128):
     blob = np.empty(L.total_bytes, np.uint8)
     _check(lib().oracle_pack(_p(W), _p(_flags(flags)), ctypes.byref(L), _p(blob),
                              ctypes.c_uint64(blob.nbytes)), "pack")
+    return blob, L
+
+
+def pack_patterns(W, flags, patterns, tile_n=128, tile_k=128):
+    """Canonical packed blob with the 2:4 mask given as one candidate index (row of S) per group."""
+    W = _u16(W)
+    N, K = W.shape
+    patterns = np.ascontiguousarray(patterns, dtype=np.uint8).reshape(-1)
+    assert patterns.size == N * K // 4
+    L = packed_size(N, K, flags, tile_n, tile_k)
+    blob = np.empty(L.total_bytes, np.uint8)
+    _check(lib().oracle_pack_patterns(_p(W), _p(_flags(flags)), _p(patterns), ctypes.byref(L), _p(blob),
+                                      ctypes.c_uint64(blob.nbytes)), "pack_patterns")
     return blob, L
 
 
@@ -180,6 +196,61 @@ def swiglu(Y_gu, block: int = 128) -> np.ndarray:
     with np.errstate(over="ignore"):
         out = g / (1.0 + np.exp(-g)) * u
     return out.reshape(M, N // 2).astype(np.float32)
+
+
+def uniform(seed, stream, idx) -> float:
+    return float(lib().oracle_uniform(ctypes.c_uint64(seed), ctypes.c_uint64(stream), ctypes.c_uint64(idx)))
+
+
+def gumbel(seed, stream, idx) -> float:
+    return float(lib().oracle_gumbel(ctypes.c_uint64(seed), ctypes.c_uint64(stream), ctypes.c_uint64(idx)))
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+def soft_mask(W, P_tile, P24, tau, kappa, seed=0, noise=True, tile_n=128, tile_k=128):
+    """Soft mask of Eq. 2-4 -> (Mt float64 [N x K], Mt (.) W as bf16 bits, sums[4] for Eq. 5)."""
+    W = _u16(W)
+    N, K = W.shape
+    P_tile, P24 = _f32(P_tile), _f32(P24)
+    assert P_tile.size == (N // tile_n) * (K // tile_k) and P24.shape == (6, N * K // 4)
+    Mt = np.empty((N, K), np.float64)
+    Wt = np.empty((N, K), np.uint16)
+    sums = np.empty(4, np.float64)
+    _check(lib().oracle_soft_mask(_p(W), ctypes.c_int64(N), ctypes.c_int64(K), _p(P_tile), _p(P24), tile_n, tile_k,
+                                  ctypes.c_double(tau), ctypes.c_double(kappa), ctypes.c_uint64(seed), int(bool(noise)),
+                                  _p(Mt), _p(Wt), _p(sums)), "soft_mask")
+    return Mt, Wt, sums
+
+
+def regularizers(sums, rho, lambda1, lambda2) -> float:
+    """The sparsity and weight regularisers of Eq. 5 from the per-matrix sums ([n x 4])."""
+    sums = np.ascontiguousarray(sums, dtype=np.float64).reshape(-1, 4)
+    return float(lib().oracle_regularizers(_p(sums), int(sums.shape[0]), ctypes.c_double(rho),
+                                           ctypes.c_double(lambda1), ctypes.c_double(lambda2)))
+
+
+def hard_mask(P_tile, P24, N, K, tile_n=128, tile_k=128):
+    """Algorithm 1's hard masks -> (tile flags uint8 [TN*TK], candidate index per group uint8 [N*K/4])."""
+    P_tile, P24 = _f32(P_tile), _f32(P24)
+    assert P_tile.size == (N // tile_n) * (K // tile_k) and P24.shape == (6, N * K // 4)
+    flags = np.empty(P_tile.size, np.uint8)
+    patterns = np.empty(N * K // 4, np.uint8)
+    _check(lib().oracle_hard_mask(_p(P_tile), _p(P24), ctypes.c_int64(N), ctypes.c_int64(K), tile_n, tile_k,
+                                  _p(flags), _p(patterns)), "hard_mask")
+    return flags, patterns
+
+
+def mask_patterns(N, K, flags, patterns, tile_n=128, tile_k=128) -> np.ndarray:
+    """Hard mask M* (uint8) with the 2:4 part given as candidate indices."""
+    patterns = np.ascontiguousarray(patterns, dtype=np.uint8).reshape(-1)
+    out = np.empty((N, K), np.uint8)
+    _check(lib().oracle_mask_patterns(ctypes.c_int64(N), ctypes.c_int64(K), _p(_flags(flags)), _p(patterns),
+                                      tile_n, tile_k, _p(out)), "mask_patterns")
+    return out
 
 
 def parity_metrics(Y_test_f32, Y_ref_f32):

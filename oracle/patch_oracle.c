@@ -18,10 +18,16 @@
  *     of the 4-bit quantisation table.
  *   - the linear layer itself, on the same bf16-rounded inputs, accumulated in double (and in
  *     plain fp32 as a cross-check) in k order.
+ *   - (last section of the file) the masks of the learning procedure: the Gumbel-softmax soft masks
+ *     of Eq. 2-4 with the noise of Eq. 1 drawn from a counter-based generator, the per-matrix sums
+ *     and the two regularisers of Eq. 5, the hard masks Algorithm 1 reads off the logits, and the
+ *     compression with that given 2:4 mask instead of the magnitude rule.
  *
  * Pins: every function here is pinned by tests that do not call it to produce their expected
  * value (brute force over the six patterns, closed-form byte counts, numpy matmul, round trips,
- * hand-written fixtures).  No function is "parity unpinned".
+ * hand-written fixtures; for the mask-learning part: scipy's softmax, closed forms, the
+ * Gumbel-max property, the tau -> 0 limit that joins soft and hard masks).  No function is
+ * "parity unpinned".
  *
  * Conventions: W is [N x K] row-major bf16 (uint16 bit patterns), N = out-features,
  * K = in-features; X is [M x K]; Y is [M x N].  flags[tn*TK + tk]: 0 = dense, 1 = 2:4.
@@ -201,8 +207,14 @@ static void write_header_and_table(const oracle_layout_t* L, const uint8_t* flag
     }
 }
 
-int oracle_pack(const uint16_t* W, const uint8_t* flags, const oracle_layout_t* L,
-                uint8_t* blob, uint64_t capacity) {
+/* S: the six 2:4 candidates ("Learnable 2:4 Mask": the matrix whose rows are the candidate masks).
+ * The paper does not print the row order; rows are taken in lexicographic order of the kept positions. */
+static const uint8_t S_24[6][4] = {
+    {1, 1, 0, 0}, {1, 0, 1, 0}, {1, 0, 0, 1}, {0, 1, 1, 0}, {0, 1, 0, 1}, {0, 0, 1, 1}};
+
+/* patterns == NULL: magnitude top-2 per group; otherwise group (n, g) keeps row patterns[n*K/4 + g] of S. */
+static int pack_impl(const uint16_t* W, const uint8_t* flags, const uint8_t* patterns,
+                     const oracle_layout_t* L, uint8_t* blob, uint64_t capacity) {
     if (!W || !flags || !L || !blob) return -1;
     if (L->magic != ORACLE_MAGIC || L->version != ORACLE_VERSION) return -7;
     if (capacity < L->total_bytes) return -6;
@@ -228,7 +240,13 @@ int oracle_pack(const uint16_t* W, const uint8_t* flags, const oracle_layout_t* 
                     for (int g = 0; g < tk_ / 4; ++g) {
                         const uint16_t* w = &W[(tn * tn_ + r) * K + tk * tk_ + 4 * g];
                         int keep[4], pos[2], cnt = 0;
-                        select_top2(w, keep);
+                        if (patterns) {
+                            uint8_t c = patterns[(tn * tn_ + r) * (K / 4) + (tk * tk_) / 4 + g];
+                            if (c > 5) return -4;
+                            for (int j = 0; j < 4; ++j) keep[j] = S_24[c][j];
+                        } else {
+                            select_top2(w, keep);
+                        }
                         for (int j = 0; j < 4; ++j) if (keep[j]) pos[cnt++] = j;
                         vals[r * (tk_ / 2) + 2 * g + 0] = w[pos[0]];
                         vals[r * (tk_ / 2) + 2 * g + 1] = w[pos[1]];
@@ -238,6 +256,19 @@ int oracle_pack(const uint16_t* W, const uint8_t* flags, const oracle_layout_t* 
             }
         }
     return 0;
+}
+
+int oracle_pack(const uint16_t* W, const uint8_t* flags, const oracle_layout_t* L,
+                uint8_t* blob, uint64_t capacity) {
+    return pack_impl(W, flags, NULL, L, blob, capacity);
+}
+
+/* The same compression with the 2:4 mask given (Algorithm 1: "select best 2:4 mask from P_2:4"),
+ * one candidate index per group of four; groups inside dense tiles ignore theirs. */
+int oracle_pack_patterns(const uint16_t* W, const uint8_t* flags, const uint8_t* patterns,
+                         const oracle_layout_t* L, uint8_t* blob, uint64_t capacity) {
+    if (!patterns) return -1;
+    return pack_impl(W, flags, patterns, L, blob, capacity);
 }
 
 /* Inverse of oracle_pack: canonical blob -> What [N x K]. */
@@ -394,5 +425,125 @@ int oracle_gemm_f64_rows(const uint16_t* X, int64_t K, const int64_t* rows, int6
             acc += (double)bf16_to_f32(X[m * K + k]) * (double)bf16_to_f32(What[n * K + k]);
         Y32[i] = (float)acc;
     }
+    return 0;
+}
+
+/* =========================================================================================== */
+/* Mask learning: soft masks (Eq. 1-4), the two regularisers of the loss (Eq. 5) and the hard   */
+/* mask read off the logits (Algorithm 1, the lines after the training loop).                   */
+/*                                                                                             */
+/* Layouts: P_tile [TN x TK] row-major, one logit per tile.  P_24 [6 x G] row-major with        */
+/* G = N*K/4 and group index n*(K/4) + g, so row c holds the logit of candidate c for every     */
+/* group ("P_2:4 in R^{6 x d1 d2 / 4}").                                                        */
+/* =========================================================================================== */
+#include <math.h>
+
+/* Counter-based uniform in (0, 1): 23 bits taken from a splitmix64-style mix of (seed, stream,
+ * idx), centred in their cell so that 0 and 1 never occur.  stream 0 = tile classes (idx = 2*t + class),
+ * stream 1 = 2:4 candidates (idx = c*G + group). */
+double oracle_uniform(uint64_t seed, uint64_t stream, uint64_t idx) {
+    uint64_t x = seed + 0x9E3779B97F4A7C15ull * (idx + 1) + 0xD1B54A32D192ED03ull * stream;
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27; x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return ((double)(x >> 41) + 0.5) / 8388608.0;
+}
+
+/* Gumbel noise z = -log(-log(u))  (Eq. 1). */
+double oracle_gumbel(uint64_t seed, uint64_t stream, uint64_t idx) {
+    return -log(-log(oracle_uniform(seed, stream, idx)));
+}
+
+/* GS(p; tau, kappa)_k = exp((kappa p_k + z_k)/tau) / sum_j exp((kappa p_j + z_j)/tau)  (Eq. 1 with the
+ * scaling factor kappa on the logits).  The largest exponent is subtracted from all of them first, which
+ * leaves the quotient unchanged and keeps exp() in range. */
+static void gumbel_softmax(const double* p, const double* z, int n, double tau, double kappa, double* out) {
+    double e[6], top = -INFINITY, sum = 0.0;
+    for (int k = 0; k < n; ++k) { e[k] = (kappa * p[k] + z[k]) / tau; if (e[k] > top) top = e[k]; }
+    for (int k = 0; k < n; ++k) { out[k] = exp(e[k] - top); sum += out[k]; }
+    for (int k = 0; k < n; ++k) out[k] /= sum;
+}
+
+/* Soft mask  Mt = Mt_tile + (1 - Mt_tile) (.) Mt_2:4  (Eq. 4) with
+ *   Mt_tile = GS([P_tile, 0])_0 broadcast over the tile (Eq. 3),
+ *   Mt_2:4  = GS(P_2:4) x S per group of four (Eq. 2),
+ * the masked weight Mt (.) W (double, and rounded once to bf16), and the four sums Eq. 5 needs from one
+ * matrix:  sums = { sum Mt, ||W||_0, ||Mt (.) W||_2^2, ||W||_2^2 }.
+ * use_noise == 0 drops z (all zeros).  Mt, Wt16 may be NULL. */
+int oracle_soft_mask(const uint16_t* W, int64_t N, int64_t K, const float* P_tile, const float* P24,
+                     int tile_n, int tile_k, double tau, double kappa, uint64_t seed, int use_noise,
+                     double* Mt, uint16_t* Wt16, double* sums) {
+    int rc = check_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    if (!W || !P_tile || !P24 || !sums) return -1;
+    if (!(tau > 0.0)) return -2;
+    int64_t TK = K / tile_k, G = N * (K / 4);
+    double s_m = 0.0, s_nz = 0.0, s_mw2 = 0.0, s_w2 = 0.0;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t g = 0; g < K / 4; ++g) {
+            int64_t t = (n / tile_n) * TK + (4 * g) / tile_k, grp = n * (K / 4) + g;
+            double p2[2] = {(double)P_tile[t], 0.0}, z2[2] = {0.0, 0.0}, gs2[2];
+            double p6[6], z6[6], gs6[6];
+            for (int c = 0; c < 6; ++c) { p6[c] = (double)P24[c * G + grp]; z6[c] = 0.0; }
+            if (use_noise) {
+                for (int c = 0; c < 2; ++c) z2[c] = oracle_gumbel(seed, 0, 2 * (uint64_t)t + c);
+                for (int c = 0; c < 6; ++c) z6[c] = oracle_gumbel(seed, 1, (uint64_t)c * G + grp);
+            }
+            gumbel_softmax(p2, z2, 2, tau, kappa, gs2);
+            gumbel_softmax(p6, z6, 6, tau, kappa, gs6);
+            for (int j = 0; j < 4; ++j) {
+                double m24 = 0.0;
+                for (int c = 0; c < 6; ++c) m24 += gs6[c] * S_24[c][j];
+                double m = gs2[0] + (1.0 - gs2[0]) * m24;
+                double w = (double)bf16_to_f32(W[n * K + 4 * g + j]), mw = m * w;
+                if (Mt) Mt[n * K + 4 * g + j] = m;
+                if (Wt16) Wt16[n * K + 4 * g + j] = f32_to_bf16_rne((float)mw);
+                s_m += m; s_nz += (w != 0.0); s_mw2 += mw * mw; s_w2 += w * w;
+            }
+        }
+    sums[0] = s_m; sums[1] = s_nz; sums[2] = s_mw2; sums[3] = s_w2;
+    return 0;
+}
+
+/* The two regularisers of Eq. 5 over matrices i = 0..n-1, from their per-matrix sums:
+ *   lambda1 * | sum_i sum(Mt_i) / sum_i ||W_i||_0 - rho |  -  lambda2 * sum_i ||Mt_i (.) W_i||^2 / sum_i ||W_i||^2 */
+double oracle_regularizers(const double* sums, int n, double rho, double lambda1, double lambda2) {
+    double a = 0, b = 0, c = 0, d = 0;
+    for (int i = 0; i < n; ++i) { a += sums[4 * i]; b += sums[4 * i + 1]; c += sums[4 * i + 2]; d += sums[4 * i + 3]; }
+    return lambda1 * fabs(a / b - rho) - lambda2 * (c / d);
+}
+
+/* Hard masks from the logits (Algorithm 1): tile t is dense iff P_tile[t] > 0 (flag 0), else 2:4 (flag 1);
+ * every group takes the candidate with the largest logit ("select best 2:4 mask"), the first of equals. */
+int oracle_hard_mask(const float* P_tile, const float* P24, int64_t N, int64_t K, int tile_n, int tile_k,
+                     uint8_t* flags, uint8_t* patterns) {
+    int rc = check_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    if (!P_tile || !P24 || !flags || !patterns) return -1;
+    int64_t T = (N / tile_n) * (K / tile_k), G = N * (K / 4);
+    for (int64_t t = 0; t < T; ++t) flags[t] = P_tile[t] > 0.0f ? KIND_DENSE : KIND_SPARSE;
+    for (int64_t grp = 0; grp < G; ++grp) {
+        int best = 0;
+        for (int c = 1; c < 6; ++c)
+            if (P24[c * G + grp] > P24[best * G + grp]) best = c;
+        patterns[grp] = (uint8_t)best;
+    }
+    return 0;
+}
+
+/* M* = M*_tile + (1 - M*_tile) (.) M*_2:4 with the 2:4 part given by candidate indices. */
+int oracle_mask_patterns(int64_t N, int64_t K, const uint8_t* flags, const uint8_t* patterns,
+                         int tile_n, int tile_k, uint8_t* mask) {
+    int rc = check_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    int64_t TK = K / tile_k;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t g = 0; g < K / 4; ++g) {
+            uint8_t c = patterns[n * (K / 4) + g];
+            if (c > 5) return -4;
+            int m_tile = flags[(n / tile_n) * TK + (4 * g) / tile_k] == KIND_DENSE;
+            for (int j = 0; j < 4; ++j)
+                mask[n * K + 4 * g + j] = (uint8_t)(m_tile + (1 - m_tile) * S_24[c][j]);
+        }
     return 0;
 }

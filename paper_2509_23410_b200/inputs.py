@@ -189,3 +189,28 @@ def make_case_inputs(case: dict, seed: int = MASTER_SEED, M: int | None = None):
     flags = case_flags(case, seed)
     X = activation(M, K, seed, *case["stream"], M)
     return W, flags, X
+
+
+# ---------------------------------------------------------------------------------------------
+# Mask-learning inputs (logits of Algorithm 1).  Draws only: no softmax, no masks here.
+
+ROLE_P_TILE, ROLE_P_24 = 5, 6
+LOGIT_STD = 0.014                # "Logits Init N(0, 0.014)" of the hyper-parameter table
+PRIOR_STRENGTH = 3.0             # "Prior(Strength) SparseGPT(3)"
+# (tau, kappa) at the start and at the end of the schedules of the hyper-parameter table
+SCHEDULE_START, SCHEDULE_END = (2.0, 25.0), (0.05, 350.0)
+
+
+def tile_logits(TN: int, TK: int, p_dense: float, seed: int, *stream) -> np.ndarray:
+    """P_tile [TN x TK] float32: N(0, LOGIT_STD^2) plus a prior of +-PRIOR_STRENGTH, positive
+    (dense) with probability ``p_dense`` -- the shape of the paper's prior-initialised logits."""
+    g = generator(seed, ROLE_P_TILE, *stream)
+    base = g.standard_normal(TN * TK, dtype=np.float32) * np.float32(LOGIT_STD)
+    sign = np.where(g.random(TN * TK) < p_dense, np.float32(1), np.float32(-1))
+    return (base + np.float32(PRIOR_STRENGTH) * sign).reshape(TN, TK).astype(np.float32)
+
+
+def pattern_logits(N: int, K: int, seed: int, *stream, std: float = LOGIT_STD) -> np.ndarray:
+    """P_2:4 [6 x N*K/4] float32 ~ N(0, std^2); row c = candidate c, column = n*(K/4) + g."""
+    g = generator(seed, ROLE_P_24, *stream)
+    return (g.standard_normal(6 * (N * K // 4), dtype=np.float32) * np.float32(std)).reshape(6, N * K // 4)
