@@ -438,15 +438,17 @@ int oracle_gemm_f64_rows(const uint16_t* X, int64_t K, const int64_t* rows, int6
 /* =========================================================================================== */
 #include <math.h>
 
-/* Counter-based uniform in (0, 1): 23 bits taken from a splitmix64-style mix of (seed, stream,
- * idx), centred in their cell so that 0 and 1 never occur.  stream 0 = tile classes (idx = 2*t + class),
- * stream 1 = 2:4 candidates (idx = c*G + group). */
+/* Counter-based uniform in (0, 1).  One 64-bit splitmix64-style mix of (seed, stream, idx / 2) serves two
+ * consecutive counters: the even one takes its top 23 bits, the odd one bits 9..31.  The 23 bits are
+ * centred in their cell, so 0 and 1 never occur and the value is exact in fp32.
+ * stream 0 = tile classes (idx = 2*t + class), stream 1 = 2:4 candidates (idx = c*G + group). */
 double oracle_uniform(uint64_t seed, uint64_t stream, uint64_t idx) {
-    uint64_t x = seed + 0x9E3779B97F4A7C15ull * (idx + 1) + 0xD1B54A32D192ED03ull * stream;
+    uint64_t x = seed + 0x9E3779B97F4A7C15ull * (idx / 2 + 1) + 0xD1B54A32D192ED03ull * stream;
     x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
     x ^= x >> 27; x *= 0x94D049BB133111EBull;
     x ^= x >> 31;
-    return ((double)(x >> 41) + 0.5) / 8388608.0;
+    uint64_t bits = (idx & 1) ? (x >> 9) & 0x7FFFFFull : x >> 41;
+    return ((double)bits + 0.5) / 8388608.0;
 }
 
 /* Gumbel noise z = -log(-log(u))  (Eq. 1). */
