@@ -440,6 +440,168 @@ def run_ours(args):
     print(json.dumps(out))
 
 
+# ---------------------------------------------------------------------------------------------
+# mask-learning workload: one training-forward evaluation of the soft masks of one transformer block
+
+
+MASK_BYTES_PER_ELEMENT = 10.0      # soft mask: 2 B of W + 6 B of 2:4 logits read, 2 B of masked weight written
+# warp instructions per group of four weights per lane of soft_mask_kernel<noise>, and its DRAM traffic per
+# algorithmic byte, from the ncu capture summarised in profiles/soft_mask_kernel_llama7b_block.md
+# (38 458 368 instructions for a 4096 x 4096 launch; 152.8 MB read + written against 167.8 MB)
+MASK_WARP_INST_PER_GROUP = 293.4
+MASK_TRAFFIC_RATIO = 0.91
+
+
+def run_masks(args):
+    """`--workload masks`: a step = patch_soft_mask (Gumbel noise on) over the seven linear weights of one
+    LLaMA-2-7B-shaped block (4 x 4096^2, 2 x 11008x4096, 4096x11008; 1.2 GB of logits per step, so every
+    byte comes from HBM).  Also times the no-noise variant, patch_hard_mask and patch_pack_patterns."""
+    import torch
+    from paper_2509_23410_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("the masks workload is a single-GPU measurement")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B.lib()
+    peaks = measured_peaks()
+    tau, kappa = 0.5, 120.0           # mid-schedule values between (2, 25) and (0.05, 350)
+    shapes = [(4096, 4096)] * 4 + [(11008, 4096)] * 2 + [(4096, 11008)]
+    mats = []
+    for i, (N, K) in enumerate(shapes):
+        W = torch.from_numpy(np.ascontiguousarray(inputs.weight(N, K, inputs.MASTER_SEED, "masks", i)).view(np.int16)).to(dev).view(torch.bfloat16)
+        PT = torch.from_numpy(inputs.tile_logits(N // 128, K // 128, 0.5, inputs.MASTER_SEED, "masks", i)).to(dev)
+        P6 = torch.from_numpy(inputs.pattern_logits(N, K, inputs.MASTER_SEED, "masks", i)).to(dev)
+        mats.append(dict(N=N, K=K, W=W, PT=PT, P6=P6, Wt=torch.empty_like(W),
+                         sums=torch.empty(4, dtype=torch.float64, device=dev),
+                         ws=torch.empty(B.patch_soft_mask_workspace_size(N, K), dtype=torch.uint8, device=dev),
+                         flags=torch.empty((N // 128) * (K // 128), dtype=torch.uint8, device=dev),
+                         patterns=torch.empty(N * K // 4, dtype=torch.uint8, device=dev)))
+    elements = sum(m["N"] * m["K"] for m in mats)
+
+    def soft(flags):
+        for i, m in enumerate(mats):
+            B.patch_soft_mask(m["W"], m["PT"], m["P6"], tau, kappa, 1000 + i, flags, Wt=m["Wt"], sums=m["sums"],
+                              workspace=m["ws"])
+
+    def hard():
+        for m in mats:
+            B.patch_hard_mask(m["PT"], m["P6"], m["N"], m["K"], flags_out=m["flags"], patterns_out=m["patterns"])
+
+    def graph_of(fn):
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            fn()
+        torch.cuda.current_stream().wait_stream(s)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g
+
+    def time_graph(g, reps, warm=3):
+        for _ in range(warm):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / reps
+
+    steps = min(args.steps, 200)
+    g_noise = graph_of(lambda: soft(0))
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    t0 = time.time()
+    step_s = time_graph(g_noise, steps, max(args.warmup, 3))
+    clocks = sampler.stop(t0, time.time())
+    t_plain = time_graph(graph_of(lambda: soft(B.MASK_NO_NOISE)), 50)
+    t_hard = time_graph(graph_of(hard), 50)
+    # packing with the hard masks just computed (flags go through the host, as the entry point requires)
+    hard()
+    torch.cuda.synchronize()
+    pk = []
+    for m in mats:
+        fl = m["flags"].cpu().numpy()
+        L = B.patch_packed_size(m["N"], m["K"], fl)
+        pk.append((m, fl, L, torch.empty(L.total_bytes, dtype=torch.uint8, device=dev)))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_pack, pack_bytes = 0.0, 0.0
+    for rep in range(4):
+        torch.cuda.synchronize()
+        e0.record()
+        for m, fl, L, out in pk:
+            B.patch_pack_patterns(m["W"], fl, m["patterns"], layout=L, out=out)
+        e1.record()
+        torch.cuda.synchronize()
+        if rep:
+            t_pack += e0.elapsed_time(e1) * 1e-3 / 3
+    pack_bytes = sum(m["N"] * m["K"] * 2.25 + L.total_bytes for m, fl, L, out in pk)
+    # end to end: logits and weights from pinned host memory every step, the four sums per matrix read back
+    host = [dict(W=m["W"].cpu().pin_memory(), PT=m["PT"].cpu().pin_memory(), P6=m["P6"].cpu().pin_memory(),
+                 sums=torch.empty(4, dtype=torch.float64).pin_memory()) for m in mats]
+    def e2e_step():
+        for m, h in zip(mats, host):
+            m["W"].copy_(h["W"], non_blocking=True)
+            m["PT"].copy_(h["PT"], non_blocking=True)
+            m["P6"].copy_(h["P6"], non_blocking=True)
+        soft(0)
+        for m, h in zip(mats, host):
+            h["sums"].copy_(m["sums"], non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_step()
+    tw = time.time()
+    for _ in range(3):
+        e2e_step()
+    e2e_s = (time.time() - tw) / 3
+    h2d = sum(h["W"].numel() * 2 + h["PT"].numel() * 4 + h["P6"].numel() * 4 for h in host)
+    reg = B.patch_mask_regularizers(np.stack([h["sums"].numpy() for h in host]), 0.75, 7.0, 10.0)
+    # the oracle on a bounded sample: one 1024 x 1024 matrix with noise
+    import oracle
+    Wc, PTc, P6c = inputs.weight(1024, 1024, 1, "masks-cpu"), inputs.tile_logits(8, 8, 0.5, 1, "masks-cpu"), \
+        inputs.pattern_logits(1024, 1024, 1, "masks-cpu")
+    tc = time.time()
+    oracle.soft_mask(Wc, PTc, P6c, tau, kappa, seed=1, noise=True)
+    tc = time.time() - tc
+    gbs = elements * MASK_BYTES_PER_ELEMENT / step_s / 1e9
+    winst = MASK_WARP_INST_PER_GROUP * elements / 4 / 32           # warp instructions per step
+    alu_peak = 148 * 4 * (clocks.get("sm_mhz") or 1965.0) * 1e6    # warp instructions per second
+    out = {
+        "metric": "soft_mask_forward_effective_gbs", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "soft-mask forward (Eq. 2-5) of one llama2-7b block's seven linear weights, Gumbel noise on",
+                   "tau": tau, "kappa": kappa, "elements": elements, "cuda_graph": True,
+                   "l2": "inputs larger than L2: 2.0 GB streamed per step"},
+        # with the noise on the kernel is bound by instruction issue (integer mixes, two logarithms and one
+        # exponential per candidate): achieved = warp instructions per second, peak = 148 SMs x 4 schedulers x
+        # one warp instruction per clock at the SM clock sampled during the run
+        "roofline": {"bound": "alu", "achieved": winst / step_s / 1e9, "peak": alu_peak / 1e9, "unit": "Gwarp-inst/s",
+                     "frac": winst / step_s / alu_peak,
+                     "traffic": MASK_TRAFFIC_RATIO * elements * MASK_BYTES_PER_ELEMENT / len(mats),
+                     "kernel": "soft_mask_kernel<noise>", "hbm_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                     "peak_source": "148 x 4 x sampled SM clock; instructions per group from ncu"},
+        "soft_mask_no_noise": {"ms_per_step": t_plain * 1e3, "gbs": elements * MASK_BYTES_PER_ELEMENT / t_plain / 1e9,
+                               "frac_of_measured_hbm": elements * MASK_BYTES_PER_ELEMENT / t_plain / 1e9 / peaks["hbm_gbs"]},
+        "hard_mask": {"ms_per_step": t_hard * 1e3, "gbs": elements * 6.25 / t_hard / 1e9,
+                      "frac_of_measured_hbm": elements * 6.25 / t_hard / 1e9 / peaks["hbm_gbs"]},
+        "pack_patterns": {"ms_per_step": t_pack * 1e3, "gbs": pack_bytes / t_pack / 1e9,
+                          "note": "includes the host-built tile table and its copy, per matrix"},
+        "e2e": {"value": elements * MASK_BYTES_PER_ELEMENT / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": 32 * len(mats), "ms_per_step": e2e_s * 1e3},
+        "regularizers_of_last_step": reg,
+        "gpu_launches": steps * 2 * len(mats),
+        "clocks": clocks,
+        "cpu_baseline": {"value": 1024 * 1024 * MASK_BYTES_PER_ELEMENT / tc / 1e9, "unit": "GB/s", "cores": 1,
+                         "kind": "oracle", "sample": "one 1024x1024 matrix, noise on"},
+    }
+    print(json.dumps(out))
+
+
 def workload_label(args):
     return {"13b": "llama2-13b linears", "stack": f"llama2-7b full linear stack, M={args.stack_m}",
             "stack-fused": f"llama2-7b full linear stack with q/k/v and gate/up stacked, M={args.stack_m}",
@@ -467,7 +629,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused", "masks"])
     ap.add_argument("--stack-m", type=int, default=1, help="tokens per GEMM of the 224-GEMM stack workload")
     ap.add_argument("--launch", default="independent", choices=["dependent", "independent"],
                     help="independent (default; true for this workload, whose GEMMs do not feed each other): "
@@ -477,7 +639,12 @@ def main():
     ap.add_argument("--detail", action="store_true", help="add the per-GEMM table (us, TFLOP/s, roofline fraction)")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "masks":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the masks workload reports the oracle in its cpu_baseline key"}))
+        else:
+            run_masks(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

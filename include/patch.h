@@ -256,6 +256,82 @@ int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M,
                        const patch_layout_t* layout, const void* packed_dev,
                        void* Y_dev, int64_t ldy, void* stream);
 
+/* =========================================================================================
+ * Mask learning (the training side of Algorithm 1): soft masks, regulariser sums, hard masks.
+ *
+ * Logit layouts (fp32, device): P_tile [N/128 x K/128] row-major, one logit per tile;
+ * P_24 [6 x G] row-major with G = N*K/4 and group index n*(K/4) + g, i.e. row c holds the
+ * logit of candidate c for every group of four ("P_2:4 in R^{6 x d1 d2 / 4}").  The six
+ * candidates (the rows of the matrix S of the 2:4 paragraph) are taken in lexicographic
+ * order of the kept positions: 0:(0,1) 1:(0,2) 2:(0,3) 3:(1,2) 4:(1,3) 5:(2,3).
+ * ========================================================================================= */
+
+/* patch_soft_mask flag: drop the Gumbel noise (z = 0), e.g. for evaluation. */
+enum { PATCH_MASK_NO_NOISE = 1 };
+
+/*
+ * Hard masks read off the logits (Algorithm 1, the lines after the loop):
+ *   tile_flags_dev[t] = PATCH_TILE_DENSE if P_tile[t] > 0 else PATCH_TILE_SPARSE_2_4
+ *                       ("positive values correspond to the dense option"; 0 and NaN are not positive);
+ *   patterns_dev[grp] = index of the largest of the group's six logits, the first of equals
+ *                       ("select best 2:4 mask from P_2:4").
+ *   tile_flags_dev  u8 [N/128 x K/128];  patterns_dev  u8 [N x K/4], 16-byte aligned.
+ * One kernel, no host synchronisation.  The flags must be copied to the host by the caller
+ * before patch_packed_size / patch_pack_patterns, which take them as host arrays.
+ */
+int patch_hard_mask(const float* P_tile_dev, const float* P24_dev, int64_t N, int64_t K,
+                    int tile_n, int tile_k, uint8_t* tile_flags_dev, uint8_t* patterns_dev,
+                    void* stream);
+
+/*
+ * patch_pack with the 2:4 mask given instead of chosen by magnitude (the deployment input of
+ * a learned or otherwise precomputed mask): in every 2:4 tile, group (n, g) keeps the two
+ * positions of candidate patterns_dev[n*(K/4) + g]; groups inside dense tiles ignore theirs.
+ *   patterns_dev  u8 [N x K/4] device, 4-byte aligned, values 0..5
+ *   status_dev    optional device int (caller zeroes it): set to PATCH_ERR_FLAG if a 2:4 tile
+ *                 holds an index above 5 (that group is then packed as candidate 0)
+ * Everything else as for patch_pack.
+ */
+int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t* tile_flags_host,
+                        const uint8_t* patterns_dev, const patch_layout_t* layout, void* packed_dev,
+                        size_t packed_capacity, int* status_dev, void* stream);
+
+/* Scratch bytes of patch_soft_mask: four doubles per tile. */
+int patch_soft_mask_workspace_size(int64_t N, int64_t K, int tile_n, int tile_k, size_t* bytes_out);
+
+/*
+ * One training-forward evaluation of the soft mask of a matrix and of everything Eq. 5 needs from it:
+ *   Mt_tile = GS([P_tile, 0]; tau, kappa)_0, one value per tile                     (Eq. 3)
+ *   Mt_2:4  = GS(P_2:4; tau, kappa) x S, four values per group                     (Eq. 2)
+ *   Mt      = Mt_tile + (1 - Mt_tile) (.) Mt_2:4                                    (Eq. 4)
+ *   Wt_dev  = Mt (.) W, rounded once to bf16 [N x ldo] -- the weight the language-model loss runs on
+ *   sums_dev[4] = { sum Mt, ||W||_0, ||Mt (.) W||_2^2 (before rounding), ||W||_2^2 }, doubles
+ * with GS(p)_k = exp((kappa p_k + z_k)/tau) / sum_j exp((kappa p_j + z_j)/tau), z = -log(-log(u)) (Eq. 1).
+ * The noise is drawn on the device from a counter-based generator keyed by `seed`, so that a
+ * call is reproducible and needs no noise buffers: u = (b + 0.5) / 2^23 with b 23 bits of
+ * x = mix(seed + 0x9E3779B97F4A7C15 * (i/2 + 1) + 0xD1B54A32D192ED03 * stream), mix = the
+ * splitmix64 finaliser (x ^= x >> 30, *= 0xBF58476D1CE4E5B9, ^= x >> 27, *= 0x94D049BB133111EB,
+ * ^= x >> 31); even counters i take b = x >> 41, odd ones b = (x >> 9) & 0x7FFFFF; stream 0,
+ * i = 2 t + class for the tiles (class 0 = dense); stream 1, i = c G + group for the candidates.
+ *   tau > 0, kappa finite; flags = 0 or PATCH_MASK_NO_NOISE
+ *   Mt_dev        optional fp32 [N x ldm] (ldm % 4 == 0): the soft mask itself, e.g. for a backward pass
+ *   workspace_dev at least patch_soft_mask_workspace_size bytes, 8-byte aligned; no initialisation needed
+ * Arithmetic is fp32 (sums: fp32 within a thread's 64 elements, double above that, in a fixed
+ * order: the result does not depend on scheduling).  Two kernels, no host synchronisation.
+ */
+int patch_soft_mask(const void* W_dev, int64_t ldw, const float* P_tile_dev, const float* P24_dev,
+                    int64_t N, int64_t K, int tile_n, int tile_k, float tau, float kappa, uint64_t seed,
+                    int flags, void* Wt_dev, int64_t ldo, float* Mt_dev, int64_t ldm, double* sums_dev,
+                    void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
+ * The two regularisers of Eq. 5 from the sums of n matrices (host arrays, [n x 4] as written by
+ * patch_soft_mask): lambda1 * | sum_i sum(Mt_i) / sum_i ||W_i||_0 - rho | - lambda2 * sum_i ||Mt_i (.) W_i||^2 / sum_i ||W_i||^2.
+ * Host only.
+ */
+int patch_mask_regularizers(const double* sums_host, int n, double rho, double lambda1, double lambda2,
+                            double* out_host);
+
 /* Human-readable text for a status code (static storage). */
 const char* patch_strerror(int status);
 

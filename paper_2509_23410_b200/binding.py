@@ -26,7 +26,10 @@ ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
            "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch",
            "patch_gemm_noalloc",
+           "patch_hard_mask", "patch_pack_patterns", "patch_soft_mask_workspace_size", "patch_soft_mask",
+           "patch_mask_regularizers",
            "patch_strerror", "patch_version"]
+MASK_NO_NOISE = 1
 
 
 class Layout(ctypes.Structure):
@@ -69,6 +72,13 @@ def lib() -> ctypes.CDLL:
         L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
         L.patch_gemm_noalloc.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp]
         L.patch_gemm_host_batch.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp]
+        L.patch_hard_mask.argtypes = [vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp]
+        L.patch_pack_patterns.argtypes = [vp, i64, vp, vp, ctypes.POINTER(Layout), vp, sz, vp, vp]
+        L.patch_soft_mask_workspace_size.argtypes = [i64, i64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(sz)]
+        L.patch_soft_mask.argtypes = [vp, i64, vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                      ctypes.c_float, ctypes.c_uint64, ctypes.c_int, vp, i64, vp, i64, vp, vp, sz, vp]
+        L.patch_mask_regularizers.argtypes = [vp, ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                              ctypes.POINTER(ctypes.c_double)]
         L.patch_strerror.argtypes = [ctypes.c_int]
         L.patch_strerror.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -241,3 +251,77 @@ def patch_gemm_noalloc(X, layout: Layout, packed, Y, stream=None):
 
 def patch_version() -> int:
     return int(lib().patch_version())
+
+
+# ---------------------------------------------------------------------------------------------
+# Mask learning: hard masks from logits, packing with a given 2:4 mask, soft-mask forward.
+
+
+def patch_hard_mask(P_tile, P24, N: int, K: int, flags_out=None, patterns_out=None, stream=None):
+    """Tile flags (uint8 [N/128 * K/128]) and candidate index per group (uint8 [N * K/4]) from the logits."""
+    import torch
+    assert P_tile.is_cuda and P_tile.dtype == torch.float32 and P_tile.is_contiguous()
+    assert P24.is_cuda and P24.dtype == torch.float32 and P24.is_contiguous() and tuple(P24.shape) == (6, N * K // 4)
+    if flags_out is None:
+        flags_out = torch.empty((N // 128) * (K // 128), dtype=torch.uint8, device=P24.device)
+    if patterns_out is None:
+        patterns_out = torch.empty(N * K // 4, dtype=torch.uint8, device=P24.device)
+    _check(lib().patch_hard_mask(_ptr(P_tile), _ptr(P24), N, K, 128, 128, _ptr(flags_out), _ptr(patterns_out),
+                                 _stream(stream)), "patch_hard_mask")
+    return flags_out, patterns_out
+
+
+def patch_pack_patterns(W, flags, patterns, layout: Layout | None = None, out=None, status=None, stream=None):
+    """patch_pack with the 2:4 mask given as candidate indices (uint8 CUDA tensor [N * K/4])."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    assert patterns.is_cuda and patterns.dtype == torch.uint8 and patterns.is_contiguous()
+    N, K = W.shape
+    assert patterns.numel() == N * K // 4
+    if layout is None:
+        layout = patch_packed_size(N, K, flags)
+    if out is None:
+        out = torch.empty(layout.total_bytes, dtype=torch.uint8, device=W.device)
+    f, fp = _flags_buf(flags)
+    _check(lib().patch_pack_patterns(_ptr(W), W.stride(0), fp, _ptr(patterns), ctypes.byref(layout), _ptr(out),
+                                     out.numel(), _ptr(status), _stream(stream)), "patch_pack_patterns")
+    return out, layout
+
+
+def patch_soft_mask_workspace_size(N: int, K: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().patch_soft_mask_workspace_size(N, K, 128, 128, ctypes.byref(n)), "patch_soft_mask_workspace_size")
+    return int(n.value)
+
+
+def patch_soft_mask(W, P_tile, P24, tau: float, kappa: float, seed: int = 0, flags: int = 0, Wt=None, Mt=None,
+                    sums=None, workspace=None, stream=None):
+    """Soft-mask forward of one matrix: returns (Wt bf16 [N x K], sums float64 CUDA tensor [4]);
+    pass a float32 ``Mt`` [N x K] to also get the soft mask itself."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    N, K = W.shape
+    assert P_tile.is_cuda and P_tile.dtype == torch.float32 and P_tile.is_contiguous()
+    assert P24.is_cuda and P24.dtype == torch.float32 and P24.is_contiguous() and tuple(P24.shape) == (6, N * K // 4)
+    if Wt is None:
+        Wt = torch.empty((N, K), dtype=torch.bfloat16, device=W.device)
+    if sums is None:
+        sums = torch.empty(4, dtype=torch.float64, device=W.device)
+    if workspace is None:
+        workspace = torch.empty(patch_soft_mask_workspace_size(N, K), dtype=torch.uint8, device=W.device)
+    assert Mt is None or (Mt.is_cuda and Mt.dtype == torch.float32 and Mt.stride(1) == 1)
+    _check(lib().patch_soft_mask(_ptr(W), W.stride(0), _ptr(P_tile), _ptr(P24), N, K, 128, 128, float(tau),
+                                 float(kappa), int(seed) & 0xFFFFFFFFFFFFFFFF, int(flags), _ptr(Wt), Wt.stride(0),
+                                 _ptr(Mt), Mt.stride(0) if Mt is not None else 0, _ptr(sums), _ptr(workspace),
+                                 workspace.numel(), _stream(stream)), "patch_soft_mask")
+    return Wt, sums
+
+
+def patch_mask_regularizers(sums, rho: float, lambda1: float, lambda2: float) -> float:
+    """The two regularisers of Eq. 5 from per-matrix sums (host array-like [n x 4])."""
+    import numpy as np
+    a = np.ascontiguousarray(sums, dtype=np.float64).reshape(-1, 4)
+    out = ctypes.c_double(0.0)
+    _check(lib().patch_mask_regularizers(ctypes.c_void_p(a.ctypes.data), int(a.shape[0]), float(rho), float(lambda1),
+                                         float(lambda2), ctypes.byref(out)), "patch_mask_regularizers")
+    return float(out.value)

@@ -70,10 +70,17 @@ __device__ __forceinline__ uint32_t top2_of_4(const uint32_t w[4], uint32_t& v0,
     return i0 | (i1 << 2);
 }
 
+// The two kept positions of candidate c (row c of the matrix S of the six 2:4 masks, rows in
+// lexicographic order of the kept positions) as the position code i0 | (i1 << 2), one nibble per candidate.
+constexpr uint32_t kCandidateCodes = 0xED9C84u;
+
 // One CTA per tile.  W is read with 16-byte loads, the payload is written with 16-byte stores.
+// GIVEN: the 2:4 mask comes from `patterns` (one candidate index per group of four, [N x K/4]
+// row-major) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
+template <bool GIVEN>
 __global__ void __launch_bounds__(256)
 pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob,
-            uint64_t table_off) {
+            uint64_t table_off, const uint8_t* __restrict__ patterns, int* status) {
     const int t = blockIdx.x;
     const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
     const int tn = t / TK, tk = t - tn * TK;
@@ -95,13 +102,26 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
             const uint16_t* src = wt + int64_t(r) * ldw + u * 16;
             const uint4 a = ld_stream(src), b = ld_stream(src + 8);
             const uint32_t in[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-            uint32_t out[4], code = 0;
+            uint32_t out[4], code = 0, given = 0;
+            if (GIVEN)   // the four candidate indices of this thread's groups: one aligned 4-byte load
+                given = *reinterpret_cast<const uint32_t*>(patterns + (int64_t(tn) * kTile + r) * (int64_t(TK) * 32) +
+                                                           tk * 32 + u * 4);
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 const uint32_t w[4] = {in[2 * g] & 0xFFFFu, in[2 * g] >> 16,
                                        in[2 * g + 1] & 0xFFFFu, in[2 * g + 1] >> 16};
-                uint32_t v0, v1;
-                code |= top2_of_4(w, v0, v1) << (4 * g);
+                uint32_t v0, v1, nib;
+                if (GIVEN) {
+                    uint32_t c = (given >> (8 * g)) & 0xFFu;
+                    if (c > 5u) { if (status) *status = PATCH_ERR_FLAG; c = 0; }
+                    nib = (kCandidateCodes >> (4 * c)) & 0xFu;
+                    const uint32_t i0 = nib & 3u, i1 = nib >> 2;
+                    v0 = i0 == 0 ? w[0] : i0 == 1 ? w[1] : w[2];
+                    v1 = i1 == 1 ? w[1] : i1 == 2 ? w[2] : w[3];
+                } else {
+                    nib = top2_of_4(w, v0, v1);
+                }
+                code |= nib << (4 * g);
                 out[g] = v0 | (v1 << 16);
             }
             *reinterpret_cast<uint4*>(pay + atom_chunk_offset(r, u)) = make_uint4(out[0], out[1], out[2], out[3]);
@@ -186,8 +206,8 @@ extern "C" int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
     return PATCH_OK;
 }
 
-extern "C" int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* flags,
-                          const patch_layout_t* L, void* packed_dev, size_t capacity, void* stream) {
+static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const uint8_t* patterns_dev,
+                     const patch_layout_t* L, void* packed_dev, size_t capacity, int* status_dev, void* stream) {
     if (!W_dev || !flags || !L || !packed_dev) return PATCH_ERR_NULL;
     int rc = validate_layout(L);
     if (rc) return rc;
@@ -217,9 +237,27 @@ extern "C" int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* flags,
     // pageable source: the runtime stages it before returning, so `head` may die at scope exit
     if (cudaMemcpyAsync(packed_dev, head.data(), head.size(), cudaMemcpyHostToDevice, s) != cudaSuccess)
         return PATCH_ERR_CUDA;
-    pack_kernel<<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
-                                            static_cast<uint8_t*>(packed_dev), L->table_off);
+    if (patterns_dev)
+        pack_kernel<true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                      static_cast<uint8_t*>(packed_dev), L->table_off, patterns_dev,
+                                                      status_dev);
+    else
+        pack_kernel<false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                       static_cast<uint8_t*>(packed_dev), L->table_off, nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* flags,
+                          const patch_layout_t* L, void* packed_dev, size_t capacity, void* stream) {
+    return pack_impl(W_dev, ldw, flags, nullptr, L, packed_dev, capacity, nullptr, stream);
+}
+
+extern "C" int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t* flags, const uint8_t* patterns_dev,
+                                   const patch_layout_t* L, void* packed_dev, size_t capacity, int* status_dev,
+                                   void* stream) {
+    if (!patterns_dev) return PATCH_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(patterns_dev) & 3u) return PATCH_ERR_ALIGN;
+    return pack_impl(W_dev, ldw, flags, patterns_dev, L, packed_dev, capacity, status_dev, stream);
 }
 
 extern "C" int patch_unpack(const patch_layout_t* L, const void* packed_dev, void* What_dev,

@@ -152,3 +152,30 @@ def test_host_batch_validates_before_enqueueing():
     assert lib.patch_gemm_host_batch(jobs, 2, 1, None) == B.ERR_NULL      # job 0 is checked first
     jobs[0].M = 0
     assert lib.patch_gemm_host_batch(jobs, 2, 1, None) == B.ERR_SHAPE
+
+
+def test_mask_entry_points_validate_on_the_host():
+    """Shape, tile, pointer and alignment errors of the mask entry points are reported before any device is touched."""
+    import ctypes
+    from paper_2509_23410_b200 import binding as B
+    lib = B.lib()
+    buf = (ctypes.c_double * 64)()
+    p = ctypes.addressof(buf)
+    assert lib.patch_hard_mask(p, p, 128, 100, 128, 128, p, p, None) == B.ERR_SHAPE
+    assert lib.patch_hard_mask(p, p, 128, 128, 128, 64, p, p, None) == B.ERR_TILE
+    assert lib.patch_hard_mask(None, p, 128, 128, 128, 128, p, p, None) == B.ERR_NULL
+    n = ctypes.c_size_t(0)
+    assert lib.patch_soft_mask_workspace_size(4096, 11008, 128, 128, ctypes.byref(n)) == 0
+    assert n.value == 32 * 86 * 32
+    assert lib.patch_soft_mask_workspace_size(4096, 11000, 128, 128, ctypes.byref(n)) == B.ERR_SHAPE
+    assert lib.patch_soft_mask(p, 128, p, p, 128, 128, 128, 128, -1.0, 1.0, 0, 0, p, 128, None, 0, p, p, 128, None) == B.ERR_SHAPE
+    assert lib.patch_soft_mask(p, 120, p, p, 128, 128, 128, 128, 1.0, 1.0, 0, 0, p, 128, None, 0, p, p, 128, None) == B.ERR_SHAPE
+    assert lib.patch_soft_mask(p, 128, p, p, 128, 128, 128, 128, 1.0, 1.0, 0, 0, p, 128, None, 0, p, p, 16, None) == B.ERR_SIZE
+    assert lib.patch_pack_patterns(p, 128, p, None, None, p, 0, None, None) == B.ERR_NULL
+    # the regularisers: 7 |75/100 - 1/2| - 10 * 30/60, and pooled sums over two matrices
+    assert B.patch_mask_regularizers([[75, 100, 30, 60]], 0.5, 7, 10) == -3.25
+    two = [[10, 40, 1, 4], [50, 60, 5, 6]]
+    assert abs(B.patch_mask_regularizers(two, 0.9, 3, 0.1) - (3 * abs(60 / 100 - 0.9) - 0.1 * 6 / 10)) < 1e-15
+    out = ctypes.c_double(0)
+    assert lib.patch_mask_regularizers(p, 0, 0.5, 1.0, 1.0, ctypes.byref(out)) == B.ERR_SHAPE
+    assert lib.patch_mask_regularizers(p, 1, 0.5, 1.0, 1.0, ctypes.byref(out)) == B.ERR_SHAPE   # all-zero sums: no weights

@@ -1,0 +1,236 @@
+"""GPU parity of the mask-learning entry points (hard masks, packing with a given 2:4 mask, the
+soft-mask forward and its sums) against the CPU oracle on the same seeded inputs.
+
+Integer and byte results are compared bit for bit.  The soft mask is fp32 arithmetic on the
+device against double in the oracle: with the exponents (kappa p + z) / tau reaching a few
+hundred at the end of the schedule, fp32 rounding of the exponent and the hardware logarithm
+leave a relative error of up to a few 1e-4 in a softmax term, hence |dMt| <= 1e-3; the masked
+weight is that times w, rounded to bf16 (one more 2^-9 relative)."""
+import numpy as np
+import pytest
+
+from paper_2509_23410_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+MT_TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("no CUDA device: GPU tests must run on a B200")
+    from paper_2509_23410_b200 import binding
+    binding.lib()
+    return torch, binding
+
+
+def to_dev(torch, bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def to_bits(t):
+    import torch
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+f32 = inputs.bf16_bits_to_f32
+
+
+def logits(N, K, p_dense, seed, *stream, std=inputs.LOGIT_STD):
+    PT = inputs.tile_logits(N // 128, K // 128, p_dense, seed, *stream)
+    P6 = inputs.pattern_logits(N, K, seed, *stream, std=std)
+    return PT, P6
+
+
+# ---------------------------------------------------------------------------------------------
+# hard masks and packing with them
+
+
+@pytest.mark.parametrize("N,K", [(128, 128), (256, 384), (640, 256), (4096, 4096)])
+def test_hard_mask_bit_exact(gpu, oracle, N, K):
+    torch, B = gpu
+    PT, P6 = logits(N, K, 0.4, 21, "hard", N, K)
+    PT.reshape(-1)[0] = 0.0                     # not positive: 2:4
+    P6[:, 5] = 0.125                            # six-way tie -> candidate 0
+    P6[[1, 3], 17] = 9.0                        # two-way tie -> the lower index
+    P6[5, 33] = 7.0                             # last candidate wins
+    flags, patterns = B.patch_hard_mask(torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), N, K)
+    rf, rp = oracle.hard_mask(PT, P6, N, K)
+    assert (flags.cpu().numpy() == rf).all()
+    got = patterns.cpu().numpy()
+    assert (got == rp).all()
+    assert got[5] == 0 and got[17] == 1 and got[33] == 5 and got.max() <= 5
+
+
+@pytest.mark.parametrize("N,K,p", [(128, 128, 0.0), (256, 384, 0.5), (1024, 1024, 0.5), (4096, 4096, 0.3)])
+def test_pack_patterns_bit_exact(gpu, oracle, N, K, p):
+    torch, B = gpu
+    W = inputs.weight(N, K, 22, "pp", N, K)
+    W[::13, ::7] = 0
+    flags = inputs.tile_flags(N, K, 1.0 - p, 22, "pp", N, K)
+    patterns = inputs.generator(22, "pp", "patterns", N, K).integers(0, 6, N * K // 4).astype(np.uint8)
+    canon, Lo = oracle.pack_patterns(W, flags, patterns)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    packed, L = B.patch_pack_patterns(to_dev(torch, W), flags, torch.from_numpy(patterns).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert (L.n_dense, L.n_sparse, L.total_bytes) == (Lo.n_dense, Lo.n_sparse, Lo.total_bytes)
+    assert (packed.cpu().numpy() == oracle.device_image(canon)).all()
+    M = oracle.mask_patterns(N, K, flags, patterns)
+    assert (to_bits(B.patch_unpack(L, packed)) == np.where(M == 1, W, 0)).all()
+
+
+def test_pack_patterns_flags_a_bad_index(gpu, oracle):
+    torch, B = gpu
+    N, K = 256, 256
+    W = inputs.weight(N, K, 23, "bad")
+    flags = np.array([[1, 0], [0, 1]], np.uint8)
+    patterns = np.zeros(N * K // 4, np.uint8)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bad = patterns.copy()
+    bad[(3 * (K // 4)) + 40] = 9                 # row 3, group 40: inside the dense tile (0, 1) -> ignored
+    B.patch_pack_patterns(to_dev(torch, W), flags, torch.from_numpy(bad).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    bad[(3 * (K // 4)) + 4] = 6                  # inside the 2:4 tile (0, 0)
+    packed, L = B.patch_pack_patterns(to_dev(torch, W), flags, torch.from_numpy(bad).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_FLAG
+    # the offending group was packed as candidate 0, everything else is unaffected
+    canon, _ = oracle.pack_patterns(W, flags, patterns)
+    assert (packed.cpu().numpy() == oracle.device_image(canon)).all()
+
+
+@pytest.mark.parametrize("M", [1, 16, 300])
+def test_learned_mask_deployment_chain(gpu, oracle, M):
+    """logits -> hard masks -> packed blob -> GEMM, all on the device, against the oracle's chain."""
+    torch, B = gpu
+    N, K = 512, 768
+    W = inputs.weight(N, K, 24, "chain")
+    X = inputs.activation(M, K, 24, "chain", M)
+    PT, P6 = logits(N, K, 0.5, 24, "chain")
+    flags_d, patterns_d = B.patch_hard_mask(torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), N, K)
+    flags = flags_d.cpu().numpy()
+    packed, L = B.patch_pack_patterns(to_dev(torch, W), flags, patterns_d)
+    ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = to_bits(B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws, status=status))
+    assert int(status.item()) == 0
+    rf, rp = oracle.hard_mask(PT, P6, N, K)
+    assert 0 < rf.sum() < rf.size
+    What = oracle.unpack(oracle.pack_patterns(W, rf, rp)[0])
+    Y32, _ = oracle.gemm_f64(X, What)
+    relF, maxrel = oracle.parity_metrics(f32(Y), Y32)
+    assert relF <= 2e-3 and maxrel <= 1e-2, (relF, maxrel)
+
+
+# ---------------------------------------------------------------------------------------------
+# soft masks
+
+
+def run_soft(gpu, W, PT, P6, tau, kappa, seed, noise, want_mt=True, ld_pad=0):
+    torch, B = gpu
+    N, K = W.shape
+    Wd = to_dev(torch, W)
+    if ld_pad:
+        buf = torch.zeros((N, K + ld_pad), dtype=torch.bfloat16, device="cuda")
+        buf[:, :K] = Wd
+        Wd = buf[:, :K]
+    Mt = torch.full((N, K), -1.0, dtype=torch.float32, device="cuda") if want_mt else None
+    Wt, sums = B.patch_soft_mask(Wd, torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), tau, kappa, seed,
+                                 0 if noise else B.MASK_NO_NOISE, Mt=Mt)
+    torch.cuda.synchronize()
+    return to_bits(Wt), (Mt.cpu().numpy() if want_mt else None), sums.cpu().numpy()
+
+
+def check_soft(oracle, W, got_Wt, got_Mt, got_sums, ref):
+    rMt, rWt, rsums = ref
+    w = f32(W).astype(np.float64)
+    if got_Mt is not None:
+        assert np.abs(got_Mt - rMt).max() <= MT_TOL
+    dW = np.abs(f32(got_Wt).astype(np.float64) - rMt * w)
+    assert (dW <= np.abs(w) * (MT_TOL + 2.0 ** -8) + 1e-30).all()
+    assert (got_Wt == rWt).mean() > 0.97
+    assert got_sums[1] == rsums[1]                                  # ||W||_0 is a count
+    assert np.allclose(got_sums[[0, 2, 3]], rsums[[0, 2, 3]], rtol=2e-4)
+    assert abs(got_sums[3] - rsums[3]) <= 2e-6 * rsums[3]           # no softmax in ||W||^2
+
+
+@pytest.mark.parametrize("tau,kappa", [inputs.SCHEDULE_START, inputs.SCHEDULE_END, (0.6, 100.0)])
+@pytest.mark.parametrize("noise", [False, True])
+def test_soft_mask_parity(gpu, oracle, tau, kappa, noise):
+    N, K = 384, 640
+    W = inputs.weight(N, K, 31, "soft")
+    W[::11, ::5] = 0
+    PT, P6 = logits(N, K, 0.5, 31, "soft")
+    PT *= np.float32(0.004)       # tile values across (0, 1) instead of saturated ones
+    ref = oracle.soft_mask(W, PT, P6, tau, kappa, seed=77, noise=noise)
+    got = run_soft(gpu, W, PT, P6, tau, kappa, 77, noise)
+    check_soft(oracle, W, *got, ref)
+    # the same through a padded leading dimension and without the optional mask output
+    got2 = run_soft(gpu, W, PT, P6, tau, kappa, 77, noise, want_mt=False, ld_pad=24)
+    assert (got2[0] == got[0]).all() and (got2[2] == got[2]).all()
+
+
+def test_soft_mask_prior_initialised_tiles_and_seeds(gpu, oracle):
+    N, K = 256, 512
+    W = inputs.weight(N, K, 32, "soft2")
+    PT, P6 = logits(N, K, 0.5, 32, "soft2")          # +-3 prior: tiles saturate as kappa grows
+    tau, kappa = 1.0, 60.0
+    a = run_soft(gpu, W, PT, P6, tau, kappa, 1, True)
+    check_soft(oracle, W, *a, oracle.soft_mask(W, PT, P6, tau, kappa, seed=1, noise=True))
+    b = run_soft(gpu, W, PT, P6, tau, kappa, 2 ** 63 + 5, True)
+    check_soft(oracle, W, *b, oracle.soft_mask(W, PT, P6, tau, kappa, seed=2 ** 63 + 5, noise=True))
+    assert np.abs(a[1] - b[1]).max() > 0.1           # a different seed is a different draw
+    c = run_soft(gpu, W, PT, P6, tau, kappa, 1, True)
+    assert (a[0] == c[0]).all() and (a[1] == c[1]).all() and (a[2] == c[2]).all()     # reproducible, sums included
+
+
+def test_soft_mask_closed_form_and_hardening(gpu, oracle):
+    torch, B = gpu
+    N, K = 256, 256
+    W = inputs.weight(N, K, 33, "soft3")
+    # equal logits, zero tile logit, no noise: Mt = 3/4 everywhere
+    Wt, Mt, sums = run_soft(gpu, W, np.zeros((2, 2), np.float32), np.full((6, N * K // 4), 0.3, np.float32),
+                            0.7, 9.0, 0, False)
+    assert np.abs(Mt - 0.75).max() < 1e-6
+    assert abs(sums[0] - 0.75 * N * K) < 1e-3 * N * K
+    # tau -> 0 without noise: the soft mask becomes the hard mask of the same logits
+    PT = np.array([[2.5, -2.5], [-1.0, 4.0]], np.float32)
+    P6 = inputs.pattern_logits(N, K, 33, "soft3", std=1.0)
+    top = np.sort(P6, axis=0)
+    clear = np.repeat(((top[-1] - top[-2]) > 1e-2).reshape(N, K // 4), 4, axis=1)
+    Wt, Mt, _ = run_soft(gpu, W, PT, P6, 1e-3, 1.0, 0, False)
+    flags, patterns = B.patch_hard_mask(torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), N, K)
+    Mstar = oracle.mask_patterns(N, K, flags.cpu().numpy(), patterns.cpu().numpy())
+    assert clear.mean() > 0.95 and np.abs(Mt - Mstar)[clear].max() < 1e-3
+
+
+def test_soft_mask_full_size(gpu, oracle):
+    """The 4096 x 4096 shape the benchmark times, against the oracle over the whole matrix."""
+    N, K = 4096, 4096
+    W = inputs.weight(N, K, 34, "soft4")
+    PT, P6 = logits(N, K, 0.5, 34, "soft4")
+    PT *= np.float32(0.004)
+    tau, kappa = 0.5, 120.0
+    got = run_soft(gpu, W, PT, P6, tau, kappa, 12345, True)
+    check_soft(oracle, W, *got, oracle.soft_mask(W, PT, P6, tau, kappa, seed=12345, noise=True))
+
+
+def test_mask_entry_points_reject_bad_arguments(gpu):
+    torch, B = gpu
+    lib = B.lib()
+    z = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    p = z.data_ptr()
+    assert lib.patch_hard_mask(p, p, 128, 100, 128, 128, p, p, None) == B.ERR_SHAPE
+    assert lib.patch_hard_mask(p, p, 128, 128, 64, 128, p, p, None) == B.ERR_TILE
+    assert lib.patch_hard_mask(p, None, 128, 128, 128, 128, p, p, None) == B.ERR_NULL
+    assert lib.patch_hard_mask(p, p + 4, 128, 128, 128, 128, p, p, None) == B.ERR_ALIGN
+    args = lambda tau=1.0, ws=128, flags=0: (p, 128, p, p, 128, 128, 128, 128, tau, 1.0, 0, flags, p, 128, None, 0,
+                                             p, p, ws, None)
+    assert lib.patch_soft_mask(*args(tau=0.0)) == B.ERR_SHAPE
+    assert lib.patch_soft_mask(*args(tau=float("nan"))) == B.ERR_SHAPE
+    assert lib.patch_soft_mask(*args(ws=8)) == B.ERR_SIZE
+    assert lib.patch_soft_mask(*args(flags=4)) == B.ERR_SHAPE
