@@ -233,6 +233,30 @@ def regularizers(sums, rho, lambda1, lambda2) -> float:
                                            ctypes.c_double(lambda1), ctypes.c_double(lambda2)))
 
 
+def regularizer_coefficients(sums, rho, lambda1, lambda2):
+    """(c1, c2): how one element's soft-mask value enters the gradient of Eq. 5's two regularisers."""
+    sums = np.ascontiguousarray(sums, dtype=np.float64).reshape(-1, 4)
+    c1, c2 = ctypes.c_double(0), ctypes.c_double(0)
+    lib().oracle_regularizer_coefficients(_p(sums), int(sums.shape[0]), ctypes.c_double(rho), ctypes.c_double(lambda1),
+                                          ctypes.c_double(lambda2), ctypes.byref(c1), ctypes.byref(c2))
+    return float(c1.value), float(c2.value)
+
+
+def soft_mask_backward(W, P_tile, P24, tau, kappa, Gw, c1, c2, seed=0, noise=True, tile_n=128, tile_k=128):
+    """Gradient of sum(Gw * Mt * W) + c1 sum(Mt) - c2/2 sum((Mt W)^2) w.r.t. the logits -> (gP_tile, gP24), float64."""
+    W = _u16(W)
+    N, K = W.shape
+    P_tile, P24, Gw = _f32(P_tile), _f32(P24), _f32(Gw)
+    assert Gw.shape == (N, K) and P24.shape == (6, N * K // 4)
+    gt = np.empty(P_tile.size, np.float64)
+    g6 = np.empty((6, N * K // 4), np.float64)
+    _check(lib().oracle_soft_mask_backward(_p(W), ctypes.c_int64(N), ctypes.c_int64(K), _p(P_tile), _p(P24), tile_n,
+                                           tile_k, ctypes.c_double(tau), ctypes.c_double(kappa), ctypes.c_uint64(seed),
+                                           int(bool(noise)), _p(Gw), ctypes.c_double(c1), ctypes.c_double(c2), _p(gt),
+                                           _p(g6)), "soft_mask_backward")
+    return gt.reshape(np.asarray(P_tile).shape), g6
+
+
 def hard_mask(P_tile, P24, N, K, tile_n=128, tile_k=128):
     """Algorithm 1's hard masks -> (tile flags uint8 [TN*TK], candidate index per group uint8 [N*K/4])."""
     P_tile, P24 = _f32(P_tile), _f32(P24)

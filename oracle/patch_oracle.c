@@ -549,3 +549,73 @@ int oracle_mask_patterns(int64_t N, int64_t K, const uint8_t* flags, const uint8
         }
     return 0;
 }
+
+/* Coefficients with which one element's soft-mask value enters the gradient of the two regularisers of
+ * Eq. 5 (pooled sums a = sum Mt, b = sum ||W||_0, d = sum ||W||^2 over all matrices):
+ *   d/dMt_e [ lambda1 |a/b - rho| ]        = lambda1 sign(a/b - rho) / b         =: c1
+ *   d/dMt_e [ -lambda2 sum (Mt W)^2 / d ]  = -(2 lambda2 / d) Mt_e W_e^2         =: -c2 Mt_e W_e^2 */
+void oracle_regularizer_coefficients(const double* sums, int n, double rho, double lambda1, double lambda2,
+                                     double* c1, double* c2) {
+    double a = 0, b = 0, d = 0;
+    for (int i = 0; i < n; ++i) { a += sums[4 * i]; b += sums[4 * i + 1]; d += sums[4 * i + 3]; }
+    double dev = a / b - rho;
+    *c1 = lambda1 * (dev > 0 ? 1.0 : dev < 0 ? -1.0 : 0.0) / b;
+    *c2 = 2.0 * lambda2 / d;
+}
+
+/* Gradient with respect to the logits ("Update P_tile, P_2:4 via backpropagation", Algorithm 1) of
+ *   F = sum_e Gw_e Mt_e W_e  +  c1 sum_e Mt_e  -  (c2 / 2) sum_e (Mt_e W_e)^2
+ * for fixed noise, where Gw = dL_LM / d(Mt (.) W) is the gradient the language-model loss hands back for
+ * the masked weight.  Chain rule through Eq. 4, Eq. 2 / Eq. 3 and the softmax of Eq. 1:
+ *   gM_e   = Gw_e W_e + c1 - c2 Mt_e W_e^2
+ *   h_c    = (1 - Mt_tile) sum_j S[c][j] gM_j                      (per group)
+ *   gP24_c = (kappa / tau) GS_c (h_c - sum_k GS_k h_k)
+ *   gP_tile = (kappa / tau) Mt_tile (1 - Mt_tile) sum_{e in tile} gM_e (1 - Mt_2:4,e)
+ * gP_tile [TN x TK], gP24 [6 x G], both double. */
+int oracle_soft_mask_backward(const uint16_t* W, int64_t N, int64_t K, const float* P_tile, const float* P24,
+                              int tile_n, int tile_k, double tau, double kappa, uint64_t seed, int use_noise,
+                              const float* Gw, double c1, double c2, double* gP_tile, double* gP24) {
+    int rc = check_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    if (!W || !P_tile || !P24 || !Gw || !gP_tile || !gP24) return -1;
+    if (!(tau > 0.0)) return -2;
+    int64_t TK = K / tile_k, T = (N / tile_n) * TK, G = N * (K / 4);
+    for (int64_t t = 0; t < T; ++t) gP_tile[t] = 0.0;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t g = 0; g < K / 4; ++g) {
+            int64_t t = (n / tile_n) * TK + (4 * g) / tile_k, grp = n * (K / 4) + g;
+            double p2[2] = {(double)P_tile[t], 0.0}, z2[2] = {0.0, 0.0}, gs2[2];
+            double p6[6], z6[6], gs6[6], m24[4], gM[4], h[6], hbar = 0.0;
+            for (int c = 0; c < 6; ++c) { p6[c] = (double)P24[c * G + grp]; z6[c] = 0.0; }
+            if (use_noise) {
+                for (int c = 0; c < 2; ++c) z2[c] = oracle_gumbel(seed, 0, 2 * (uint64_t)t + c);
+                for (int c = 0; c < 6; ++c) z6[c] = oracle_gumbel(seed, 1, (uint64_t)c * G + grp);
+            }
+            gumbel_softmax(p2, z2, 2, tau, kappa, gs2);
+            gumbel_softmax(p6, z6, 6, tau, kappa, gs6);
+            double mt = gs2[0];
+            for (int j = 0; j < 4; ++j) {
+                m24[j] = 0.0;
+                for (int c = 0; c < 6; ++c) m24[j] += gs6[c] * S_24[c][j];
+                double m = mt + (1.0 - mt) * m24[j];
+                double w = (double)bf16_to_f32(W[n * K + 4 * g + j]);
+                gM[j] = (double)Gw[n * K + 4 * g + j] * w + c1 - c2 * m * w * w;
+                gP_tile[t] += gM[j] * (1.0 - m24[j]);
+            }
+            for (int c = 0; c < 6; ++c) {
+                h[c] = 0.0;
+                for (int j = 0; j < 4; ++j) h[c] += S_24[c][j] * gM[j];
+                h[c] *= 1.0 - mt;
+                hbar += gs6[c] * h[c];
+            }
+            for (int c = 0; c < 6; ++c) gP24[c * G + grp] = kappa / tau * gs6[c] * (h[c] - hbar);
+        }
+    for (int64_t t = 0; t < T; ++t) {
+        double p2[2] = {(double)P_tile[t], 0.0}, z2[2] = {0.0, 0.0}, gs2[2];
+        if (use_noise)
+            for (int c = 0; c < 2; ++c) z2[c] = oracle_gumbel(seed, 0, 2 * (uint64_t)t + c);
+        gumbel_softmax(p2, z2, 2, tau, kappa, gs2);
+        gP_tile[t] *= kappa / tau * gs2[0] * (1.0 - gs2[0]);
+    }
+    return 0;
+}

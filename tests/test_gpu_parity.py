@@ -272,7 +272,8 @@ def test_decode_shapes_full_output(gpu, oracle, shape, p):
 @pytest.mark.parametrize("N,K,M,p", [(4096, 4096, 2048, 0.5), (11008, 4096, 512, 0.5), (4096, 11008, 4096, 1.0),
                                      (5120, 13824, 64, 0.6), (13824, 5120, 8, 0.3)])
 def test_prefill_shapes_sampled(gpu, oracle, N, K, M, p):
-    """Large M: compare 64 random token rows over all N, plus the four corner tiles' rows."""
+    """Large M: compare 64 random token rows over all N (first / last rows included) and two whole row-blocks of N
+    over all tokens."""
     torch, B = gpu
     stream = ("prefill", N, K, p)
     W = inputs.weight(N, K, inputs.MASTER_SEED, *stream)
@@ -285,6 +286,11 @@ def test_prefill_shapes_sampled(gpu, oracle, N, K, M, p):
     rows = np.unique(np.concatenate([rng.integers(0, M, 60), [0, M - 1, min(M - 1, 127), min(M - 1, 128)]]))
     Y32 = oracle.gemm_f64_rows(X, rows, What)
     check_parity(oracle, Y[rows], Y32, f"sampled rows N={N} K={K} M={M}")
+    # two whole 128-row blocks of N over all tokens: every token tile of the schedule is touched
+    for tn in np.unique(rng.integers(0, N // 128, 2)):
+        cols = slice(int(tn) * 128, int(tn) * 128 + 128)
+        Yb, _ = oracle.gemm_f64(X, What[cols], want_bf16=False)
+        check_parity(oracle, Y[:, cols], Yb, f"row-block {tn} N={N} K={K} M={M}")
     # property that holds at any size: doubling X doubles every output exactly
     Y2 = run_gemm(gpu, inputs.f32_to_bf16_bits(2.0 * f32(X)), L, packed, B.VARIANT_AUTO)
     assert (f32(Y2) == 2.0 * f32(Y)).all()

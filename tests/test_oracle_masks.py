@@ -274,3 +274,57 @@ def test_regularizers_closed_form(oracle):
     assert oracle.regularizers(two, 0.9, 3, 0.1) == pytest.approx(3 * abs(60 / 100 - 0.9) - 0.1 * 6 / 10, abs=1e-15)
     assert oracle.regularizers(two, 0.9, 3, 0.1) != pytest.approx(
         3 * abs((10 / 40 + 50 / 60) / 2 - 0.9) - 0.1 * (1 / 4 + 5 / 6) / 2)
+
+
+# ---------------------------------------------------------------------------------------------
+# backward
+
+
+def _objective(oracle, W, PT, P6, tau, kappa, seed, noise, Gw, c1, c2, tn, tk):
+    Mt, _, _ = oracle.soft_mask(W, PT, P6, tau, kappa, seed=seed, noise=noise, tile_n=tn, tile_k=tk)
+    w = f32(W).astype(np.float64)
+    return (Gw.astype(np.float64) * Mt * w).sum() + c1 * Mt.sum() - 0.5 * c2 * ((Mt * w) ** 2).sum()
+
+
+@pytest.mark.parametrize("noise", [False, True])
+def test_backward_against_finite_differences(oracle, noise):
+    """The analytic gradient against central differences of the (separately pinned) forward."""
+    N, K, tn, tk = 8, 16, 4, 8
+    W = inputs.weight(N, K, 9, "bw")
+    g = inputs.generator(9, "bw", "gw")
+    Gw = g.standard_normal((N, K)).astype(np.float32)
+    PT = (g.standard_normal((2, 2)) * 0.05).astype(np.float32)
+    P6 = (g.standard_normal((6, N * K // 4)) * 0.05).astype(np.float32)
+    tau, kappa, c1, c2 = 0.8, 12.0, 0.3, 40.0
+    gt, g6 = oracle.soft_mask_backward(W, PT, P6, tau, kappa, Gw, c1, c2, seed=3, noise=noise, tile_n=tn, tile_k=tk)
+    F = lambda pt, p6: _objective(oracle, W, pt, p6, tau, kappa, 3, noise, Gw, c1, c2, tn, tk)
+    d = np.float32(2.0 ** -12)
+    for (i, j) in [(0, 0), (0, 1), (1, 0), (1, 1)]:
+        a, b = PT.copy(), PT.copy()
+        a[i, j] += d
+        b[i, j] -= d
+        fd = (F(a, P6) - F(b, P6)) / (float(a[i, j]) - float(b[i, j]))
+        assert fd == pytest.approx(gt[i, j], rel=2e-4, abs=1e-7)
+    for (c, grp) in [(0, 0), (5, 0), (2, 7), (3, 13), (1, 31), (4, 18)]:
+        a, b = P6.copy(), P6.copy()
+        a[c, grp] += d
+        b[c, grp] -= d
+        fd = (F(PT, a) - F(PT, b)) / (float(a[c, grp]) - float(b[c, grp]))
+        assert fd == pytest.approx(g6[c, grp], rel=2e-4, abs=1e-7)
+    # a softmax gradient sums to zero over the classes of a group
+    assert np.abs(g6.sum(axis=0)).max() < 1e-12 * max(1.0, np.abs(g6).max())
+
+
+def test_regularizer_coefficients_are_the_derivative_of_the_regularizers(oracle):
+    sums = np.array([[60.0, 100, 30, 60], [20.0, 50, 8, 20]])
+    rho, l1, l2 = 0.4, 7.0, 10.0
+    c1, c2 = oracle.regularizer_coefficients(sums, rho, l1, l2)
+    assert c1 == pytest.approx(7.0 / 150) and c2 == pytest.approx(2 * 10.0 / 80)
+    # raising one element's Mt by e raises sum Mt by e and sum (Mt W)^2 by 2 e Mt W^2: compare with the regularisers
+    e, mt, w = 1e-6, 0.7, 1.3
+    s2 = sums.copy()
+    s2[0, 0] += e
+    s2[0, 2] += 2 * e * mt * w * w
+    fd = (oracle.regularizers(s2, rho, l1, l2) - oracle.regularizers(sums, rho, l1, l2)) / e
+    assert fd == pytest.approx(c1 - c2 * mt * w * w, rel=1e-5)
+    assert oracle.regularizer_coefficients(sums, 0.9, l1, l2)[0] == pytest.approx(-7.0 / 150)   # below the target
