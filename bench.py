@@ -473,7 +473,8 @@ def run_masks(args):
         W = torch.from_numpy(np.ascontiguousarray(inputs.weight(N, K, inputs.MASTER_SEED, "masks", i)).view(np.int16)).to(dev).view(torch.bfloat16)
         PT = torch.from_numpy(inputs.tile_logits(N // 128, K // 128, 0.5, inputs.MASTER_SEED, "masks", i)).to(dev)
         P6 = torch.from_numpy(inputs.pattern_logits(N, K, inputs.MASTER_SEED, "masks", i)).to(dev)
-        mats.append(dict(N=N, K=K, W=W, PT=PT, P6=P6, Wt=torch.empty_like(W),
+        Gw = torch.from_numpy(np.ascontiguousarray(inputs.normal_bf16((N, K), 1.0, inputs.MASTER_SEED, "masks-gw", i)).view(np.int16)).to(dev).view(torch.bfloat16)
+        mats.append(dict(N=N, K=K, W=W, PT=PT, P6=P6, Wt=torch.empty_like(W), Gw=Gw, gPT=torch.empty_like(PT), gP6=torch.empty_like(P6),
                          sums=torch.empty(4, dtype=torch.float64, device=dev),
                          ws=torch.empty(B.patch_soft_mask_workspace_size(N, K), dtype=torch.uint8, device=dev),
                          flags=torch.empty((N // 128) * (K // 128), dtype=torch.uint8, device=dev),
@@ -484,6 +485,11 @@ def run_masks(args):
         for i, m in enumerate(mats):
             B.patch_soft_mask(m["W"], m["PT"], m["P6"], tau, kappa, 1000 + i, flags, Wt=m["Wt"], sums=m["sums"],
                               workspace=m["ws"])
+
+    def backward():
+        for i, m in enumerate(mats):
+            B.patch_soft_mask_backward(m["W"], m["PT"], m["P6"], tau, kappa, m["Gw"], 1e-9, 1e-3, seed=1000 + i,
+                                       gP_tile=m["gPT"], gP24=m["gP6"])
 
     def hard():
         for m in mats:
@@ -521,6 +527,7 @@ def run_masks(args):
     clocks = sampler.stop(t0, time.time())
     t_plain = time_graph(graph_of(lambda: soft(B.MASK_NO_NOISE)), 50)
     t_hard = time_graph(graph_of(hard), 50)
+    t_bwd = time_graph(graph_of(backward), 50)
     # packing with the hard masks just computed (flags go through the host, as the entry point requires)
     hard()
     torch.cuda.synchronize()
@@ -589,6 +596,9 @@ def run_masks(args):
                                "frac_of_measured_hbm": elements * MASK_BYTES_PER_ELEMENT / t_plain / 1e9 / peaks["hbm_gbs"]},
         "hard_mask": {"ms_per_step": t_hard * 1e3, "gbs": elements * 6.25 / t_hard / 1e9,
                       "frac_of_measured_hbm": elements * 6.25 / t_hard / 1e9 / peaks["hbm_gbs"]},
+        "soft_mask_backward": {"ms_per_step": t_bwd * 1e3, "gbs": elements * 16.0 / t_bwd / 1e9,
+                               "frac_of_measured_hbm": elements * 16.0 / t_bwd / 1e9 / peaks["hbm_gbs"],
+                               "note": "16 B per element: W, Gw and six logits read, six logit gradients written; noise on"},
         "pack_patterns": {"ms_per_step": t_pack * 1e3, "gbs": pack_bytes / t_pack / 1e9,
                           "note": "includes the host-built tile table and its copy, per matrix"},
         "e2e": {"value": elements * MASK_BYTES_PER_ELEMENT / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,

@@ -332,6 +332,35 @@ int patch_soft_mask(const void* W_dev, int64_t ldw, const float* P_tile_dev, con
 int patch_mask_regularizers(const double* sums_host, int n, double rho, double lambda1, double lambda2,
                             double* out_host);
 
+/*
+ * Coefficients with which one element's soft-mask value enters the gradient of the regularisers of
+ * Eq. 5, from the pooled sums of n matrices (host arrays as for patch_mask_regularizers):
+ *   *c1_host = lambda1 * sign(sum Mt / sum ||W||_0 - rho) / sum ||W||_0
+ *   *c2_host = 2 * lambda2 / sum ||W||^2
+ * so that d(regularisers)/dMt_e = c1 - c2 * Mt_e * W_e^2.  Host only.
+ */
+int patch_mask_regularizer_coefficients(const double* sums_host, int n, double rho, double lambda1,
+                                        double lambda2, double* c1_host, double* c2_host);
+
+/*
+ * Backward of patch_soft_mask ("Update P_tile, P_2:4 via backpropagation", Algorithm 1): gradient with
+ * respect to the logits of
+ *   F = sum_e Gw_e Mt_e W_e + c1 sum_e Mt_e - (c2 / 2) sum_e (Mt_e W_e)^2,
+ * where Gw = dL_LM / d(Mt (.) W) is the gradient the language-model loss returns for the masked weight
+ * and c1, c2 come from patch_mask_regularizer_coefficients.  The forward is recomputed on the fly with
+ * the same (seed, flags), so nothing has to be kept from the forward call:
+ *   gM_e = Gw_e W_e + c1 - c2 Mt_e W_e^2;   h_c = (1 - Mt_tile) sum_j S[c][j] gM_j   (per group)
+ *   gP24_dev[c][grp] = (kappa / tau) GS_c (h_c - sum_k GS_k h_k)
+ *   gP_tile_dev[t]   = (kappa / tau) Mt_tile (1 - Mt_tile) sum_{e in tile t} gM_e (1 - Mt_2:4,e)
+ *   Gw_dev  bf16 [N x ldg];  gP_tile_dev fp32 [N/128 x K/128];  gP24_dev fp32 [6 x G], 16-byte aligned.
+ * Every output element is written (no accumulation into the buffers).  fp32 arithmetic, the tile sum in
+ * a fixed order.  One kernel, no workspace, no host synchronisation.
+ */
+int patch_soft_mask_backward(const void* W_dev, int64_t ldw, const float* P_tile_dev, const float* P24_dev,
+                             int64_t N, int64_t K, int tile_n, int tile_k, float tau, float kappa,
+                             uint64_t seed, int flags, const void* Gw_dev, int64_t ldg, double c1, double c2,
+                             float* gP_tile_dev, float* gP24_dev, void* stream);
+
 /* Human-readable text for a status code (static storage). */
 const char* patch_strerror(int status);
 

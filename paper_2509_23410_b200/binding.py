@@ -27,7 +27,7 @@ EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_worksp
            "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch",
            "patch_gemm_noalloc",
            "patch_hard_mask", "patch_pack_patterns", "patch_soft_mask_workspace_size", "patch_soft_mask",
-           "patch_mask_regularizers",
+           "patch_mask_regularizers", "patch_mask_regularizer_coefficients", "patch_soft_mask_backward",
            "patch_strerror", "patch_version"]
 MASK_NO_NOISE = 1
 
@@ -79,6 +79,12 @@ def lib() -> ctypes.CDLL:
                                       ctypes.c_float, ctypes.c_uint64, ctypes.c_int, vp, i64, vp, i64, vp, vp, sz, vp]
         L.patch_mask_regularizers.argtypes = [vp, ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                               ctypes.POINTER(ctypes.c_double)]
+        L.patch_mask_regularizer_coefficients.argtypes = [vp, ctypes.c_int, ctypes.c_double, ctypes.c_double,
+                                                          ctypes.c_double, ctypes.POINTER(ctypes.c_double),
+                                                          ctypes.POINTER(ctypes.c_double)]
+        L.patch_soft_mask_backward.argtypes = [vp, i64, vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                               ctypes.c_float, ctypes.c_uint64, ctypes.c_int, vp, i64, ctypes.c_double,
+                                               ctypes.c_double, vp, vp, vp]
         L.patch_strerror.argtypes = [ctypes.c_int]
         L.patch_strerror.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -325,3 +331,34 @@ def patch_mask_regularizers(sums, rho: float, lambda1: float, lambda2: float) ->
     _check(lib().patch_mask_regularizers(ctypes.c_void_p(a.ctypes.data), int(a.shape[0]), float(rho), float(lambda1),
                                          float(lambda2), ctypes.byref(out)), "patch_mask_regularizers")
     return float(out.value)
+
+
+def patch_mask_regularizer_coefficients(sums, rho: float, lambda1: float, lambda2: float):
+    """(c1, c2) of the regularisers' gradient from per-matrix sums (host array-like [n x 4])."""
+    import numpy as np
+    a = np.ascontiguousarray(sums, dtype=np.float64).reshape(-1, 4)
+    c1, c2 = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib().patch_mask_regularizer_coefficients(ctypes.c_void_p(a.ctypes.data), int(a.shape[0]), float(rho),
+                                                     float(lambda1), float(lambda2), ctypes.byref(c1), ctypes.byref(c2)),
+           "patch_mask_regularizer_coefficients")
+    return float(c1.value), float(c2.value)
+
+
+def patch_soft_mask_backward(W, P_tile, P24, tau: float, kappa: float, Gw, c1: float, c2: float, seed: int = 0,
+                             flags: int = 0, gP_tile=None, gP24=None, stream=None):
+    """Gradient of the soft-mask objective w.r.t. the logits: returns (gP_tile float32, gP24 float32 [6 x G])."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    assert Gw.is_cuda and Gw.dtype == torch.bfloat16 and Gw.shape == W.shape and Gw.stride(1) == 1
+    N, K = W.shape
+    assert P_tile.is_cuda and P_tile.dtype == torch.float32 and P_tile.is_contiguous()
+    assert P24.is_cuda and P24.dtype == torch.float32 and P24.is_contiguous() and tuple(P24.shape) == (6, N * K // 4)
+    if gP_tile is None:
+        gP_tile = torch.empty_like(P_tile)
+    if gP24 is None:
+        gP24 = torch.empty_like(P24)
+    _check(lib().patch_soft_mask_backward(_ptr(W), W.stride(0), _ptr(P_tile), _ptr(P24), N, K, 128, 128, float(tau),
+                                          float(kappa), int(seed) & 0xFFFFFFFFFFFFFFFF, int(flags), _ptr(Gw), Gw.stride(0),
+                                          float(c1), float(c2), _ptr(gP_tile), _ptr(gP24), _stream(stream)),
+           "patch_soft_mask_backward")
+    return gP_tile, gP24

@@ -76,7 +76,7 @@ soft_mask_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __res
                  const float* __restrict__ P24, int TK, int64_t G, float sp, float sz, uint64_t seed,
                  uint64_t candidate_step /* kGolden * (G / 2) */, uint16_t* __restrict__ Wt, int64_t ldo, float* __restrict__ Mt, int64_t ldm,
                  double* __restrict__ partials) {
-    __shared__ float s_mt;
+    __shared__ float s_mt, s_omt;
     __shared__ double s_red[8][4];
     const int t = blockIdx.x, tn = t / TK, tk = t - tn * TK;
     if (threadIdx.x == 0) {
@@ -88,9 +88,10 @@ soft_mask_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __res
         }
         const float inv = softmax2_terms(a);
         s_mt = a[0] * inv;
+        s_omt = a[1] * inv;     // 1 - Mt_tile as the other softmax term: no cancellation when Mt_tile is next to 1
     }
     __syncthreads();
-    const float mt = s_mt, one_minus_mt = 1.0f - mt;
+    const float mt = s_mt, one_minus_mt = s_omt;
     float acc_mw2 = 0.f, acc_w2 = 0.f;
     uint32_t acc_nz = 0;
 #pragma unroll 1
@@ -170,6 +171,102 @@ soft_mask_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __res
         double s = 0.0;
         for (int w = 0; w < 8; ++w) s += s_red[w][threadIdx.x];
         partials[int64_t(t) * 4 + threadIdx.x] = s;
+    }
+}
+
+// Gradient with respect to the logits of  F = sum Gw Mt W + c1 sum Mt - (c2 / 2) sum (Mt W)^2  ("Update
+// P_tile, P_2:4 via backpropagation", Algorithm 1), the forward recomputed on the fly with the same noise.
+// Same work split as the forward: one CTA per tile, four groups per thread and iteration.  Per element it
+// reads 2 B of W, 2 B of Gw and 6 B of logits and writes 6 B of logit gradient.
+template <bool NOISE>
+__global__ void __launch_bounds__(256)
+soft_mask_backward_kernel(const uint16_t* __restrict__ W, int64_t ldw, const uint16_t* __restrict__ Gw, int64_t ldg,
+                          const float* __restrict__ P_tile, const float* __restrict__ P24, int TK, int64_t G, float sp,
+                          float sz, float kappa_over_tau, uint64_t seed, uint64_t candidate_step, float c1, float c2,
+                          float* __restrict__ gP_tile, float* __restrict__ gP24) {
+    __shared__ float s_mt, s_omt;
+    __shared__ double s_red[8];
+    const int t = blockIdx.x, tn = t / TK, tk = t - tn * TK;
+    if (threadIdx.x == 0) {
+        float a[2] = {P_tile[t] * sp, 0.f};
+        if (NOISE) {
+            const uint64_t h = mix_final(seed + kGolden * (uint64_t(t) + 1));
+            a[0] += gumbel_log2(uint32_t(h >> 41)) * sz;
+            a[1] += gumbel_log2(uint32_t(h >> 9) & 0x7FFFFFu) * sz;
+        }
+        const float inv = softmax2_terms(a);
+        s_mt = a[0] * inv;
+        s_omt = a[1] * inv;     // 1 - Mt_tile as the other softmax term: no cancellation when Mt_tile is next to 1
+    }
+    __syncthreads();
+    const float mt = s_mt, one_minus_mt = s_omt;
+    float acc_gmt = 0.f;     // sum of gM (1 - Mt_2:4) over this thread's elements
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+        const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 3, u = idx & 7u;
+        const int64_t n = int64_t(tn) * kTile + r;
+        const int64_t grp = n * (int64_t(TK) * 32) + tk * 32 + u * 4;
+        const uint16_t* src = W + n * ldw + int64_t(tk) * kTile + u * 16;
+        const uint16_t* gsrc = Gw + n * ldg + int64_t(tk) * kTile + u * 16;
+        const uint4 wa = *reinterpret_cast<const uint4*>(src), wb = *reinterpret_cast<const uint4*>(src + 8);
+        const uint4 ga = *reinterpret_cast<const uint4*>(gsrc), gb = *reinterpret_cast<const uint4*>(gsrc + 8);
+        float a[4][6];
+        uint64_t x0 = seed + kStreamStep + kGolden * (uint64_t(grp >> 1) + 1);
+#pragma unroll
+        for (int c = 0; c < 6; ++c) {
+            const float4 p = *reinterpret_cast<const float4*>(P24 + int64_t(c) * G + grp);
+            a[0][c] = p.x * sp; a[1][c] = p.y * sp; a[2][c] = p.z * sp; a[3][c] = p.w * sp;
+            if (NOISE) {
+                const uint64_t h0 = mix_final(x0), h1 = mix_final(x0 + kGolden);
+                x0 += candidate_step;
+                a[0][c] += gumbel_log2(uint32_t(h0 >> 41)) * sz;
+                a[1][c] += gumbel_log2(uint32_t(h0 >> 9) & 0x7FFFFFu) * sz;
+                a[2][c] += gumbel_log2(uint32_t(h1 >> 41)) * sz;
+                a[3][c] += gumbel_log2(uint32_t(h1 >> 9) & 0x7FFFFFu) * sz;
+            }
+        }
+        const uint32_t win[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+        const uint32_t gin[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+        float gout[6][4];   // gout[candidate][group]
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const float inv = softmax2_terms(a[g]);
+#pragma unroll
+            for (int c = 0; c < 6; ++c) a[g][c] *= inv;                        // GS_c
+            const float m24[4] = {a[g][0] + a[g][1] + a[g][2], a[g][0] + a[g][3] + a[g][4],
+                                  a[g][1] + a[g][3] + a[g][5], a[g][2] + a[g][4] + a[g][5]};
+            float gM[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t wbits = j & 1 ? win[2 * g + (j >> 1)] >> 16 : win[2 * g + (j >> 1)] & 0xFFFFu;
+                const uint32_t gbits = j & 1 ? gin[2 * g + (j >> 1)] >> 16 : gin[2 * g + (j >> 1)] & 0xFFFFu;
+                const float w = bf16_bits_to_float(wbits), gw = bf16_bits_to_float(gbits);
+                const float m = fmaf(one_minus_mt, m24[j], mt);
+                gM[j] = fmaf(gw, w, c1) - c2 * m * w * w;
+                acc_gmt = fmaf(gM[j], 1.0f - m24[j], acc_gmt);
+            }
+            // h_c = (1 - Mt_tile) (gM of the two kept positions of candidate c); gP_c = kappa/tau GS_c (h_c - sum GS h)
+            const float h[6] = {gM[0] + gM[1], gM[0] + gM[2], gM[0] + gM[3], gM[1] + gM[2], gM[1] + gM[3], gM[2] + gM[3]};
+            float hbar = 0.f;
+#pragma unroll
+            for (int c = 0; c < 6; ++c) hbar = fmaf(a[g][c], h[c], hbar);
+            const float scale = kappa_over_tau * one_minus_mt;
+#pragma unroll
+            for (int c = 0; c < 6; ++c) gout[c][g] = scale * a[g][c] * (h[c] - hbar);
+        }
+#pragma unroll
+        for (int c = 0; c < 6; ++c)
+            *reinterpret_cast<float4*>(gP24 + int64_t(c) * G + grp) = make_float4(gout[c][0], gout[c][1], gout[c][2], gout[c][3]);
+    }
+    double v = double(acc_gmt);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (int w = 0; w < 8; ++w) s += s_red[w];
+        gP_tile[t] = float(s * double(kappa_over_tau) * double(mt) * double(one_minus_mt));
     }
 }
 
@@ -297,6 +394,51 @@ extern "C" int patch_soft_mask(const void* W_dev, int64_t ldw, const float* P_ti
     if (cudaGetLastError() != cudaSuccess) return PATCH_ERR_CUDA;
     reduce_partials_kernel<<<1, 256, 0, s>>>(partials, T, sums_dev);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_soft_mask_backward(const void* W_dev, int64_t ldw, const float* P_tile_dev, const float* P24_dev,
+                                        int64_t N, int64_t K, int tile_n, int tile_k, float tau, float kappa,
+                                        uint64_t seed, int flags, const void* Gw_dev, int64_t ldg, double c1, double c2,
+                                        float* gP_tile_dev, float* gP24_dev, void* stream) {
+    int rc = check_mask_shape(N, K, tile_n, tile_k);
+    if (rc) return rc;
+    if (!W_dev || !P_tile_dev || !P24_dev || !Gw_dev || !gP_tile_dev || !gP24_dev) return PATCH_ERR_NULL;
+    if (!(tau > 0.0f) || !std::isfinite(tau) || !std::isfinite(kappa) || !std::isfinite(c1) || !std::isfinite(c2))
+        return PATCH_ERR_SHAPE;
+    if (flags & ~PATCH_MASK_NO_NOISE) return PATCH_ERR_SHAPE;
+    if (ldw < K || ldg < K || ldw % 8 || ldg % 8) return PATCH_ERR_SHAPE;
+    if (!aligned16(W_dev) || !aligned16(Gw_dev) || !aligned16(P24_dev) || !aligned16(gP24_dev) ||
+        (reinterpret_cast<uintptr_t>(P_tile_dev) & 3u) || (reinterpret_cast<uintptr_t>(gP_tile_dev) & 3u))
+        return PATCH_ERR_ALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    const int64_t TK = K / kTile, T = (N / kTile) * TK, G = N * (K / 4);
+    const float sz = 1.0f / tau, sp = kappa * 1.44269504f * sz;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint16_t* W = static_cast<const uint16_t*>(W_dev);
+    const uint16_t* Gw = static_cast<const uint16_t*>(Gw_dev);
+    if (flags & PATCH_MASK_NO_NOISE)
+        soft_mask_backward_kernel<false><<<unsigned(T), 256, 0, s>>>(W, ldw, Gw, ldg, P_tile_dev, P24_dev, int(TK), G, sp, sz,
+                                                                     kappa * sz, seed, kGolden * uint64_t(G / 2), float(c1),
+                                                                     float(c2), gP_tile_dev, gP24_dev);
+    else
+        soft_mask_backward_kernel<true><<<unsigned(T), 256, 0, s>>>(W, ldw, Gw, ldg, P_tile_dev, P24_dev, int(TK), G, sp, sz,
+                                                                    kappa * sz, seed, kGolden * uint64_t(G / 2), float(c1),
+                                                                    float(c2), gP_tile_dev, gP24_dev);
+    return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_mask_regularizer_coefficients(const double* sums_host, int n, double rho, double lambda1,
+                                                   double lambda2, double* c1_host, double* c2_host) {
+    if (!sums_host || !c1_host || !c2_host) return PATCH_ERR_NULL;
+    if (n <= 0) return PATCH_ERR_SHAPE;
+    double m = 0, nz = 0, w2 = 0;
+    for (int i = 0; i < n; ++i) { m += sums_host[4 * i]; nz += sums_host[4 * i + 1]; w2 += sums_host[4 * i + 3]; }
+    if (!(nz > 0) || !(w2 > 0)) return PATCH_ERR_SHAPE;
+    const double dev = m / nz - rho;
+    *c1_host = lambda1 * (dev > 0 ? 1.0 : dev < 0 ? -1.0 : 0.0) / nz;
+    *c2_host = 2.0 * lambda2 / w2;
+    return PATCH_OK;
 }
 
 extern "C" int patch_mask_regularizers(const double* sums_host, int n, double rho, double lambda1, double lambda2,

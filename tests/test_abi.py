@@ -179,3 +179,22 @@ def test_mask_entry_points_validate_on_the_host():
     out = ctypes.c_double(0)
     assert lib.patch_mask_regularizers(p, 0, 0.5, 1.0, 1.0, ctypes.byref(out)) == B.ERR_SHAPE
     assert lib.patch_mask_regularizers(p, 1, 0.5, 1.0, 1.0, ctypes.byref(out)) == B.ERR_SHAPE   # all-zero sums: no weights
+
+
+def test_mask_backward_validates_on_the_host():
+    import ctypes
+    from paper_2509_23410_b200 import binding as B
+    lib = B.lib()
+    buf = (ctypes.c_double * 64)()
+    p = ctypes.addressof(buf)
+    ok = (p, 128, p, p, 128, 128, 128, 128, 1.0, 1.0, 0, 0, p, 128, 0.0, 0.0, p, p, None)
+    bad = lambda i, v: ok[:i] + (v,) + ok[i + 1:]
+    assert lib.patch_soft_mask_backward(*bad(8, 0.0)) == B.ERR_SHAPE            # tau
+    assert lib.patch_soft_mask_backward(*bad(14, float("inf"))) == B.ERR_SHAPE  # c1
+    assert lib.patch_soft_mask_backward(*bad(13, 100)) == B.ERR_SHAPE           # ldg < K
+    assert lib.patch_soft_mask_backward(*bad(12, None)) == B.ERR_NULL           # Gw
+    assert lib.patch_soft_mask_backward(*bad(17, p + 4)) == B.ERR_ALIGN         # gP24
+    assert lib.patch_soft_mask_backward(*bad(6, 64)) == B.ERR_TILE
+    c1, c2 = B.patch_mask_regularizer_coefficients([[60.0, 100, 30, 60], [20.0, 50, 8, 20]], 0.4, 7.0, 10.0)
+    assert abs(c1 - 7.0 / 150) < 1e-15 and abs(c2 - 0.25) < 1e-15
+    assert B.patch_mask_regularizer_coefficients([[60.0, 100, 30, 60]], 0.9, 7.0, 10.0)[0] == -0.07

@@ -14,6 +14,8 @@ from paper_2509_23410_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 MT_TOL = 1e-3
+# gradients of saturated tiles are e^-|d| with |d| in the hundreds: below fp32's range the device returns 0
+TINY = 1e-20
 
 
 @pytest.fixture(scope="module")
@@ -234,3 +236,79 @@ def test_mask_entry_points_reject_bad_arguments(gpu):
     assert lib.patch_soft_mask(*args(tau=float("nan"))) == B.ERR_SHAPE
     assert lib.patch_soft_mask(*args(ws=8)) == B.ERR_SIZE
     assert lib.patch_soft_mask(*args(flags=4)) == B.ERR_SHAPE
+
+
+# ---------------------------------------------------------------------------------------------
+# backward
+
+
+@pytest.mark.parametrize("tau,kappa", [inputs.SCHEDULE_START, (0.6, 100.0), inputs.SCHEDULE_END])
+@pytest.mark.parametrize("noise", [False, True])
+def test_soft_mask_backward_parity(gpu, oracle, tau, kappa, noise):
+    """fp32 on the device against the oracle's double gradient: relative Frobenius error <= 1e-3 and
+    max |d| <= 2e-3 max |g| (the same exponent-rounding argument as for the forward, times the few terms
+    of the chain rule)."""
+    torch, B = gpu
+    N, K = 384, 640
+    W = inputs.weight(N, K, 41, "bwd")
+    W[::11, ::5] = 0
+    Gw = inputs.normal_bf16((N, K), 1.0, 41, "bwd", "gw")
+    PT, P6 = logits(N, K, 0.5, 41, "bwd")
+    PT *= np.float32(0.004)
+    c1, c2 = 3.0e-6, 0.8
+    rt, r6 = oracle.soft_mask_backward(W, PT, P6, tau, kappa, f32(Gw), c1, c2, seed=55, noise=noise)
+    gt, g6 = B.patch_soft_mask_backward(to_dev(torch, W), torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), tau,
+                                        kappa, to_dev(torch, Gw), c1, c2, seed=55, flags=0 if noise else B.MASK_NO_NOISE)
+    torch.cuda.synchronize()
+    # at the end of the schedule (kappa / tau = 7000) the tiles are saturated: their gradient is e^-|d| with
+    # |d| in the tens to hundreds, so an absolute error of 1e-3 in the fp32 exponent is a relative error of
+    # 1e-3 in the gradient
+    tol = 3.0 if kappa / tau > 1000 else 1.0
+    for got, ref in ((gt.cpu().numpy().astype(np.float64), rt), (g6.cpu().numpy().astype(np.float64), r6)):
+        assert np.isfinite(got).all()
+        assert np.abs(got - ref).max() <= tol * 2e-3 * np.abs(ref).max() + TINY
+        assert np.sqrt(((got - ref) ** 2).sum()) <= tol * 1e-3 * np.sqrt((ref ** 2).sum()) + TINY
+    assert np.abs(r6).max() > 0 and np.abs(rt).max() > 0
+
+
+def test_soft_mask_backward_full_size_and_determinism(gpu, oracle):
+    torch, B = gpu
+    N, K = 2048, 4096
+    W = inputs.weight(N, K, 42, "bwd2")
+    Gw = inputs.normal_bf16((N, K), 1.0, 42, "bwd2", "gw")
+    PT, P6 = logits(N, K, 0.5, 42, "bwd2")
+    tau, kappa, c1, c2 = 0.5, 120.0, -2.0e-7, 0.05
+    args = (to_dev(torch, W), torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), tau, kappa, to_dev(torch, Gw), c1, c2)
+    gt, g6 = B.patch_soft_mask_backward(*args, seed=9)
+    gt2, g62 = B.patch_soft_mask_backward(*args, seed=9)
+    torch.cuda.synchronize()
+    assert torch.equal(gt, gt2) and torch.equal(g6, g62)
+    rt, r6 = oracle.soft_mask_backward(W, PT, P6, tau, kappa, f32(Gw), c1, c2, seed=9, noise=True)
+    for got, ref in ((gt.cpu().numpy().astype(np.float64), rt), (g6.cpu().numpy().astype(np.float64), r6)):
+        assert np.abs(got - ref).max() <= 2e-3 * np.abs(ref).max() + TINY
+        assert np.sqrt(((got - ref) ** 2).sum()) <= 1e-3 * np.sqrt((ref ** 2).sum()) + TINY
+
+
+def test_forward_backward_step_lowers_the_objective(gpu, oracle):
+    """One gradient step on the logits, all on the device, lowers F = sum(Gw Mt W) + regularisers' linearisation."""
+    torch, B = gpu
+    N, K = 256, 512
+    W = to_dev(torch, inputs.weight(N, K, 43, "step"))
+    Gw = to_dev(torch, inputs.normal_bf16((N, K), 1.0, 43, "step", "gw"))
+    PT0, P60 = logits(N, K, 0.5, 43, "step")
+    PT = torch.from_numpy(PT0 * np.float32(0.004)).cuda()
+    P6 = torch.from_numpy(P60).cuda()
+    tau, kappa = 1.0, 30.0
+
+    def objective(pt, p6):
+        Mt = torch.empty((N, K), dtype=torch.float32, device="cuda")
+        B.patch_soft_mask(W, pt, p6, tau, kappa, 7, 0, Mt=Mt)
+        return float((Gw.float() * Mt * W.float()).double().sum())
+
+    f0 = objective(PT, P6)
+    gt, g6 = B.patch_soft_mask_backward(W, PT, P6, tau, kappa, Gw, 0.0, 0.0, seed=7)
+    lr = 1e-3 / float(g6.abs().max())
+    f1 = objective(PT - lr * gt, P6 - lr * g6)
+    predicted = -lr * float((gt.double() ** 2).sum() + (g6.double() ** 2).sum())
+    assert f1 < f0
+    assert (f1 - f0) == pytest.approx(predicted, rel=0.15)       # a small step follows the linearisation
