@@ -296,6 +296,33 @@ int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t* tile_flag
                         const uint8_t* patterns_dev, const patch_layout_t* layout, void* packed_dev,
                         size_t packed_capacity, int* status_dev, void* stream);
 
+/*
+ * patch_pack / patch_pack_patterns with the tile flags in DEVICE memory (e.g. as written by
+ * patch_hard_mask) and no host work at all: every CTA of the pack kernel derives its tile's offset
+ * from the flags (sum of the payload sizes before it) and writes its table entry; CTA 0 writes the
+ * header.  The blob is byte for byte the one patch_pack writes for the same flags.
+ *   tile_flags_dev  u8 [N/128 x K/128] device
+ *   patterns_dev    NULL (magnitude top-2, as patch_pack) or u8 [N x K/4] device (as patch_pack_patterns)
+ *   packed_capacity must hold the blob the flags imply; N/128 * K/128 * 32768 + table always does.
+ *                   The host checks only the smallest possible size (all tiles 2:4).
+ *   status_dev      optional device int (caller zeroes it): PATCH_ERR_SIZE if the blob did not fit
+ *                   (then nothing but a header without magic number is written), PATCH_ERR_FLAG for
+ *                   a flag other than 0 / 1 (packed as dense) or a candidate index above 5.
+ * Enqueues one kernel; no copy, no synchronisation.  The host-side layout that patch_gemm
+ * needs comes from patch_packed_size when the flags are also known on the host, else from
+ * patch_read_layout.
+ */
+int patch_pack_dev(const void* W_dev, int64_t ldw, const uint8_t* tile_flags_dev, const uint8_t* patterns_dev,
+                   int64_t N, int64_t K, int tile_n, int tile_k, void* packed_dev, size_t packed_capacity,
+                   int* status_dev, void* stream);
+
+/*
+ * Reads the header of a packed blob back into a host layout struct and validates it
+ * (PATCH_ERR_FORMAT if it is not a valid header, e.g. after a patch_pack_dev that did not fit).
+ * Copies 80 bytes device->host on `stream` and synchronises it.
+ */
+int patch_read_layout(const void* packed_dev, patch_layout_t* layout_out, void* stream);
+
 /* Scratch bytes of patch_soft_mask: four doubles per tile. */
 int patch_soft_mask_workspace_size(int64_t N, int64_t K, int tile_n, int tile_k, size_t* bytes_out);
 

@@ -26,7 +26,7 @@ ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
            "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch",
            "patch_gemm_noalloc",
-           "patch_hard_mask", "patch_pack_patterns", "patch_soft_mask_workspace_size", "patch_soft_mask",
+           "patch_hard_mask", "patch_pack_patterns", "patch_pack_dev", "patch_read_layout", "patch_soft_mask_workspace_size", "patch_soft_mask",
            "patch_mask_regularizers", "patch_mask_regularizer_coefficients", "patch_soft_mask_backward",
            "patch_strerror", "patch_version"]
 MASK_NO_NOISE = 1
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.patch_soft_mask_backward.argtypes = [vp, i64, vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_float,
                                                ctypes.c_float, ctypes.c_uint64, ctypes.c_int, vp, i64, ctypes.c_double,
                                                ctypes.c_double, vp, vp, vp]
+        L.patch_pack_dev.argtypes = [vp, i64, vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, sz, vp, vp]
+        L.patch_read_layout.argtypes = [vp, ctypes.POINTER(Layout), vp]
         L.patch_strerror.argtypes = [ctypes.c_int]
         L.patch_strerror.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -362,3 +364,25 @@ def patch_soft_mask_backward(W, P_tile, P24, tau: float, kappa: float, Gw, c1: f
                                           float(c1), float(c2), _ptr(gP_tile), _ptr(gP24), _stream(stream)),
            "patch_soft_mask_backward")
     return gP_tile, gP24
+
+
+def patch_pack_dev(W, flags_dev, patterns=None, out=None, status=None, stream=None):
+    """Pack with the tile flags in device memory (uint8 CUDA tensor); returns the packed uint8 tensor.
+    ``out`` defaults to a buffer that fits any flags; get the layout with ``patch_read_layout``."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    assert flags_dev.is_cuda and flags_dev.dtype == torch.uint8 and flags_dev.is_contiguous()
+    N, K = W.shape
+    T = (N // 128) * (K // 128)
+    assert flags_dev.numel() == T
+    if out is None:
+        out = torch.empty((256 + 16 * T + 1023) // 1024 * 1024 + T * 32768, dtype=torch.uint8, device=W.device)
+    _check(lib().patch_pack_dev(_ptr(W), W.stride(0), _ptr(flags_dev), _ptr(patterns), N, K, 128, 128, _ptr(out),
+                                out.numel(), _ptr(status), _stream(stream)), "patch_pack_dev")
+    return out
+
+
+def patch_read_layout(packed, stream=None) -> Layout:
+    L = Layout()
+    _check(lib().patch_read_layout(_ptr(packed), ctypes.byref(L), _stream(stream)), "patch_read_layout")
+    return L

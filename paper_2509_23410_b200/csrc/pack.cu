@@ -74,15 +74,86 @@ __device__ __forceinline__ uint32_t top2_of_4(const uint32_t w[4], uint32_t& v0,
 // lexicographic order of the kept positions) as the position code i0 | (i1 << 2), one nibble per candidate.
 constexpr uint32_t kCandidateCodes = 0xED9C84u;
 
+// Tile flags in device memory (patch_pack_dev): what the pack kernel needs to know about the blob.
+struct DeviceFlags {
+    const uint8_t* flags;   // [T]; NULL = the table in the blob was written by the host
+    int64_t T, N, K;
+    uint64_t capacity;
+};
+
+// Descriptor of tile t from the flags alone: the CTA sums the payload sizes of the tiles before t (its
+// offset) and of all tiles (does the blob fit?).  A few KB of flags per CTA, served by L2.  CTA 0 also
+// writes the header and the padding behind the table; every CTA writes its own table entry.
+// Returns false if the blob does not fit `capacity` (then only a header without magic number is written).
+__device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int t, uint8_t* blob, int* status, TileDesc& d) {
+    __shared__ unsigned long long s_part[8][3];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned long long before = 0, total = 0, dense = 0;
+    bool bad = false;
+    for (int64_t i = tid; i < F.T; i += 256) {
+        const uint8_t f = F.flags[i];
+        bad |= f > 1;
+        const unsigned long long b = f == PATCH_TILE_SPARSE_2_4 ? kSparseBytes : kDenseBytes;
+        total += b;
+        before += i < t ? b : 0;
+        dense += f == PATCH_TILE_SPARSE_2_4 ? 0 : 1;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
+        total += __shfl_xor_sync(0xFFFFFFFFu, total, off);
+        dense += __shfl_xor_sync(0xFFFFFFFFu, dense, off);
+    }
+    if (lane == 0) { s_part[warp][0] = before; s_part[warp][1] = total; s_part[warp][2] = dense; }
+    bad = __syncthreads_or(bad) != 0;
+    before = total = dense = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { before += s_part[w][0]; total += s_part[w][1]; dense += s_part[w][2]; }
+    const uint64_t payload_off = (kHeaderBytes + 16 * uint64_t(F.T) + 1023) / 1024 * 1024;
+    const uint64_t size = payload_off + total;
+    const bool fits = size <= F.capacity && size / 16 <= 0xFFFFFFF0ull;
+    if (t == 0) {
+        if (bad && status && tid == 0) *status = PATCH_ERR_FLAG;     // every CTA sees all flags; one reports
+        if (!fits && status && tid == 0) *status = PATCH_ERR_SIZE;
+        if (tid == 0) {
+            patch_layout_t L;
+            L.magic = fits ? kMagic : 0u; L.version = kVersion;
+            L.N = F.N; L.K = F.K; L.tile_n = kTile; L.tile_k = kTile;
+            L.n_dense = int64_t(dense); L.n_sparse = F.T - int64_t(dense);
+            L.table_off = kHeaderBytes; L.payload_off = payload_off; L.payload_bytes = total; L.total_bytes = size;
+            uint32_t* h = reinterpret_cast<uint32_t*>(blob);
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(&L);
+            for (uint32_t i = 0; i < kHeaderBytes / 4; ++i) h[i] = i < sizeof(L) / 4 ? src[i] : 0u;
+        }
+        if (fits) {
+            uint32_t* pad = reinterpret_cast<uint32_t*>(blob + kHeaderBytes + 16 * uint64_t(F.T));
+            for (uint64_t i = tid; i < (payload_off - kHeaderBytes - 16 * uint64_t(F.T)) / 4; i += 256) pad[i] = 0u;
+        }
+    }
+    if (!fits) return false;
+    const uint64_t off = payload_off + before;
+    if (F.flags[t] == PATCH_TILE_SPARSE_2_4) d = TileDesc{PATCH_TILE_SPARSE_2_4, uint32_t(off / 16), uint32_t((off + kAtomBytes) / 16), 0};
+    else d = TileDesc{PATCH_TILE_DENSE, uint32_t(off / 16), 0xFFFFFFFFu, 0};
+    if (tid == 0) reinterpret_cast<TileDesc*>(blob + kHeaderBytes)[t] = d;
+    return true;
+}
+
 // One CTA per tile.  W is read with 16-byte loads, the payload is written with 16-byte stores.
 // GIVEN: the 2:4 mask comes from `patterns` (one candidate index per group of four, [N x K/4]
 // row-major) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
-template <bool GIVEN>
+// DEVFLAGS: the tile's descriptor is computed from tile flags in device memory instead of read
+// from a table the host wrote.
+template <bool GIVEN, bool DEVFLAGS>
 __global__ void __launch_bounds__(256)
 pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob,
-            uint64_t table_off, const uint8_t* __restrict__ patterns, int* status) {
+            uint64_t table_off, const uint8_t* __restrict__ patterns, int* status, DeviceFlags F) {
     const int t = blockIdx.x;
-    const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+    TileDesc d;
+    if (DEVFLAGS) {
+        if (!descriptor_from_flags(F, t, blob, status, d)) return;
+    } else {
+        d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+    }
     const int tn = t / TK, tk = t - tn * TK;
     const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
     uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
@@ -237,13 +308,15 @@ static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const
     // pageable source: the runtime stages it before returning, so `head` may die at scope exit
     if (cudaMemcpyAsync(packed_dev, head.data(), head.size(), cudaMemcpyHostToDevice, s) != cudaSuccess)
         return PATCH_ERR_CUDA;
+    const DeviceFlags none = {nullptr, 0, 0, 0, 0};
     if (patterns_dev)
-        pack_kernel<true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
-                                                      static_cast<uint8_t*>(packed_dev), L->table_off, patterns_dev,
-                                                      status_dev);
+        pack_kernel<true, false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                             static_cast<uint8_t*>(packed_dev), L->table_off, patterns_dev,
+                                                             status_dev, none);
     else
-        pack_kernel<false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
-                                                       static_cast<uint8_t*>(packed_dev), L->table_off, nullptr, nullptr);
+        pack_kernel<false, false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                              static_cast<uint8_t*>(packed_dev), L->table_off, nullptr,
+                                                              nullptr, none);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
@@ -258,6 +331,45 @@ extern "C" int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t
     if (!patterns_dev) return PATCH_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(patterns_dev) & 3u) return PATCH_ERR_ALIGN;
     return pack_impl(W_dev, ldw, flags, patterns_dev, L, packed_dev, capacity, status_dev, stream);
+}
+
+extern "C" int patch_pack_dev(const void* W_dev, int64_t ldw, const uint8_t* flags_dev, const uint8_t* patterns_dev,
+                              int64_t N, int64_t K, int tile_n, int tile_k, void* packed_dev, size_t capacity,
+                              int* status_dev, void* stream) {
+    if (!W_dev || !flags_dev || !packed_dev) return PATCH_ERR_NULL;
+    if (tile_n != kTile || tile_k != kTile) return PATCH_ERR_TILE;
+    if (N <= 0 || K <= 0 || N % kTile || K % kTile) return PATCH_ERR_SHAPE;
+    if (ldw < K || ldw % 8) return PATCH_ERR_SHAPE;
+    const int64_t TK = K / kTile, T = (N / kTile) * TK;
+    if (T > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
+    if (!aligned16(W_dev) || !aligned16(packed_dev) || (patterns_dev && (reinterpret_cast<uintptr_t>(patterns_dev) & 3u)))
+        return PATCH_ERR_ALIGN;
+    const uint64_t payload_off = (kHeaderBytes + 16 * uint64_t(T) + 1023) / 1024 * 1024;
+    if (capacity < payload_off + uint64_t(T) * kSparseBytes) return PATCH_ERR_SIZE;   // below the smallest possible blob
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* blob = static_cast<uint8_t*>(packed_dev);
+    const DeviceFlags F = {flags_dev, T, N, K, uint64_t(capacity)};
+    if (patterns_dev)
+        pack_kernel<true, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
+                                                            kHeaderBytes, patterns_dev, status_dev, F);
+    else
+        pack_kernel<false, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
+                                                             kHeaderBytes, nullptr, status_dev, F);
+    return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_read_layout(const void* packed_dev, patch_layout_t* layout_out, void* stream) {
+    if (!packed_dev || !layout_out) return PATCH_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    patch_layout_t L;
+    if (cudaMemcpyAsync(&L, packed_dev, sizeof L, cudaMemcpyDeviceToHost, s) != cudaSuccess) return PATCH_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return PATCH_ERR_CUDA;
+    const int rc = validate_layout(&L);
+    if (rc) return rc;
+    *layout_out = L;
+    return PATCH_OK;
 }
 
 extern "C" int patch_unpack(const patch_layout_t* L, const void* packed_dev, void* What_dev,

@@ -198,3 +198,18 @@ def test_mask_backward_validates_on_the_host():
     c1, c2 = B.patch_mask_regularizer_coefficients([[60.0, 100, 30, 60], [20.0, 50, 8, 20]], 0.4, 7.0, 10.0)
     assert abs(c1 - 7.0 / 150) < 1e-15 and abs(c2 - 0.25) < 1e-15
     assert B.patch_mask_regularizer_coefficients([[60.0, 100, 30, 60]], 0.9, 7.0, 10.0)[0] == -0.07
+
+
+def test_pack_dev_validates_on_the_host():
+    import ctypes
+    from paper_2509_23410_b200 import binding as B
+    lib = B.lib()
+    buf = (ctypes.c_double * 64)()
+    p = ctypes.addressof(buf)
+    assert lib.patch_pack_dev(p, 128, None, None, 128, 128, 128, 128, p, 1 << 20, None, None) == B.ERR_NULL
+    assert lib.patch_pack_dev(p, 128, p, None, 128, 192, 128, 128, p, 1 << 20, None, None) == B.ERR_SHAPE
+    assert lib.patch_pack_dev(p, 120, p, None, 128, 128, 128, 128, p, 1 << 20, None, None) == B.ERR_SHAPE
+    assert lib.patch_pack_dev(p, 128, p, None, 128, 128, 128, 64, p, 1 << 20, None, None) == B.ERR_TILE
+    assert lib.patch_pack_dev(p, 128, p, p + 2, 128, 128, 128, 128, p, 1 << 20, None, None) == B.ERR_ALIGN
+    assert lib.patch_pack_dev(p, 128, p, None, 128, 128, 128, 128, p, 1024 + 18431, None, None) == B.ERR_SIZE
+    assert lib.patch_read_layout(None, None, None) == B.ERR_NULL

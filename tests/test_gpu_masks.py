@@ -312,3 +312,80 @@ def test_forward_backward_step_lowers_the_objective(gpu, oracle):
     predicted = -lr * float((gt.double() ** 2).sum() + (g6.double() ** 2).sum())
     assert f1 < f0
     assert (f1 - f0) == pytest.approx(predicted, rel=0.15)       # a small step follows the linearisation
+
+
+# ---------------------------------------------------------------------------------------------
+# packing with the tile flags on the device
+
+
+@pytest.mark.parametrize("N,K,p", [(128, 128, 1.0), (256, 384, 0.5), (1024, 1024, 0.0), (4096, 11008, 0.6), (11008, 4096, 0.3)])
+def test_pack_dev_equals_pack(gpu, oracle, N, K, p):
+    """The device-built header and table, and the payloads behind them, are byte for byte those of patch_pack
+    (which the other tests compare with the oracle)."""
+    torch, B = gpu
+    W = to_dev(torch, inputs.weight(N, K, 51, "pdev", N, K))
+    flags = inputs.tile_flags(N, K, p, 51, "pdev", N, K)
+    ref, L = B.patch_pack(W, flags)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fd = torch.from_numpy(np.ascontiguousarray(flags).reshape(-1)).cuda()
+    out = B.patch_pack_dev(W, fd, status=status)
+    Ld = B.patch_read_layout(out)
+    assert int(status.item()) == 0
+    assert bytes(Ld) == bytes(L)
+    assert torch.equal(out[:L.total_bytes], ref)
+    # an exactly sized buffer works too, and so does the given-mask variant
+    out2 = B.patch_pack_dev(W, fd, out=torch.empty(L.total_bytes, dtype=torch.uint8, device="cuda"), status=status)
+    assert int(status.item()) == 0 and torch.equal(out2, ref)
+    patterns = torch.from_numpy(inputs.generator(51, "pdev", "pat", N, K).integers(0, 6, N * K // 4).astype(np.uint8)).cuda()
+    ref_p, _ = B.patch_pack_patterns(W, flags, patterns)
+    out_p = B.patch_pack_dev(W, fd, patterns=patterns, status=status)
+    assert int(status.item()) == 0 and torch.equal(out_p[:L.total_bytes], ref_p)
+
+
+def test_pack_dev_reports_size_and_flag_errors(gpu):
+    torch, B = gpu
+    N, K = 512, 512
+    W = to_dev(torch, inputs.weight(N, K, 52, "pdev2"))
+    flags = np.zeros(16, np.uint8)
+    flags[[1, 5, 6]] = 1
+    L = B.patch_packed_size(N, K, flags)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fd = torch.from_numpy(flags).cuda()
+    small = torch.full((L.total_bytes - 1024,), 0xAB, dtype=torch.uint8, device="cuda")   # above the all-2:4 minimum, below the need
+    B.patch_pack_dev(W, fd, out=small, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_SIZE
+    assert (small[L.payload_off:] == 0xAB).all()               # no payload was written
+    with pytest.raises(B.PatchError) as e:
+        B.patch_read_layout(small)
+    assert e.value.status == B.ERR_FORMAT
+    with pytest.raises(B.PatchError) as e:                      # below the smallest possible blob: refused on the host
+        B.patch_pack_dev(W, fd, out=torch.empty(16 * 18432, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == B.ERR_SIZE
+    status.zero_()
+    bad = flags.copy()
+    bad[3] = 7
+    out = B.patch_pack_dev(W, torch.from_numpy(bad).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_FLAG
+    ref, _ = B.patch_pack(W, flags)                             # the bad flag was packed as dense, which flags[3] is
+    assert torch.equal(out[:L.total_bytes], ref)
+
+
+def test_device_only_deployment_chain(gpu, oracle):
+    """logits -> hard masks -> blob -> GEMM with no flag ever visiting the host before the layout read-back."""
+    torch, B = gpu
+    N, K, M = 768, 512, 5
+    W = inputs.weight(N, K, 53, "chain2")
+    X = inputs.activation(M, K, 53, "chain2", M)
+    PT, P6 = logits(N, K, 0.5, 53, "chain2")
+    flags_d, patterns_d = B.patch_hard_mask(torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), N, K)
+    packed = B.patch_pack_dev(to_dev(torch, W), flags_d, patterns=patterns_d)
+    L = B.patch_read_layout(packed)
+    ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+    Y = to_bits(B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws))
+    rf, rp = oracle.hard_mask(PT, P6, N, K)
+    assert (L.n_dense, L.n_sparse) == (int((rf == 0).sum()), int((rf == 1).sum()))
+    Y32, _ = oracle.gemm_f64(X, oracle.unpack(oracle.pack_patterns(W, rf, rp)[0]))
+    relF, maxrel = oracle.parity_metrics(f32(Y), Y32)
+    assert relF <= 2e-3 and maxrel <= 1e-2, (relF, maxrel)
