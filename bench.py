@@ -542,7 +542,7 @@ def run_masks(args):
     t_plain = time_graph(graph_of(lambda: soft(B.MASK_NO_NOISE)), 50)
     t_hard = time_graph(graph_of(hard), 50)
     t_bwd = time_graph(graph_of(backward), 50)
-    # packing with the hard masks just computed (flags go through the host, as the entry point requires)
+    # packing with the hard masks just computed (the flags visit the host only to size the buffers)
     hard()
     torch.cuda.synchronize()
     pk = []
@@ -556,7 +556,7 @@ def run_masks(args):
         torch.cuda.synchronize()
         e0.record()
         for m, fl, L, out in pk:
-            B.patch_pack_patterns(m["W"], fl, m["patterns"], layout=L, out=out)
+            B.patch_pack_dev(m["W"], m["flags"], patterns=m["patterns"], out=out)
         e1.record()
         torch.cuda.synchronize()
         if rep:
@@ -614,7 +614,7 @@ def run_masks(args):
                                "frac_of_measured_hbm": elements * 16.0 / t_bwd / 1e9 / peaks["hbm_gbs"],
                                "note": "16 B per element: W, Gw and six logits read, six logit gradients written; noise on"},
         "pack_patterns": {"ms_per_step": t_pack * 1e3, "gbs": pack_bytes / t_pack / 1e9,
-                          "note": "includes the host-built tile table and its copy, per matrix"},
+                          "note": "patch_pack_dev with the flags and candidates patch_hard_mask left on the device"},
         "e2e": {"value": elements * MASK_BYTES_PER_ELEMENT / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": 32 * len(mats), "ms_per_step": e2e_s * 1e3},
         "regularizers_of_last_step": reg,
