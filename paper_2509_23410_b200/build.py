@@ -15,7 +15,8 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f != "mma_rate_probe.cu"]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)
+            if f != "mma_rate_probe.cu" and os.path.isfile(os.path.join(CSRC, f))]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "patch.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
