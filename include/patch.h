@@ -17,7 +17,7 @@
  *   - Entry points may be called from several host threads (on different streams or devices);
  *     calls that share a workspace must be ordered on one stream.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
- *     and return; patch_pack, patch_gemm_host and patch_gemm_host_batch are the exceptions noted below.
+ *     and return; patch_pack, patch_gemm_host and the patch_gemm_host_batch pair are the exceptions noted below.
  *   - Supported: tile_n = tile_k = 128, N % 128 == 0, K % 128 == 0, device pointers 16-byte
  *     aligned, leading dimensions multiples of 8 elements.  Device must be sm_100
  *     (PATCH_ERR_ARCH otherwise; there is no fallback path).
@@ -215,6 +215,9 @@ int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* layout,
  * launches carry PATCH_GEMM_INPUT_STATIC whenever `weights_static` is non-zero (the caller's
  * promise that no packed weight is written on this stream meanwhile).  Jobs are independent:
  * no job's X_stage_dev, Y_stage_dev or Y_host may alias another's; jobs may share a workspace.
+ * Copies of consecutive jobs whose host buffers AND staging buffers are both adjacent in memory
+ * (job i+1's begin where job i's end) are issued as one copy, so a step whose activations live
+ * in one pinned arena, staged in one device arena in the same order, costs one transfer each way.
  */
 typedef struct {
     const void* X_host;             /* bf16 [M x K] contiguous */
@@ -228,6 +231,19 @@ typedef struct {
     size_t workspace_bytes;
 } patch_host_job_t;
 int patch_gemm_host_batch(const patch_host_job_t* jobs, int n_jobs, int weights_static, void* stream);
+
+/*
+ * The same step with the transfers overlapped with the GEMMs.  The jobs are cut into `n_chunks`
+ * runs of consecutive jobs (by bytes moved); run c's activations are copied on `copy_in_stream`,
+ * its GEMMs run on `stream` once they have landed, its results are copied back on
+ * `copy_out_stream` once they are computed -- so run c+1's copy in, run c's GEMMs and run c-1's
+ * copy out proceed at the same time (PCIe is full duplex).  The three streams must be distinct
+ * and are all synchronised before the call returns (also when it returns an error after having
+ * enqueued part of the work).  2 * n_chunks events are created and destroyed inside the call;
+ * 1 <= n_chunks <= 64 (clamped to n_jobs).  Everything else as for patch_gemm_host_batch.
+ */
+int patch_gemm_host_batch_pipelined(const patch_host_job_t* jobs, int n_jobs, int weights_static, int n_chunks,
+                                    void* stream, void* copy_in_stream, void* copy_out_stream);
 
 /*
  * patch_gemm for callers that cannot allocate device memory.  (The paper has no counterpart;

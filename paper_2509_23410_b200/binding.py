@@ -24,7 +24,7 @@ ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
-           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch",
+           "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch", "patch_gemm_host_batch_pipelined",
            "patch_gemm_noalloc",
            "patch_hard_mask", "patch_pack_patterns", "patch_pack_dev", "patch_read_layout", "patch_soft_mask_workspace_size", "patch_soft_mask",
            "patch_mask_regularizers", "patch_mask_regularizer_coefficients", "patch_soft_mask_backward",
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         L.patch_gemm_host.argtypes = [vp, i64, ctypes.POINTER(Layout), vp, vp, vp, vp, vp, sz, vp]
         L.patch_gemm_noalloc.argtypes = [vp, i64, i64, ctypes.POINTER(Layout), vp, vp, i64, vp]
         L.patch_gemm_host_batch.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp]
+        L.patch_gemm_host_batch_pipelined.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp]
         L.patch_hard_mask.argtypes = [vp, vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp]
         L.patch_pack_patterns.argtypes = [vp, i64, vp, vp, ctypes.POINTER(Layout), vp, sz, vp, vp]
         L.patch_soft_mask_workspace_size.argtypes = [i64, i64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(sz)]
@@ -244,6 +245,14 @@ def patch_gemm_host_batch(batch, weights_static: bool = False, stream=None):
     """One step of GEMMs with host X / Y: all copies in, all launches, all copies out, one synchronisation."""
     _check(lib().patch_gemm_host_batch(batch, len(batch), 1 if weights_static else 0, _stream(stream)),
            "patch_gemm_host_batch")
+
+
+def patch_gemm_host_batch_pipelined(batch, copy_in_stream, copy_out_stream, n_chunks: int = 4,
+                                    weights_static: bool = False, stream=None):
+    """The same step with copies in, GEMMs and copies out overlapped over ``n_chunks`` runs of jobs (three streams)."""
+    _check(lib().patch_gemm_host_batch_pipelined(batch, len(batch), 1 if weights_static else 0, int(n_chunks),
+                                                 _stream(stream), _stream(copy_in_stream), _stream(copy_out_stream)),
+           "patch_gemm_host_batch_pipelined")
 
 
 def patch_gemm_noalloc(X, layout: Layout, packed, Y, stream=None):

@@ -124,11 +124,12 @@ extern "C" int patch_gemm_host(const void* X_host, int64_t M, const patch_layout
     return cudaStreamSynchronize(s) == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
-extern "C" int patch_gemm_host_batch(const patch_host_job_t* jobs, int n_jobs, int weights_static, void* stream) {
+// Validation shared by the batched host entry points: everything is checked before anything is enqueued.
+static int check_host_jobs(const patch_host_job_t* jobs, int n_jobs) {
     if (n_jobs < 0) return PATCH_ERR_SHAPE;
     if (n_jobs == 0) return PATCH_OK;
     if (!jobs) return PATCH_ERR_NULL;
-    for (int i = 0; i < n_jobs; ++i) {      // everything is checked before anything is enqueued
+    for (int i = 0; i < n_jobs; ++i) {
         const patch_host_job_t& j = jobs[i];
         if (!j.layout) return PATCH_ERR_NULL;
         int rc = validate_layout(j.layout);
@@ -136,26 +137,109 @@ extern "C" int patch_gemm_host_batch(const patch_host_job_t* jobs, int n_jobs, i
         if (j.M < 0) return PATCH_ERR_SHAPE;
         if (j.M > 0 && (!j.X_host || !j.Y_host || !j.X_stage_dev || !j.Y_stage_dev || !j.packed_dev)) return PATCH_ERR_NULL;
     }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    for (int i = 0; i < n_jobs; ++i) {
+    return PATCH_OK;
+}
+
+// Copies of jobs [first, last) in one direction.  Consecutive jobs whose host buffers and staging buffers are
+// both adjacent in memory are issued as one copy: a step whose activations live in one host arena costs one
+// transfer each way.
+static bool copy_jobs(const patch_host_job_t* jobs, int first, int last, bool inbound, cudaStream_t s) {
+    const char* run_host = nullptr; const char* run_dev = nullptr; size_t run_bytes = 0;
+    auto flush = [&]() -> bool {
+        if (!run_bytes) return true;
+        const cudaError_t e = inbound
+            ? cudaMemcpyAsync(const_cast<char*>(run_dev), run_host, run_bytes, cudaMemcpyHostToDevice, s)
+            : cudaMemcpyAsync(const_cast<char*>(run_host), run_dev, run_bytes, cudaMemcpyDeviceToHost, s);
+        run_bytes = 0;
+        return e == cudaSuccess;
+    };
+    for (int i = first; i < last; ++i) {
         const patch_host_job_t& j = jobs[i];
-        if (j.M && cudaMemcpyAsync(j.X_stage_dev, j.X_host, size_t(j.M) * j.layout->K * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
-            return PATCH_ERR_CUDA;
+        if (!j.M) continue;
+        const char* h = static_cast<const char*>(inbound ? j.X_host : j.Y_host);
+        const char* d = static_cast<const char*>(inbound ? j.X_stage_dev : j.Y_stage_dev);
+        const size_t bytes = size_t(j.M) * size_t(inbound ? j.layout->K : j.layout->N) * 2;
+        if (run_bytes && h == run_host + run_bytes && d == run_dev + run_bytes) { run_bytes += bytes; continue; }
+        if (!flush()) return false;
+        run_host = h; run_dev = d; run_bytes = bytes;
     }
-    // with two or more jobs the operation before any launch is another launch or the copy of a different X
-    const int flags = weights_static ? (PATCH_GEMM_WEIGHTS_STATIC | (n_jobs >= 2 ? PATCH_GEMM_INPUT_STATIC : 0)) : 0;
-    for (int i = 0; i < n_jobs; ++i) {
+    return flush();
+}
+
+static int launch_jobs(const patch_host_job_t* jobs, int first, int last, int flags, void* stream) {
+    for (int i = first; i < last; ++i) {
         const patch_host_job_t& j = jobs[i];
         int rc = patch_gemm_ex(j.X_stage_dev, j.layout->K, j.M, j.layout, j.packed_dev, j.Y_stage_dev, j.layout->N,
                                j.workspace_dev, j.workspace_bytes, nullptr, stream, PATCH_VARIANT_AUTO | flags);
         if (rc) return rc;
     }
-    for (int i = 0; i < n_jobs; ++i) {
-        const patch_host_job_t& j = jobs[i];
-        if (j.M && cudaMemcpyAsync(j.Y_host, j.Y_stage_dev, size_t(j.M) * j.layout->N * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-            return PATCH_ERR_CUDA;
-    }
+    return PATCH_OK;
+}
+
+extern "C" int patch_gemm_host_batch(const patch_host_job_t* jobs, int n_jobs, int weights_static, void* stream) {
+    int rc = check_host_jobs(jobs, n_jobs);
+    if (rc || n_jobs == 0) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!copy_jobs(jobs, 0, n_jobs, true, s)) return PATCH_ERR_CUDA;
+    // with two or more jobs the operation before any launch is another launch or the copy of a different X
+    const int flags = weights_static ? (PATCH_GEMM_WEIGHTS_STATIC | (n_jobs >= 2 ? PATCH_GEMM_INPUT_STATIC : 0)) : 0;
+    rc = launch_jobs(jobs, 0, n_jobs, flags, stream);
+    if (rc) return rc;
+    if (!copy_jobs(jobs, 0, n_jobs, false, s)) return PATCH_ERR_CUDA;
     return cudaStreamSynchronize(s) == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
+extern "C" int patch_gemm_host_batch_pipelined(const patch_host_job_t* jobs, int n_jobs, int weights_static, int n_chunks,
+                                               void* stream, void* copy_in_stream, void* copy_out_stream) {
+    int rc = check_host_jobs(jobs, n_jobs);
+    if (rc || n_jobs == 0) return rc;
+    if (n_chunks < 1 || n_chunks > 64) return PATCH_ERR_SHAPE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream), sin = static_cast<cudaStream_t>(copy_in_stream),
+                 sout = static_cast<cudaStream_t>(copy_out_stream);
+    if (s == sin || s == sout || sin == sout) return PATCH_ERR_SHAPE;      // three distinct streams
+    if (n_chunks > n_jobs) n_chunks = n_jobs;
+    // chunk boundaries by output bytes, so that the last copy out (the only one nothing overlaps) is short
+    int bound[65];
+    {
+        double total = 0, acc = 0;
+        for (int i = 0; i < n_jobs; ++i) total += double(jobs[i].M) * double(jobs[i].layout->N + jobs[i].layout->K);
+        int c = 0;
+        bound[0] = 0;
+        for (int i = 0; i < n_jobs && c + 1 < n_chunks; ++i) {
+            acc += double(jobs[i].M) * double(jobs[i].layout->N + jobs[i].layout->K);
+            if (acc >= total * (c + 1) / n_chunks && n_jobs - (i + 1) >= n_chunks - (c + 1)) bound[++c] = i + 1;
+        }
+        while (c + 1 < n_chunks) { bound[c + 1] = bound[c] + 1; ++c; }
+        bound[n_chunks] = n_jobs;
+    }
+    cudaEvent_t landed[64], done[64];
+    int n_events = 0;
+    auto cleanup = [&]() { for (int i = 0; i < n_events; ++i) { cudaEventDestroy(landed[i]); cudaEventDestroy(done[i]); } };
+    for (; n_events < n_chunks; ++n_events)
+        if (cudaEventCreateWithFlags(&landed[n_events], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&done[n_events], cudaEventDisableTiming) != cudaSuccess) {
+            cleanup();
+            return PATCH_ERR_CUDA;
+        }
+    // every X is on the device before the GEMM that reads it (event), and is written by a copy on another stream
+    const int flags = weights_static ? (PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC) : 0;
+    rc = PATCH_OK;
+    bool ok = true;
+    for (int c = 0; c < n_chunks && ok && !rc; ++c) {
+        ok = copy_jobs(jobs, bound[c], bound[c + 1], true, sin) && cudaEventRecord(landed[c], sin) == cudaSuccess &&
+             cudaStreamWaitEvent(s, landed[c], 0) == cudaSuccess;
+        if (!ok) break;
+        rc = launch_jobs(jobs, bound[c], bound[c + 1], flags, stream);
+        if (rc) break;
+        ok = cudaEventRecord(done[c], s) == cudaSuccess && cudaStreamWaitEvent(sout, done[c], 0) == cudaSuccess &&
+             copy_jobs(jobs, bound[c], bound[c + 1], false, sout);
+    }
+    // whatever was enqueued is waited for, also on failure: the caller's buffers are then quiescent
+    const bool synced = cudaStreamSynchronize(sin) == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess &&
+                        cudaStreamSynchronize(sout) == cudaSuccess;
+    cleanup();
+    if (rc) return rc;
+    return ok && synced ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
 extern "C" const char* patch_strerror(int status) {

@@ -213,3 +213,13 @@ def test_pack_dev_validates_on_the_host():
     assert lib.patch_pack_dev(p, 128, p, p + 2, 128, 128, 128, 128, p, 1 << 20, None, None) == B.ERR_ALIGN
     assert lib.patch_pack_dev(p, 128, p, None, 128, 128, 128, 128, p, 1024 + 18431, None, None) == B.ERR_SIZE
     assert lib.patch_read_layout(None, None, None) == B.ERR_NULL
+
+
+def test_pipelined_host_batch_validates_before_enqueueing():
+    import ctypes
+    from paper_2509_23410_b200 import binding as B
+    lib = B.lib()
+    assert lib.patch_gemm_host_batch_pipelined(None, 0, 0, 4, None, None, None) == 0        # empty batch: nothing to do
+    assert lib.patch_gemm_host_batch_pipelined(None, 3, 0, 4, None, None, None) == B.ERR_NULL
+    jobs = (B.HostJob * 1)()
+    assert lib.patch_gemm_host_batch_pipelined(jobs, 1, 0, 4, None, None, None) == B.ERR_NULL   # no layout

@@ -581,3 +581,46 @@ def test_host_batch_entry_point(gpu, oracle):
         B.patch_gemm_host_batch(batch, weights_static=weights_static)      # returns after the stream is synchronised
         for j, ref in zip(jobs, refs):
             check_parity(oracle, j["Yh"].view(torch.int16).numpy().view(np.uint16), ref, "host batch")
+
+
+def test_host_batch_merges_adjacent_buffers(gpu, oracle):
+    """Jobs whose host and staging buffers are adjacent (one arena each) are copied in one transfer; a job in
+    between with separate buffers breaks the run.  Results must not depend on how the copies were grouped."""
+    torch, B = gpu
+    shapes = [(1024, 768, 4, 0.5), (512, 768, 16, 1.0), (768, 512, 7, 0.0), (640, 1024, 2, 0.4), (256, 256, 33, 0.6)]
+    cases = []
+    for i, (N, K, M, p) in enumerate(shapes):
+        W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=p, stream=("arena", i)), 52, M)
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        cases.append((N, K, M, X, L, packed, oracle.gemm_f64(X, oracle.prune(W, flags))[0]))
+    nx, ny = sum(M * K for N, K, M, *_ in cases), sum(M * N for N, K, M, *_ in cases)
+    xh, yh = torch.empty(nx, dtype=torch.bfloat16).pin_memory(), torch.zeros(ny, dtype=torch.bfloat16).pin_memory()
+    xd, yd = torch.empty(nx, dtype=torch.bfloat16, device="cuda"), torch.empty(ny, dtype=torch.bfloat16, device="cuda")
+    jobs, ox, oy = [], 0, 0
+    for i, (N, K, M, X, L, packed, ref) in enumerate(cases):
+        ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+        j = dict(layout=L, packed=packed, ws=ws, Xh=xh[ox:ox + M * K].view(M, K), Yh=yh[oy:oy + M * N].view(M, N),
+                 X=xd[ox:ox + M * K].view(M, K), Y=yd[oy:oy + M * N].view(M, N))
+        if i == 2:      # separate buffers in the middle of the arena run
+            j.update(Xh=torch.empty((M, K), dtype=torch.bfloat16).pin_memory(), Yh=torch.zeros((M, N), dtype=torch.bfloat16).pin_memory(),
+                     X=torch.empty((M, K), dtype=torch.bfloat16, device="cuda"), Y=torch.empty((M, N), dtype=torch.bfloat16, device="cuda"))
+        j["Xh"].copy_(torch.from_numpy(np.ascontiguousarray(X).view(np.int16)).view(torch.bfloat16))
+        jobs.append(j)
+        ox, oy = ox + M * K, oy + M * N
+    batch = B.make_host_batch(jobs)
+    B.patch_gemm_host_batch(batch, weights_static=True)
+    for j, c in zip(jobs, cases):
+        check_parity(oracle, j["Yh"].contiguous().view(torch.int16).numpy().view(np.uint16), c[6], "arena batch")
+    # the pipelined form: copies in, GEMMs and copies out on three streams, any number of chunks
+    first = [j["Yh"].clone() for j in jobs]
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    for n_chunks in (1, 2, 3, 5, 64):
+        for j in jobs:
+            j["Yh"].zero_()
+        B.patch_gemm_host_batch_pipelined(batch, s_in, s_out, n_chunks=n_chunks, weights_static=True)
+        for j, f in zip(jobs, first):
+            assert torch.equal(j["Yh"], f), n_chunks          # the kernels are deterministic: same bits
+    lib = B.lib()
+    cur = torch.cuda.current_stream().cuda_stream
+    assert lib.patch_gemm_host_batch_pipelined(batch, len(batch), 1, 2, cur, cur, s_out.cuda_stream) == B.ERR_SHAPE
+    assert lib.patch_gemm_host_batch_pipelined(batch, len(batch), 1, 0, cur, s_in.cuda_stream, s_out.cuda_stream) == B.ERR_SHAPE
