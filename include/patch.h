@@ -324,6 +324,8 @@ int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t* tile_flag
  *   status_dev      optional device int (caller zeroes it): PATCH_ERR_SIZE if the blob did not fit
  *                   (then nothing but a header without magic number is written), PATCH_ERR_FLAG for
  *                   a flag other than 0 / 1 (packed as dense) or a candidate index above 5.
+ * Every CTA reads the whole flag array (one byte per tile, from L2), so the extra work grows with the
+ * square of the tile count: negligible for the tens of thousands of tiles of an LLM weight.
  * Enqueues one kernel; no copy, no synchronisation.  The host-side layout that patch_gemm
  * needs comes from patch_packed_size when the flags are also known on the host, else from
  * patch_read_layout.
