@@ -49,24 +49,25 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) {
 
 // Keep the two largest magnitudes of four bf16 values (ties: lower index first).
 // Returns the 4-bit position code i0 | (i1 << 2), i0 < i1, and the two kept bit patterns.
+// Each value becomes one sort key  magnitude << 3 | (3 - index) << 1 | sign : keys are distinct, order by
+// magnitude and then by lower index (the sign sits below the index bits and cannot decide), and a key holds
+// everything needed to rebuild its value and position.  The two largest of four keys come out of a
+// five-comparator network.
 __device__ __forceinline__ uint32_t top2_of_4(const uint32_t w[4], uint32_t& v0, uint32_t& v1) {
-    // distinct sort keys: magnitude in the high bits, reversed index in the low two bits
     uint32_t key[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) key[j] = ((w[j] & 0x7FFFu) << 2) | uint32_t(3 - j);
-    bool keep[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        int before = 0;  // number of elements ordered before j
-#pragma unroll
-        for (int l = 0; l < 4; ++l) before += key[l] > key[j];
-        keep[j] = before < 2;
-    }
-    // exactly two are kept: the first kept index is at most 2, the second at least 1
-    const uint32_t i0 = keep[0] ? 0u : (keep[1] ? 1u : 2u);
-    const uint32_t i1 = keep[3] ? 3u : (keep[2] ? 2u : 1u);
-    v0 = keep[0] ? w[0] : (keep[1] ? w[1] : w[2]);
-    v1 = keep[3] ? w[3] : (keep[2] ? w[2] : w[1]);
+    for (int j = 0; j < 4; ++j) key[j] = ((w[j] << 3) & 0x3FFF8u) | (w[j] >> 15) | (uint32_t(3 - j) << 1);
+    const uint32_t hi01 = max(key[0], key[1]), lo01 = min(key[0], key[1]);
+    const uint32_t hi23 = max(key[2], key[3]), lo23 = min(key[2], key[3]);
+    const uint32_t first = max(hi01, hi23);
+    // the runner-up is the loser of the final or the partner the winner beat in its own pair
+    const uint32_t second = max(min(hi01, hi23), hi01 > hi23 ? lo01 : lo23);
+    // position order: the larger index field (3 - index) is the lower position
+    const bool swap = (first & 6u) < (second & 6u);
+    const uint32_t ka = swap ? second : first, kb = swap ? first : second;
+    v0 = (ka >> 3) | ((ka & 1u) << 15);
+    v1 = (kb >> 3) | ((kb & 1u) << 15);
+    const uint32_t i0 = 3u - ((ka >> 1) & 3u), i1 = 3u - ((kb >> 1) & 3u);
     return i0 | (i1 << 2);
 }
 
