@@ -47,28 +47,25 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) {
     return v;
 }
 
-// Keep the two largest magnitudes of four bf16 values (ties: lower index first).
-// Returns the 4-bit position code i0 | (i1 << 2), i0 < i1, and the two kept bit patterns.
-// Each value becomes one sort key  magnitude << 3 | (3 - index) << 1 | sign : keys are distinct, order by
-// magnitude and then by lower index (the sign sits below the index bits and cannot decide), and a key holds
-// everything needed to rebuild its value and position.  The two largest of four keys come out of a
-// five-comparator network.
-__device__ __forceinline__ uint32_t top2_of_4(const uint32_t w[4], uint32_t& v0, uint32_t& v1) {
-    uint32_t key[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) key[j] = ((w[j] << 3) & 0x3FFF8u) | (w[j] >> 15) | (uint32_t(3 - j) << 1);
-    const uint32_t hi01 = max(key[0], key[1]), lo01 = min(key[0], key[1]);
-    const uint32_t hi23 = max(key[2], key[3]), lo23 = min(key[2], key[3]);
+// The two kept positions i0 < i1 of a group whose four bf16 values are the halves of (x0, x1):
+// the two largest magnitudes, equal magnitudes ordered by position (lower first).  Each value gets the
+// sort key  magnitude << 2 | (3 - position): keys are distinct, and the two largest of four come out of a
+// five-comparator network with their positions in the low bits.
+__device__ __forceinline__ void top2_positions(uint32_t x0, uint32_t x1, uint32_t& i0, uint32_t& i1) {
+    const uint32_t k0 = ((x0 & 0x7FFFu) << 2) | 3u, k1 = ((x0 >> 14) & 0x1FFFCu) | 2u;
+    const uint32_t k2 = ((x1 & 0x7FFFu) << 2) | 1u, k3 = (x1 >> 14) & 0x1FFFCu;
+    const uint32_t hi01 = max(k0, k1), lo01 = min(k0, k1), hi23 = max(k2, k3), lo23 = min(k2, k3);
     const uint32_t first = max(hi01, hi23);
     // the runner-up is the loser of the final or the partner the winner beat in its own pair
     const uint32_t second = max(min(hi01, hi23), hi01 > hi23 ? lo01 : lo23);
-    // position order: the larger index field (3 - index) is the lower position
-    const bool swap = (first & 6u) < (second & 6u);
-    const uint32_t ka = swap ? second : first, kb = swap ? first : second;
-    v0 = (ka >> 3) | ((ka & 1u) << 15);
-    v1 = (kb >> 3) | ((kb & 1u) << 15);
-    const uint32_t i0 = 3u - ((ka >> 1) & 3u), i1 = 3u - ((kb >> 1) & 3u);
-    return i0 | (i1 << 2);
+    const uint32_t pa = 3u - (first & 3u), pb = 3u - (second & 3u);
+    i0 = min(pa, pb);
+    i1 = max(pa, pb);
+}
+
+// {value at position i1 : value at position i0} of the group (x0, x1): element j is bytes 2j, 2j + 1 of the pair
+__device__ __forceinline__ uint32_t gather_pair(uint32_t x0, uint32_t x1, uint32_t i0, uint32_t i1) {
+    return __byte_perm(x0, x1, (i0 | (i1 << 8)) * 0x22u + 0x1010u);
 }
 
 // The two kept positions of candidate c (row c of the matrix S of the six 2:4 masks, rows in
@@ -87,29 +84,47 @@ struct DeviceFlags {
 // writes the header and the padding behind the table; every CTA writes its own table entry.
 // Returns false if the blob does not fit `capacity` (then only a header without magic number is written).
 __device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int t, uint8_t* blob, int* status, TileDesc& d) {
-    __shared__ unsigned long long s_part[8][3];
+    __shared__ unsigned long long s_part[8][2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    unsigned long long before = 0, total = 0, dense = 0;
+    // count the 2:4 flags before tile t and in total; four flags per load where the array is word aligned
+    unsigned long long sparse_before = 0, sparse_total = 0;
     bool bad = false;
-    for (int64_t i = tid; i < F.T; i += 256) {
+    const int64_t words = (reinterpret_cast<uintptr_t>(F.flags) & 3u) == 0 ? F.T / 4 : 0;
+    for (int64_t i = tid; i < words; i += 256) {
+        const uint32_t w = reinterpret_cast<const uint32_t*>(F.flags)[i];
+        uint32_t ones = w & 0x01010101u;
+        if (w & 0xFEFEFEFEu) {          // a byte that is neither 0 nor 1: an error, packed as dense
+            bad = true;
+            ones = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) ones |= ((w >> (8 * q)) & 0xFFu) == 1u ? 1u << (8 * q) : 0u;
+        }
+        const int64_t first = 4 * i;                      // flags first .. first + 3; those below t count as "before"
+        const uint32_t below = first + 4 <= t ? 0xFFFFFFFFu : first >= t ? 0u : (1u << (8 * uint32_t(t - first))) - 1u;
+        sparse_total += __popc(ones);
+        sparse_before += __popc(ones & below);
+    }
+    for (int64_t i = 4 * words + tid; i < F.T; i += 256) {
         const uint8_t f = F.flags[i];
         bad |= f > 1;
-        const unsigned long long b = f == PATCH_TILE_SPARSE_2_4 ? kSparseBytes : kDenseBytes;
-        total += b;
-        before += i < t ? b : 0;
-        dense += f == PATCH_TILE_SPARSE_2_4 ? 0 : 1;
+        sparse_total += f == PATCH_TILE_SPARSE_2_4;
+        sparse_before += (f == PATCH_TILE_SPARSE_2_4) && i < t;
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
-        before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
-        total += __shfl_xor_sync(0xFFFFFFFFu, total, off);
-        dense += __shfl_xor_sync(0xFFFFFFFFu, dense, off);
+        sparse_total += __shfl_xor_sync(0xFFFFFFFFu, sparse_total, off);
+        sparse_before += __shfl_xor_sync(0xFFFFFFFFu, sparse_before, off);
     }
-    if (lane == 0) { s_part[warp][0] = before; s_part[warp][1] = total; s_part[warp][2] = dense; }
+    if (lane == 0) { s_part[warp][0] = sparse_total; s_part[warp][1] = sparse_before; }
     bad = __syncthreads_or(bad) != 0;
-    before = total = dense = 0;
+    sparse_total = sparse_before = 0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) { before += s_part[w][0]; total += s_part[w][1]; dense += s_part[w][2]; }
+    for (int w = 0; w < 8; ++w) { sparse_total += s_part[w][0]; sparse_before += s_part[w][1]; }
+    // as payload bytes: every tile a dense one, minus the saving of each 2:4 tile
+    constexpr unsigned long long kSaving = kDenseBytes - kSparseBytes;
+    const unsigned long long before = (unsigned long long)t * kDenseBytes - sparse_before * kSaving;
+    const unsigned long long total = (unsigned long long)F.T * kDenseBytes - sparse_total * kSaving;
+    const unsigned long long dense = (unsigned long long)F.T - sparse_total;
     const uint64_t payload_off = (kHeaderBytes + 16 * uint64_t(F.T) + 1023) / 1024 * 1024;
     const uint64_t size = payload_off + total;
     const bool fits = size <= F.capacity && size / 16 <= 0xFFFFFFF0ull;
@@ -167,34 +182,41 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
         }
     } else {
         uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
+        // all of the thread's loads are issued before any of the selection work: 128 bytes in flight per thread
+        uint4 va[4], vb[4];
+        uint32_t vgiven[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 3, u = idx & 7u;
+            const uint16_t* src = wt + int64_t(r) * ldw + u * 16;
+            va[it] = ld_stream(src);
+            vb[it] = ld_stream(src + 8);
+            if (GIVEN)   // the four candidate indices of this thread's groups: one aligned 4-byte load
+                vgiven[it] = *reinterpret_cast<const uint32_t*>(patterns + (int64_t(tn) * kTile + r) * (int64_t(TK) * 32) +
+                                                                tk * 32 + u * 4);
+        }
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             // 16 consecutive elements of one row: four groups -> 8 kept values + 16 metadata bits
             const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 3, u = idx & 7u;
-            const uint16_t* src = wt + int64_t(r) * ldw + u * 16;
-            const uint4 a = ld_stream(src), b = ld_stream(src + 8);
+            const uint4 a = va[it], b = vb[it];
             const uint32_t in[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-            uint32_t out[4], code = 0, given = 0;
-            if (GIVEN)   // the four candidate indices of this thread's groups: one aligned 4-byte load
-                given = *reinterpret_cast<const uint32_t*>(patterns + (int64_t(tn) * kTile + r) * (int64_t(TK) * 32) +
-                                                           tk * 32 + u * 4);
+            uint32_t out[4], code = 0;
+            const uint32_t given = vgiven[it];
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-                const uint32_t w[4] = {in[2 * g] & 0xFFFFu, in[2 * g] >> 16,
-                                       in[2 * g + 1] & 0xFFFFu, in[2 * g + 1] >> 16};
-                uint32_t v0, v1, nib;
+                uint32_t i0, i1;
                 if (GIVEN) {
                     uint32_t c = (given >> (8 * g)) & 0xFFu;
                     if (c > 5u) { if (status) *status = PATCH_ERR_FLAG; c = 0; }
-                    nib = (kCandidateCodes >> (4 * c)) & 0xFu;
-                    const uint32_t i0 = nib & 3u, i1 = nib >> 2;
-                    v0 = i0 == 0 ? w[0] : i0 == 1 ? w[1] : w[2];
-                    v1 = i1 == 1 ? w[1] : i1 == 2 ? w[2] : w[3];
+                    const uint32_t nib = (kCandidateCodes >> (4 * c)) & 0xFu;
+                    i0 = nib & 3u;
+                    i1 = nib >> 2;
                 } else {
-                    nib = top2_of_4(w, v0, v1);
+                    top2_positions(in[2 * g], in[2 * g + 1], i0, i1);
                 }
-                code |= nib << (4 * g);
-                out[g] = v0 | (v1 << 16);
+                code |= (i0 | (i1 << 2)) << (4 * g);
+                out[g] = gather_pair(in[2 * g], in[2 * g + 1], i0, i1);
             }
             *reinterpret_cast<uint4*>(pay + atom_chunk_offset(r, u)) = make_uint4(out[0], out[1], out[2], out[3]);
             // metadata row L = 16q + 8h + i, word j, low half for tile rows 16q+i, high for 16q+8+i
