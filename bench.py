@@ -475,8 +475,8 @@ def run_ours(args):
 MASK_BYTES_PER_ELEMENT = 10.0      # soft mask: 2 B of W + 6 B of 2:4 logits read, 2 B of masked weight written
 # warp instructions per group of four weights per lane of soft_mask_kernel<noise>, and its DRAM traffic per
 # algorithmic byte, from the ncu capture summarised in profiles/soft_mask_kernel_llama7b_block.md
-# (38 458 368 instructions for a 4096 x 4096 launch; 152.8 MB read + written against 167.8 MB)
-MASK_WARP_INST_PER_GROUP = 293.4
+# (32 287 744 instructions for a 4096 x 4096 launch; 152.3 MB read + written against 167.8 MB)
+MASK_WARP_INST_PER_GROUP = 246.3
 MASK_TRAFFIC_RATIO = 0.91
 
 

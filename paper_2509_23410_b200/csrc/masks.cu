@@ -31,12 +31,18 @@ __device__ __forceinline__ uint64_t mix_final(uint64_t x) {
 // logarithm elsewhere.  u and v are built from the bits without an integer-to-float conversion:
 // 1.b (binary) minus 1 is b / 2^23 exactly, and adding 2^-24 centres it in its cell; both stay
 // within 24 significant bits, so both are exact.
+__device__ __forceinline__ float lg2_approx(float x) {   // log2 of a normal positive number
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ float gumbel_log2(uint32_t bits) {
     const float u = (__uint_as_float(0x3F800000u | bits) - 1.0f) + 5.9604645e-8f;
     const float v = (__uint_as_float(0x3F800000u | (bits ^ 0x7FFFFFu)) - 1.0f) + 5.9604645e-8f;
-    const float series = v * (1.0f + v * (0.5f + v * (0.33333334f + v * 0.25f)));
-    const float direct = -0.69314718f * __log2f(u);
-    return -__log2f(v < 0.015625f ? series : direct);
+    const float series = v * (1.0f + v * (0.5f + v * 0.33333334f));      // v < 2^-6: the next term is below 2^-20 relative
+    const float direct = -0.69314718f * lg2_approx(u);
+    return -lg2_approx(v < 0.015625f ? series : direct);
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {   // 2^x; results below 2^-126 flush to zero
@@ -57,7 +63,9 @@ __device__ __forceinline__ float softmax2_terms(float (&a)[NCLS]) {
     float sum = 0.f;
 #pragma unroll
     for (int k = 0; k < NCLS; ++k) { a[k] = ex2_approx(a[k] - top); sum += a[k]; }
-    return __fdividef(1.0f, sum);
+    float inv;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(sum));      // sum is in [1, NCLS]
+    return inv;
 }
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
@@ -131,12 +139,12 @@ soft_mask_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __res
             float mw[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t bits = j & 1 ? in[2 * g + (j >> 1)] >> 16 : in[2 * g + (j >> 1)] & 0xFFFFu;
-                const float w = bf16_bits_to_float(bits);
+                const uint32_t pair = in[2 * g + (j >> 1)];               // a bf16 is the upper half of its fp32
+                const float w = __uint_as_float(j & 1 ? pair & 0xFFFF0000u : pair << 16);
                 const float m = fmaf(scale, m24[j], mt);                   // Eq. 4
                 mw[j] = m * w;
                 mvals[4 * g + j] = m;
-                acc_nz += (bits & 0x7FFFu) != 0;
+                acc_nz += w != 0.0f;                                       // -0 is zero
                 acc_mw2 = fmaf(mw[j], mw[j], acc_mw2);
                 acc_w2 = fmaf(w, w, acc_w2);
             }
