@@ -157,9 +157,15 @@ def oracle_sample(cases, budget_s):
             if secs >= budget_s:
                 break
         passes += 1
+    # the oracle's pack (single-threaded C loops) on the first matrix, next to patch_pack's GB/s
+    W, flags, _ = inputs.make_case_inputs(cases[0])
+    t = time.perf_counter()
+    blob, _ = oracle.pack(W, flags)
+    t_pack = time.perf_counter() - t
     return dict(value=flops / secs / 1e12, unit="TFLOP/s", cores=oracle.num_threads(), kind="oracle",
                 sample=f"oracle GEMM (double accumulation) over the step's first {len(done)} GEMMs "
-                       f"({done[0]} .. {done[-1]}), repeated for {secs:.1f} s of CPU time"), secs
+                       f"({done[0]} .. {done[-1]}), repeated for {secs:.1f} s of CPU time",
+                pack_gbs=(W.nbytes + blob.nbytes) / t_pack / 1e9, pack_sample=f"oracle pack of {cases[0]['name']}, one thread"), secs
 
 
 def run_reference(args):
