@@ -26,6 +26,7 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports
 // PATCH_ERR_TIMEOUT through status_dev, drains its copies in flight, frees TMEM and returns.
+#include <cstdlib>
 #include "sm100_ptx.cuh"
 
 namespace patch {
@@ -687,6 +688,18 @@ static int launch_decode_f(bool wstatic, bool xstatic, const CUtensorMap& map, c
     return launch_decode_t<N_TOK, STAGES, false, false>(map, L, packed, M, Y, ldy, workspace, status_dev, stream);
 }
 
+// Which small-M schedule serves a launch: stream-K over all SMs (a lone or dependent GEMM gets the whole
+// GPU's bandwidth) or one CTA per row-block / small cluster (independent GEMMs: several of them are resident
+// at once and together stream faster).  PATCH_DECODE_SCHEDULE=streamk|rowblock forces one (experiments).
+static bool use_rowblock_schedule(bool wstatic, bool xstatic) {
+    static const int forced = [] {
+        const char* e = getenv("PATCH_DECODE_SCHEDULE");
+        return !e ? 0 : e[0] == 's' ? 1 : e[0] == 'r' ? 2 : 0;
+    }();
+    if (forced) return forced == 2;
+    return wstatic && xstatic;
+}
+
 int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                   __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream,
                   bool wstatic, bool xstatic) {
@@ -694,6 +707,8 @@ int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_la
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
+    if (use_rowblock_schedule(wstatic, xstatic))
+        return launch_decode_cluster(map, L, packed, int(M), n_tok, Y, ldy, status_dev, stream, wstatic, xstatic);
     switch (n_tok) {
         case 16:
             if (wstatic && xstatic)

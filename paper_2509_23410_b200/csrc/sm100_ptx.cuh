@@ -231,6 +231,12 @@ __device__ __forceinline__ void store_fragment_transposed(const uint32_t (&v)[16
 // 128-byte swizzle, zero fill outside the matrix.
 int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok);
 
+// Row-block / cluster split-K schedule for M <= 64 (gemm_decode_cluster_sm100.cu), used for GEMMs the caller
+// declared independent of their predecessor (`map`: X tensor map with a box of `n_tok` token rows).
+int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int n_tok,
+                          __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic,
+                          bool xstatic);
+
 #ifdef PATCH_TRACE
 // Debug build only: status_dev is reinterpreted as a buffer of 16 timestamps (ns) per CTA.
 #define PATCH_TRACE_AT(slot) do { if ((threadIdx.x & 31) == 0) reinterpret_cast<unsigned long long*>(status_dev)[(blockIdx.y * gridDim.x + blockIdx.x) * 16 + (slot)] = global_timer_ns(); } while (0)

@@ -624,3 +624,52 @@ def test_host_batch_merges_adjacent_buffers(gpu, oracle):
     cur = torch.cuda.current_stream().cuda_stream
     assert lib.patch_gemm_host_batch_pipelined(batch, len(batch), 1, 2, cur, cur, s_out.cuda_stream) == B.ERR_SHAPE
     assert lib.patch_gemm_host_batch_pipelined(batch, len(batch), 1, 0, cur, s_in.cuda_stream, s_out.cuda_stream) == B.ERR_SHAPE
+
+
+# ---------------------------------------------------------------------------------------------
+# the schedule for GEMMs declared independent of their predecessor (one CTA per row-block, or a
+# small cluster splitting K where the weight has few row-blocks)
+
+
+@pytest.mark.parametrize("N,K", [(128, 128), (128, 256), (256, 1024), (512, 2304), (1024, 1024), (2048, 640), (4224, 1152)])
+@pytest.mark.parametrize("M", [1, 5, 16, 17, 33, 64])
+def test_independent_launch_schedule(gpu, oracle, N, K, M):
+    """Row-block counts 1 .. 33: cluster sizes 8, 4, 2 and 1 (capped by the number of K tiles), all token tiles."""
+    torch, B = gpu
+    p = [0.0, 0.5, 1.0][(N // 128 + K // 128 + M) % 3]
+    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=p, stream=("indep", N, K)), 61, M)
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y32, _ = oracle.gemm_f64(X, What)
+    got = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
+    check_parity(oracle, got, Y32, f"independent N={N} K={K} M={M} p={p}")
+    # the stream-K schedule (no promise) rounds the same sums: both are deterministic, and close
+    other = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO)
+    check_parity(oracle, other, Y32, "stream-K")
+    again = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
+    assert (again == got).all()
+
+
+def test_independent_launches_back_to_back(gpu, oracle):
+    """A stream of independent GEMMs of different shapes and token counts, launched without any
+    synchronisation in between (several kernels are resident at once), twice over the same outputs."""
+    torch, B = gpu
+    shapes = [(1024, 768, 1), (4096, 512, 16), (256, 2048, 40), (2304, 1024, 3), (512, 512, 64), (1536, 1280, 9)]
+    jobs = []
+    for i, (N, K, M) in enumerate(shapes):
+        W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=0.5, stream=("indep-b2b", i)), 62, M)
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        jobs.append(dict(X=to_dev(torch, X), L=L, packed=packed, Y=torch.zeros((M, N), dtype=torch.bfloat16, device="cuda"),
+                         ref=oracle.gemm_f64(X, oracle.prune(W, flags))[0]))
+    ws = torch.zeros(B.patch_gemm_workspace_size(jobs[0]["L"], 64), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for rep in range(3):
+        for j in jobs:
+            B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Y"], workspace=ws, status=status,
+                         variant=B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
+        # a dependent GEMM in the middle of the stream (stream-K schedule, same workspace)
+        B.patch_gemm(jobs[0]["X"], jobs[0]["L"], jobs[0]["packed"], Y=jobs[0]["Y"], workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for j in jobs:
+        check_parity(oracle, to_bits(j["Y"]), j["ref"], "independent stream")
