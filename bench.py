@@ -373,7 +373,7 @@ def run_ours(args):
         if dom is None or t > dom[1]:
             dom = (M, t, js)
     dM, dt, djs = dom
-    kernel_name = B_kernel_name(dM)
+    kernel_name = B_kernel_name(dM, args.launch)
     bound = roofline_seconds(djs[0]["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)[1]
     per_launch = dt / len(djs)
     if bound == "hbm":
@@ -674,14 +674,17 @@ def workload_label(args):
             "single": "single 1024x1024 GEMM"}.get(args.workload, f"llama2-7b {args.workload} linears")
 
 
-def B_kernel_name(M):
-    return "decode_kernel" if M <= 64 else "prefill2_kernel (two row-blocks per CTA) or prefill_kernel, chosen per shape"
+def B_kernel_name(M, launch="independent"):
+    if M <= 64:
+        return "decode_cluster_kernel" if launch == "independent" else "decode_kernel"
+    return "prefill2_kernel (two row-blocks per CTA) or prefill_kernel, chosen per shape"
 
 
-# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes per launch, from the ncu
-# captures summarised in profiles/decode_kernel_llama7b_decode.md (three launches: 1.035, 1.029, 1.008).
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes per launch, from the ncu captures
+# summarised in profiles/decode_cluster_kernel_llama7b_decode.md (1.055, 1.018, 1.007) and
+# profiles/decode_kernel_llama7b_decode.md (1.035, 1.029, 1.008).
 # Traffic grows in proportion to the payload, so the ratio scales to any launch of the kernel.
-NCU_TRAFFIC_RATIO = {"decode_kernel": 1.03}
+NCU_TRAFFIC_RATIO = {"decode_kernel": 1.03, "decode_cluster_kernel": 1.03}
 
 
 def load_traffic(kernel, algorithmic):

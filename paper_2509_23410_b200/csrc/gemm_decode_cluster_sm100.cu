@@ -285,9 +285,10 @@ static int launch_dc_t(const CUtensorMap& map, const patch_layout_t* L, const ui
 // The environment variable PATCH_DECODE_CLUSTER_S forces a size (experiments).
 int decode_cluster_split(int TN, int TK) {
     static const int forced = [] { const char* e = getenv("PATCH_DECODE_CLUSTER_S"); return e ? atoi(e) : 0; }();
+    static const int max_tiles = [] { const char* e = getenv("PATCH_DECODE_CLUSTER_TILES"); return e ? atoi(e) : 48; }();
     int S = 1;
     if (forced) S = forced;
-    else while (S < 8 && TN * S < 32) S *= 2;
+    else while (S < 8 && (TN * S < 32 || TK > max_tiles * S)) S *= 2;
     while (S > 1 && S > TK) S /= 2;
     return S;
 }
