@@ -61,6 +61,11 @@ enum { PATCH_GEMM_WEIGHTS_STATIC = 0x100 };
  * which read the same X).  Activations are then fetched without waiting for the previous
  * kernel; writes to Y and to the workspace still wait for it. */
 enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
+/* With BOTH promises a GEMM of M <= 64 tokens is independent of its predecessor, and the library runs
+ * it on a schedule made for streams of such GEMMs: one CTA per row-block (a small cluster splitting K
+ * where row-blocks are few), so that several consecutive GEMMs are resident on the GPU at once; without
+ * them it runs stream-K over all SMs, which is the faster choice for a GEMM that has the GPU to itself.
+ * Both are deterministic; their results may differ in the last bit (different fp32 summation order). */
 
 /*
  * Description of a packed blob.  Plain host struct, caller-owned, filled by patch_packed_size.
