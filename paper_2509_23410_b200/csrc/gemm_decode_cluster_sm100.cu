@@ -32,19 +32,22 @@
 namespace patch {
 
 namespace dc {
-template <int N_TOK, int STAGES>
+template <int N_TOK, int STAGES, bool GATED = false>
 struct Cfg {
     static constexpr uint32_t kXAtomBytes = N_TOK * 128;                  // N_TOK rows x 64 bf16
     static constexpr uint32_t kXBytes = 2 * kXAtomBytes;
     static constexpr uint32_t kStageBytes = kDenseBytes + kXBytes;
     static constexpr uint32_t kBarrierOffset = STAGES * kStageBytes;
     static constexpr uint32_t kSmemBytes = kBarrierOffset + 256 + 1024;   // + barriers + alignment slack
-    static constexpr uint32_t kTmemNeeded = N_TOK + 4 * STAGES;           // one accumulator + metadata (4 columns per stage)
+    static constexpr int kAccs = GATED ? 2 : 1;                           // gated: gate and up accumulators
+    static constexpr uint32_t kTmemNeeded = kAccs * N_TOK + 4 * STAGES;   // accumulators + metadata (4 columns per stage)
     static constexpr uint32_t kTmemCols = kTmemNeeded <= 32 ? 32 : kTmemNeeded <= 64 ? 64 : 128;
     static constexpr uint32_t kPartialRowBytes = N_TOK * 4;               // fp32 partial: [128 rows][N_TOK]
     static_assert(N_TOK == 16 || N_TOK == 32 || N_TOK == 64, "MMA N in {16, 32, 64}");
     static_assert(STAGES >= 2 && STAGES <= 4, "ring depth");
-    static_assert(128 * kPartialRowBytes <= kDenseBytes, "the partial takes the place of the first stage's weight tile");
+    static constexpr uint32_t kPartialBytes = 128 * kPartialRowBytes;     // per accumulator
+    static_assert(kAccs * kPartialBytes <= kDenseBytes, "the partials take the place of the first stage's weight tile");
+    static_assert(!GATED || N_TOK == 16, "the gated product exists for the 16-token schedule");
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -65,12 +68,15 @@ __device__ __forceinline__ float4 ld_peer_f4(uint32_t saddr, uint32_t rank) {
 }
 }  // namespace dc
 
-template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC>
+// GATED: the weight stacks a gate and an up projection with their row-blocks interleaved (2j: gate, 2j + 1: up);
+// a cluster owns the pair j, streams the gate tiles of its K-slice into one accumulator and the up tiles into a
+// second one, and writes silu(gate) * up for out-feature block j of Y [M x N / 2].
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
 __global__ void __launch_bounds__(192)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                       int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
     using namespace dc;
-    using C = Cfg<N_TOK, STAGES>;
+    using C = Cfg<N_TOK, STAGES, GATED>;
     constexpr uint32_t kStageBytes = C::kStageBytes, kXAtomBytes = C::kXAtomBytes, kXBytes = C::kXBytes;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -90,8 +96,10 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
     const uint32_t s = cluster_ctarank();
     const int tn = blockIdx.x / S;
     // K-slice of this CTA: tiles [k0, k1) of row-block tn
-    const int k0 = int(int64_t(s) * TK / S), k1 = int(int64_t(s + 1) * TK / S), n_tiles = k1 - k0;
-    const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off) + int64_t(tn) * TK + k0;
+    const int k0 = int(int64_t(s) * TK / S), k1 = int(int64_t(s + 1) * TK / S), n_slice = k1 - k0;
+    constexpr int kAccs = C::kAccs;
+    const int n_tiles = kAccs * n_slice;             // gated: the slice of the gate row-block, then of the up row-block
+    const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off) + int64_t(kAccs) * tn * TK + k0;
 
     if (threadIdx.x == 64) {
         for (int i = 0; i < STAGES; ++i) {
@@ -108,7 +116,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_meta = tmem_base + N_TOK;                 // 4 columns per stage behind the accumulator
+    const uint32_t tmem_meta = tmem_base + kAccs * N_TOK;         // 4 columns per stage behind the accumulators
 
     if (warp == 0) {
         // ---------------- producer ----------------
@@ -121,9 +129,10 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
         // resolved (WSTATIC); their activations follow once it is (unless XSTATIC)
         const int n_early = (WSTATIC && !XSTATIC) ? (n_tiles < STAGES ? n_tiles : STAGES) : 0;
         for (int i = 0; i < n_tiles && ok; ++i) {
-            if ((i & 31) == 0 && i + lane < n_tiles) mine = table[i + lane];
-            const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
-            const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
+            const int half = (GATED && i >= n_slice) ? 1 : 0, idx = i - half * n_slice;   // tile idx of row-block `half`
+            if ((idx & 31) == 0 && idx + lane < n_slice) mine = table[int64_t(half) * TK + idx + lane];
+            const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, idx & 31);
+            const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, idx & 31);
             if (lane == 0) {
                 const int stage = i % STAGES;
                 const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
@@ -139,14 +148,14 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
                             grid_dependency_wait();
                             for (int j = 0; j < n_early; ++j) {
                                 const uint32_t sX = smem_base + j * kStageBytes + kDenseBytes;
-                                const int k = (k0 + j) * kTile;
+                                const int k = (k0 + (GATED && j >= n_slice ? j - n_slice : j)) * kTile;
                                 tma_tile_load(sX, &tmap_x, k, 0, bar_full + 8 * j, pol_x);
                                 tma_tile_load(sX + kXAtomBytes, &tmap_x, k + 64, 0, bar_full + 8 * j, pol_x);
                             }
                         }
                     } else {
                         const uint32_t sX = sW + kDenseBytes;
-                        const int k = (k0 + i) * kTile;
+                        const int k = (k0 + idx) * kTile;
                         tma_tile_load(sX, &tmap_x, k, 0, full, pol_x);
                         tma_tile_load(sX + kXAtomBytes, &tmap_x, k + 64, 0, full, pol_x);
                     }
@@ -173,8 +182,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sW = smem_base + stage * kStageBytes;
-                issue_tile_mma<N_TOK>(stage_kind[stage], sW, sW + kDenseBytes, kXAtomBytes, tmem_base, tmem_meta + 4 * stage,
-                                     i == 0);
+                const int half = (GATED && i >= n_slice) ? 1 : 0;
+                issue_tile_mma<N_TOK>(stage_kind[stage], sW, sW + kDenseBytes, kXAtomBytes, tmem_base + uint32_t(half) * N_TOK,
+                                      tmem_meta + 4 * stage, i == half * n_slice);
                 mma_commit(bar_empty + 8 * stage);
             }
             if (ok && n_tiles > 0) mma_commit(bar_acc_full);      // every MMA of the slice has completed
@@ -191,9 +201,11 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             tc_fence_after();
         }
-        float4* dst = reinterpret_cast<float4*>(smem + row * C::kPartialRowBytes);
 #pragma unroll
-        for (int c0 = 0; c0 < N_TOK; c0 += 16) {
+        for (int c0 = 0; c0 < kAccs * N_TOK; c0 += 16) {
+            // accumulator c0 / N_TOK, its columns (c0 % N_TOK) .. + 15: partial [acc][row][token]
+            float4* dst = reinterpret_cast<float4*>(smem + (c0 / N_TOK) * C::kPartialBytes + row * C::kPartialRowBytes) +
+                          (c0 % N_TOK) / 4;
             uint32_t v[16];
             if (n_tiles > 0 && ok) {
                 tmem_ld16(tmem_base + ((quad * 32u) << 16) + uint32_t(c0), v);
@@ -204,7 +216,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-                dst[c0 / 4 + q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
                                               __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
         }
         tc_fence_before();
@@ -231,7 +243,17 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
                 const float4 p = dc::ld_peer_f4(addr, uint32_t(q));
                 acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
             }
-            const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+            float a[4] = {acc.x, acc.y, acc.z, acc.w};
+            if (GATED) {
+                float4 up = dc::ld_peer_f4(addr + C::kPartialBytes, 0);
+                for (int q = 1; q < S; ++q) {
+                    const float4 p = dc::ld_peer_f4(addr + C::kPartialBytes, uint32_t(q));
+                    up.x += p.x; up.y += p.y; up.z += p.z; up.w += p.w;
+                }
+                const float u[4] = {up.x, up.y, up.z, up.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) a[j] = __fdividef(a[j], 1.0f + __expf(-a[j])) * u[j];   // silu(gate) * up
+            }
             __nv_bfloat16* y = Y + int64_t(tn) * kTile + r;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -250,18 +272,18 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
     if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
 }
 
-template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC>
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
 static int launch_dc_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int S,
                        __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
-    using C = dc::Cfg<N_TOK, STAGES>;
-    auto kern = decode_cluster_kernel<N_TOK, STAGES, WSTATIC, XSTATIC>;
+    using C = dc::Cfg<N_TOK, STAGES, GATED>;
+    auto kern = decode_cluster_kernel<N_TOK, STAGES, WSTATIC, XSTATIC, GATED>;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
             return PATCH_ERR_CUDA;
         configured = true;
     }
-    const int TN = int(L->N / kTile), TK = int(L->K / kTile);
+    const int TN = int(L->N / kTile) / (GATED ? 2 : 1), TK = int(L->K / kTile);     // gated: pairs of row-blocks
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     cfg.gridDim = dim3(unsigned(TN) * unsigned(S), 1, 1);
@@ -310,6 +332,15 @@ int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const
         case 32: return launch_dc_f<32, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
         default: return launch_dc_f<64, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
     }
+}
+
+// silu(gate) * up on a stacked gate/up weight (row-blocks interleaved), M <= 16, independent launches.
+int launch_decode_cluster_gated(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
+                                __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+    const int TK = int(L->K / kTile);
+    int S = decode_cluster_split(int(L->N / kTile) / 2, 2 * TK);      // a CTA streams the slices of two row-blocks
+    while (S > 1 && S > TK) S /= 2;
+    return launch_dc_t<16, 3, true, true, true>(map, L, packed, M, S, Y, ldy, status_dev, stream);
 }
 
 }  // namespace patch

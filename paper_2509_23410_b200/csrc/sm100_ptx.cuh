@@ -236,6 +236,8 @@ int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int
 int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int n_tok,
                           __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic,
                           bool xstatic);
+int launch_decode_cluster_gated(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
+                                __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
 
 #ifdef PATCH_TRACE
 // Debug build only: status_dev is reinterpreted as a buffer of 16 timestamps (ns) per CTA.

@@ -525,6 +525,9 @@ def test_gated_product_small_m_schedule(gpu, oracle, M, shape):
     Nh, K = shape
     for flags_arg in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC):
         _gated_case(gpu, oracle, Nh, K, M, 0.3, 0.8, ws="own", flags_arg=flags_arg)
+    # declared independent of its predecessor: a cluster per (gate, up) pair of row-blocks, no workspace needed
+    _gated_case(gpu, oracle, Nh, K, M, 0.3, 0.8, ws=None, flags_arg=B.WEIGHTS_STATIC | B.INPUT_STATIC)
+    _gated_case(gpu, oracle, Nh, K, M, 1.0, 0.0, ws=None, flags_arg=B.WEIGHTS_STATIC | B.INPUT_STATIC)
 
 
 def test_gated_and_plain_calls_share_a_workspace(gpu, oracle):
