@@ -168,7 +168,7 @@ int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
 /* patch_gemm with an explicit kernel choice and options.
  *   PATCH_VARIANT_GEMV  CUDA-core decode kernel, M <= 4 only (PATCH_ERR_SHAPE otherwise)
  *   PATCH_VARIANT_MMA   tcgen05 tensor-core kernel, any M
- *   | PATCH_GEMM_WEIGHTS_STATIC  see above */
+ *   | PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC  see above */
 int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
                   const patch_layout_t* layout, const void* packed_dev,
                   void* Y_dev, int64_t ldy,
@@ -193,6 +193,8 @@ int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
  *           fp32 values, the finisher of the matching up row-block multiplies.  Otherwise (or for
  *           larger M) the large-M schedule runs, whose CTA holds both accumulators.
  *   flags   0 or PATCH_GEMM_WEIGHTS_STATIC [| PATCH_GEMM_INPUT_STATIC], as for patch_gemm_ex.
+ *           With both flags and M <= 16 the call needs no workspace at all: a cluster of CTAs owns a
+ *           (gate, up) pair of row-blocks, holds both accumulators and applies the product itself.
  * Other arguments and error behaviour as patch_gemm.
  */
 int patch_gemm_gated_workspace_size(const patch_layout_t* layout, int64_t M, size_t* bytes_out);
