@@ -58,7 +58,7 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
     if (variant == PATCH_VARIANT_GEMV) return launch_gemv(X, ldx, int(M), L, packed, Y, ldy, status_dev, s);
     if (M <= 64) return launch_decode(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s, wstatic, xstatic);
-    return launch_prefill(X, ldx, M, L, packed, Y, ldy, status_dev, s);
+    return launch_prefill(X, ldx, M, L, packed, Y, ldy, status_dev, s, wstatic && xstatic);
 }
 
 extern "C" int patch_gemm(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,
@@ -108,7 +108,8 @@ extern "C" int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M, const
     if (need > 0 && workspace_dev && workspace_bytes >= need && !(reinterpret_cast<uintptr_t>(workspace_dev) & 255u))
         return launch_decode_gated(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s,
                                    (flags & PATCH_GEMM_WEIGHTS_STATIC) != 0, (flags & PATCH_GEMM_INPUT_STATIC) != 0);
-    return launch_prefill_gated(X, ldx, M, L, packed, Y, ldy, status_dev, s);
+    return launch_prefill_gated(X, ldx, M, L, packed, Y, ldy, status_dev, s,
+                                (flags & PATCH_GEMM_WEIGHTS_STATIC) && (flags & PATCH_GEMM_INPUT_STATIC));
 }
 
 extern "C" int patch_gemm_host(const void* X_host, int64_t M, const patch_layout_t* L, const void* packed_dev,

@@ -46,7 +46,7 @@ constexpr uint32_t kSparse = 2;
 __global__ void __launch_bounds__(320)
 prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                 int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev,
-                int gated) {
+                int gated, int independent) {
     using namespace p2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -64,7 +64,9 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
     volatile uint32_t* slot_kind = misc + 2;                      // NA words
 
     grid_launch_dependents();
-    grid_dependency_wait();     // X, the packed weight and Y may belong to the previous kernel until here
+    // X, the packed weight and Y may belong to the previous kernel until here -- unless the caller declared
+    // this GEMM independent of its predecessor: then only the Y stores (and the exit) wait
+    if (!independent) grid_dependency_wait();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int TP = (TN + 1) / 2;                                   // row-block pairs
@@ -255,6 +257,7 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
 #ifdef PATCH_TRACE
             const long long te0 = clock64();
 #endif
+            if (independent && j == 0) grid_dependency_wait();     // Y may be in use by the preceding kernel
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             const int chunks = (valid + 15) / 16, c_begin = half == 0 ? 0 : (chunks + 1) / 2,
                       c_end = half == 0 ? (chunks + 1) / 2 : chunks;
@@ -303,13 +306,15 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
         }
     }
 
+    if (independent) grid_dependency_wait();      // every thread passes the dependency before the CTA exits
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
-                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated) {
+                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated,
+                    bool independent) {
     static bool configured = false;   // per-process attribute, idempotent
     if (!configured) {
         if (cudaFuncSetAttribute(prefill2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p2::kSmemBytes) != cudaSuccess)
@@ -330,7 +335,7 @@ int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, prefill2_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
-                                       Y, ldy, status_dev, gated ? 1 : 0);
+                                       Y, ldy, status_dev, gated ? 1 : 0, independent ? 1 : 0);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

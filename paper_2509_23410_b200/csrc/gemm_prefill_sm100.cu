@@ -40,7 +40,8 @@ struct PrefillConfig {
 
 __global__ void __launch_bounds__(192)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
-               int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
+               int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev,
+               int independent) {
     using Cfg = PrefillConfig;
     const uint32_t stage_bytes = kDenseBytes + uint32_t(n_tok) * 256u;
     const int STAGES = int(Cfg::kRingBytes / stage_bytes) < Cfg::kMaxStages ? int(Cfg::kRingBytes / stage_bytes) : Cfg::kMaxStages;
@@ -57,7 +58,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
     volatile uint32_t* stage_kind = reinterpret_cast<volatile uint32_t*>(tmem_slot + 2);  // kMaxStages words
 
     grid_launch_dependents();
-    grid_dependency_wait();     // X, the packed weight and Y may belong to the previous kernel until here
+    // X, the packed weight and Y may belong to the previous kernel until here -- unless the caller declared
+    // this GEMM independent of its predecessor: then only the Y stores (and the exit) wait, and this kernel's
+    // CTAs start on whatever SMs the tail of the previous kernel leaves idle
+    if (!independent) grid_dependency_wait();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0) PATCH_TRACE_AT(0);
@@ -164,6 +168,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
             const uint32_t acc = tmem_base + (j & 1 ? Cfg::kAcc1Col : 0u) + ((quad * 32u) << 16);
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             __nv_bfloat16* ytile = Y + int64_t(m0) * ldy + int64_t(tn) * kTile + quad * 32;
+            if (independent && j == 0) grid_dependency_wait();      // Y may be in use by the preceding kernel
 #pragma unroll 1
             for (int c0 = 0; c0 < valid; c0 += 16) {
                 uint32_t v[16];
@@ -179,6 +184,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
         if (warp == 2) PATCH_TRACE_AT(5);
     }
 
+    if (independent) grid_dependency_wait();      // every thread passes the dependency before the CTA exits
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, Cfg::kTmemCols);
@@ -228,7 +234,8 @@ static int sm_count_prefill() {
 }
 
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
-                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated);
+                    int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated,
+                    bool independent);
 
 // Testing / tuning aid: PATCH_PREFILL_SCHEDULE=1|2 in the environment pins the schedule (one or two
 // row-blocks per CTA); anything else lets the cost model choose.
@@ -277,7 +284,7 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row
 }
 
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                   __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+                   __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent) {
     if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
     const int sms = sm_count_prefill();
     if (sms <= 0) return PATCH_ERR_CUDA;
@@ -287,7 +294,7 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
-    if (plan.schedule == 2) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream, false);
+    if (plan.schedule == 2) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream, false, independent);
     static bool configured = false;   // per-process attribute, idempotent
     if (!configured) {
         if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -308,14 +315,14 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
-                                       Y, ldy, status_dev);
+                                       Y, ldy, status_dev, independent ? 1 : 0);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
 // Gated product of a stacked gate/up weight whose row-blocks alternate (gate j, up j): always the
 // two-row-block kernel, whose CTA holds both accumulators of an output row-block.
 int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                         __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+                         __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent) {
     if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
     const int sms = sm_count_prefill();
     if (sms <= 0) return PATCH_ERR_CUDA;
@@ -324,7 +331,7 @@ int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const p
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, plan.n_tok);
     if (rc) return rc;
-    return launch_prefill2(map, L, packed, M, plan.n_tok, sms, Y, ldy, status_dev, stream, true);
+    return launch_prefill2(map, L, packed, M, plan.n_tok, sms, Y, ldy, status_dev, stream, true, independent);
 }
 
 }  // namespace patch

@@ -48,10 +48,14 @@ int launch_gemv(const __nv_bfloat16* X, int64_t ldx, int M, const patch_layout_t
 int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                   const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev,
                   cudaStream_t stream, bool wstatic, bool xstatic);
+// `independent`: the caller declared the GEMM independent of its predecessor (weights and X static): only its
+// Y stores wait for the preceding kernel.
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
-                   const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+                   const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream,
+                   bool independent);
 int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
-                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream,
+                         bool independent);
 size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M);
 int launch_decode_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev,
