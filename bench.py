@@ -493,6 +493,20 @@ def run_ours(args):
         out["cpu_baseline"] = cpu
     if table:
         out["cases"] = table
+        # speed-up of every hybrid / 2:4 case over the all-dense tile configuration of the same shape and M
+        # (the comparison the prefill workload asks for; for a bandwidth-bound linear the ceiling is 1 / (1 - 0.4375 f))
+        dense = {}
+        for c in table:
+            if c["f_sparse"] == 0.0:
+                dense[(c["name"].split(".p")[0], c["name"].rsplit(".M", 1)[1])] = c["us"]
+        sp = []
+        for c in table:
+            base = dense.get((c["name"].split(".p")[0], c["name"].rsplit(".M", 1)[1]))
+            if base and c["f_sparse"] > 0.0:
+                sp.append(dict(name=c["name"], f_sparse=c["f_sparse"], speedup_vs_all_dense=round(base / c["us"], 3),
+                               bandwidth_ceiling=round(1.0 / (1.0 - 0.4375 * c["f_sparse"]), 3)))
+        if sp:
+            out["speedup_vs_all_dense"] = sp
     print(json.dumps(out))
 
 
