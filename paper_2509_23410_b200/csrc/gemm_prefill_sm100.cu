@@ -255,7 +255,8 @@ static int forced_schedule() {
 // pipeline), plus a per-tile prologue/epilogue cost.
 struct PrefillPlan { int n_tok; int schedule; };   // schedule: row-blocks per CTA (1 or 2)
 
-static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row_blocks_only = false) {
+static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row_blocks_only = false,
+                                bool independent = false) {
     PrefillPlan best = {240, 1};
     double best_cost = 1e300;
     const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : kPrefillMaxTok, n_lo = M <= 128 ? n_hi : 128;
@@ -276,7 +277,10 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row
             const double load2_ns = (65536.0 + n * 256.0) / 120.0 > 1200.0 ? (65536.0 + n * 256.0) / 120.0 : 1200.0;
             const double load_ns = sched == 1 ? load1_ns : load2_ns;
             const double tile_ns = TK * (mma_ns > load_ns ? mma_ns : load_ns) + (sched == 1 ? 6000.0 : 10000.0);
-            const double cost = double(waves) * tile_ns + n;      // at equal time, the narrower tile (less padding)
+            // a GEMM whose successor may start on the SMs its last wave leaves idle pays only part of that wave
+            const double frac = double(tiles) / sms > 1.0 ? double(tiles) / sms : 1.0;
+            const double eff_waves = independent ? frac : double(waves);
+            const double cost = eff_waves * tile_ns + n;          // at equal time, the narrower tile (less padding)
             if (cost < best_cost) { best_cost = cost; best = {n, sched}; }
         }
     }
@@ -289,7 +293,7 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     const int sms = sm_count_prefill();
     if (sms <= 0) return PATCH_ERR_CUDA;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
-    const PrefillPlan plan = plan_prefill(M, TN, TK, sms);
+    const PrefillPlan plan = plan_prefill(M, TN, TK, sms, false, independent);
     const int n_tok = plan.n_tok;
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
@@ -327,7 +331,7 @@ int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const p
     const int sms = sm_count_prefill();
     if (sms <= 0) return PATCH_ERR_CUDA;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
-    const PrefillPlan plan = plan_prefill(M, TN, TK, sms, true);
+    const PrefillPlan plan = plan_prefill(M, TN, TK, sms, true, independent);
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, plan.n_tok);
     if (rc) return rc;
