@@ -51,21 +51,34 @@ enum {
 
 /* Kernel choice for patch_gemm_ex (low bits), optionally OR-ed with PATCH_GEMM_WEIGHTS_STATIC. */
 enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2 };
-/* Promise that the packed weight was NOT written by the operation that precedes this call in
- * the stream (the serving case: weights are packed once, offline).  The kernel is launched with
- * programmatic dependent launch either way; with this flag it also requests its first weight
- * tiles before the previous kernel has finished.  Activations and outputs always wait. */
+/*
+ * Launch promises.  Every GEMM kernel is launched with programmatic dependent launch and lets its
+ * successor become resident as soon as it has started itself; each kernel orders itself against
+ * what came before with a device-side wait.  A promise lets it do part of its work before that wait.
+ * Since the kernels before it may have started early in the same way, a GEMM can be running at the
+ * same time as ANY of the GEMMs of this library that were enqueued directly before it, one after the
+ * other, on the same stream -- however those were launched.  Call that run of consecutive GEMM calls,
+ * back to the nearest operation that is not one of this library's GEMMs (a copy, a memset, any other
+ * kernel: those complete before the next kernel starts), the GEMM's "overlap window".
+ *
+ * PATCH_GEMM_WEIGHTS_STATIC: no operation in the overlap window writes the packed weight (the serving
+ *   case: weights are packed once, offline).  The kernel then requests weight tiles before its wait.
+ * PATCH_GEMM_INPUT_STATIC (only honoured together with the first): no operation in the overlap window
+ *   writes X either (e.g. q, k and v projections enqueued one after the other behind the kernel that
+ *   produced their common X; not a GEMM whose X is the Y of a GEMM enqueued directly before it).
+ *   Activations are then fetched without waiting too.
+ * Writes to Y and to the workspace always wait for everything before them, and no kernel completes
+ * before its predecessors, so stream order as seen from later operations is unchanged.
+ *
+ * With BOTH promises a GEMM of M <= 64 tokens runs on a schedule made for streams of independent
+ * GEMMs: one CTA per row-block (a small cluster splitting K where row-blocks are few), so that several
+ * consecutive GEMMs are resident on the GPU at once; without them it runs stream-K over all SMs, which
+ * is the faster choice for a GEMM that has the GPU to itself.  For M > 64 both promises let the kernel
+ * start on the SMs that the tail of the previous kernel leaves idle.  All schedules are deterministic;
+ * their results may differ in the last bit (different fp32 summation order).
+ */
 enum { PATCH_GEMM_WEIGHTS_STATIC = 0x100 };
-/* Promise (only honoured together with PATCH_GEMM_WEIGHTS_STATIC) that X was NOT written by the
- * operation that precedes this call in the stream (e.g. the k projection after the q projection,
- * which read the same X).  Activations are then fetched without waiting for the previous
- * kernel; writes to Y and to the workspace still wait for it. */
 enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
-/* With BOTH promises a GEMM of M <= 64 tokens is independent of its predecessor, and the library runs
- * it on a schedule made for streams of such GEMMs: one CTA per row-block (a small cluster splitting K
- * where row-blocks are few), so that several consecutive GEMMs are resident on the GPU at once; without
- * them it runs stream-K over all SMs, which is the faster choice for a GEMM that has the GPU to itself.
- * Both are deterministic; their results may differ in the last bit (different fp32 summation order). */
 
 /*
  * Description of a packed blob.  Plain host struct, caller-owned, filled by patch_packed_size.
