@@ -676,3 +676,32 @@ def test_independent_launches_back_to_back(gpu, oracle):
     assert int(status.item()) == 0
     for j in jobs:
         check_parity(oracle, to_bits(j["Y"]), j["ref"], "independent stream")
+
+
+@pytest.mark.parametrize("M", [4, 48, 300])
+def test_promises_are_bounded_by_other_operations(gpu, oracle, M):
+    """A GEMM launched with both promises behind an operation that is not one of the library's GEMMs
+    (here: the copy that produces its X) must see that operation's result: the overlap window ends there.
+    Five rounds without any synchronisation, each with a different X in the same buffer."""
+    torch, B = gpu
+    N, K = 1024, 768
+    W, flags, _ = inputs.make_case_inputs(dict(N=N, K=K, p=0.5, stream=("window",)), 63, M)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    What = oracle.prune(W, flags)
+    Xs = [inputs.activation(M, K, 63, "window", M, i) for i in range(5)]
+    Xd = [to_dev(torch, x) for x in Xs]
+    Xbuf = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
+    Ys = [torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(5)]
+    ws = torch.zeros(max(B.patch_gemm_workspace_size(L, M), 1), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    for i in range(5):
+        Xbuf.copy_(Xd[i])                                        # not a library GEMM: fully ordered
+        B.patch_gemm(Xbuf, L, packed, Y=Ys[i], workspace=ws, variant=B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
+    torch.cuda.synchronize()
+    for i in range(5):
+        if M <= 64:
+            ref = oracle.gemm_f64(Xs[i], What)[0]
+            check_parity(oracle, to_bits(Ys[i]), ref, f"window round {i}")
+        else:
+            rows = np.array([0, 1, M // 2, M - 1])
+            check_parity(oracle, to_bits(Ys[i])[rows], oracle.gemm_f64_rows(Xs[i], rows, What), f"window round {i}")
