@@ -347,6 +347,18 @@ def run_ours(args):
     step_flops = sum(j["cost"]["flops"] for j in jobs)
     value = world * step_flops / step_s / 1e12
 
+    # ---- spread: 50 more replays of the timed graph, each between its own pair of events (median and minimum;
+    # every replay ends with a drain here, so these sit slightly above the back-to-back mean of the timed region)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(50)]
+    for a, b in evs:
+        a.record()
+        multi_graph.replay()
+        b.record()
+    torch.cuda.synchronize()
+    per_step = sorted(a.elapsed_time(b) / spg for a, b in evs)
+    replay_stats = {"replays": len(per_step), "steps_per_replay": spg, "median_ms_per_step": per_step[len(per_step) // 2],
+                    "min_ms_per_step": per_step[0], "max_ms_per_step": per_step[-1]}
+
     # ---- one step per graph replay, for comparison: every step then ends with a full drain of the GPU
     single_s = step_s
     if spg > 1:
@@ -487,6 +499,7 @@ def run_ours(args):
                             "ms_per_step": other_s * 1e3, "frac_of_roofline_measured": meas_t / other_s},
         "one_step_per_graph": {"value": world * step_flops / single_s / 1e12, "unit": "TFLOP/s", "ms_per_step": single_s * 1e3,
                                "frac_of_roofline_spec": spec_t / single_s, "frac_of_roofline_measured": meas_t / single_s},
+        "replay_stats": replay_stats,
         "gpu_launches": args.steps * len(jobs),
         "clocks": clocks,
         # whole calls, one per matrix, read + written bytes: patch_pack_dev (flags on the device, two kernels) and
