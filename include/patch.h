@@ -6,14 +6,17 @@
  * (two kept values of every four consecutive elements along K, plus two position bits per
  * kept value).  This is the deployment format of PATCH (arXiv 2509.23410): the hard mask
  * M* = M*_tile + (1 - M*_tile) (.) M*_2:4 of Algorithm 1 applied to W, compressed per tile
- * ("Efficient deployment", Appendix A), and the matmul in which "tiles within a matrix
- * [are] either dense or sparse" within one multiplication.
+ * (deployment section, Appendix A), and the matmul that mixes dense and 2:4 tiles inside one
+ * multiplication.
  *
  * General rules
  *   - Every function returns a status (PATCH_OK = 0, errors negative).  Nothing throws,
  *     prints or exits.  All argument validation happens on the host before any launch.
  *   - Pointers named *_dev are device pointers, *_host are host pointers.  The library
- *     allocates no device memory and keeps no global state; every buffer is the caller's.
+ *     allocates no device memory; every buffer is the caller's.  What it remembers between
+ *     calls is per device and read-mostly: the SM count and which kernels already had their
+ *     shared-memory limit raised there (plus patch_gemm_noalloc's scratch array, see there).
+ *     No environment variable changes its behaviour.
  *   - Entry points may be called from several host threads (on different streams or devices);
  *     calls that share a workspace must be ordered on one stream.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
@@ -114,7 +117,7 @@ typedef struct patch_layout_t {
 
 /*
  * Size and layout of the packed blob for a weight of N x K with the given tile flags.
- * (Appendix A: compression "determined by the chosen tile size"; here fixed at 128 x 128.)
+ * (Appendix A: the tile size fixes the compressed format; here it is 128 x 128.)
  *   tile_flags_host  [N/128 x K/128] row-major bytes, PATCH_TILE_DENSE or PATCH_TILE_SPARSE_2_4
  *   layout_out       filled on success
  * Host only; touches no device.
@@ -146,8 +149,8 @@ int patch_unpack(const patch_layout_t* layout, const void* packed_dev, void* Wha
 
 /*
  * Scratch memory patch_gemm needs for `M` tokens (may be 0 bytes).  The scratch holds fp32
- * split-K partial sums and arrival counters of the small-M schedules ("alternative kernel
- * execution schemes such as split-K parallelism", Appendix A).
+ * split-K partial sums and arrival counters of the small-M schedules (split-K is the schedule
+ * Appendix A names for decode).
  */
 int patch_gemm_workspace_size(const patch_layout_t* layout, int64_t M, size_t* bytes_out);
 
@@ -190,8 +193,8 @@ int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
 
 /*
  * Gated product of the MLP's gate and up projections in one launch (a first step of the
- * block-level fusion that follows the per-matrix matmul; the paper studies the "up, gate, and
- * down matrices of the MLP" separately, and in the LLaMA models it measures the MLP computes
+ * block-level fusion that follows the per-matrix matmul; the paper treats the MLP's up, gate and
+ * down matrices separately, and in the LLaMA models it measures the MLP computes
  * down(silu(gate x) * up x)):
  *     Y[m][128 j + r] = silu(G[m][128 j + r]) * U[m][128 j + r],   silu(x) = x / (1 + exp(-x)),
  * where G = X Wgate^T and U = X Wup^T come from ONE packed weight that stacks the two matrices
@@ -278,12 +281,15 @@ int patch_gemm_host_batch_pipelined(const patch_host_job_t* jobs, int n_jobs, in
  * cudaFree or any allocating routine.
  *
  *   Arguments as for patch_gemm, without workspace and status.  Result and rounding are those
- *   of patch_gemm (same kernel, same summation order).
+ *   of patch_gemm (same kernel, same summation order).  There is no status word: a bounded
+ *   device-side wait that expires (PATCH_ERR_TIMEOUT in patch_gemm) is NOT reported here and
+ *   leaves Y undefined; a caller that needs to know uses patch_gemm.
  *   Limits: M <= 16 tokens and N <= 131072; beyond them the call returns PATCH_ERR_SIZE and
  *   launches nothing (use patch_gemm with a caller-owned workspace instead).
  *   The first call on each device looks up the array's device address; make that first call
  *   with the device current and before any stream capture.  Every call enqueues a memset of
- *   the scratch array (it must start empty) followed by the kernel.
+ *   the whole scratch array followed by the kernel: the array must start empty, also after a
+ *   call that was cut short or that raced with another one.
  *   All calls on a device share the one array, which keeps the last call's contents: calls that
  *   may overlap on the GPU (different streams) race with each other -- issue them on one stream
  *   or order them with events.
@@ -308,9 +314,9 @@ enum { PATCH_MASK_NO_NOISE = 1 };
 /*
  * Hard masks read off the logits (Algorithm 1, the lines after the loop):
  *   tile_flags_dev[t] = PATCH_TILE_DENSE if P_tile[t] > 0 else PATCH_TILE_SPARSE_2_4
- *                       ("positive values correspond to the dense option"; 0 and NaN are not positive);
+ *                       (a positive tile logit means dense; 0 and NaN are not positive);
  *   patterns_dev[grp] = index of the largest of the group's six logits, the first of equals
- *                       ("select best 2:4 mask from P_2:4").
+ *                       (the candidate Algorithm 1 keeps for deployment).
  *   tile_flags_dev  u8 [N/128 x K/128];  patterns_dev  u8 [N x K/4], 16-byte aligned.
  * One kernel, no host synchronisation.  The flags must be copied to the host by the caller
  * before patch_packed_size / patch_pack_patterns, which take them as host arrays.
@@ -408,7 +414,7 @@ int patch_mask_regularizer_coefficients(const double* sums_host, int n, double r
                                         double lambda2, double* c1_host, double* c2_host);
 
 /*
- * Backward of patch_soft_mask ("Update P_tile, P_2:4 via backpropagation", Algorithm 1): gradient with
+ * Backward of patch_soft_mask (the logit update step of Algorithm 1): gradient with
  * respect to the logits of
  *   F = sum_e Gw_e Mt_e W_e + c1 sum_e Mt_e - (c2 / 2) sum_e (Mt_e W_e)^2,
  * where Gw = dL_LM / d(Mt (.) W) is the gradient the language-model loss returns for the masked weight

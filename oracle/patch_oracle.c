@@ -10,10 +10,10 @@
  *     consecutive elements along K (Preliminaries, "Learnable 2:4 Mask": six candidate patterns
  *     per group of four).  The 2:4 mask itself is magnitude top-2 per group, the selection the
  *     workloads fix; ties go to the lower index.
- *   - pruned weight  What = W (.) M*  (Algorithm 1, "Final pruned weights"), done as a select so
+ *   - pruned weight  What = W (.) M*  (last line of Algorithm 1), done as a select so
  *     that a pruned element is +0.
  *   - compression of the mixed matrix into kept values + metadata, per tile (Appendix A:
- *     "Matrix compression and metadata generation are determined by the chosen tile size");
+ *     the tile size fixes how the matrix is compressed and its metadata laid out);
  *     two metadata bits per kept value, the cost that reproduces the compression-ratio column
  *     of the 4-bit quantisation table.
  *   - the linear layer itself, on the same bf16-rounded inputs, accumulated in double (and in
@@ -263,7 +263,7 @@ int oracle_pack(const uint16_t* W, const uint8_t* flags, const oracle_layout_t* 
     return pack_impl(W, flags, NULL, L, blob, capacity);
 }
 
-/* The same compression with the 2:4 mask given (Algorithm 1: "select best 2:4 mask from P_2:4"),
+/* The same compression with the 2:4 mask given (the per-group candidate that Algorithm 1 keeps at the end),
  * one candidate index per group of four; groups inside dense tiles ignore theirs. */
 int oracle_pack_patterns(const uint16_t* W, const uint8_t* flags, const uint8_t* patterns,
                          const oracle_layout_t* L, uint8_t* blob, uint64_t capacity) {
@@ -393,7 +393,7 @@ int oracle_gemm_f64(const uint16_t* X, int64_t M, int64_t K, const uint16_t* Wha
     return 0;
 }
 
-/* plain fp32 accumulation in k order: "an fp32 matmul on the same bf16-rounded inputs" */
+/* plain fp32 accumulation in k order on the same bf16-rounded inputs */
 int oracle_gemm_f32(const uint16_t* X, int64_t M, int64_t K, const uint16_t* What, int64_t N,
                     float* Y32) {
     if (!X || !What || !Y32) return -1;
@@ -563,7 +563,7 @@ void oracle_regularizer_coefficients(const double* sums, int n, double rho, doub
     *c2 = 2.0 * lambda2 / d;
 }
 
-/* Gradient with respect to the logits ("Update P_tile, P_2:4 via backpropagation", Algorithm 1) of
+/* Gradient with respect to the logits (the logit update step of Algorithm 1) of
  *   F = sum_e Gw_e Mt_e W_e  +  c1 sum_e Mt_e  -  (c2 / 2) sum_e (Mt_e W_e)^2
  * for fixed noise, where Gw = dL_LM / d(Mt (.) W) is the gradient the language-model loss hands back for
  * the masked weight.  Chain rule through Eq. 4, Eq. 2 / Eq. 3 and the softmax of Eq. 1:

@@ -15,8 +15,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)
-            if f != "mma_rate_probe.cu" and os.path.isfile(os.path.join(CSRC, f))]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if os.path.isfile(os.path.join(CSRC, f))]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "patch.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
@@ -29,23 +28,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("PATCH_NVCC_FLAGS", "").split()     # tuning experiments, e.g. -DNAME=value
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
     return LIB
 
 
-def build_probe() -> str:
-    """Standalone tensor-pipe rate probe (csrc/mma_rate_probe.cu); not needed by the library."""
-    out = os.path.join(HERE, "mma_rate_probe")
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-o", out,
-                    os.path.join(CSRC, "mma_rate_probe.cu")], check=True)
-    return out
-
-
 if __name__ == "__main__":
-    if "--probe" in sys.argv:
-        print(build_probe())
-    else:
-        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

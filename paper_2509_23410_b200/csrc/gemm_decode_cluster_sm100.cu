@@ -12,8 +12,7 @@
 //   -> cluster barrier -> every CTA sums 128 / S rows over the S partials (ld.shared::cluster, in K
 //   order: deterministic) -> wait for the predecessor kernel -> bf16 stores -> cluster barrier.
 // Nothing but Y is written to global memory, so only the Y stores wait for the predecessor.
-// "Alternative kernel execution schemes such as split-K parallelism" (Appendix A) in the form
-// the hardware offers for it.
+// This is the split-K schedule Appendix A mentions for decode, in the form the hardware offers for it.
 //
 // Measured (B200, the 24 decode GEMMs of the LLaMA-2-7B workload launched back to back as independent
 // GEMMs): with S chosen as small as possible -- S = 1 wherever the weight has 32 or more row-blocks, i.e. one
@@ -26,7 +25,6 @@
 //
 // Same operand roles, tile format, ring of whole-tile stages, bounded waits and launch flags as the
 // stream-K kernel; M <= 64 tokens (MMA N = 16, 32 or 64).
-#include <cstdlib>
 #include "sm100_ptx.cuh"
 
 namespace patch {
@@ -277,12 +275,8 @@ static int launch_dc_t(const CUtensorMap& map, const patch_layout_t* L, const ui
                        __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
     using C = dc::Cfg<N_TOK, STAGES, GATED>;
     auto kern = decode_cluster_kernel<N_TOK, STAGES, WSTATIC, XSTATIC, GATED>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-            return PATCH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (int rc = allow_dynamic_smem(kern, C::kSmemBytes, configured)) return rc;
     const int TN = int(L->N / kTile) / (GATED ? 2 : 1), TK = int(L->K / kTile);     // gated: pairs of row-blocks
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
@@ -303,14 +297,12 @@ static int launch_dc_t(const CUtensorMap& map, const patch_layout_t* L, const ui
 }
 
 // Cluster size for a weight of TN x TK tiles: the smallest power of two that gives the kernel at least 32
-// CTAs (fewer would leave a short stream of GEMMs without enough bytes in flight), at most 8 and at most TK.
-// The environment variable PATCH_DECODE_CLUSTER_S forces a size (experiments).
+// CTAs (fewer would leave a short stream of GEMMs without enough bytes in flight) and at most 48 tiles per CTA
+// (a longer run holds back the completion of every kernel behind it), at most 8 and at most TK.
 int decode_cluster_split(int TN, int TK) {
-    static const int forced = [] { const char* e = getenv("PATCH_DECODE_CLUSTER_S"); return e ? atoi(e) : 0; }();
-    static const int max_tiles = [] { const char* e = getenv("PATCH_DECODE_CLUSTER_TILES"); return e ? atoi(e) : 48; }();
+    constexpr int kMaxTilesPerCta = 48;
     int S = 1;
-    if (forced) S = forced;
-    else while (S < 8 && (TN * S < 32 || TK > max_tiles * S)) S *= 2;
+    while (S < 8 && (TN * S < 32 || TK > kMaxTilesPerCta * S)) S *= 2;
     while (S > 1 && S > TK) S /= 2;
     return S;
 }

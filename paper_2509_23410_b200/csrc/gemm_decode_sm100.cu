@@ -1,7 +1,7 @@
 // Small-M (decode) schedule of the hybrid dense / 2:4 tile matmul on the sm_100a tensor cores.
 //
-// The paper names decode as "the primary bottleneck" of generation and split-K as the schedule
-// its inspector picks there (Appendix A).  At M <= 64 tokens the layer is bound by the bytes of
+// Appendix A singles out decode as the stage that limits generation and split-K as the schedule
+// its inspector picks there.  At M <= 64 tokens the layer is bound by the bytes of
 // the packed weight, so the whole design serves one purpose: keep HBM busy.
 //
 //   * Work = the T = TN x TK weight tiles in (tn, tk) order.  One CTA per SM; CTA c streams the
@@ -26,7 +26,6 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports
 // PATCH_ERR_TIMEOUT through status_dev, drains its copies in flight, frees TMEM and returns.
-#include <cstdlib>
 #include "sm100_ptx.cuh"
 
 namespace patch {
@@ -258,7 +257,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = blockIdx.x, G = gridDim.x;
-    if (warp == 0) PATCH_TRACE_AT(0);
     const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off);
 
     if (warp == 0) {
@@ -305,7 +303,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const int t0 = range[0], t1 = range[1], n_tiles = t1 - t0;
-    if (warp == 0) PATCH_TRACE_AT(1);
     const uint32_t tmem_meta = tmem_base + 2 * N_TOK;    // 4 columns per stage; accumulators at 0 and N_TOK
 
     if (warp == 0) {
@@ -332,7 +329,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                     stage_kind[stage] = kind;
                     mbar_expect_tx(full, wbytes + Cfg::kXBytes);
                     tma_bulk_load(sW, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
-                    if (i == 0) PATCH_TRACE_AT(2);
                     if (i < n_early) {
                         if (i + 1 == n_early) {
                             grid_dependency_wait();
@@ -373,7 +369,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                     ok = mbar_wait(bar_acc_empty + 8 * (seg & 1), (uint32_t(seg >> 1) & 1u) ^ 1u, abort_flag, status_dev);
                 if (ok) ok = mbar_wait(bar_full + 8 * stage, uint32_t(i / STAGES) & 1u, abort_flag, status_dev);
                 if (!ok) break;
-                if (i == 0) PATCH_TRACE_AT(3);
                 tc_fence_after();
                 const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
                 issue_tile_mma<N_TOK>(stage_kind[stage], sW, sW + kDenseBytes, Cfg::kXAtomBytes,
@@ -384,7 +379,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                 first = last;
                 tk = (tk == TK - 1) ? 0 : tk + 1;
             }
-            PATCH_TRACE_AT(4);
         }
         __syncwarp();
     } else {
@@ -406,11 +400,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
             ok = epilogue_all(ok);      // same decision in all 128 threads: they share barriers below
             if (!ok) break;
             tc_fence_after();
-            if (seg == 0 && warp == 2) PATCH_TRACE_AT(5);
             if (!waited) {              // Y and the workspace may be in use by the previous kernel until here
                 grid_dependency_wait();
                 waited = true;
-                if (warp == 2) PATCH_TRACE_AT(8);
             }
             const uint32_t acc = tmem_base + uint32_t(seg & 1) * N_TOK + ((quad * 32u) << 16);
             if (GATED && ntiles == TK) {
@@ -458,7 +450,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                     for (int j = 0; j < 16; j += 4)
                         st_relaxed_gpu_v4(mine + j, make_uint4(nonempty(v[j]), nonempty(v[j + 1]), nonempty(v[j + 2]),
                                                                nonempty(v[j + 3])));
-                    if (warp == 2) PATCH_TRACE_AT(9);
                 } else {
                     // this run owns the row-block's first tile and ends inside it: add the following CTAs'
                     // partials in ascending K order, five contributors in flight at a time
@@ -516,7 +507,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                         for (int j = 0; j < 16; ++j)
                             if (j < M) ycol[int64_t(j) * ldy] = __float2bfloat16_rn(a[j]);
                     }
-                    if (warp == 2) PATCH_TRACE_AT(14);
                 }
             } else {
                 // partial row-block: write fp32 partial sums ([slot][row][token]), then count in
@@ -535,7 +525,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (seg & 1));
                 asm volatile("bar.sync 1, 128;" ::: "memory");      // all 128 epilogue threads have written
-                if (warp == 2) PATCH_TRACE_AT(k == 0 ? 9 : 12);
                 part_tn[k] = tn;
                 if (et == 32 * k) {
                     // {tiles : 16, contributors : 16, first contributor's slot + 1 : 16, finished readers : 16}
@@ -587,14 +576,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                 }
             }
         }
-        if (warp == 2) PATCH_TRACE_AT(6);
     }
 
     grid_dependency_wait();     // completion of this grid implies completion of its predecessors
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, Cfg::kTmemCols);
-    if (warp == 0) PATCH_TRACE_AT(7);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -629,27 +616,13 @@ size_t decode_workspace_bytes(const patch_layout_t* L, int64_t M) {
     return counters_bytes(L) + kFlaggedBytes + (n_tok > 16 ? size_t(2) * kMaxDecodeCtas * n_tok * kTile * sizeof(float) : 0);
 }
 
-static int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        return v;
-    }();
-    return n;
-}
-
 template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
 static int launch_decode_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
                            __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream) {
     using Cfg = DecodeConfig<N_TOK, STAGES>;
     auto kern = decode_kernel<N_TOK, STAGES, WSTATIC, XSTATIC, GATED>;
-    static bool configured = false;   // per-process attribute, idempotent
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
-            return PATCH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (int rc = allow_dynamic_smem(kern, Cfg::kSmemBytes, configured)) return rc;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     if (TK > 65535) return PATCH_ERR_SHAPE;
     int G = sm_count();
@@ -690,15 +663,8 @@ static int launch_decode_f(bool wstatic, bool xstatic, const CUtensorMap& map, c
 
 // Which small-M schedule serves a launch: stream-K over all SMs (a lone or dependent GEMM gets the whole
 // GPU's bandwidth) or one CTA per row-block / small cluster (independent GEMMs: several of them are resident
-// at once and together stream faster).  PATCH_DECODE_SCHEDULE=streamk|rowblock forces one (experiments).
-static bool use_rowblock_schedule(bool wstatic, bool xstatic) {
-    static const int forced = [] {
-        const char* e = getenv("PATCH_DECODE_SCHEDULE");
-        return !e ? 0 : e[0] == 's' ? 1 : e[0] == 'r' ? 2 : 0;
-    }();
-    if (forced) return forced == 2;
-    return wstatic && xstatic;
-}
+// at once and together stream faster).
+static bool use_rowblock_schedule(bool wstatic, bool xstatic) { return wstatic && xstatic; }
 
 int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                   __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream,
@@ -749,8 +715,7 @@ constexpr size_t kNoAllocScratchBytes =
 // In host code this name is only a handle; the device address comes from cudaGetSymbolAddress.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
-constexpr int kMaxDevices = 64;
-void* g_noalloc_ptr[kMaxDevices];             // device address of the array, per device, once known
+std::atomic<void*> g_noalloc_ptr[patch::kMaxDevices];   // device address of the array, per device, once known
 
 }  // namespace
 
@@ -768,17 +733,17 @@ extern "C" int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M, con
     if (!aligned16(X_dev) || !aligned16(Y_dev) || !aligned16(packed_dev)) return PATCH_ERR_ALIGN;
     rc = check_device();
     if (rc) return rc;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PATCH_ERR_CUDA;
-    if (!g_noalloc_ptr[dev]) {
-        // set-up, once per device, with that device current
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return PATCH_ERR_CUDA;
-        g_noalloc_ptr[dev] = p;
+    const int dev = current_device();
+    if (dev < 0) return PATCH_ERR_CUDA;
+    void* scratch = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        // set-up, once per device, with that device current (two threads racing here store the same address)
+        if (cudaGetSymbolAddress(&scratch, g_noalloc_scratch) != cudaSuccess || !scratch) return PATCH_ERR_CUDA;
+        g_noalloc_ptr[dev].store(scratch, std::memory_order_release);
     }
-    void* scratch = g_noalloc_ptr[dev];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // counters and partial-sum flags must start at zero; the array keeps whatever the last call left
+    // The whole array is cleared on every call: counters and partial-sum flags must start at zero, and the array
+    // keeps whatever the last call left -- also a call that was aborted or that raced with another one.
     if (cudaMemsetAsync(scratch, 0, kNoAllocScratchBytes, s) != cudaSuccess) return PATCH_ERR_CUDA;
     return launch_decode(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
                          static_cast<__nv_bfloat16*>(Y_dev), ldy, scratch, nullptr, s, false, false);

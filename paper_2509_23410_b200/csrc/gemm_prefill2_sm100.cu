@@ -163,14 +163,6 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             const uint32_t idesc_s = idesc_d | (1u << 2);
             bool ok = true;
             int ia = 0, ib = 0, j = 0;
-#ifdef PATCH_TRACE
-            long long wA = 0, wB = 0, tbeg = clock64(), tw;
-#define TW_BEGIN tw = clock64()
-#define TW_END(acc) acc += clock64() - tw
-#else
-#define TW_BEGIN
-#define TW_END(acc)
-#endif
             for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x, ++j) {
                 const bool has1 = 2 * (t % TP) + 1 < TN;
                 // the epilogue must have drained both accumulators of the previous tile
@@ -180,9 +172,7 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
 #pragma unroll
                     for (int h = 0; h < 2 && ok; ++h) {
                         const int bslot = ib % NB;
-                        TW_BEGIN;
                         ok = mbar_wait(bar_fullB + 8 * bslot, uint32_t(ib / NB) & 1u, abort_flag, status_dev);
-                        TW_END(wB);
                         if (!ok) break;
                         const uint64_t dB = desc_kmajor_sw128(smem_base + kBOffset + bslot * kBSlotBytes);
 #pragma unroll
@@ -192,9 +182,7 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
                             if (h == 0 || sp_slot[rb] < 0) {
                                 // next A slot in ring order: a dense half, or (at h = 0) a whole 2:4 tile
                                 const int slot = ia % NA;
-                                TW_BEGIN;
                                 ok = mbar_wait(bar_fullA + 8 * slot, uint32_t(ia / NA) & 1u, abort_flag, status_dev);
-                                TW_END(wA);
                                 if (!ok) break;
                                 ++ia;
                                 tc_fence_after();
@@ -234,12 +222,6 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
                 }
                 if (ok) mma_commit(bar_acc_full);
             }
-#ifdef PATCH_TRACE
-            {
-                unsigned long long* tr = reinterpret_cast<unsigned long long*>(status_dev) + blockIdx.x * 16;
-                tr[0] = 1; tr[1] = clock64() - tbeg; tr[2] = wA; tr[3] = wB;
-            }
-#endif
         }
         __syncwarp();
     } else {
@@ -254,9 +236,6 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             ok = mbar_wait(bar_acc_full, uint32_t(j) & 1u, abort_flag, status_dev);
             if (!ok) break;
             tc_fence_after();
-#ifdef PATCH_TRACE
-            const long long te0 = clock64();
-#endif
             if (independent && j == 0) grid_dependency_wait();     // Y may be in use by the preceding kernel
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             const int chunks = (valid + 15) / 16, c_begin = half == 0 ? 0 : (chunks + 1) / 2,
@@ -300,9 +279,6 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty);
-#ifdef PATCH_TRACE
-            if (warp == 2 && lane == 0) reinterpret_cast<unsigned long long*>(status_dev)[blockIdx.x * 16 + 5] += clock64() - te0;
-#endif
         }
     }
 
@@ -315,12 +291,8 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
                     int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated,
                     bool independent) {
-    static bool configured = false;   // per-process attribute, idempotent
-    if (!configured) {
-        if (cudaFuncSetAttribute(prefill2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p2::kSmemBytes) != cudaSuccess)
-            return PATCH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (int rc = allow_dynamic_smem(prefill2_kernel, p2::kSmemBytes, configured)) return rc;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const int64_t n_out = int64_t((TN + 1) / 2) * ((M + n_tok - 1) / n_tok);
     if (n_out > 0x7FFFFFFF) return PATCH_ERR_SHAPE;

@@ -4,8 +4,8 @@
 // (the only operand tcgen05.mma.sp accepts in compressed form), out-features ride the 128 TMEM
 // lanes, tokens ride the MMA N dimension.  An output tile is (row-block tn) x (n_tok tokens); its
 // mainloop walks the TK weight tiles of the row-block and issues, per tile, eight dense
-// tcgen05.mma or four tcgen05.mma.sp into one fp32 TMEM accumulator -- the paper's mixed
-// execution "within a single matrix multiplication" (Appendix A).
+// tcgen05.mma or four tcgen05.mma.sp into one fp32 TMEM accumulator -- dense and 2:4 tiles
+// mixed inside one multiplication, as Appendix A describes the deployed kernels.
 //
 // Persistent kernel: one CTA per SM loops over output tiles (tile index = mt * TN + tn, so CTAs
 // running side by side share an X tile in L2 and stream different row-blocks).  Two TMEM
@@ -19,7 +19,6 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports
 // PATCH_ERR_TIMEOUT through status_dev, drains its copies in flight, frees TMEM and returns.
-#include <cstdlib>
 #include "sm100_ptx.cuh"
 
 namespace patch {
@@ -64,7 +63,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
     if (!independent) grid_dependency_wait();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (warp == 0) PATCH_TRACE_AT(0);
     const int MT = (M + n_tok - 1) / n_tok;
     const int n_out = TN * MT;                                    // output tiles, index = mt * TN + tn
     const uint32_t x_atom_bytes = uint32_t(n_tok) * 128u;
@@ -87,7 +85,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    if (warp == 0) PATCH_TRACE_AT(1);
 
     if (warp == 0) {
         // ---------------- producer ----------------
@@ -142,7 +139,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
                     const int stage = step % STAGES;
                     ok = mbar_wait(bar_full + 8 * stage, uint32_t(step / STAGES) & 1u, abort_flag, status_dev);
                     if (!ok) break;
-                    if (step == 0) PATCH_TRACE_AT(2);
                     tc_fence_after();
                     const uint32_t sW = smem_base + stage * stage_bytes;
                     issue_tile_mma_n(stage_kind[stage], sW, sW + kDenseBytes, x_atom_bytes, acc,
@@ -151,7 +147,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
                 }
                 if (ok) mma_commit(bar_acc_full + 8 * (j & 1));      // accumulator complete
             }
-            PATCH_TRACE_AT(3);
         }
         __syncwarp();
     } else {
@@ -164,7 +159,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
             ok = mbar_wait(bar_acc_full + 8 * (j & 1), uint32_t(j >> 1) & 1u, abort_flag, status_dev);
             if (!ok) break;
             tc_fence_after();
-            if (j == 0 && warp == 2) PATCH_TRACE_AT(4);
             const uint32_t acc = tmem_base + (j & 1 ? Cfg::kAcc1Col : 0u) + ((quad * 32u) << 16);
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             __nv_bfloat16* ytile = Y + int64_t(m0) * ldy + int64_t(tn) * kTile + quad * 32;
@@ -181,14 +175,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty + 8 * (j & 1));
         }
-        if (warp == 2) PATCH_TRACE_AT(5);
     }
 
     if (independent) grid_dependency_wait();      // every thread passes the dependency before the CTA exits
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, Cfg::kTmemCols);
-    if (warp == 0) PATCH_TRACE_AT(6);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -223,29 +215,9 @@ int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int
     return r == CUDA_SUCCESS ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
-static int sm_count_prefill() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        return v;
-    }();
-    return n;
-}
-
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
                     int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated,
                     bool independent);
-
-// Testing / tuning aid: PATCH_PREFILL_SCHEDULE=1|2 in the environment pins the schedule (one or two
-// row-blocks per CTA); anything else lets the cost model choose.
-static int forced_schedule() {
-    static int v = [] {
-        const char* e = getenv("PATCH_PREFILL_SCHEDULE");
-        return (e && e[0] >= '1' && e[0] <= '2' && e[1] == 0) ? e[0] - '0' : 0;
-    }();
-    return v;
-}
 
 // Schedule choice: token-tile width n (a multiple of 16 in [128, 240]) and one or two row-blocks
 // per CTA, by a small cost model -- waves of output tiles over the SMs times the time of one tile,
@@ -260,11 +232,10 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row
     PrefillPlan best = {240, 1};
     double best_cost = 1e300;
     const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : kPrefillMaxTok, n_lo = M <= 128 ? n_hi : 128;
-    const int forced = forced_schedule();
     for (int n = n_hi; n >= n_lo; n -= 16) {
         const int64_t MT = (M + n - 1) / n;
         for (int sched = 1; sched <= 2; ++sched) {
-            if (two_row_blocks_only ? sched != 2 : (forced && sched != forced)) continue;
+            if (two_row_blocks_only && sched != 2) continue;
             const int64_t tiles = int64_t(sched == 1 ? TN : (TN + 1) / 2) * MT;
             const int64_t waves = (tiles + sms - 1) / sms;
             const double mma_ns = (sched == 1 ? 550.0 : 1100.0) * n / 256.0;
@@ -290,7 +261,7 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                    __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent) {
     if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
-    const int sms = sm_count_prefill();
+    const int sms = sm_count();
     if (sms <= 0) return PATCH_ERR_CUDA;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const PrefillPlan plan = plan_prefill(M, TN, TK, sms, false, independent);
@@ -299,13 +270,8 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
     if (plan.schedule == 2) return launch_prefill2(map, L, packed, M, n_tok, sms, Y, ldy, status_dev, stream, false, independent);
-    static bool configured = false;   // per-process attribute, idempotent
-    if (!configured) {
-        if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 PrefillConfig::kSmemBytes) != cudaSuccess)
-            return PATCH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (int rc = allow_dynamic_smem(prefill_kernel, PrefillConfig::kSmemBytes, configured)) return rc;
     const int64_t n_out = int64_t(TN) * ((M + n_tok - 1) / n_tok);
     if (n_out > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
     cudaLaunchConfig_t cfg = {};
@@ -328,7 +294,7 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
 int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                          __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent) {
     if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
-    const int sms = sm_count_prefill();
+    const int sms = sm_count();
     if (sms <= 0) return PATCH_ERR_CUDA;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const PrefillPlan plan = plan_prefill(M, TN, TK, sms, true, independent);

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <atomic>
 #include "../../include/patch.h"
 
 namespace patch {
@@ -38,6 +39,37 @@ int validate_layout(const patch_layout_t* L);
 int check_device();
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// What the library remembers between calls is per device: which kernels had their shared-memory limit
+// raised there, and the device's SM count.  A process may drive several GPUs from several threads.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+    int d = -1;
+    return (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < kMaxDevices) ? d : -1;
+}
+// Number of SMs of the current device (0 on failure).
+inline int sm_count() {
+    static std::atomic<int> cache[kMaxDevices];
+    const int d = current_device();
+    if (d < 0) return 0;
+    int n = cache[d].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, d) != cudaSuccess) return 0;
+        cache[d].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+// Raises a kernel's dynamic shared-memory limit once per device; `done` is that kernel's bit mask of devices.
+template <class Kernel>
+inline int allow_dynamic_smem(Kernel kern, uint32_t bytes, std::atomic<uint64_t>& done) {
+    const int d = current_device();
+    if (d < 0) return PATCH_ERR_CUDA;
+    if ((done.load(std::memory_order_acquire) >> d) & 1u) return PATCH_OK;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes)) != cudaSuccess)
+        return PATCH_ERR_CUDA;
+    done.fetch_or(uint64_t(1) << d, std::memory_order_release);
+    return PATCH_OK;
+}
 
 // Kernel launchers implemented in the .cu files; all return a PATCH_* status.
 // `wstatic` / `xstatic`: the packed weight / X was not written by the operation preceding this

@@ -239,11 +239,5 @@ int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const
 int launch_decode_cluster_gated(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
                                 __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
 
-#ifdef PATCH_TRACE
-// Debug build only: status_dev is reinterpreted as a buffer of 16 timestamps (ns) per CTA.
-#define PATCH_TRACE_AT(slot) do { if ((threadIdx.x & 31) == 0) reinterpret_cast<unsigned long long*>(status_dev)[(blockIdx.y * gridDim.x + blockIdx.x) * 16 + (slot)] = global_timer_ns(); } while (0)
-#else
-#define PATCH_TRACE_AT(slot) do {} while (0)
-#endif
 
 }  // namespace patch

@@ -95,6 +95,16 @@ def test_product_package_does_not_import_the_oracle():
                 assert "patch_oracle" not in text, fn
 
 
+def test_library_reads_no_environment_variable():
+    """The schedules are fixed in the source: no knob such as PATCH_DECODE_CLUSTER_S can change a launch."""
+    csrc = os.path.join(ROOT, "paper_2509_23410_b200", "csrc")
+    for fn in os.listdir(csrc):
+        text = open(os.path.join(csrc, fn)).read()
+        assert "getenv" not in text and "environ" not in text, fn
+    build_py = open(os.path.join(ROOT, "paper_2509_23410_b200", "build.py")).read()
+    assert "NVCC_FLAGS" not in build_py
+
+
 def test_stacked_case_flags_concatenate_parts():
     """Input recipe of the stacked-matrix workload: flags of q/k/v (gate/up) stacked along N."""
     import numpy as np
