@@ -53,7 +53,7 @@ enum {
 };
 
 /* Kernel choice for patch_gemm_ex (low bits), optionally OR-ed with PATCH_GEMM_WEIGHTS_STATIC. */
-enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2 };
+enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2, PATCH_VARIANT_PAIR = 3 };
 /*
  * Launch promises.  Every GEMM kernel is launched with programmatic dependent launch and lets its
  * successor become resident as soon as it has started itself; each kernel orders itself against
@@ -184,6 +184,8 @@ int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
 /* patch_gemm with an explicit kernel choice and options.
  *   PATCH_VARIANT_GEMV  CUDA-core decode kernel, M <= 4 only (PATCH_ERR_SHAPE otherwise)
  *   PATCH_VARIANT_MMA   tcgen05 tensor-core kernel, any M
+ *   PATCH_VARIANT_PAIR  the CTA-pair (cta_group::2) large-M kernel: M > 64 and a weight whose tiles are all
+ *                       of one kind (PATCH_ERR_SHAPE otherwise); AUTO picks it where it is the fastest
  *   | PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC  see above */
 int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
                   const patch_layout_t* layout, const void* packed_dev,

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpatch_b200.so")
 
 TILE_DENSE, TILE_SPARSE_2_4 = 0, 1
-VARIANT_AUTO, VARIANT_GEMV, VARIANT_MMA = 0, 1, 2
+VARIANT_AUTO, VARIANT_GEMV, VARIANT_MMA, VARIANT_PAIR = 0, 1, 2, 3
 WEIGHTS_STATIC = 0x100   # OR into `variant`: the packed weight is not produced by the preceding kernel
 INPUT_STATIC = 0x200     # OR into `variant`: X is not produced by the preceding kernel
 OK = 0

@@ -41,9 +41,11 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     const bool wstatic = (variant & PATCH_GEMM_WEIGHTS_STATIC) != 0;
     const bool xstatic = (variant & PATCH_GEMM_INPUT_STATIC) != 0;
     variant &= ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC);
-    if (variant != PATCH_VARIANT_AUTO && variant != PATCH_VARIANT_GEMV && variant != PATCH_VARIANT_MMA)
+    if (variant != PATCH_VARIANT_AUTO && variant != PATCH_VARIANT_GEMV && variant != PATCH_VARIANT_MMA &&
+        variant != PATCH_VARIANT_PAIR)
         return PATCH_ERR_SHAPE;
     if (variant == PATCH_VARIANT_GEMV && M > 4) return PATCH_ERR_SHAPE;
+    if (variant == PATCH_VARIANT_PAIR && (M <= 64 || (L->n_dense && L->n_sparse))) return PATCH_ERR_SHAPE;
     const size_t need = decode_workspace_bytes(L, M);
     if (need > 0) {
         if (!workspace_dev) return PATCH_ERR_NULL;
@@ -58,7 +60,7 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
     if (variant == PATCH_VARIANT_GEMV) return launch_gemv(X, ldx, int(M), L, packed, Y, ldy, status_dev, s);
     if (M <= 64) return launch_decode(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s, wstatic, xstatic);
-    return launch_prefill(X, ldx, M, L, packed, Y, ldy, status_dev, s, wstatic && xstatic);
+    return launch_prefill(X, ldx, M, L, packed, Y, ldy, status_dev, s, wstatic && xstatic, variant == PATCH_VARIANT_PAIR);
 }
 
 extern "C" int patch_gemm(const void* X_dev, int64_t ldx, int64_t M, const patch_layout_t* L,

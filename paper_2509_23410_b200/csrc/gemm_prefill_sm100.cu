@@ -215,6 +215,20 @@ int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int
     return r == CUDA_SUCCESS ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
+int make_blob_tensor_map(CUtensorMap* map, const uint8_t* blob, uint64_t total_bytes, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return PATCH_ERR_CUDA;
+    if (total_bytes % 256 || box_rows < 1 || box_rows > 256) return PATCH_ERR_FORMAT;
+    const cuuint64_t dims[2] = {256, cuuint64_t(total_bytes / 256)};
+    const cuuint64_t strides[1] = {256};
+    const cuuint32_t box[2] = {256, cuuint32_t(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(blob), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
 int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int64_t M, int n_tok,
                     int sms, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool gated,
                     bool independent);
@@ -225,11 +239,11 @@ int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8
 // what one SM pulls from L2 (measured: a step's copies land ~1.75 us after they are issued, so
 // the one-row-block ring sustains one step per 1.75 us / stages; ~120 GB/s with the two-ring
 // pipeline), plus a per-tile prologue/epilogue cost.
-struct PrefillPlan { int n_tok; int schedule; };   // schedule: row-blocks per CTA (1 or 2)
+struct PrefillPlan { int n_tok; int schedule; double cost_ns; };   // schedule: row-blocks per CTA (1 or 2), 3 = CTA pairs
 
 static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row_blocks_only = false,
                                 bool independent = false) {
-    PrefillPlan best = {240, 1};
+    PrefillPlan best = {240, 1, 1e300};
     double best_cost = 1e300;
     const int n_hi = M <= 128 ? int((M + 15) / 16 * 16) : kPrefillMaxTok, n_lo = M <= 128 ? n_hi : 128;
     for (int n = n_hi; n >= n_lo; n -= 16) {
@@ -252,19 +266,49 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row
             const double frac = double(tiles) / sms > 1.0 ? double(tiles) / sms : 1.0;
             const double eff_waves = independent ? frac : double(waves);
             const double cost = eff_waves * tile_ns + n;          // at equal time, the narrower tile (less padding)
-            if (cost < best_cost) { best_cost = cost; best = {n, sched}; }
+            if (cost < best_cost) { best_cost = cost; best = {n, sched, cost}; }
         }
     }
     return best;
 }
 
+// CTA-pair schedule (weights whose tiles are all of one kind): a cluster takes four row-blocks x n tokens, so the
+// waves are those of the two-row-block schedule; what a K step costs is the tensor time alone (per CTA the same
+// two accumulators, but half the activation bytes), 2:4 tiles at twice the dense rate.
+int prefill_pair_clusters(bool sparse);
+int prefill_pair_max_tok(bool sparse);
+int launch_prefill_pair(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
+                        int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+
+static PrefillPlan plan_prefill_pair(int64_t M, int TN, int TK, bool sparse) {
+    PrefillPlan best = {0, 3, 1e300};
+    const int clusters = prefill_pair_clusters(sparse);
+    if (clusters <= 0) return best;
+    const int n_max = prefill_pair_max_tok(sparse);
+    const int n_hi = M < n_max ? int((M + 15) / 16 * 16 < 32 ? 32 : (M + 15) / 16 * 16) : n_max, n_lo = n_hi < 128 ? n_hi : 128;
+    for (int n = n_hi; n >= n_lo; n -= 16) {
+        const int64_t tiles = int64_t((TN + 3) / 4) * ((M + n - 1) / n);
+        const int64_t waves = (tiles + clusters - 1) / clusters;
+        const double step_ns = (sparse ? 600.0 : 1100.0) * n / 256.0;
+        const double cost = double(waves) * (TK * step_ns + 8000.0) + n;
+        if (cost < best.cost_ns) best = {n, 3, cost};
+    }
+    return best;
+}
+
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                   __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent) {
+                   __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent, bool force_pair) {
     if (M > 0x7FFFFFFF) return PATCH_ERR_SHAPE;
     const int sms = sm_count();
     if (sms <= 0) return PATCH_ERR_CUDA;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const PrefillPlan plan = plan_prefill(M, TN, TK, sms, false, independent);
+    if (L->n_dense == 0 || L->n_sparse == 0) {
+        const PrefillPlan pair = plan_prefill_pair(M, TN, TK, L->n_dense == 0);
+        if (pair.n_tok && (force_pair || pair.cost_ns < plan.cost_ns))
+            return launch_prefill_pair(X, ldx, M, L, packed, pair.n_tok, Y, ldy, status_dev, stream);
+    }
+    if (force_pair) return PATCH_ERR_SHAPE;      // tiles of both kinds, or the schedule is unavailable on this device
     const int n_tok = plan.n_tok;
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);

@@ -82,9 +82,10 @@ int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_la
                   cudaStream_t stream, bool wstatic, bool xstatic);
 // `independent`: the caller declared the GEMM independent of its predecessor (weights and X static): only its
 // Y stores wait for the preceding kernel.
+// `force_pair`: only the CTA-pair schedule will do (PATCH_ERR_SHAPE if the weight mixes tile kinds).
 int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                    const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream,
-                   bool independent);
+                   bool independent, bool force_pair = false);
 int launch_prefill_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                          const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream,
                          bool independent);

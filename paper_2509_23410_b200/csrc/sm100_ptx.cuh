@@ -131,6 +131,72 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- CTA pairs (cluster of two CTAs on the two SMs of one TPC; cta_group::2 instructions) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// 2-D tiled copy global -> own shared memory whose completion is counted on a barrier that may live in the
+// other CTA of the pair (`bar` is a shared::cluster address).  No multicast: every CTA fetches its own box.
+__device__ __forceinline__ void tma_tile_load_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                                   uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
+}
+// Tensor memory of both CTAs of the pair, same columns in each; executed by one warp of EACH CTA.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// 256 x N x 16 (dense) / 256 x N x 32 (2:4): each CTA supplies its 128 rows of A and N/2 rows of B and
+// receives its 128 rows of D; issued by ONE thread of the leader CTA (rank 0), same addresses in both CTAs.
+__device__ __forceinline__ void mma_dense_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_sparse_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t e_tmem,
+                                                uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+// each CTA's 128 rows x 16 B of shared memory -> its own TMEM, 4 columns
+__device__ __forceinline__ void tmem_copy_pair_128x128b(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// one arrival on the barrier at this shared-memory offset in BOTH CTAs once all tcgen05 operations issued so
+// far by this thread have completed
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(uint16_t(3)) : "memory");
+}
+// Instruction descriptor of the pair MMA: bf16 x bf16 -> fp32, K-major operands, M = 256, N = n_tok.
+__host__ __device__ constexpr uint32_t instr_desc_pair(int n_tok, bool sparse) {
+    return (sparse ? (1u << 2) : 0u) | (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n_tok >> 3) << 17) |
+           (uint32_t(256 >> 4) << 24);
+}
+
 // programmatic dependent launch: allow the next kernel to start / wait for the previous one
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -230,6 +296,9 @@ __device__ __forceinline__ void store_fragment_transposed(const uint32_t (&v)[16
 // Host: tensor map over X [M x ldx] bf16 with a box of 64 columns (128 B) x n_tok rows,
 // 128-byte swizzle, zero fill outside the matrix.
 int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok);
+// Host: tensor map over a packed blob seen as rows of 256 bytes, box = `box_rows` whole rows, no swizzle: a
+// tiled copy at row (byte offset / 256) lands in shared memory exactly like a linear copy of box_rows * 256 bytes.
+int make_blob_tensor_map(CUtensorMap* map, const uint8_t* blob, uint64_t total_bytes, int box_rows);
 
 // Row-block / cluster split-K schedule for M <= 64 (gemm_decode_cluster_sm100.cu), used for GEMMs the caller
 // declared independent of their predecessor (`map`: X tensor map with a box of `n_tok` token rows).
