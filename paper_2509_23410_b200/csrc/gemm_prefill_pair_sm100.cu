@@ -32,6 +32,13 @@
 // 320 threads: warp 0 producer, warp 1 MMA issuer (leader) and TMEM owner, warps 2..9 epilogue (two warps
 // per TMEM lane quadrant, each taking half of the token columns).  Persistent over output tiles.
 //
+// Tried and dropped (each measured against this form on the LLaMA-2-7B shapes at M = 2048 / 4096, same GPU, runs
+// interleaved): cutting the token axis into nearly equal tiles whose count is a multiple of the cluster count (the
+// K steps are bound by the latency of the copies, not by the tensor time of the tile's width, so narrower tiles cost
+// the same per step and balance bought nothing); and an epilogue of sixteen warps that pulls both accumulators into
+// registers, hands them back at once and writes Y while the next tile's MMAs run (no gain on dense, a loss on 2:4
+// weights, whose short stages are the most sensitive to anything else that runs on the SM).
+//
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports PATCH_ERR_TIMEOUT through
 // status_dev, and every role still runs to the common cluster barrier at the end before TMEM is freed.
 #include "sm100_ptx.cuh"
@@ -66,11 +73,21 @@ __device__ __forceinline__ uint32_t meta_col(int stage, int j) {
 }
 }  // namespace pp
 
+// Barrier over the 256 epilogue threads that also ORs a predicate (the same give-up decision in all of them).
+__device__ __forceinline__ bool epilogue_any(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+        "barrier.cta.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"(uint32_t(pred)) : "memory");
+    return out != 0;
+}
+
 template <class C>
 __global__ void __launch_bounds__(pp::kThreads)
 prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     uint32_t pay0_256, int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy,
-                    int* status_dev) {
+                    int* status_dev, int independent) {
     using namespace pp;
     constexpr int KIND = C::KIND, NST = C::NST;
     constexpr uint32_t kTileRows256 = (KIND == kDense ? kDenseBytes : kSparseBytes) / 256;   // blob rows per tile
@@ -114,6 +131,13 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     cluster_sync_all();     // both CTAs' barriers and tensor memory exist before anything crosses the pair
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+
+    // Programmatic dependent launch: the next kernel in the stream may become resident from here on (its CTAs fit
+    // on an SM only once this kernel's have left it).  X, the packed weight and Y may belong to the previous
+    // kernel until the wait -- unless the caller declared this GEMM independent of its predecessor: then only the
+    // Y stores (and the exit) wait.
+    grid_launch_dependents();
+    if (!independent) grid_dependency_wait();
 
     if (warp == 0) {
         // ---------------- producer: this CTA's two weight tiles and its half of the tokens, per stage ----------------
@@ -246,9 +270,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         int jt = 0;
         for (int t = cluster_id; t < n_out && ok; t += n_clusters, ++jt) {
             const int q = t % TQ, m0 = (t / TQ) * n_tok;
-            ok = mbar_wait(bar_acc_full, uint32_t(jt) & 1u, abort_flag, status_dev);
+            // one thread polls the barrier (sleeping in between); the other 255 wait on a hardware barrier, which
+            // costs the shared-memory port nothing while the MMAs run
+            bool failed = false;
+            if (warp == 2 && lane == 0) failed = !mbar_wait_relaxed(bar_acc_full, uint32_t(jt) & 1u, abort_flag, status_dev);
+            ok = !epilogue_any(failed);
             if (!ok) break;
             tc_fence_after();
+            if (independent && jt == 0) grid_dependency_wait();     // Y may be in use by the preceding kernel
             const int valid = M - m0 < n_tok ? M - m0 : n_tok;      // tokens of this tile that exist
             const int chunks = (valid + 15) / 16, c_begin = half == 0 ? 0 : (chunks + 1) / 2,
                       c_end = half == 0 ? (chunks + 1) / 2 : chunks;
@@ -274,6 +303,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     }
 
+    if (independent) grid_dependency_wait();      // every thread passes the dependency before the CTA exits
     // every role of both CTAs ends here: nothing crosses the pair after this barrier
     tc_fence_before();
     __syncthreads();
@@ -318,7 +348,8 @@ int prefill_pair_max_tok(bool sparse) { return sparse ? pp::Cfg<pp::kSparse>::kM
 
 template <class C>
 static int launch_pair_t(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                         int n_tok, int clusters, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+                         int n_tok, int clusters, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream,
+                         bool independent) {
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const int64_t n_out = int64_t((TN + 3) / 4) * ((M + n_tok - 1) / n_tok);
     if (n_out > 0x3FFFFFFF || L->total_bytes / 256 > 0x7FFFFFFFull) return PATCH_ERR_SHAPE;
@@ -329,7 +360,7 @@ static int launch_pair_t(const __nv_bfloat16* X, int64_t ldx, int64_t M, const p
     rc = make_blob_tensor_map(&map_w, packed, L->total_bytes, int(C::kARegionBytes / 256));
     if (rc) return rc;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     cfg.gridDim = dim3(2u * unsigned(n_out < clusters ? n_out : clusters), 1, 1);
     cfg.blockDim = dim3(pp::kThreads, 1, 1);
     cfg.dynamicSmemBytes = C::kSmemBytes;
@@ -338,22 +369,24 @@ static int launch_pair_t(const __nv_bfloat16* X, int64_t ldx, int64_t M, const p
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_pair_kernel<C>, map_x, map_w, uint32_t(L->payload_off / 256), TN, TK,
-                                       int(M), n_tok, Y, ldy, status_dev);
+                                       int(M), n_tok, Y, ldy, status_dev, independent ? 1 : 0);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
 // The weight must hold tiles of one kind only (n_dense == 0 or n_sparse == 0).
 int launch_prefill_pair(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                        int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
+                        int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent) {
     if (L->n_dense && L->n_sparse) return PATCH_ERR_FORMAT;
     const bool sparse = L->n_sparse != 0;
     const int clusters = prefill_pair_clusters(sparse);
     if (clusters <= 0) return PATCH_ERR_CUDA;
-    if (sparse) return launch_pair_t<pp::Cfg<pp::kSparse>>(X, ldx, M, L, packed, n_tok, clusters, Y, ldy, status_dev, stream);
-    return launch_pair_t<pp::Cfg<pp::kDense>>(X, ldx, M, L, packed, n_tok, clusters, Y, ldy, status_dev, stream);
+    if (sparse) return launch_pair_t<pp::Cfg<pp::kSparse>>(X, ldx, M, L, packed, n_tok, clusters, Y, ldy, status_dev, stream, independent);
+    return launch_pair_t<pp::Cfg<pp::kDense>>(X, ldx, M, L, packed, n_tok, clusters, Y, ldy, status_dev, stream, independent);
 }
 
 }  // namespace patch

@@ -278,7 +278,7 @@ static PrefillPlan plan_prefill(int64_t M, int TN, int TK, int sms, bool two_row
 int prefill_pair_clusters(bool sparse);
 int prefill_pair_max_tok(bool sparse);
 int launch_prefill_pair(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                        int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+                        int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent);
 
 static PrefillPlan plan_prefill_pair(int64_t M, int TN, int TK, bool sparse) {
     PrefillPlan best = {0, 3, 1e300};
@@ -289,8 +289,10 @@ static PrefillPlan plan_prefill_pair(int64_t M, int TN, int TK, bool sparse) {
     for (int n = n_hi; n >= n_lo; n -= 16) {
         const int64_t tiles = int64_t((TN + 3) / 4) * ((M + n - 1) / n);
         const int64_t waves = (tiles + clusters - 1) / clusters;
-        const double step_ns = (sparse ? 600.0 : 1100.0) * n / 256.0;
-        const double cost = double(waves) * (TK * step_ns + 8000.0) + n;
+        // a K step costs the tensor time of n tokens, but not less than the pipeline's latency floor (measured with every
+        // SM busy: ~1.3 us on dense, ~0.8 us on 2:4 tiles, whatever the width): at equal cost the wider tile wins
+        const double mma_ns = (sparse ? 550.0 : 1100.0) * n / 256.0, floor_ns = sparse ? 800.0 : 1300.0;
+        const double cost = double(waves) * (TK * (mma_ns > floor_ns ? mma_ns : floor_ns) + 8000.0) - 1e-3 * n;
         if (cost < best.cost_ns) best = {n, 3, cost};
     }
     return best;
@@ -305,8 +307,11 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     const PrefillPlan plan = plan_prefill(M, TN, TK, sms, false, independent);
     if (L->n_dense == 0 || L->n_sparse == 0) {
         const PrefillPlan pair = plan_prefill_pair(M, TN, TK, L->n_dense == 0);
-        if (pair.n_tok && (force_pair || pair.cost_ns < plan.cost_ns))
-            return launch_prefill_pair(X, ldx, M, L, packed, pair.n_tok, Y, ldy, status_dev, stream);
+        // the pair schedule wins wherever every cluster gets a tile of a useful width (measured on the LLaMA shapes:
+        // all M >= 2048, and M = 512 on the 11008-row weights)
+        const bool enough = M * int64_t((TN + 3) / 4) >= int64_t(sms / 2) * 128;
+        if (pair.n_tok && (force_pair || enough))
+            return launch_prefill_pair(X, ldx, M, L, packed, pair.n_tok, Y, ldy, status_dev, stream, independent);
     }
     if (force_pair) return PATCH_ERR_SHAPE;      // tiles of both kinds, or the schedule is unavailable on this device
     const int n_tok = plan.n_tok;

@@ -57,6 +57,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// The same for a wait that is expected to last long (tens of microseconds): the thread sleeps between polls, so
+// that its polling does not compete for the shared-memory port with the operand traffic of the running MMAs.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  int* status_dev) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        __nanosleep(200);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 15u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
 // L2 eviction policies for streamed-once (weights) and reused (activations) data.
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t p;

@@ -81,7 +81,10 @@ def test_pair_schedule_back_to_back(gpu, oracle, p):
     outs = []
     for i in range(12):
         What, packed, L, X, Xd = cases[i % 2]
-        outs.append(B.patch_gemm(Xd, L, packed, status=status, variant=B.VARIANT_PAIR))
+        # every other launch declared independent of its predecessor (weights and X are not written here): it may
+        # start while the launch before it still runs, and only its Y stores wait
+        promise = (B.WEIGHTS_STATIC | B.INPUT_STATIC) if i % 2 else 0
+        outs.append(B.patch_gemm(Xd, L, packed, status=status, variant=B.VARIANT_PAIR | promise))
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     refs = [oracle.gemm_f64(c[3], c[0])[0] for c in cases]
