@@ -207,6 +207,188 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------
+# our arm: helpers shared by the headline workload and the prefill section
+
+
+def launch_flags(B, mode):
+    # weights are packed once, before any step; "independent": no GEMM of the step reads another GEMM's output
+    return B.WEIGHTS_STATIC | (B.INPUT_STATIC if mode == "independent" else 0)
+
+
+def launch_all(B, js, mode, variant=0):
+    for j in js:
+        B.patch_gemm(j["X"], j["layout"], j["packed"], Y=j["Y"], workspace=j["ws"], variant=variant | launch_flags(B, mode))
+
+
+def make_graph(torch, B, js, mode, variant=0):
+    launch_all(B, js, mode, variant)        # first call sets kernel attributes; must precede capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        launch_all(B, js, mode, variant)
+    return g
+
+
+def time_graph(torch, g, reps):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e-3 / reps
+
+
+def per_case_table(torch, B, jobs, mode, peaks, variant=0):
+    """Each GEMM on rotating copies of its packed weight (>= 3 x L2 of them), so that its weight reads come from HBM."""
+    table = []
+    for j in jobs:
+        blob = j["packed"]
+        n_copies = int(min(max(3 * L2_BYTES // blob.numel() + 1, 2), 24))
+        copies = [blob.clone() for _ in range(n_copies)]
+        js = [dict(j, packed=cp) for cp in copies]
+        g = make_graph(torch, B, js, mode, variant)
+        for _ in range(3):
+            g.replay()
+        t = time_graph(torch, g, 3) / n_copies
+        # enough launches per graph (about 2 ms worth, at most 48 rounds) that the drain at its end does not show
+        rounds = int(min(max(round(2e-3 / (t * n_copies)), 1), 48))
+        if rounds > 1:
+            g = make_graph(torch, B, js * rounds, mode, variant)
+            g.replay()
+        t = time_graph(torch, g, 10) / (n_copies * rounds)
+        rs, b = roofline_seconds(j["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)
+        rm, _ = roofline_seconds(j["cost"], peaks["hbm_gbs"], peaks["bf16_tflops_sustained"],
+                                 2 * peaks["bf16_tflops_sustained"])
+        table.append(dict(name=j["case"]["name"], us=round(t * 1e6, 2),
+                          eff_tflops=round(j["cost"]["flops"] / t / 1e12, 2), bound=b,
+                          frac_spec=round(rs / t, 3), frac_measured=round(rm / t, 3),
+                          f_sparse=round(j["layout"].n_sparse / (j["layout"].n_sparse + j["layout"].n_dense), 3)))
+        del copies, js, g
+    return table
+
+
+def speedup_table(table):
+    """Speed-up of every hybrid / 2:4 case over the all-dense tile configuration of the same shape and M
+    (the comparison the prefill workload asks for)."""
+    dense = {}
+    for c in table:
+        if c["f_sparse"] == 0.0:
+            dense[(c["name"].split(".p")[0], c["name"].rsplit(".M", 1)[1])] = c["us"]
+    sp = []
+    for c in table:
+        base = dense.get((c["name"].split(".p")[0], c["name"].rsplit(".M", 1)[1]))
+        if base and c["f_sparse"] > 0.0:
+            # ceiling: 18 432 instead of 32 768 bytes per 2:4 tile where HBM binds, half the tensor time where the MMAs do
+            ceiling = 1.0 / (1.0 - (0.4375 if c["bound"] == "hbm" else 0.5) * c["f_sparse"])
+            sp.append(dict(name=c["name"], f_sparse=c["f_sparse"], speedup_vs_all_dense=round(base / c["us"], 3),
+                           ceiling=round(ceiling, 3), bound=c["bound"]))
+    return sp
+
+
+def parity_check(torch, jobs, seed_rows=8):
+    """`--check sampled`: the outputs the timed graph left behind against the oracle (rank 0, one GPU).  GEMMs of up to
+    64 tokens are compared in full, larger ones on `seed_rows` token rows spread over the token tiles plus the first and
+    the last row.  Returns the worst relative Frobenius error and the worst max |dY| / max |Yref| over the GEMMs."""
+    import oracle
+    oracle.build()
+    to_bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    pruned, worst_f, worst_m, n_out = {}, 0.0, 0.0, 0
+    for j in jobs:
+        key = id(j["packed"])
+        if key not in pruned:
+            pruned[key] = oracle.prune(j["W_bits"]() if callable(j["W_bits"]) else j["W_bits"], j["flags"])
+        What = pruned[key]
+        M = j["case"]["M"]
+        Xb, Yb = to_bits(j["X"]), to_bits(j["Y"])
+        if M <= 64:
+            ref, _ = oracle.gemm_f64(Xb, What)
+            got = inputs.bf16_bits_to_f32(Yb)
+        else:
+            rows = np.unique(np.concatenate([np.linspace(0, M - 1, seed_rows).astype(np.int64), [0, M - 1]]))
+            ref = oracle.gemm_f64_rows(Xb, rows, What)
+            got = inputs.bf16_bits_to_f32(Yb[rows])
+        relF, maxrel = oracle.parity_metrics(got, ref)
+        worst_f, worst_m, n_out = max(worst_f, float(relF)), max(worst_m, float(maxrel)), n_out + ref.size
+    return dict(relF=worst_f, maxrel=worst_m, gemms=len(jobs), outputs_compared=int(n_out),
+                tolerance={"relF": 2e-3, "maxrel": 1e-2}, ok=bool(worst_f <= 2e-3 and worst_m <= 1e-2),
+                how="timed graph's outputs vs the CPU oracle (double accumulation); M <= 64 in full, larger M on sampled token rows")
+
+
+def prefill_section(args, torch, B, dev, peaks):
+    """The tensor-core half of the metric on the default line: the 27 LLaMA-2-7B prefill GEMMs (3 shapes x
+    M in {512, 2048, 4096} x 2:4-tile fraction in {0, .5, 1}) as one step from a CUDA graph.  Weights and activations
+    are drawn on the device (torch Philox, seeded per matrix); the tile flags are the seeded Bernoulli draws of
+    inputs.prefill_cases()."""
+    cases = sorted(inputs.prefill_cases(), key=lambda c: c["M"])
+    mats, xs, jobs = {}, {}, []
+    for c in cases:
+        key = (c["N"], c["K"], c["stream"])
+        if key not in mats:
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(inputs.MASTER_SEED * 1000 + 500 + len(mats))
+            W = torch.empty((c["N"], c["K"]), dtype=torch.bfloat16, device=dev).normal_(0.0, 0.02, generator=gen)
+            flags = inputs.case_flags(c)
+            layout = B.patch_packed_size(c["N"], c["K"], flags)
+            packed = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
+            B.patch_pack(W, flags, layout=layout, out=packed)
+            Wh = W.view(torch.int16).cpu().numpy().view(np.uint16) if args.check != "none" else None
+            mats[key] = (layout, packed, flags, Wh)
+            del W
+        layout, packed, flags, Wh = mats[key]
+        xkey = (c["M"], c["K"])
+        if xkey not in xs:
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(inputs.MASTER_SEED * 1000 + 900 + len(xs))
+            xs[xkey] = torch.empty(xkey, dtype=torch.bfloat16, device=dev).normal_(0.0, 1.0, generator=gen)
+        Y = torch.empty((c["M"], c["N"]), dtype=torch.bfloat16, device=dev)
+        jobs.append(dict(case=c, layout=layout, packed=packed, X=xs[xkey], Y=Y, ws=None, cost=case_costs(c, layout),
+                         W_bits=Wh, flags=flags))
+    g = make_graph(torch, B, jobs, args.launch)
+    # the step is power-capped: warm up until the clocks have settled (~0.3 s of back-to-back steps), then time
+    steps, warm = max(3, min(100, args.steps)), max(3, min(100, args.steps))
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    for _ in range(warm):
+        g.replay()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    step_s = time_graph(torch, g, steps)
+    clocks = sampler.stop(t0, time.time())
+    flops = sum(j["cost"]["flops"] for j in jobs)
+    fd, fs = sum(j["cost"]["f_dense"] for j in jobs), sum(j["cost"]["f_sparse"] for j in jobs)
+    sus = peaks["bf16_tflops_sustained"]
+    peak_meas = (fd + fs) / (fd / sus + fs / (2 * sus))                 # flop-weighted mix, 2:4 tiles at twice the dense rate
+    peak_spec = (fd + fs) / (fd / DENSE_SPEC_TFLOPS + fs / SPARSE_SPEC_TFLOPS)
+    spec_t = sum(roofline_seconds(j["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)[0] for j in jobs)
+    achieved = flops / step_s / 1e12
+    out = {
+        "workload": "llama2-7b prefill linears", "gemms_per_step": len(jobs), "steps": steps, "warmup": warm,
+        "ms_per_step": step_s * 1e3, "value": achieved, "unit": "TFLOP/s", "launch": args.launch, "cuda_graph": True,
+        "data": "synthetic (weights and activations drawn on the device)",
+        "l2": "inputs larger than L2: a step streams 9 packed matrices (~0.5 GB) and 0.77 GB of outputs",
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak_meas, "unit": "TFLOP/s", "frac": achieved / peak_meas,
+                     "frac_of_spec": spec_t / step_s, "peak_spec": peak_spec, "peak_source": peaks["source"] + " (sustained bf16; 2:4 tiles x2)",
+                     "traffic": None,
+                     "kernels": "prefill_pair_kernel (weights of one tile kind), prefill2_kernel / prefill_kernel (mixed weights, M = 512)"},
+        "clocks": clocks,
+        # the step is power-capped: its time times the sampled SM clock separates kernel changes from clock drift
+        "ms_x_sm_ghz": step_s * 1e3 * (clocks.get("sm_mhz") or 0.0) / 1e3,
+        "gpu_launches": steps * len(jobs),
+    }
+    table = per_case_table(torch, B, jobs, args.launch, peaks)
+    out["cases"] = table
+    out["speedup_vs_all_dense"] = speedup_table(table)
+    if args.check != "none":
+        g.replay()
+        torch.cuda.synchronize()
+        for j in jobs:
+            j["ws"] = None
+        out["parity"] = parity_check(torch, jobs)
+    return out
+
+
+# ---------------------------------------------------------------------------------------------
 # our arm
 
 
@@ -267,11 +449,12 @@ def run_ours(args):
         pack_dev_secs += e0.elapsed_time(e1) * 1e-3
         if not torch.equal(packed, packed2):
             raise SystemExit("patch_pack_dev and patch_pack disagree")
-        mats[key] = (layout, packed)
+        keep_w = args.check != "none" and not args.workload.startswith("stack")
+        mats[key] = (layout, packed, flags, inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]) if keep_w else None)
         del W, packed2
     jobs, stack_x, shared_ws = [], {}, {}
     for c in cases:
-        layout, packed = mats[(c["N"], c["K"], c["stream"])]
+        layout, packed, flags, w_bits = mats[(c["N"], c["K"], c["stream"])]
         xkey = (c["M"], c["K"]) if args.workload.startswith("stack") else None
         if xkey is not None and xkey in stack_x:
             X = stack_x[xkey]                # the stack shares one activation per (M, K); outputs are not chained
@@ -284,26 +467,12 @@ def run_ours(args):
         if wkey not in shared_ws:            # GEMMs on one stream are ordered, so they may share a workspace
             shared_ws[wkey] = torch.zeros(max(B.patch_gemm_workspace_size(layout, c["M"]), 256), dtype=torch.uint8, device=dev)
         ws = shared_ws[wkey]
-        jobs.append(dict(case=c, layout=layout, packed=packed, X=X, Y=Y, ws=ws, cost=case_costs(c, layout)))
+        jobs.append(dict(case=c, layout=layout, packed=packed, X=X, Y=Y, ws=ws, cost=case_costs(c, layout),
+                         W_bits=w_bits, flags=flags))
     weight_bytes = sum(m[0].total_bytes for m in mats.values())
 
-    # weights are packed once, before any step; in this workload no GEMM reads another GEMM's output
-    def flags_for(mode):
-        return B.WEIGHTS_STATIC | (B.INPUT_STATIC if mode == "independent" else 0)
-
-    def launch_all(js, mode):
-        for j in js:
-            B.patch_gemm(j["X"], j["layout"], j["packed"], Y=j["Y"], workspace=j["ws"],
-                         variant=args.variant | flags_for(mode))
-
-    def make_graph(js, mode=None):
-        mode = mode or args.launch
-        launch_all(js, mode)                # first call sets kernel attributes; must precede capture
-        torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            launch_all(js, mode)
-        return g
+    def mk_graph(js, mode=None):
+        return make_graph(torch, B, js, mode or args.launch, args.variant)
 
     def barrier():
         if world > 1:
@@ -311,20 +480,14 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def time_graph(g, reps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
-            g.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) * 1e-3 / reps
+    def tm_graph(g, reps):
+        return time_graph(torch, g, reps)
 
-    step_graph = make_graph(jobs)
+    step_graph = mk_graph(jobs)
     # several consecutive steps may be captured into one graph (a serving loop enqueues step after step on
     # one stream; a graph per step would end every step with a full drain that such a loop does not have)
     spg = max(1, min(args.steps_per_graph, args.steps))
-    multi_graph = make_graph(jobs * spg) if spg > 1 else step_graph
+    multi_graph = mk_graph(jobs * spg) if spg > 1 else step_graph
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
     sampler.start()
     for _ in range(max(args.warmup, 3)):
@@ -362,14 +525,14 @@ def run_ours(args):
     # ---- one step per graph replay, for comparison: every step then ends with a full drain of the GPU
     single_s = step_s
     if spg > 1:
-        single_s = replicas.max_over_ranks(time_graph(step_graph, max(10, args.steps // 5)), dev)
+        single_s = replicas.max_over_ranks(tm_graph(step_graph, max(10, args.steps // 5)), dev)
 
     # ---- the same step under the other launch promise (context for the headline number)
     other = "dependent" if args.launch == "independent" else "independent"
-    g_other = make_graph(jobs * spg, other)
+    g_other = mk_graph(jobs * spg, other)
     for _ in range(3):
         g_other.replay()
-    other_s = time_graph(g_other, max(10, args.steps // 5 // spg)) / spg
+    other_s = tm_graph(g_other, max(10, args.steps // 5 // spg)) / spg
     del g_other
 
     # ---- dominant kernel: the launches that take the largest share of the step, timed on their own
@@ -378,10 +541,10 @@ def run_ours(args):
         groups.setdefault(j["case"]["M"], []).append(j)
     dom = None
     for M, js in groups.items():
-        g = make_graph(js * spg)            # the same number of passes per graph as the timed step
+        g = mk_graph(js * spg)              # the same number of passes per graph as the timed step
         for _ in range(3):
             g.replay()
-        t = time_graph(g, max(10, args.steps // 10 // spg)) / spg
+        t = tm_graph(g, max(10, args.steps // 10 // spg)) / spg
         if dom is None or t > dom[1]:
             dom = (M, t, js)
     dM, dt, djs = dom
@@ -450,31 +613,18 @@ def run_ours(args):
     d2h = sum(j["Y"].numel() * 2 for j in jobs)
 
     # ---- per-case table (each GEMM on rotating copies of its packed weight so reads come from HBM)
-    table = []
-    if args.detail and rank == 0:
-        for j in jobs:
-            blob = j["packed"]
-            n_copies = int(min(max(3 * L2_BYTES // blob.numel() + 1, 2), 24))
-            copies = [blob.clone() for _ in range(n_copies)]
-            js = [dict(j, packed=cp) for cp in copies]
-            g = make_graph(js)
-            for _ in range(3):
-                g.replay()
-            t = time_graph(g, 3) / n_copies
-            # enough launches per graph (about 2 ms worth, at most 48 rounds) that the drain at its end does not show
-            rounds = int(min(max(round(2e-3 / (t * n_copies)), 1), 48))
-            if rounds > 1:
-                g = make_graph(js * rounds)
-                g.replay()
-            t = time_graph(g, 10) / (n_copies * rounds)
-            rs, b = roofline_seconds(j["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)
-            rm, _ = roofline_seconds(j["cost"], peaks["hbm_gbs"], peaks["bf16_tflops_sustained"],
-                                     2 * peaks["bf16_tflops_sustained"])
-            table.append(dict(name=j["case"]["name"], us=round(t * 1e6, 2),
-                              eff_tflops=round(j["cost"]["flops"] / t / 1e12, 2), bound=b,
-                              frac_spec=round(rs / t, 3), frac_measured=round(rm / t, 3),
-                              f_sparse=round(j["layout"].n_sparse / (j["layout"].n_sparse + j["layout"].n_dense), 3)))
-            del copies, js, g
+    table = per_case_table(torch, B, jobs, args.launch, peaks, args.variant) if args.detail and rank == 0 else []
+
+    # ---- parity of what the timed graph computed (opt-in), and the tensor-core half of the metric
+    parity = None
+    if args.check != "none" and rank == 0 and world == 1 and not args.workload.startswith("stack"):
+        step_graph.replay()
+        torch.cuda.synchronize()
+        parity = parity_check(torch, jobs)
+    prefill = None
+    if args.workload == "decode" and not args.no_prefill and rank == 0:
+        del step_graph, multi_graph
+        prefill = prefill_section(args, torch, B, dev, peaks)
 
     if rank != 0:
         return
@@ -511,22 +661,13 @@ def run_ours(args):
         out["cpu_baseline"] = cpu
     if table:
         out["cases"] = table
-        # speed-up of every hybrid / 2:4 case over the all-dense tile configuration of the same shape and M
-        # (the comparison the prefill workload asks for)
-        dense = {}
-        for c in table:
-            if c["f_sparse"] == 0.0:
-                dense[(c["name"].split(".p")[0], c["name"].rsplit(".M", 1)[1])] = c["us"]
-        sp = []
-        for c in table:
-            base = dense.get((c["name"].split(".p")[0], c["name"].rsplit(".M", 1)[1]))
-            if base and c["f_sparse"] > 0.0:
-                # ceiling: 18 432 instead of 32 768 bytes per 2:4 tile where HBM binds, half the tensor time where the MMAs do
-                ceiling = 1.0 / (1.0 - (0.4375 if c["bound"] == "hbm" else 0.5) * c["f_sparse"])
-                sp.append(dict(name=c["name"], f_sparse=c["f_sparse"], speedup_vs_all_dense=round(base / c["us"], 3),
-                               ceiling=round(ceiling, 3), bound=c["bound"]))
+        sp = speedup_table(table)
         if sp:
             out["speedup_vs_all_dense"] = sp
+    if parity is not None:
+        out["parity"] = parity
+    if prefill is not None:
+        out["prefill"] = prefill
     print(json.dumps(out))
 
 
@@ -743,6 +884,11 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--steps-per-graph", type=int, default=8,
                     help="consecutive steps captured into one CUDA graph (the timed region still runs exactly --steps steps)")
+    ap.add_argument("--check", default="none", choices=["none", "sampled"],
+                    help="sampled: after timing, compare the outputs of the timed graph with the CPU oracle and print "
+                         "parity {relF, maxrel} on the line (adds the oracle's run time)")
+    ap.add_argument("--no-prefill", action="store_true",
+                    help="default workload only: skip the prefill section (the tensor-core half of the metric)")
     ap.add_argument("--e2e-chunks", type=int, default=0,
                     help="runs of jobs the end-to-end leg pipelines over its three streams (0: 2 for steps that move "
                          "less than 32 MB, where each extra run costs more in event traffic than it hides, else 8)")

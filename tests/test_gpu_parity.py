@@ -336,10 +336,94 @@ def _check_case(gpu, oracle, W, flags, X, what, n_rows=16):
         Y32, _ = oracle.gemm_f64(X, What)
         check_parity(oracle, Y, Y32, what)
     else:
+        # sampled: random token rows, one row out of every 128 tokens (so that every token tile of every schedule,
+        # whose tiles are at least 128 tokens wide, has a sampled row), the corners of the usual tile widths ...
         rng = inputs.generator(inputs.MASTER_SEED, "rows", what)
-        rows = np.unique(np.concatenate([rng.integers(0, M, n_rows), [0, M - 1, 239, 240, M // 2]]))
+        stride_rows = np.arange(0, M, 128) + rng.integers(0, 128, (M + 127) // 128)
+        rows = np.unique(np.concatenate([rng.integers(0, M, n_rows), stride_rows[stride_rows < M],
+                                         [0, M - 1, 239, 240, 255, 256, M // 2]]))
         check_parity(oracle, Y[rows], oracle.gemm_f64_rows(X, rows, What), what)
+        # ... and two whole row-blocks of out-features over ALL tokens (the last one and a random one)
+        N = W.shape[0]
+        for tn in {N // 128 - 1, int(rng.integers(0, N // 128))}:
+            cols = slice(tn * 128, tn * 128 + 128)
+            Yb, _ = oracle.gemm_f64(X, What[cols], want_bf16=False)
+            check_parity(oracle, Y[:, cols], Yb, f"{what} row-block {tn}")
     return packed, L
+
+
+@pytest.fixture(scope="module")
+def decode_workload(gpu, oracle):
+    """The 24 GEMMs of the decode workload as bench.py sets them up: 12 packed matrices (3 shapes x four 2:4-tile
+    fractions), M = 1 and 16, with the oracle's result for each."""
+    torch, B = gpu
+    cases = sorted(inputs.decode_cases(), key=lambda c: c["M"])
+    mats, jobs = {}, []
+    for c in cases:
+        key = c["stream"]
+        if key not in mats:
+            W = inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"])
+            flags = inputs.case_flags(c)
+            packed, L = B.patch_pack(to_dev(torch, W), flags)
+            mats[key] = (oracle.prune(W, flags), packed, L)
+        What, packed, L = mats[key]
+        X = inputs.activation(c["M"], c["K"], inputs.MASTER_SEED, *c["stream"], c["M"])
+        Y32, Y16 = oracle.gemm_f64(X, What)
+        jobs.append(dict(case=c, L=L, packed=packed, X=to_dev(torch, X), Y32=Y32, Y16=Y16,
+                         Y=torch.zeros((c["M"], c["N"]), dtype=torch.bfloat16, device="cuda")))
+    ws = torch.zeros(B.patch_gemm_workspace_size(jobs[0]["L"], 64), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    return jobs, ws
+
+
+def test_decode_workload_all_cases_bench_flags(gpu, oracle, decode_workload):
+    """Every one of the 24 decode cases, whole output, launched as the benchmark launches them
+    (automatic kernel choice with both promises: the row-block / cluster schedule)."""
+    torch, B = gpu
+    jobs, ws = decode_workload
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for j in jobs:
+        j["Y"].zero_()
+        B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Y"], workspace=ws, status=status,
+                     variant=B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got = to_bits(j["Y"])
+        check_parity(oracle, got, j["Y32"], j["case"]["name"])
+        assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
+
+
+@pytest.mark.parametrize("mode", ["independent", "dependent"])
+def test_decode_workload_graph_replay(gpu, oracle, decode_workload, mode):
+    """The regime the headline number is timed in: two consecutive steps of the 24 GEMMs captured into one CUDA
+    graph (several kernels resident at once, ordered only by their device-side waits), replayed twice; then
+    every one of the 24 outputs is compared with the oracle.  Once with both promises, once with the weights
+    promise only (every GEMM waits for its predecessor before reading X)."""
+    torch, B = gpu
+    jobs, ws = decode_workload
+    flags = B.WEIGHTS_STATIC | (B.INPUT_STATIC if mode == "independent" else 0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step():
+        for j in jobs:
+            B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Y"], workspace=ws, status=status, variant=B.VARIANT_AUTO | flags)
+    step()                                   # kernel attributes are set outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+        step()
+    for j in jobs:
+        j["Y"].zero_()
+    torch.cuda.synchronize()
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for j in jobs:
+        got = to_bits(j["Y"])
+        check_parity(oracle, got, j["Y32"], f"{j['case']['name']} ({mode}, graph)")
+        assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
 
 
 _PREFILL = [(s, p) for s in inputs.LLAMA2_7B_SHAPES for p in (0.0, 0.5, 1.0)]
