@@ -184,8 +184,10 @@ int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
 /* patch_gemm with an explicit kernel choice and options.
  *   PATCH_VARIANT_GEMV  CUDA-core decode kernel, M <= 4 only (PATCH_ERR_SHAPE otherwise)
  *   PATCH_VARIANT_MMA   tcgen05 tensor-core kernel, any M
- *   PATCH_VARIANT_PAIR  the CTA-pair (cta_group::2) large-M kernel: M > 64 and a weight whose tiles are all
- *                       of one kind (PATCH_ERR_SHAPE otherwise); AUTO picks it where it is the fastest
+ *   PATCH_VARIANT_PAIR  the CTA-pair (cta_group::2) large-M kernels, M > 64 (PATCH_ERR_SHAPE otherwise).  AUTO
+ *                       picks the pair schedule for weights whose tiles are all of one kind wherever every CTA
+ *                       pair gets a tile of a useful width; for weights that mix kinds it is slower than the
+ *                       one-CTA schedule and runs only when asked for
  *   | PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC  see above */
 int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
                   const patch_layout_t* layout, const void* packed_dev,

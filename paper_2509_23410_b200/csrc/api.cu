@@ -45,7 +45,7 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
         variant != PATCH_VARIANT_PAIR)
         return PATCH_ERR_SHAPE;
     if (variant == PATCH_VARIANT_GEMV && M > 4) return PATCH_ERR_SHAPE;
-    if (variant == PATCH_VARIANT_PAIR && (M <= 64 || (L->n_dense && L->n_sparse))) return PATCH_ERR_SHAPE;
+    if (variant == PATCH_VARIANT_PAIR && M <= 64) return PATCH_ERR_SHAPE;
     const size_t need = decode_workspace_bytes(L, M);
     if (need > 0) {
         if (!workspace_dev) return PATCH_ERR_NULL;

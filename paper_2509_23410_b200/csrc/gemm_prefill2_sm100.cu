@@ -233,7 +233,8 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
         for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x, ++j) {
             const int tn0 = 2 * (t % TP), m0 = (t / TP) * n_tok;
             const bool has1 = tn0 + 1 < TN;
-            ok = mbar_wait(bar_acc_full, uint32_t(j) & 1u, abort_flag, status_dev);
+            // one thread polls, the other 255 epilogue threads sleep on a hardware barrier
+            ok = group_wait(bar_acc_full, uint32_t(j) & 1u, warp == 2 && lane == 0, 1, 256, abort_flag, status_dev);
             if (!ok) break;
             tc_fence_after();
             if (independent && j == 0) grid_dependency_wait();     // Y may be in use by the preceding kernel

@@ -73,16 +73,6 @@ __device__ __forceinline__ uint32_t meta_col(int stage, int j) {
 }
 }  // namespace pp
 
-// Barrier over the 256 epilogue threads that also ORs a predicate (the same give-up decision in all of them).
-__device__ __forceinline__ bool epilogue_any(bool pred) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
-        "barrier.cta.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out) : "r"(uint32_t(pred)) : "memory");
-    return out != 0;
-}
-
 template <class C>
 __global__ void __launch_bounds__(pp::kThreads)
 prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -272,9 +262,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const int q = t % TQ, m0 = (t / TQ) * n_tok;
             // one thread polls the barrier (sleeping in between); the other 255 wait on a hardware barrier, which
             // costs the shared-memory port nothing while the MMAs run
-            bool failed = false;
-            if (warp == 2 && lane == 0) failed = !mbar_wait_relaxed(bar_acc_full, uint32_t(jt) & 1u, abort_flag, status_dev);
-            ok = !epilogue_any(failed);
+            ok = group_wait(bar_acc_full, uint32_t(jt) & 1u, warp == 2 && lane == 0, 1, 256, abort_flag, status_dev);
             if (!ok) break;
             tc_fence_after();
             if (independent && jt == 0) grid_dependency_wait();     // Y may be in use by the preceding kernel

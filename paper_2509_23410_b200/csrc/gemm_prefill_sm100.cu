@@ -156,7 +156,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
         int j = 0;
         for (int t = blockIdx.x; t < n_out && ok; t += gridDim.x, ++j) {
             const int tn = t % TN, m0 = (t / TN) * n_tok;
-            ok = mbar_wait(bar_acc_full + 8 * (j & 1), uint32_t(j >> 1) & 1u, abort_flag, status_dev);
+            // one thread polls, the other 127 epilogue threads sleep on a hardware barrier
+            ok = group_wait(bar_acc_full + 8 * (j & 1), uint32_t(j >> 1) & 1u, warp == 2 && lane == 0, 1, 128, abort_flag, status_dev);
             if (!ok) break;
             tc_fence_after();
             const uint32_t acc = tmem_base + (j & 1 ? Cfg::kAcc1Col : 0u) + ((quad * 32u) << 16);
@@ -280,11 +281,18 @@ int prefill_pair_max_tok(bool sparse);
 int launch_prefill_pair(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                         int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent);
 
-static PrefillPlan plan_prefill_pair(int64_t M, int TN, int TK, bool sparse) {
+int prefill_pair_mixed_clusters();
+int prefill_pair_mixed_max_tok();
+int launch_prefill_pair_mixed(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
+                              int n_tok, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool independent);
+
+// kind: 0 all dense, 1 all 2:4, 2 mixed (gemm_prefill_pair_mixed_sm100.cu)
+static PrefillPlan plan_prefill_pair(int64_t M, int TN, int TK, int kind) {
     PrefillPlan best = {0, 3, 1e300};
-    const int clusters = prefill_pair_clusters(sparse);
+    const bool sparse = kind == 1;
+    const int clusters = kind == 2 ? prefill_pair_mixed_clusters() : prefill_pair_clusters(sparse);
     if (clusters <= 0) return best;
-    const int n_max = prefill_pair_max_tok(sparse);
+    const int n_max = kind == 2 ? prefill_pair_mixed_max_tok() : prefill_pair_max_tok(sparse);
     const int n_hi = M < n_max ? int((M + 15) / 16 * 16 < 32 ? 32 : (M + 15) / 16 * 16) : n_max, n_lo = n_hi < 128 ? n_hi : 128;
     for (int n = n_hi; n >= n_lo; n -= 16) {
         const int64_t tiles = int64_t((TN + 3) / 4) * ((M + n - 1) / n);
@@ -305,15 +313,22 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     if (sms <= 0) return PATCH_ERR_CUDA;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const PrefillPlan plan = plan_prefill(M, TN, TK, sms, false, independent);
-    if (L->n_dense == 0 || L->n_sparse == 0) {
-        const PrefillPlan pair = plan_prefill_pair(M, TN, TK, L->n_dense == 0);
+    {
+        const int kind = L->n_sparse == 0 ? 0 : L->n_dense == 0 ? 1 : 2;
+        const PrefillPlan pair = plan_prefill_pair(M, TN, TK, kind);
         // the pair schedule wins wherever every cluster gets a tile of a useful width (measured on the LLaMA shapes:
         // all M >= 2048, and M = 512 on the 11008-row weights)
         const bool enough = M * int64_t((TN + 3) / 4) >= int64_t(sms / 2) * 128;
-        if (pair.n_tok && (force_pair || enough))
+        // Weights that mix kinds go to the pair schedule only on request: every 2:4 tile whose pair partner is dense
+        // has to be expanded first, and the chain [tile lands -> helper warps rewrite it -> arrival crosses the pair]
+        // is longer than the four stages can hide (measured on the LLaMA-2-7B shapes at half 2:4 tiles:
+        // 900-1020 TFLOP/s against 1200-1640 on the two-row-block schedule).
+        if (pair.n_tok && (force_pair || (enough && kind != 2))) {
+            if (kind == 2) return launch_prefill_pair_mixed(X, ldx, M, L, packed, pair.n_tok, Y, ldy, status_dev, stream, independent);
             return launch_prefill_pair(X, ldx, M, L, packed, pair.n_tok, Y, ldy, status_dev, stream, independent);
+        }
     }
-    if (force_pair) return PATCH_ERR_SHAPE;      // tiles of both kinds, or the schedule is unavailable on this device
+    if (force_pair) return PATCH_ERR_CUDA;       // the schedule is unavailable on this device
     const int n_tok = plan.n_tok;
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);

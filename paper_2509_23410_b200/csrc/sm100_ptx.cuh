@@ -77,6 +77,24 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
     }
 }
 
+// Hardware barrier `id` over `threads` threads of the CTA that also ORs a predicate (the same decision in all of them).
+__device__ __forceinline__ bool barrier_any(bool pred, int id, int threads) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+        "barrier.cta.red.or.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"(uint32_t(pred)), "r"(id), "r"(threads) : "memory");
+    return out != 0;
+}
+// A group of warps waits for an mbarrier: the thread with `poller` set polls it (sleeping in between), the others
+// wait on hardware barrier `id`, which costs the shared-memory port nothing while the MMAs run.  False if given up.
+__device__ __forceinline__ bool group_wait(uint32_t bar, uint32_t parity, bool poller, int id, int threads,
+                                           volatile int* abort_flag, int* status_dev) {
+    bool failed = false;
+    if (poller) failed = !mbar_wait_relaxed(bar, parity, abort_flag, status_dev);
+    return !barrier_any(failed, id, threads);
+}
+
 // L2 eviction policies for streamed-once (weights) and reused (activations) data.
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t p;
