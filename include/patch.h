@@ -170,9 +170,12 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  *   Y_dev   bf16 [M x ldy], ldy >= N, ldy % 8 == 0
  *   workspace_dev / workspace_bytes   at least patch_gemm_workspace_size(layout, M) bytes,
  *           256-byte aligned, initialised once with patch_workspace_init; may be NULL if 0
- *   status_dev   optional device int, must be zero before the call; receives
- *           PATCH_ERR_TIMEOUT if a bounded device-side wait expired (the kernel then stops
- *           early and Y is undefined).  NULL = not reported.
+ *   status_dev   optional device int, must be zero before the call; receives the first device-side
+ *           error: PATCH_ERR_TIMEOUT if a bounded wait expired (the kernel then stops early), or
+ *           PATCH_ERR_FORMAT if an entry of the blob's tile table is not a dense or 2:4 tile lying
+ *           inside the blob (every entry is checked before a byte of its tile is requested; the
+ *           kernel reads the blob's first payload in its place, so nothing is read out of range).
+ *           In both cases Y is undefined.  NULL = not reported.
  * M == 0 returns PATCH_OK without launching.  Calls sharing a workspace must be ordered on
  * one stream.
  */

@@ -51,14 +51,14 @@ class PatchError(RuntimeError):
 _lib = None
 
 
-def lib() -> ctypes.CDLL:
-    """Load the CUDA library; fails loudly if it has not been built."""
-    global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2509_23410_b200.build` "
+def load(path: str) -> ctypes.CDLL:
+    """Load a build of the library from ``path`` and declare its argument types (``lib()`` is the product build;
+    the tests also load the fault-injection build this way)."""
+    if True:
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run `python -m paper_2509_23410_b200.build` "
                                "(there is no CPU fallback)")
-        L = ctypes.CDLL(LIB_PATH)
+        L = ctypes.CDLL(path)
         vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
         L.patch_packed_size.argtypes = [i64, i64, ctypes.c_int, ctypes.c_int, vp, ctypes.POINTER(Layout)]
         L.patch_pack.argtypes = [vp, i64, vp, ctypes.POINTER(Layout), vp, sz, vp]
@@ -93,7 +93,14 @@ def lib() -> ctypes.CDLL:
         for name in EXPORTS:
             if name != "patch_strerror":
                 getattr(L, name).restype = ctypes.c_int
-        _lib = L
+    return L
+
+
+def lib() -> ctypes.CDLL:
+    """The product build of the CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        _lib = load(LIB_PATH)
     return _lib
 
 

@@ -67,7 +67,8 @@ __device__ __forceinline__ float4 ld_peer_f4(uint32_t saddr, uint32_t rank) {
 template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
 __global__ void __launch_bounds__(192)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
-                      int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
+                      uint32_t pay0_16, uint32_t end16, int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy,
+                      int* status_dev) {
     using namespace dc;
     using C = Cfg<N_TOK, STAGES, GATED>;
     constexpr uint32_t kStageBytes = C::kStageBytes, kXAtomBytes = C::kXAtomBytes, kXBytes = C::kXBytes;
@@ -124,10 +125,11 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
         for (int i = 0; i < n_tiles && ok; ++i) {
             const int half = (GATED && i >= n_slice) ? 1 : 0, idx = i - half * n_slice;   // tile idx of row-block `half`
             if ((idx & 31) == 0 && idx + lane < n_slice) mine = table[int64_t(half) * TK + idx + lane];
-            const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, idx & 31);
-            const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, idx & 31);
+            uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, idx & 31);
+            uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, idx & 31);
             if (lane == 0) {
                 const int stage = i % STAGES;
+                sanitize_tile(kind, off16, pay0_16, end16, status_dev);
                 const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
                 const uint32_t sW = smem_base + stage * kStageBytes, full = bar_full + 8 * stage;
                 if (i >= STAGES)
@@ -287,7 +289,8 @@ static int launch_dc_t(const CUtensorMap& map, const patch_layout_t* L, const ui
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, packed, uint64_t(L->table_off), TK, S, M, Y, ldy, status_dev);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, packed, uint64_t(L->table_off), uint32_t(L->payload_off / 16),
+                                       uint32_t(L->total_bytes / 16), TK, S, M, Y, ldy, status_dev);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

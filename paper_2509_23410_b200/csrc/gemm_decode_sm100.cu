@@ -163,7 +163,7 @@ __device__ __forceinline__ bool finish_gated_row(const float (&a)[16], int tn, i
         for (int q = 0; q < 4; ++q) all = all && w[q].x != 0u && w[q].y != 0u && w[q].z != 0u && w[q].w != 0u;
         if (!all && (*abort_flag || global_timer_ns() - tstart > kWaitLimitNs)) {
             *abort_flag = 1;
-            if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+            if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_TIMEOUT);
             return false;
         }
     }
@@ -278,7 +278,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
             const int tn_b = (t1 - 1) / TK;
             if (t1 > t0 && t1 < (tn_b + 1) * TK && t0 <= tn_b * TK) {
                 const uint32_t d = off_last - pay0_16;
-                const int c_last = int(((uint64_t(d) + 1) * uint64_t(G) - 1) / pay_total_16);
+                int c_last = int(((uint64_t(d) + 1) * uint64_t(G) - 1) / pay_total_16);
+                c_last = c_last < c ? c : c_last > G - 1 ? G - 1 : c_last;     // whatever the table says, a CTA of this grid
                 n_others = c_last - c;
             }
         }
@@ -311,15 +312,26 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
         TileDesc mine = TileDesc{0, 0, 0, 0};
         int issued = 0;
         bool ok = true;
+#ifdef PATCH_FAULT_INJECTION
+        uint32_t inject_bytes = 0u;
+        if (c == 0 && status_dev && *status_dev == kInjectMagic) {
+            inject_bytes = 16u;
+            __syncwarp();
+            if (lane == 0) *status_dev = PATCH_OK;       // the word then reports like any other launch's
+        }
+#else
+        constexpr uint32_t inject_bytes = 0u;
+#endif
         // Weight tiles of the first STAGES steps may be requested before the grid dependency is
         // resolved (WSTATIC); their activations follow once it is (unless XSTATIC).
         const int n_early = (WSTATIC && !XSTATIC) ? (n_tiles < STAGES ? n_tiles : STAGES) : 0;
         for (int i = 0; i < n_tiles && ok; ++i) {
             if ((i & 31) == 0 && i + lane < n_tiles) mine = table[t0 + i + lane];   // 32 descriptors per load
-            const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
-            const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
+            uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
+            uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
             if (lane == 0) {
                 const int stage = i % STAGES;
+                sanitize_tile(kind, off16, pay0_16, pay0_16 + pay_total_16, status_dev);
                 const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
                 const uint32_t sW = smem_base + stage * Cfg::kStageBytes;
                 const uint32_t full = bar_full + 8 * stage;
@@ -327,7 +339,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                     ok = mbar_wait(bar_empty + 8 * stage, (uint32_t(i / STAGES) & 1u) ^ 1u, abort_flag, status_dev);
                 if (ok) {
                     stage_kind[stage] = kind;
-                    mbar_expect_tx(full, wbytes + Cfg::kXBytes);
+                    mbar_expect_tx(full, wbytes + Cfg::kXBytes + (i == 0 ? inject_bytes : 0u));
                     tma_bulk_load(sW, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
                     if (i < n_early) {
                         if (i + 1 == n_early) {
@@ -478,7 +490,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                                     all = all && w[jj][q].x != 0u && w[jj][q].y != 0u && w[jj][q].z != 0u && w[jj][q].w != 0u;
                             if (!all && (*abort_flag || global_timer_ns() - tstart > kWaitLimitNs)) {
                                 *abort_flag = 1;
-                                if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                                if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_TIMEOUT);
                                 ok = false;
                                 break;
                             }
@@ -551,7 +563,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
                         cur = ld_acquire_gpu(ctr);
                         if (*abort_flag || global_timer_ns() - tstart > kWaitLimitNs) {
                             *abort_flag = 1;
-                            if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                            if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_TIMEOUT);
                             cur = 0ull;
                             break;
                         }

@@ -45,8 +45,8 @@ constexpr uint32_t kSparse = 2;
 
 __global__ void __launch_bounds__(320)
 prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
-                int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev,
-                int gated, int independent) {
+                uint32_t pay0_16, uint32_t end16, int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy,
+                int* status_dev, int gated, int independent) {
     using namespace p2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -115,6 +115,8 @@ prefill2_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __res
                 kind[1] = __shfl_sync(0xFFFFFFFFu, mine.kind, 16 + (k & 15));
                 off16[1] = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, 16 + (k & 15));
                 if (lane == 0) {
+                    sanitize_tile(kind[0], off16[0], pay0_16, end16, status_dev);
+                    if (has1) sanitize_tile(kind[1], off16[1], pay0_16, end16, status_dev);
 #pragma unroll
                     for (int h = 0; h < 2 && ok; ++h) {
 #pragma unroll
@@ -307,8 +309,9 @@ int launch_prefill2(const CUtensorMap& map, const patch_layout_t* L, const uint8
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill2_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
-                                       Y, ldy, status_dev, gated ? 1 : 0, independent ? 1 : 0);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill2_kernel, map, packed, uint64_t(L->table_off), uint32_t(L->payload_off / 16),
+                                       uint32_t(L->total_bytes / 16), TN, TK, int(M), n_tok, Y, ldy, status_dev, gated ? 1 : 0,
+                                       independent ? 1 : 0);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

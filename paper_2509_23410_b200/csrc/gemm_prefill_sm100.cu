@@ -39,8 +39,8 @@ struct PrefillConfig {
 
 __global__ void __launch_bounds__(192)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
-               int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev,
-               int independent) {
+               uint32_t pay0_16, uint32_t end16, int TN, int TK, int M, int n_tok, __nv_bfloat16* __restrict__ Y, int64_t ldy,
+               int* status_dev, int independent) {
     using Cfg = PrefillConfig;
     const uint32_t stage_bytes = kDenseBytes + uint32_t(n_tok) * 256u;
     const int STAGES = int(Cfg::kRingBytes / stage_bytes) < Cfg::kMaxStages ? int(Cfg::kRingBytes / stage_bytes) : Cfg::kMaxStages;
@@ -98,10 +98,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __rest
             TileDesc mine = TileDesc{0, 0, 0, 0};
             for (int i = 0; i < TK && ok; ++i) {
                 if ((i & 31) == 0 && i + lane < TK) mine = table[i + lane];   // 32 descriptors per warp load
-                const uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
-                const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
+                uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
+                uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
                 if (lane == 0) {
                     const int stage = issued % STAGES;
+                    sanitize_tile(kind, off16, pay0_16, end16, status_dev);
                     ok = mbar_wait(bar_empty + 8 * stage, (uint32_t(issued / STAGES) & 1u) ^ 1u, abort_flag, status_dev);
                     if (ok) {
                         const uint32_t wbytes = kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes;
@@ -348,8 +349,8 @@ int launch_prefill(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_l
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel, map, packed, uint64_t(L->table_off), TN, TK, int(M), n_tok,
-                                       Y, ldy, status_dev, independent ? 1 : 0);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel, map, packed, uint64_t(L->table_off), uint32_t(L->payload_off / 16),
+                                       uint32_t(L->total_bytes / 16), TN, TK, int(M), n_tok, Y, ldy, status_dev, independent ? 1 : 0);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

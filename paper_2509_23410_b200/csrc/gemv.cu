@@ -73,7 +73,7 @@ __device__ __forceinline__ void load_tile(TileRegs<M_MAX>& t, const TileDesc& d,
                                   : zero4;
         }
     } else {
-        const uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
+        const uint8_t* meta = pay + kAtomBytes;      // the metadata block follows the kept values
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
             const uint32_t r = row0 + 32u * p;
@@ -125,8 +125,8 @@ __device__ __forceinline__ void fma_tile(const TileRegs<M_MAX>& t, float (&acc)[
 template <int M_MAX>
 __global__ void __launch_bounds__(256)
 gemv_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int M,
-            const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
-            __nv_bfloat16* __restrict__ Y, int64_t ldy) {
+            const uint8_t* __restrict__ blob, uint64_t table_off, uint32_t pay0_16, uint32_t end16, int TK,
+            __nv_bfloat16* __restrict__ Y, int64_t ldy, int* status_dev) {
     cg::cluster_group cluster = cg::this_cluster();
     // programmatic dependent launch: let the next kernel start its prologue, then wait until the
     // previous kernel's results (X, and the last readers of Y) are complete
@@ -153,7 +153,11 @@ gemv_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int M,
     for (int base = tk0; base < tk1; base += 256) {
         const int n = tk1 - base < 256 ? tk1 - base : 256;
         __syncthreads();
-        if (int(threadIdx.x) < n) descs[threadIdx.x] = table[base + threadIdx.x];
+        if (int(threadIdx.x) < n) {
+            TileDesc d = table[base + threadIdx.x];
+            sanitize_tile(d.kind, d.payload_off16, pay0_16, end16, status_dev);     // checked once, before any tile byte is read
+            descs[threadIdx.x] = d;
+        }
         __syncthreads();
         load_tile<M_MAX>(cur, descs[0], blob, X, ldx, M, base, row0, c);
         for (int i = 0; i < n; ++i) {
@@ -195,7 +199,7 @@ static int pick_splits(int TN, int TK) {
 
 template <int M_MAX>
 static int launch_gemv_t(const __nv_bfloat16* X, int64_t ldx, int M, const patch_layout_t* L,
-                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, cudaStream_t stream) {
+                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     const int S = pick_splits(TN, TK);
     cudaLaunchConfig_t cfg = {};
@@ -212,19 +216,19 @@ static int launch_gemv_t(const __nv_bfloat16* X, int64_t ldx, int M, const patch
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_kernel<M_MAX>, X, ldx, M, packed,
-                                       uint64_t(L->table_off), TK, Y, ldy);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_kernel<M_MAX>, X, ldx, M, packed, uint64_t(L->table_off),
+                                       uint32_t(L->payload_off / 16), uint32_t(L->total_bytes / 16), TK, Y, ldy, status_dev);
     return e == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
 int launch_gemv(const __nv_bfloat16* X, int64_t ldx, int M, const patch_layout_t* L,
-                const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* /*status_dev*/,
+                const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, int* status_dev,
                 cudaStream_t stream) {
     if (M < 1 || M > 4) return PATCH_ERR_SHAPE;
     if (L->N / kTile > 65535) return PATCH_ERR_SHAPE;
-    if (M == 1) return launch_gemv_t<1>(X, ldx, M, L, packed, Y, ldy, stream);
-    if (M == 2) return launch_gemv_t<2>(X, ldx, M, L, packed, Y, ldy, stream);
-    return launch_gemv_t<4>(X, ldx, M, L, packed, Y, ldy, stream);
+    if (M == 1) return launch_gemv_t<1>(X, ldx, M, L, packed, Y, ldy, status_dev, stream);
+    if (M == 2) return launch_gemv_t<2>(X, ldx, M, L, packed, Y, ldy, status_dev, stream);
+    return launch_gemv_t<4>(X, ldx, M, L, packed, Y, ldy, status_dev, stream);
 }
 
 }  // namespace patch

@@ -32,6 +32,22 @@ __host__ __device__ inline uint32_t atom_chunk_offset(uint32_t r, uint32_t c) {
     return (r >> 3) * 1024u + (r & 7u) * 128u + ((c ^ (r & 7u)) << 4);
 }
 
+// Trap-free check of a tile-table entry read from device memory, made before any byte of the tile is requested.
+// The host validates the layout struct, but the table inside the blob is the caller's device memory: an entry
+// whose kind is unknown or whose payload does not lie inside [first payload, end of blob) is reported
+// (PATCH_ERR_FORMAT in status_dev) and replaced by the first payload read as a 2:4 tile -- 18 432 bytes that lie
+// inside every blob -- so that the launch runs to its end with a defined status and an undefined Y instead of
+// reading out of range.
+__device__ __forceinline__ void sanitize_tile(uint32_t& kind, uint32_t& off16, uint32_t pay0_16, uint32_t end16,
+                                              int* status_dev) {
+    const uint32_t len16 = (kind == PATCH_TILE_DENSE ? kDenseBytes : kSparseBytes) / 16;
+    if (kind > PATCH_TILE_SPARSE_2_4 || off16 < pay0_16 || off16 > end16 || len16 > end16 - off16) {
+        if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_FORMAT);
+        kind = PATCH_TILE_SPARSE_2_4;
+        off16 = pay0_16;
+    }
+}
+
 // Host-side checks of a layout struct handed in by the caller.
 int validate_layout(const patch_layout_t* L);
 

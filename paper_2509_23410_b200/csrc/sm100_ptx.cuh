@@ -35,7 +35,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     return t;
 }
 
+#ifdef PATCH_FAULT_INJECTION
+// Test build (libpatch_b200_fi.so, see build.py): waits give up after 300 us, and a launch of the stream-K decode
+// kernel whose status word holds kInjectMagic announces, in CTA 0, sixteen bytes more than its first stage will
+// ever receive -- the one way the tests make a bounded wait run out.  Nothing faults, traps or spins for ever.
+constexpr uint64_t kWaitLimitNs = 300000ull;
+constexpr int kInjectMagic = 0x7E57;
+#else
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
+#endif
 constexpr uint64_t kDrainLimitNs = 2000000ull;    // 2 ms for copies already in flight
 
 // Bounded wait.  Returns false if the wait was given up (own timeout, or another role of this
@@ -50,7 +58,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kWaitLimitNs) {
                 *abort_flag = 1;
-                if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_TIMEOUT);
                 return false;
             }
         }
@@ -70,7 +78,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kWaitLimitNs) {
                 *abort_flag = 1;
-                if (status_dev) atomicExch(status_dev, PATCH_ERR_TIMEOUT);
+                if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_TIMEOUT);
                 return false;
             }
         }
