@@ -75,8 +75,9 @@ enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2, PA
  *
  * With BOTH promises a GEMM of M <= 64 tokens runs on a schedule made for streams of independent
  * GEMMs: one CTA per row-block (a small cluster splitting K where row-blocks are few), so that several
- * consecutive GEMMs are resident on the GPU at once; without them it runs stream-K over all SMs, which
- * is the faster choice for a GEMM that has the GPU to itself.  For M > 64 both promises let the kernel
+ * consecutive GEMMs are resident on the GPU at once.  With the weights promise alone it runs on the same
+ * row-block schedule with larger clusters (at least 128 CTAs: it streams alone once its predecessor is
+ * done); without any promise it runs stream-K over all SMs.  For M > 64 both promises let the kernel
  * start on the SMs that the tail of the previous kernel leaves idle.  All schedules are deterministic;
  * their results may differ in the last bit (different fp32 summation order).
  */

@@ -316,7 +316,16 @@ static int launch_dc_f(const CUtensorMap& map, const patch_layout_t* L, const ui
 int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int n_tok,
                           __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic,
                           bool xstatic) {
-    const int S = decode_cluster_split(int(L->N / kTile), int(L->K / kTile));
+    const int TN = int(L->N / kTile), TK = int(L->K / kTile);
+    int S = decode_cluster_split(TN, TK);
+    if (!xstatic) {
+        // a GEMM that waits for its predecessor streams alone for a while: at least 128 CTAs, so that its own loads
+        // can keep HBM busy (the independent schedule wants few CTAs per GEMM and several GEMMs resident instead).
+        // Tried on top of this and dropped: asking L2 for the rest of the CTA's weight tiles before the wait
+        // (0.332 against 0.322 ms on the 24-GEMM step) -- a three-stage ring drains L2 hardly faster than HBM.
+        S = 1;
+        while (S < 8 && TN * S < 128 && 2 * S <= TK) S *= 2;
+    }
     switch (n_tok) {
         case 16: return launch_dc_f<16, 3>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
         case 32: return launch_dc_f<32, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
