@@ -672,6 +672,125 @@ def run_ours(args):
 
 
 # ---------------------------------------------------------------------------------------------
+# block workload: the linear layers of a decoder stack chained the way a decoder chains them
+
+
+def run_block(args):
+    """`--workload block`: 32 LLaMA-2-7B-shaped blocks, four launches per block, M tokens (`--stack-m`):
+      qkv   one stacked weight (N = 12288), X = the block's input buffer, which no GEMM writes: both promises;
+      o     X = the v slice of what the qkv launch just wrote (row pitch 12288): weights promise only;
+      mlp   silu(gate) * up from one stacked, interleaved gate/up weight (patch_gemm_gated), X = o's output: weights promise;
+      down  X = the gated product: weights promise only.
+    Three of the four launches of a block read what the launch before them wrote, as in a decoder (what sits between
+    them there -- attention, norms, residuals -- is not part of this path).  Per-matrix 2:4-tile fractions ~ U[0, 1] as in
+    the stack workloads; weights drawn on the device.  Reported beside it: the same launches all declared independent
+    (what the stack workloads time; not a valid promise here) and all without any promise."""
+    import torch
+    from paper_2509_23410_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("the block workload is a single-GPU measurement")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B.lib()
+    peaks = measured_peaks()
+    M = args.stack_m
+    cases = inputs.stack_fused_cases()
+    gen = torch.Generator(device=dev)
+    h = torch.empty((M, 4096), dtype=torch.bfloat16, device=dev).normal_(0.0, 1.0, generator=gen)
+    launches, nbytes, flops, weight_bytes = [], 0.0, 0.0, 0
+    ws = None
+    for i, c in enumerate(cases):
+        gen.manual_seed(inputs.MASTER_SEED * 1000 + i)
+        W = torch.empty((c["N"], c["K"]), dtype=torch.bfloat16, device=dev).normal_(0.0, 0.02, generator=gen)
+        flags = inputs.case_flags(c)
+        role = c["name"].rsplit(".", 1)[1]
+        if role == "gate_up":
+            half = c["N"] // 2
+            W = B.interleave_row_blocks(W[:half], W[half:]).contiguous()
+            flags = B.interleave_row_blocks(flags[:half // 128], flags[half // 128:], block=1)
+        layout = B.patch_packed_size(c["N"], c["K"], flags)
+        packed = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
+        B.patch_pack(W, flags, layout=layout, out=packed)
+        del W
+        n_out = c["N"] // 2 if role == "gate_up" else c["N"]
+        Y = torch.empty((M, n_out), dtype=torch.bfloat16, device=dev)
+        if role == "qkv":
+            X = h
+        elif role == "o":
+            X = launches[-1]["Y"][:, 8192:12288]          # the v slice of the stacked qkv output
+        else:
+            X = launches[-1]["Y"]
+        if ws is None:
+            ws = torch.zeros(max(B.patch_gemm_workspace_size(layout, M), 256), dtype=torch.uint8, device=dev)
+        gws = None
+        if role == "gate_up":
+            gws = torch.zeros(max(B.patch_gemm_gated_workspace_size(layout, M), 256), dtype=torch.uint8, device=dev)
+        launches.append(dict(role=role, layout=layout, packed=packed, X=X, Y=Y, gws=gws))
+        T = (c["N"] // 128) * (c["K"] // 128)
+        nbytes += layout.payload_bytes + 16 * T + M * c["K"] * 2 + M * n_out * 2
+        flops += 2.0 * M * 16384 * T
+        weight_bytes += layout.total_bytes
+
+    def enqueue(mode):
+        for L in launches:
+            if mode == "faithful":
+                fl = B.WEIGHTS_STATIC | (B.INPUT_STATIC if L["role"] == "qkv" else 0)
+            else:
+                fl = {"independent": B.WEIGHTS_STATIC | B.INPUT_STATIC, "no-promise": 0}[mode]
+            if L["role"] == "gate_up":
+                B.patch_gemm_gated(L["X"], L["layout"], L["packed"], Y=L["Y"], workspace=L["gws"], flags=fl)
+            else:
+                B.patch_gemm(L["X"], L["layout"], L["packed"], Y=L["Y"], workspace=ws, variant=fl)
+
+    def graph_of(mode):
+        enqueue(mode)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            enqueue(mode)
+        return g
+
+    steps, warm = max(3, min(args.steps, 200)), max(args.warmup, 3)
+    g = graph_of("faithful")
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    for _ in range(warm):
+        g.replay()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    step_s = time_graph(torch, g, steps)
+    clocks = sampler.stop(t0, time.time())
+    others = {}
+    for mode in ("independent", "no-promise"):
+        go = graph_of(mode)
+        for _ in range(3):
+            go.replay()
+        others[mode] = time_graph(torch, go, max(3, steps // 4))
+        del go
+    roof_spec = nbytes / (HBM_SPEC_GBS * 1e9) if M <= 64 else None
+    out = {
+        "metric": "hybrid_tile_gemm_effective_tflops", "value": flops / step_s / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": steps, "warmup": warm, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (weights drawn on the device)",
+        "config": {"workload": f"llama2-7b decoder-block chain of linears (qkv -> o -> silu(gate)*up -> down, 32 blocks), M={M}",
+                   "launches_per_step": len(launches), "packed_weight_bytes": weight_bytes, "cuda_graph": True,
+                   "l2": "inputs larger than L2: a step streams every packed matrix once",
+                   "launch": "qkv with both promises; o, mlp and down with the weights promise only (each reads what the launch before it wrote)"},
+        "gbs": nbytes / step_s / 1e9,
+        "frac_of_roofline_spec": (roof_spec / step_s) if roof_spec else None,
+        "frac_of_roofline_measured": (nbytes / (peaks["hbm_gbs"] * 1e9) / step_s) if M <= 64 else None,
+        "all_declared_independent": {"ms_per_step": others["independent"] * 1e3,
+                                     "note": "what the stack workloads time; not a valid promise for this chain"},
+        "no_promise": {"ms_per_step": others["no-promise"] * 1e3},
+        "gpu_launches": steps * len(launches),
+        "clocks": clocks,
+    }
+    print(json.dumps(out))
+
+
+# ---------------------------------------------------------------------------------------------
 # mask-learning workload: one training-forward evaluation of the soft masks of one transformer block
 
 
@@ -873,7 +992,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused", "masks"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused", "block", "masks"])
     ap.add_argument("--stack-m", type=int, default=1, help="tokens per GEMM of the 224-GEMM stack workload")
     ap.add_argument("--launch", default="independent", choices=["dependent", "independent"],
                     help="independent (default; true for this workload, whose GEMMs do not feed each other): "
@@ -898,6 +1017,11 @@ def main():
             print(json.dumps({"impl": "reference", "unavailable": "the masks workload reports the oracle in its cpu_baseline key"}))
         else:
             run_masks(args)
+    elif args.workload == "block":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the block workload has no oracle arm; see the decode workload"}))
+        else:
+            run_block(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -789,3 +789,56 @@ def test_promises_are_bounded_by_other_operations(gpu, oracle, M):
         else:
             rows = np.array([0, 1, M // 2, M - 1])
             check_parity(oracle, to_bits(Ys[i])[rows], oracle.gemm_f64_rows(Xs[i], rows, What), f"window round {i}")
+
+
+@pytest.mark.parametrize("M", [1, 16, 40, 300])
+def test_decoder_block_chain(gpu, oracle, M):
+    """The chain `bench.py --workload block` times, on small matrices and without any synchronisation, three blocks
+    deep: a stacked q/k/v GEMM with both promises (its X is written by no GEMM), then o on the v slice of that output
+    (row pitch 3 d), the gated gate/up product on o's output and down on the gated product, each with the weights
+    promise only because it reads what the launch before it wrote.  Every intermediate is checked against the oracle
+    fed with the GPU's own bf16 output of the step before."""
+    torch, B = gpu
+    d, dff = 512, 1024
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(B.patch_gemm_workspace_size(B.patch_packed_size(3 * d, d, np.zeros((12, 4), np.uint8)), 64),
+                     dtype=torch.uint8, device="cuda")
+    blocks = []
+    for b in range(3):
+        mats = {}
+        for role, N, K, scale in (("qkv", 3 * d, d, 2.0), ("o", d, d, 2.0), ("gate", dff, d, 40.0), ("up", dff, d, 2.0),
+                                  ("down", d, dff, 2.0)):
+            W = inputs.f32_to_bf16_bits(f32(inputs.weight(N, K, inputs.MASTER_SEED, "block", b, role)) * scale)
+            mats[role] = (W, inputs.tile_flags(N, K, 0.5, inputs.MASTER_SEED, "block", b, role))
+        Wgu = B.interleave_row_blocks(mats["gate"][0], mats["up"][0])
+        fgu = B.interleave_row_blocks(mats["gate"][1], mats["up"][1], block=1)
+        packed = {}
+        for role, (W, fl) in (("qkv", mats["qkv"]), ("o", mats["o"]), ("mlp", (Wgu, fgu)), ("down", mats["down"])):
+            blob, L = B.patch_pack(to_dev(torch, W), fl)
+            packed[role] = (blob, L, oracle.prune(W, fl))
+        gws = torch.zeros(max(B.patch_gemm_gated_workspace_size(packed["mlp"][1], M), 256), dtype=torch.uint8, device="cuda")
+        X = inputs.activation(M, d, inputs.MASTER_SEED, "block", b, M)
+        blocks.append(dict(packed=packed, gws=gws, X=X, Xd=to_dev(torch, X),
+                           qkv=torch.zeros((M, 3 * d), dtype=torch.bfloat16, device="cuda"),
+                           o=torch.zeros((M, d), dtype=torch.bfloat16, device="cuda"),
+                           mlp=torch.zeros((M, dff), dtype=torch.bfloat16, device="cuda"),
+                           down=torch.zeros((M, d), dtype=torch.bfloat16, device="cuda")))
+    torch.cuda.synchronize()
+    both, weights_only = B.WEIGHTS_STATIC | B.INPUT_STATIC, B.WEIGHTS_STATIC
+    for blk in blocks:
+        p = blk["packed"]
+        B.patch_gemm(blk["Xd"], p["qkv"][1], p["qkv"][0], Y=blk["qkv"], workspace=ws, status=status, variant=both)
+        B.patch_gemm(blk["qkv"][:, 2 * d:], p["o"][1], p["o"][0], Y=blk["o"], workspace=ws, status=status, variant=weights_only)
+        B.patch_gemm_gated(blk["o"], p["mlp"][1], p["mlp"][0], Y=blk["mlp"], workspace=blk["gws"], status=status, flags=weights_only)
+        B.patch_gemm(blk["mlp"], p["down"][1], p["down"][0], Y=blk["down"], workspace=ws, status=status, variant=weights_only)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for b, blk in enumerate(blocks):
+        p = blk["packed"]
+        qkv = to_bits(blk["qkv"])
+        check_parity(oracle, qkv, oracle.gemm_f64(blk["X"], p["qkv"][2])[0], f"block {b} qkv")
+        o = to_bits(blk["o"])
+        check_parity(oracle, o, oracle.gemm_f64(np.ascontiguousarray(qkv[:, 2 * d:]), p["o"][2])[0], f"block {b} o")
+        mlp = to_bits(blk["mlp"])
+        check_parity(oracle, mlp, oracle.swiglu(oracle.gemm_f64(o, p["mlp"][2])[0]), f"block {b} mlp")
+        check_parity(oracle, to_bits(blk["down"]), oracle.gemm_f64(mlp, p["down"][2])[0], f"block {b} down")
