@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "patch_oracle.c")
 _LIB = os.path.join(_HERE, "libpatch_oracle.so")
 
-KIND_DENSE, KIND_SPARSE = 0, 1
+KIND_DENSE, KIND_SPARSE, KIND_DENSE_Q4, KIND_SPARSE_Q4 = 0, 1, 2, 3
 MAGIC = 0x48435450
 
 
@@ -28,7 +28,8 @@ class Layout(ctypes.Structure):
                 ("tile_n", ctypes.c_int32), ("tile_k", ctypes.c_int32),
                 ("n_dense", ctypes.c_int64), ("n_sparse", ctypes.c_int64),
                 ("table_off", ctypes.c_uint64), ("payload_off", ctypes.c_uint64),
-                ("payload_bytes", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64)]
+                ("payload_bytes", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64),
+                ("n_dense_q4", ctypes.c_int64), ("n_sparse_q4", ctypes.c_int64)]
 
 
 def build(force: bool = False) -> str:
@@ -75,6 +76,16 @@ def _check(rc, what):
 
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
+
+
+def q4_group(values):
+    """4-bit quantiser of one group of stored values (bf16 bits): (scale bits, codes q + 8, dequantised bits)."""
+    v = _u16(values).reshape(-1)
+    scale = np.zeros(1, np.uint16)
+    codes = np.empty(v.size, np.uint8)
+    deq = np.empty(v.size, np.uint16)
+    _check(lib().oracle_q4_group(_p(v), int(v.size), _p(scale), _p(codes), _p(deq)), "q4_group")
+    return int(scale[0]), codes, deq
 
 
 def mask(W, flags, tile_n=128, tile_k=128) -> np.ndarray:

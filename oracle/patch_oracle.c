@@ -16,6 +16,13 @@
  *     the tile size fixes how the matrix is compressed and its metadata laid out);
  *     two metadata bits per kept value, the cost that reproduces the compression-ratio column
  *     of the 4-bit quantisation table.
+ *   - 4-bit weight-only quantisation of the stored values of a tile (section "Combination with other
+ *     compression methods", the 4-bit quantisation table).  The paper prints only the compression-ratio
+ *     column -- 4 bits per stored value plus the 2 metadata bits per kept value, 16 / (4 - f) -- and no
+ *     quantiser; the reading taken here: symmetric, round to nearest even, one bf16 scale per tile row
+ *     (the 128 weights of a dense tile's row, the 64 kept values of a 2:4 tile's row),
+ *         s = bf16(max|v| / 7),  q = clamp(rint(v / s), -7, 7)  (q = 0 where s = 0),  v^ = bf16(q * s),
+ *     all in fp32 on bf16 inputs; the 2:4 selection is made first, on the unquantised weights.
  *   - the linear layer itself, on the same bf16-rounded inputs, accumulated in double (and in
  *     plain fp32 as a cross-check) in k order.
  *   - (last section of the file) the masks of the learning procedure: the Gumbel-softmax soft masks
@@ -30,12 +37,14 @@
  * "parity unpinned".
  *
  * Conventions: W is [N x K] row-major bf16 (uint16 bit patterns), N = out-features,
- * K = in-features; X is [M x K]; Y is [M x N].  flags[tn*TK + tk]: 0 = dense, 1 = 2:4.
+ * K = in-features; X is [M x K]; Y is [M x N].  flags[tn*TK + tk]: 0 = dense, 1 = 2:4,
+ * 2 = dense with 4-bit values, 3 = 2:4 with 4-bit values.
  */
 #include <stdint.h>
 #include <stddef.h>
 #include <string.h>
 #include <stdlib.h>
+#include <math.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -44,6 +53,8 @@
 #define ORACLE_VERSION 1u
 #define KIND_DENSE  0u
 #define KIND_SPARSE 1u
+#define KIND_DENSE_Q4  2u     /* kind & 1: 2:4;  kind & 2: values stored as 4-bit codes + one scale per tile row */
+#define KIND_SPARSE_Q4 3u
 
 typedef struct {
     uint32_t magic, version;
@@ -51,6 +62,7 @@ typedef struct {
     int32_t  tile_n, tile_k;
     int64_t  n_dense, n_sparse;
     uint64_t table_off, payload_off, payload_bytes, total_bytes;
+    int64_t  n_dense_q4, n_sparse_q4;
 } oracle_layout_t;
 
 /* ------------------------------------------------------------------------------------------- */
@@ -70,6 +82,40 @@ static uint16_t f32_to_bf16_rne(float f) {
     uint32_t lsb = (u >> 16) & 1u;
     u += 0x7FFFu + lsb;
     return (uint16_t)(u >> 16);
+}
+
+/* ------------------------------------------------------------------------------------------- */
+/* 4-bit quantiser of one group of stored values (see the header): scale, codes, dequantised values. */
+
+static uint16_t q4_scale(const uint16_t* v, int n) {
+    float m = 0.0f;
+    for (int i = 0; i < n; ++i) {
+        float a = fabsf(bf16_to_f32(v[i]));
+        if (a > m) m = a;
+    }
+    return f32_to_bf16_rne(m / 7.0f);
+}
+static int q4_code(uint16_t v, uint16_t scale) {            /* q in [-7, 7] */
+    float s = bf16_to_f32(scale);
+    if (s == 0.0f) return 0;
+    float r = rintf(bf16_to_f32(v) / s);                    /* nearest, ties to even */
+    if (r > 7.0f) r = 7.0f;
+    if (r < -7.0f) r = -7.0f;
+    return (int)r;
+}
+static uint16_t q4_value(int q, uint16_t scale) {           /* bf16(q * s): the product is exact in fp32 */
+    return f32_to_bf16_rne((float)q * bf16_to_f32(scale));
+}
+/* exported for the tests: quantise n values -> scale, codes (q + 8 in 1..15), dequantised values */
+int oracle_q4_group(const uint16_t* v, int n, uint16_t* scale, uint8_t* codes, uint16_t* deq) {
+    if (!v || !scale || n <= 0) return -1;
+    *scale = q4_scale(v, n);
+    for (int i = 0; i < n; ++i) {
+        int q = q4_code(v[i], *scale);
+        if (codes) codes[i] = (uint8_t)(q + 8);
+        if (deq) deq[i] = q4_value(q, *scale);
+    }
+    return 0;
 }
 
 int oracle_num_threads(void) {
@@ -111,11 +157,11 @@ int oracle_mask(const uint16_t* W, int64_t N, int64_t K, const uint8_t* flags,
     if (rc) return rc;
     int64_t TK = K / tile_k;
     for (int64_t t = 0; t < (N / tile_n) * TK; ++t)
-        if (flags[t] > 1) return -4;
+        if (flags[t] > 3) return -4;
     for (int64_t n = 0; n < N; ++n) {
         for (int64_t g = 0; g < K / 4; ++g) {
             int64_t k0 = 4 * g;
-            int m_tile = flags[(n / tile_n) * TK + k0 / tile_k] == KIND_DENSE; /* 1 = dense tile */
+            int m_tile = (flags[(n / tile_n) * TK + k0 / tile_k] & 1u) == 0;   /* 1 = dense tile (bf16 or 4-bit) */
             int keep[4];
             select_top2(&W[n * K + k0], keep);
             for (int j = 0; j < 4; ++j)
@@ -133,6 +179,25 @@ int oracle_prune(const uint16_t* W, int64_t N, int64_t K, const uint8_t* flags,
     int rc = oracle_mask(W, N, K, flags, tile_n, tile_k, mask);
     if (rc == 0)
         for (int64_t i = 0; i < N * K; ++i) What[i] = mask[i] ? W[i] : (uint16_t)0;
+    /* tiles with 4-bit values: what the layer multiplies is the dequantised kept value; the group that shares a
+     * scale is the tile row's stored values (all of them in a dense tile, the kept ones in a 2:4 tile) */
+    if (rc == 0) {
+        int64_t TK = K / tile_k;
+        uint16_t* v = (uint16_t*)malloc((size_t)tile_k * 2);
+        if (!v) { free(mask); return -6; }
+        for (int64_t n = 0; n < N; ++n)
+            for (int64_t tk = 0; tk < TK; ++tk) {
+                if ((flags[(n / tile_n) * TK + tk] & 2u) == 0) continue;
+                int cnt = 0;
+                for (int c = 0; c < tile_k; ++c)
+                    if (mask[n * K + tk * tile_k + c]) v[cnt++] = W[n * K + tk * tile_k + c];
+                uint16_t s = q4_scale(v, cnt);
+                for (int c = 0; c < tile_k; ++c)
+                    if (mask[n * K + tk * tile_k + c])
+                        What[n * K + tk * tile_k + c] = q4_value(q4_code(W[n * K + tk * tile_k + c], s), s);
+            }
+        free(v);
+    }
     free(mask);
     return rc;
 }
@@ -163,23 +228,44 @@ static uint64_t vals_bytes(int tile_n, int tile_k) {
 static uint64_t sparse_bytes(int tile_n, int tile_k) {
     return vals_bytes(tile_n, tile_k) + (uint64_t)tile_n * meta_words(tile_k) * 4;
 }
+/* 4-bit kinds: [codes: value c of row r in byte r * (vals / 2) + c / 2, even c in the low nibble, code = q + 8;
+ * padded to 16 B | metadata as for the 2:4 kind (2:4 only) | scales: tile_n bf16, padded to 16 B].
+ * Payloads of 128x128 tiles are aligned to 256 B (8 448 B and 6 400 B), 16 B otherwise. */
+static uint64_t q4_codes_bytes(int tile_n, int vals_per_row) { return round_up((uint64_t)tile_n * vals_per_row / 2, 16); }
+static uint64_t q4_scales_bytes(int tile_n) { return round_up((uint64_t)tile_n * 2, 16); }
+static uint64_t dense_q4_bytes(int tile_n, int tile_k) { return q4_codes_bytes(tile_n, tile_k) + q4_scales_bytes(tile_n); }
+static uint64_t sparse_q4_bytes(int tile_n, int tile_k) {
+    return q4_codes_bytes(tile_n, tile_k / 2) + (uint64_t)tile_n * meta_words(tile_k) * 4 + q4_scales_bytes(tile_n);
+}
+static uint64_t q4_align(int tile_n, int tile_k) { return (tile_n == 128 && tile_k == 128) ? 256u : 16u; }
+static uint64_t kind_bytes(uint32_t kind, int tile_n, int tile_k) {       /* aligned size of a payload */
+    switch (kind) {
+        case KIND_DENSE: return round_up(dense_bytes(tile_n, tile_k), payload_align(tile_n, tile_k));
+        case KIND_SPARSE: return round_up(sparse_bytes(tile_n, tile_k), payload_align(tile_n, tile_k));
+        case KIND_DENSE_Q4: return round_up(dense_q4_bytes(tile_n, tile_k), q4_align(tile_n, tile_k));
+        default: return round_up(sparse_q4_bytes(tile_n, tile_k), q4_align(tile_n, tile_k));
+    }
+}
 
 int oracle_packed_size(int64_t N, int64_t K, int tile_n, int tile_k, const uint8_t* flags,
                        oracle_layout_t* L) {
     int rc = check_shape(N, K, tile_n, tile_k);
     if (rc) return rc;
     int64_t T = (N / tile_n) * (K / tile_k);
-    int64_t nd = 0, ns = 0;
-    uint64_t al = payload_align(tile_n, tile_k), bytes = 0;
+    int64_t nd = 0, ns = 0, ndq = 0, nsq = 0;
+    uint64_t bytes = 0;
     for (int64_t t = 0; t < T; ++t) {
-        if (flags[t] == KIND_DENSE) { ++nd; bytes += round_up(dense_bytes(tile_n, tile_k), al); }
-        else if (flags[t] == KIND_SPARSE) { ++ns; bytes += round_up(sparse_bytes(tile_n, tile_k), al); }
+        if (flags[t] == KIND_DENSE) ++nd;
+        else if (flags[t] == KIND_SPARSE) ++ns;
+        else if (flags[t] == KIND_DENSE_Q4) ++ndq;
+        else if (flags[t] == KIND_SPARSE_Q4) ++nsq;
         else return -4;
+        bytes += kind_bytes(flags[t], tile_n, tile_k);
     }
     memset(L, 0, sizeof *L);
     L->magic = ORACLE_MAGIC; L->version = ORACLE_VERSION;
     L->N = N; L->K = K; L->tile_n = tile_n; L->tile_k = tile_k;
-    L->n_dense = nd; L->n_sparse = ns;
+    L->n_dense = nd; L->n_sparse = ns; L->n_dense_q4 = ndq; L->n_sparse_q4 = nsq;
     L->table_off = 256;
     L->payload_off = round_up(256 + 16 * (uint64_t)T, 1024);
     L->payload_bytes = bytes;
@@ -191,19 +277,25 @@ static void write_header_and_table(const oracle_layout_t* L, const uint8_t* flag
     memset(blob, 0, (size_t)L->payload_off);
     memcpy(blob, L, sizeof *L);
     int64_t T = (L->N / L->tile_n) * (L->K / L->tile_k);
-    uint64_t al = payload_align(L->tile_n, L->tile_k), off = L->payload_off;
+    uint64_t off = L->payload_off;
+    int tn_ = L->tile_n, tk_ = L->tile_k;
     uint32_t* table = (uint32_t*)(blob + L->table_off);
     for (int64_t t = 0; t < T; ++t) {
+        /* { kind, payload / 16, metadata / 16 (0xFFFFFFFF if none), scales / 16 (0 if none) } */
         table[4 * t + 0] = flags[t];
         table[4 * t + 1] = (uint32_t)(off / 16);
-        if (flags[t] == KIND_DENSE) {
-            table[4 * t + 2] = 0xFFFFFFFFu;
-            off += round_up(dense_bytes(L->tile_n, L->tile_k), al);
-        } else {
-            table[4 * t + 2] = (uint32_t)((off + vals_bytes(L->tile_n, L->tile_k)) / 16);
-            off += round_up(sparse_bytes(L->tile_n, L->tile_k), al);
-        }
+        table[4 * t + 2] = 0xFFFFFFFFu;
         table[4 * t + 3] = 0;
+        if (flags[t] == KIND_SPARSE) {
+            table[4 * t + 2] = (uint32_t)((off + vals_bytes(tn_, tk_)) / 16);
+        } else if (flags[t] == KIND_DENSE_Q4) {
+            table[4 * t + 3] = (uint32_t)((off + q4_codes_bytes(tn_, tk_)) / 16);
+        } else if (flags[t] == KIND_SPARSE_Q4) {
+            uint64_t m = off + q4_codes_bytes(tn_, tk_ / 2);
+            table[4 * t + 2] = (uint32_t)(m / 16);
+            table[4 * t + 3] = (uint32_t)((m + (uint64_t)tn_ * meta_words(tk_) * 4) / 16);
+        }
+        off += kind_bytes(flags[t], tn_, tk_);
     }
 }
 
@@ -227,13 +319,19 @@ static int pack_impl(const uint16_t* W, const uint8_t* flags, const uint8_t* pat
         for (int64_t tk = 0; tk < TK; ++tk) {
             int64_t t = tn * TK + tk;
             uint8_t* pay = blob + (uint64_t)table[4 * t + 1] * 16;
-            if (table[4 * t + 0] == KIND_DENSE) {
-                uint16_t* d = (uint16_t*)pay;
+            uint32_t kind = table[4 * t + 0];
+            uint16_t* rowbuf = NULL;     /* 4-bit kinds: the stored values of the tile, row by row, before quantisation */
+            if (kind & 2u) {
+                rowbuf = (uint16_t*)malloc((size_t)tn_ * tk_ * 2);
+                if (!rowbuf) return -6;
+            }
+            if ((kind & 1u) == 0) {
+                uint16_t* d = (kind & 2u) ? rowbuf : (uint16_t*)pay;
                 for (int r = 0; r < tn_; ++r)
                     for (int c = 0; c < tk_; ++c)
                         d[r * tk_ + c] = W[(tn * tn_ + r) * K + tk * tk_ + c];
             } else {
-                uint16_t* vals = (uint16_t*)pay;
+                uint16_t* vals = (kind & 2u) ? rowbuf : (uint16_t*)pay;
                 uint32_t* meta = (uint32_t*)(blob + (uint64_t)table[4 * t + 2] * 16);
                 int words = (int)meta_words(tk_);
                 for (int r = 0; r < tn_; ++r)
@@ -253,6 +351,21 @@ static int pack_impl(const uint16_t* W, const uint8_t* flags, const uint8_t* pat
                         uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
                         meta[r * words + g / 8] |= nib << (4 * (g % 8));
                     }
+            }
+            if (kind & 2u) {
+                /* quantise the stored values row by row: codes into the payload, one scale per row behind them */
+                int n_vals = (kind & 1u) ? tk_ / 2 : tk_;
+                uint16_t* scales = (uint16_t*)(blob + (uint64_t)table[4 * t + 3] * 16);
+                for (int r = 0; r < tn_; ++r) {
+                    const uint16_t* v = &rowbuf[r * n_vals];
+                    uint16_t s = q4_scale(v, n_vals);
+                    scales[r] = s;
+                    for (int c = 0; c < n_vals; ++c) {
+                        uint8_t code = (uint8_t)(q4_code(v[c], s) + 8);
+                        pay[(r * n_vals + c) / 2] |= (uint8_t)(code << (4 * (c & 1)));
+                    }
+                }
+                free(rowbuf);
             }
         }
     return 0;
@@ -305,6 +418,27 @@ int oracle_unpack(const uint8_t* blob, uint64_t blob_bytes, uint16_t* What) {
                         w[i0] = vals[r * (tk_ / 2) + 2 * g + 0];
                         w[i1] = vals[r * (tk_ / 2) + 2 * g + 1];
                     }
+            } else if (table[4 * t + 0] == KIND_DENSE_Q4 || table[4 * t + 0] == KIND_SPARSE_Q4) {
+                int sparse = table[4 * t + 0] == KIND_SPARSE_Q4;
+                int n_vals = sparse ? tk_ / 2 : tk_;
+                const uint16_t* scales = (const uint16_t*)(blob + (uint64_t)table[4 * t + 3] * 16);
+                const uint32_t* meta = sparse ? (const uint32_t*)(blob + (uint64_t)table[4 * t + 2] * 16) : NULL;
+                int words = (int)meta_words(tk_);
+                for (int r = 0; r < tn_; ++r) {
+                    uint16_t* wrow = &What[(tn * tn_ + r) * K + tk * tk_];
+                    for (int c = 0; c < tk_; ++c) wrow[c] = 0;
+                    for (int c = 0; c < n_vals; ++c) {
+                        int code = (pay[(r * n_vals + c) / 2] >> (4 * (c & 1))) & 0xF;
+                        if (code == 0) return -7;                       /* q + 8 lies in 1..15 */
+                        uint16_t v = q4_value(code - 8, scales[r]);
+                        if (!sparse) { wrow[c] = v; continue; }
+                        int g = c / 2;
+                        uint32_t nib = (meta[r * words + g / 8] >> (4 * (g % 8))) & 0xFu;
+                        int i0 = (int)(nib & 3u), i1 = (int)(nib >> 2);
+                        if (i0 >= i1) return -7;
+                        wrow[4 * g + ((c & 1) ? i1 : i0)] = v;
+                    }
+                }
             } else return -7;
         }
     return 0;
@@ -343,7 +477,25 @@ int oracle_device_image(const uint8_t* canon, uint64_t blob_bytes, uint8_t* imag
     const uint32_t* table = (const uint32_t*)(canon + L.table_off);
     for (int64_t t = 0; t < T; ++t) {
         uint64_t off = (uint64_t)table[4 * t + 1] * 16;
-        if (table[4 * t + 0] == KIND_DENSE) {
+        if (table[4 * t + 0] == KIND_DENSE_Q4 || table[4 * t + 0] == KIND_SPARSE_Q4) {
+            /* 4-bit kinds: codes and scales are stored as they are; the metadata of the 2:4 kind takes the same
+             * order as below */
+            uint64_t size = kind_bytes(table[4 * t + 0], 128, 128);
+            memcpy(image + off, canon + off, (size_t)size);
+            if (table[4 * t + 0] == KIND_SPARSE_Q4) {
+                uint64_t moff = (uint64_t)table[4 * t + 2] * 16;
+                const uint32_t* cm = (const uint32_t*)(canon + moff);
+                for (int Lr = 0; Lr < 128; ++Lr) {
+                    int q = Lr / 16, h = (Lr / 8) % 2, i = Lr % 8;
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t lo = (cm[(16 * q + i) * 4 + j] >> (16 * h)) & 0xFFFFu;
+                        uint32_t hi = (cm[(16 * q + 8 + i) * 4 + j] >> (16 * h)) & 0xFFFFu;
+                        uint32_t word = lo | (hi << 16);
+                        memcpy(image + moff + (uint64_t)Lr * 16 + (uint64_t)j * 4, &word, 4);
+                    }
+                }
+            }
+        } else if (table[4 * t + 0] == KIND_DENSE) {
             const uint16_t* src = (const uint16_t*)(canon + off);
             for (int r = 0; r < 128; ++r)
                 for (int c = 0; c < 128; ++c) {

@@ -368,7 +368,7 @@ def test_device_image_structure(oracle):
 def test_rejects_bad_arguments(oracle):
     W = inputs.weight(128, 128, 9, "bad")
     with pytest.raises(ValueError):
-        oracle.pack(W, np.array([[2]], np.uint8))
+        oracle.pack(W, np.array([[4]], np.uint8))
     with pytest.raises(ValueError):
         oracle.packed_size(100, 128, np.zeros(1, np.uint8))
     with pytest.raises(ValueError):
