@@ -35,8 +35,16 @@
 extern "C" {
 #endif
 
-/* Tile kinds.  The flag is 1 - M*_tile of Algorithm 1 (the paper's tile mask is 1 = dense). */
-enum { PATCH_TILE_DENSE = 0, PATCH_TILE_SPARSE_2_4 = 1 };
+/* Tile kinds.  Bit 0 is 1 - M*_tile of Algorithm 1 (the paper's tile mask is 1 = dense).  Bit 1 selects the
+ * 4-bit payload of the section "Combination with other compression methods" (the 4-bit weight-only
+ * quantisation table): the tile's stored values -- all 128 of a row in a dense tile, the 64 kept ones in a 2:4
+ * tile -- are 4-bit codes with one bf16 scale per tile row.  The paper prints the compression ratio of this
+ * combination, 16 / (4 - f) (four bits per stored value, two metadata bits per kept value), and no quantiser;
+ * this library's reading is symmetric round-to-nearest-even,
+ *     s = bf16(max|v| / 7),  q = clamp(rint(v / s), -7, 7)  (0 where s = 0),  v^ = bf16(q * s),
+ * evaluated in fp32 on the bf16 values, the 2:4 selection made first on the unquantised weights.  The layer
+ * then multiplies by the dequantised values v^. */
+enum { PATCH_TILE_DENSE = 0, PATCH_TILE_SPARSE_2_4 = 1, PATCH_TILE_DENSE_Q4 = 2, PATCH_TILE_SPARSE_2_4_Q4 = 3 };
 
 enum {
     PATCH_OK = 0,
@@ -89,9 +97,10 @@ enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
  * The blob in device memory is position independent (offsets only):
  *   [ header 256 B (a copy of this struct, zero padded)
  *   | tile table: 16 B per tile in (tn, tk) row-major order, zero padded to a multiple of 1024 B
- *   | payloads at offsets that are multiples of 1024: 32 768 B per dense tile, 18 432 B per 2:4 tile ]
- * Table entry: { u32 kind, u32 payload_off / 16, u32 meta_off / 16 (0xFFFFFFFF if dense), u32 0 },
- * offsets counted from the start of the blob.
+ *   | payloads: 32 768 B per dense tile, 18 432 B per 2:4 tile (offsets multiples of 1024 while only these two
+ *     kinds occur), 8 448 B / 6 400 B per dense / 2:4 tile with 4-bit values (offsets multiples of 256) ]
+ * Table entry: { u32 kind, u32 payload_off / 16, u32 meta_off / 16 (0xFFFFFFFF if the kind has no metadata),
+ * u32 scales_off / 16 (0 if the kind has no scales) }, offsets counted from the start of the blob.
  *
  * Payload bytes (the "device image"):
  *   values are stored in 16 384-byte atoms of 128 rows x 64 bf16; inside an atom the 16-byte
@@ -103,6 +112,9 @@ enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
  *   (i < 8), word j: low 16 bits = the four 4-bit position codes (i0 | i1 << 2, i0 < i1) of
  *   tile row 16q+i for columns [32j + 16h, 32j + 16h + 16), high 16 bits = the same for tile
  *   row 16q+8+i.
+ *   4-bit kinds: [ codes: value c of tile row r in byte r * (V / 2) + c / 2, even c in the low nibble, code = q + 8
+ *   (1..15), V = 128 (dense) or 64 (2:4: the kept values in position order) | 2:4 only: 2 048 B of metadata in
+ *   the order above | scales: 128 bf16, one per tile row ].
  */
 typedef struct patch_layout_t {
     uint32_t magic;          /* 0x48435450 */
@@ -114,12 +126,13 @@ typedef struct patch_layout_t {
     uint64_t payload_off;    /* first payload byte */
     uint64_t payload_bytes;  /* 32768 * n_dense + 18432 * n_sparse */
     uint64_t total_bytes;    /* payload_off + payload_bytes = size of the blob */
+    int64_t  n_dense_q4, n_sparse_q4;   /* tiles of the 4-bit kinds (payload_bytes includes 8448 / 6400 B for each) */
 } patch_layout_t;
 
 /*
  * Size and layout of the packed blob for a weight of N x K with the given tile flags.
  * (Appendix A: the tile size fixes the compressed format; here it is 128 x 128.)
- *   tile_flags_host  [N/128 x K/128] row-major bytes, PATCH_TILE_DENSE or PATCH_TILE_SPARSE_2_4
+ *   tile_flags_host  [N/128 x K/128] row-major bytes, one of the four tile kinds
  *   layout_out       filled on success
  * Host only; touches no device.
  */
@@ -132,6 +145,7 @@ int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
  * In every 2:4 tile, each group of four consecutive elements along K keeps its two largest
  * magnitudes (equal magnitudes: lower index first; magnitude = bit pattern without sign);
  * dense tiles are copied.  A weight that is already 2:4 inside those tiles is packed losslessly.
+ * Tiles of the 4-bit kinds are quantised as described at the tile kinds (a second kernel).
  *   W_dev            bf16 [N x ldw], ldw >= K elements, ldw % 8 == 0
  *   tile_flags_host  as for patch_packed_size; must be the flags `layout` was computed from
  *   packed_dev       destination, packed_capacity >= layout->total_bytes, 16-byte aligned
@@ -143,7 +157,8 @@ int patch_pack(const void* W_dev, int64_t ldw, const uint8_t* tile_flags_host,
                void* stream);
 
 /*
- * Inverse of patch_pack: writes What = W (.) M* (pruned elements are +0) as bf16 [N x ldw].
+ * Inverse of patch_pack: writes What = W (.) M* (pruned elements are +0) as bf16 [N x ldw]; for tiles of the
+ * 4-bit kinds the dequantised values, i.e. exactly the matrix the layer multiplies by.
  */
 int patch_unpack(const patch_layout_t* layout, const void* packed_dev, void* What_dev,
                  int64_t ldw, void* stream);
@@ -179,6 +194,11 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  *           In both cases Y is undefined.  NULL = not reported.
  * M == 0 returns PATCH_OK without launching.  Calls sharing a workspace must be ordered on
  * one stream.
+ * Weights with 4-bit tiles: served for M <= 16 tokens (the decode case, where the bytes of the weight are
+ * what the layer costs) and only if every tile is of a 4-bit kind; a dequantising kernel of its own, no
+ * workspace.  Other M, and weights that mix bf16 and 4-bit tiles, return PATCH_ERR_SHAPE -- as do
+ * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated, patch_gemm_noalloc and the host entry points
+ * for such weights; patch_pack_dev / patch_pack_patterns report flags above 1 as PATCH_ERR_FLAG.
  */
 int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
                const patch_layout_t* layout, const void* packed_dev,

@@ -478,10 +478,23 @@ int oracle_device_image(const uint8_t* canon, uint64_t blob_bytes, uint8_t* imag
     for (int64_t t = 0; t < T; ++t) {
         uint64_t off = (uint64_t)table[4 * t + 1] * 16;
         if (table[4 * t + 0] == KIND_DENSE_Q4 || table[4 * t + 0] == KIND_SPARSE_Q4) {
-            /* 4-bit kinds: codes and scales are stored as they are; the metadata of the 2:4 kind takes the same
-             * order as below */
+            /* 4-bit kinds: scales are stored as they are; the metadata of the 2:4 kind takes the same order as
+             * below; the codes keep their 32-bit word (stored values 8w .. 8w+7 of a row in word w of the row)
+             * but inside the word the even values take nibbles 0..3 and the odd ones nibbles 4..7:
+             * value 8w + i sits in nibble (i % 2) * 4 + i / 2.  (A choice of byte order only: the paper fixes none
+             * for 4-bit payloads; with this one (word >> 4j) & 0x000F000F is the pair of neighbours 2j, 2j+1.) */
             uint64_t size = kind_bytes(table[4 * t + 0], 128, 128);
             memcpy(image + off, canon + off, (size_t)size);
+            uint64_t n_words = (table[4 * t + 0] == KIND_SPARSE_Q4 ? 4096u : 8192u) / 4;
+            for (uint64_t w = 0; w < n_words; ++w) {
+                uint32_t word = 0;
+                for (int i = 0; i < 8; ++i) {
+                    uint8_t byte = canon[off + 4 * w + (uint64_t)(i / 2)];
+                    uint32_t nib = (i % 2) ? (uint32_t)(byte >> 4) : (uint32_t)(byte & 0xF);
+                    word |= nib << (4 * ((i % 2) * 4 + i / 2));
+                }
+                memcpy(image + off + 4 * w, &word, 4);
+            }
             if (table[4 * t + 0] == KIND_SPARSE_Q4) {
                 uint64_t moff = (uint64_t)table[4 * t + 2] * 16;
                 const uint32_t* cm = (const uint32_t*)(canon + moff);

@@ -15,7 +15,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpatch_b200.so")
 
-TILE_DENSE, TILE_SPARSE_2_4 = 0, 1
+TILE_DENSE, TILE_SPARSE_2_4, TILE_DENSE_Q4, TILE_SPARSE_2_4_Q4 = 0, 1, 2, 3
 VARIANT_AUTO, VARIANT_GEMV, VARIANT_MMA, VARIANT_PAIR = 0, 1, 2, 3
 WEIGHTS_STATIC = 0x100   # OR into `variant`: the packed weight is not produced by the preceding kernel
 INPUT_STATIC = 0x200     # OR into `variant`: X is not produced by the preceding kernel
@@ -39,7 +39,8 @@ class Layout(ctypes.Structure):
                 ("tile_n", ctypes.c_int32), ("tile_k", ctypes.c_int32),
                 ("n_dense", ctypes.c_int64), ("n_sparse", ctypes.c_int64),
                 ("table_off", ctypes.c_uint64), ("payload_off", ctypes.c_uint64),
-                ("payload_bytes", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64)]
+                ("payload_bytes", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64),
+                ("n_dense_q4", ctypes.c_int64), ("n_sparse_q4", ctypes.c_int64)]
 
 
 class PatchError(RuntimeError):

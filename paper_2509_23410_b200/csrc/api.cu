@@ -21,7 +21,7 @@ extern "C" int patch_gemm_workspace_size(const patch_layout_t* L, int64_t M, siz
     int rc = validate_layout(L);
     if (rc) return rc;
     if (M < 0) return PATCH_ERR_SHAPE;
-    *bytes_out = decode_workspace_bytes(L, M);
+    *bytes_out = has_q4_tiles(L) ? 0 : decode_workspace_bytes(L, M);    // the 4-bit schedule needs none
     return PATCH_OK;
 }
 
@@ -46,6 +46,15 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
         return PATCH_ERR_SHAPE;
     if (variant == PATCH_VARIANT_GEMV && M > 4) return PATCH_ERR_SHAPE;
     if (variant == PATCH_VARIANT_PAIR && M <= 64) return PATCH_ERR_SHAPE;
+    if (has_q4_tiles(L)) {
+        // 4-bit tiles: the dequantising decode kernel, for weights made of such tiles only
+        if (L->n_dense || L->n_sparse || M > 16 || variant == PATCH_VARIANT_GEMV) return PATCH_ERR_SHAPE;
+        rc = check_device();
+        if (rc) return rc;
+        return launch_decode_q4(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
+                                static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, static_cast<cudaStream_t>(stream),
+                                wstatic, xstatic);
+    }
     const size_t need = decode_workspace_bytes(L, M);
     if (need > 0) {
         if (!workspace_dev) return PATCH_ERR_NULL;
@@ -75,6 +84,7 @@ extern "C" int patch_gemm_gated_workspace_size(const patch_layout_t* L, int64_t 
     int rc = validate_layout(L);
     if (rc) return rc;
     if (L->N % (2 * kTile) || M < 0) return PATCH_ERR_SHAPE;
+    if (has_q4_tiles(L)) return PATCH_ERR_SHAPE;
     *bytes_out = decode_gated_workspace_bytes(L, M);
     return PATCH_OK;
 }
@@ -86,7 +96,7 @@ extern "C" int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M, const
     int rc = validate_layout(L);
     if (rc) return rc;
     if (L->N % (2 * kTile)) return PATCH_ERR_SHAPE;      // whole (gate, up) pairs of row-blocks
-    if (M < 0) return PATCH_ERR_SHAPE;
+    if (M < 0 || has_q4_tiles(L)) return PATCH_ERR_SHAPE;
     if (flags & ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC)) return PATCH_ERR_SHAPE;
     if (M == 0) return PATCH_OK;
     if (!X_dev || !packed_dev || !Y_dev) return PATCH_ERR_NULL;

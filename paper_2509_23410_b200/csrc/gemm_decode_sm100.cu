@@ -741,6 +741,7 @@ extern "C" int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M, con
     if (rc) return rc;
     if (M < 0) return PATCH_ERR_SHAPE;
     if (M == 0) return PATCH_OK;
+    if (has_q4_tiles(L)) return PATCH_ERR_SHAPE;
     if (M > kNoAllocMaxTokens || L->N / kTile > kNoAllocMaxRowBlocks) return PATCH_ERR_SIZE;
     if (!X_dev || !packed_dev || !Y_dev) return PATCH_ERR_NULL;
     if (ldx < L->K || ldy < L->N || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;

@@ -5,6 +5,9 @@
 // group of four along K, and Appendix A's "compress" step (values + metadata per tile).
 // Both kernels are pure data movement plus integer compares, bound by HBM bandwidth:
 // per element of W they read 2 B and write 2 B (dense tile) or 1.125 B (2:4 tile).
+// Tiles of the 4-bit kinds (the 4-bit weight-only quantisation table of the paper's section on combining the
+// method with other compression; the quantiser is this library's reading, stated in the public header) are
+// written by a kernel of their own: one warp per tile row, 0.52 B (dense) or 0.39 B (2:4) per element.
 #include <vector>
 #include <cstring>
 #include "patch_internal.cuh"
@@ -16,13 +19,15 @@ int validate_layout(const patch_layout_t* L) {
     if (L->magic != kMagic || L->version != kVersion) return PATCH_ERR_FORMAT;
     if (L->tile_n != kTile || L->tile_k != kTile) return PATCH_ERR_TILE;
     if (L->N <= 0 || L->K <= 0 || L->N % kTile || L->K % kTile) return PATCH_ERR_SHAPE;
-    if (L->n_dense < 0 || L->n_sparse < 0) return PATCH_ERR_FORMAT;
+    if (L->n_dense < 0 || L->n_sparse < 0 || L->n_dense_q4 < 0 || L->n_sparse_q4 < 0) return PATCH_ERR_FORMAT;
     uint64_t T = uint64_t(L->N / kTile) * uint64_t(L->K / kTile);
-    if (uint64_t(L->n_dense) + uint64_t(L->n_sparse) != T) return PATCH_ERR_FORMAT;
+    if (uint64_t(L->n_dense) + uint64_t(L->n_sparse) + uint64_t(L->n_dense_q4) + uint64_t(L->n_sparse_q4) != T)
+        return PATCH_ERR_FORMAT;
     if (L->table_off != kHeaderBytes) return PATCH_ERR_FORMAT;
     uint64_t pay = (kHeaderBytes + 16 * T + 1023) / 1024 * 1024;
     if (L->payload_off != pay) return PATCH_ERR_FORMAT;
-    if (L->payload_bytes != uint64_t(kDenseBytes) * L->n_dense + uint64_t(kSparseBytes) * L->n_sparse)
+    if (L->payload_bytes != uint64_t(kDenseBytes) * L->n_dense + uint64_t(kSparseBytes) * L->n_sparse +
+                                uint64_t(kDenseQ4Bytes) * L->n_dense_q4 + uint64_t(kSparseQ4Bytes) * L->n_sparse_q4)
         return PATCH_ERR_FORMAT;
     if (L->total_bytes != L->payload_off + L->payload_bytes) return PATCH_ERR_FORMAT;
     if (L->total_bytes / 16 > 0xFFFFFFF0ull) return PATCH_ERR_SHAPE;  // offsets are stored as u32 * 16
@@ -136,6 +141,7 @@ __device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int 
             L.magic = fits ? kMagic : 0u; L.version = kVersion;
             L.N = F.N; L.K = F.K; L.tile_n = kTile; L.tile_k = kTile;
             L.n_dense = int64_t(dense); L.n_sparse = F.T - int64_t(dense);
+            L.n_dense_q4 = 0; L.n_sparse_q4 = 0;
             L.table_off = kHeaderBytes; L.payload_off = payload_off; L.payload_bytes = total; L.total_bytes = size;
             uint32_t* h = reinterpret_cast<uint32_t*>(blob);
             const uint32_t* src = reinterpret_cast<const uint32_t*>(&L);
@@ -169,6 +175,7 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
         if (!descriptor_from_flags(F, t, blob, status, d)) return;
     } else {
         d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+        if (d.kind > PATCH_TILE_SPARSE_2_4) return;      // a 4-bit kind: pack_q4_kernel writes it
     }
     const int tn = t / TK, tk = t - tn * TK;
     const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
@@ -226,6 +233,115 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// 4-bit kinds.  One warp per tile row, lane g holds the row's g-th group of four consecutive elements.
+//   scale  s = bf16(max|v| / 7) over the row's stored values (all 128, or the 64 the 2:4 selection keeps)
+//   code   q + 8 with q = clamp(rint(v / s), -7, 7), 0 where s = 0; fp32 arithmetic, IEEE division
+// Codes are stored eight to a 32-bit word, values 8w .. 8w + 7 of the row's stored values in word w: the even
+// ones in nibbles 0..3, the odd ones in nibbles 4..7, so that (word >> 4j) & 0x000F000F is the pair (2j, 2j + 1)
+// in the two halves of a register -- what the dequantising GEMM kernel turns into two bf16 with one instruction.
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
+__device__ __forceinline__ uint32_t q4_nibble(float v, float s) {
+    if (s == 0.0f) return 8u;
+    const float r = fminf(fmaxf(rintf(__fdiv_rn(v, s)), -7.0f), 7.0f);
+    return uint32_t(int(r) + 8);
+}
+// nibble index inside its 32-bit word of stored value c (c & 7 decides)
+__device__ __forceinline__ uint32_t q4_nibble_slot(uint32_t c) { return ((c & 1u) << 2) | ((c & 7u) >> 1); }
+
+__global__ void __launch_bounds__(256)
+pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob, uint64_t table_off) {
+    const int t = blockIdx.x;
+    const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+    if (d.kind < PATCH_TILE_DENSE_Q4) return;
+    const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
+    const int tn = t / TK, tk = t - tn * TK;
+    const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
+    uint8_t* codes = blob + uint64_t(d.payload_off16) * 16;
+    uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;                    // only used if sparse
+    uint16_t* scales = reinterpret_cast<uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    for (uint32_t rr = 0; rr < 16; ++rr) {
+        const uint32_t r = rr * 8 + warp;
+        const uint2 x = *reinterpret_cast<const uint2*>(wt + int64_t(r) * ldw + lane * 4);
+        float v[4] = {bf16_bits_to_f32(x.x & 0xFFFFu), bf16_bits_to_f32(x.x >> 16),
+                      bf16_bits_to_f32(x.y & 0xFFFFu), bf16_bits_to_f32(x.y >> 16)};
+        uint32_t i0 = 0, i1 = 1;
+        float m;
+        if (sparse) {
+            top2_positions(x.x, x.y, i0, i1);
+            const uint32_t kept = gather_pair(x.x, x.y, i0, i1);
+            v[0] = bf16_bits_to_f32(kept & 0xFFFFu);
+            v[1] = bf16_bits_to_f32(kept >> 16);
+            m = fmaxf(fabsf(v[0]), fabsf(v[1]));
+        } else {
+            m = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+        const __nv_bfloat16 sb = __float2bfloat16_rn(__fdiv_rn(m, 7.0f));
+        const float s = __bfloat162float(sb);
+        if (lane == 0) scales[r] = __bfloat16_as_ushort(sb);
+        // this lane's nibbles, each shifted to its slot of the 32-bit word it belongs to; the lanes of a word
+        // (two for a dense row, four for a 2:4 row) combine them with shuffles and the first one stores
+        uint32_t word = 0;
+        if (sparse) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) word |= q4_nibble(v[i], s) << (4 * q4_nibble_slot(2 * lane + i));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+            if ((lane & 3u) == 0) reinterpret_cast<uint32_t*>(codes)[r * 8 + (lane >> 2)] = word;
+            // position codes of the four groups of a 16-column chunk -> 16 bits of metadata (hardware order)
+            uint32_t code = (i0 | (i1 << 2)) << (4 * (lane & 3u));
+            code |= __shfl_xor_sync(0xFFFFFFFFu, code, 1);
+            code |= __shfl_xor_sync(0xFFFFFFFFu, code, 2);
+            const uint32_t u = lane >> 2;
+            const uint32_t Lr = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
+            if ((lane & 3u) == 0) *reinterpret_cast<uint16_t*>(meta + Lr * 16 + j * 4 + hi * 2) = uint16_t(code);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) word |= q4_nibble(v[i], s) << (4 * q4_nibble_slot(4 * lane + i));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            if ((lane & 1u) == 0) reinterpret_cast<uint32_t*>(codes)[r * 16 + (lane >> 1)] = word;
+        }
+    }
+}
+
+// Dequantised value of the code nibble n with the row's scale s: bf16(q * s), q = n - 8 (the product is exact in fp32)
+__device__ __forceinline__ uint32_t q4_dequant_bits(uint32_t n, float s) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(float(int(n) - 8) * s));
+}
+
+__device__ __forceinline__ void unpack_q4_tile(const TileDesc& d, const uint8_t* __restrict__ blob, uint16_t* wt, int64_t ldw) {
+    const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
+    const uint32_t* codes = reinterpret_cast<const uint32_t*>(blob + uint64_t(d.payload_off16) * 16);
+    const uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;
+    const uint16_t* scales = reinterpret_cast<const uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    for (uint32_t rr = 0; rr < 16; ++rr) {
+        const uint32_t r = rr * 8 + warp;
+        const float s = bf16_bits_to_f32(scales[r]);
+        uint32_t out[4] = {0, 0, 0, 0};
+        if (sparse) {
+            const uint32_t word = codes[r * 8 + (lane >> 2)];
+            const uint32_t u = lane >> 2;
+            const uint32_t Lr = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
+            const uint32_t code = *reinterpret_cast<const uint16_t*>(meta + Lr * 16 + j * 4 + hi * 2);
+            const uint32_t nib = (code >> (4 * (lane & 3u))) & 0xFu, i0 = nib & 3u, i1 = nib >> 2;
+            const uint32_t a = q4_dequant_bits((word >> (4 * q4_nibble_slot(2 * lane))) & 0xFu, s);
+            const uint32_t b = q4_dequant_bits((word >> (4 * q4_nibble_slot(2 * lane + 1))) & 0xFu, s);
+#pragma unroll
+            for (uint32_t p = 0; p < 4; ++p) out[p] = p == i0 ? a : p == i1 ? b : 0u;
+        } else {
+            const uint32_t word = codes[r * 16 + (lane >> 1)];
+#pragma unroll
+            for (uint32_t p = 0; p < 4; ++p) out[p] = q4_dequant_bits((word >> (4 * q4_nibble_slot(4 * lane + p))) & 0xFu, s);
+        }
+        *reinterpret_cast<uint2*>(wt + int64_t(r) * ldw + lane * 4) = make_uint2(out[0] | (out[1] << 16), out[2] | (out[3] << 16));
+    }
+}
+
 __global__ void __launch_bounds__(256)
 unpack_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
               uint16_t* __restrict__ What, int64_t ldw) {
@@ -234,7 +350,9 @@ unpack_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
     const int tn = t / TK, tk = t - tn * TK;
     uint16_t* wt = What + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
     const uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
-    if (d.kind == PATCH_TILE_DENSE) {
+    if (d.kind >= PATCH_TILE_DENSE_Q4) {
+        unpack_q4_tile(d, blob, wt, ldw);
+    } else if (d.kind == PATCH_TILE_DENSE) {
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
             const uint32_t idx = it * 256 + threadIdx.x, r = idx >> 4, c = idx & 15u;
@@ -280,20 +398,21 @@ extern "C" int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
     if (tile_n != kTile || tile_k != kTile) return PATCH_ERR_TILE;
     if (N <= 0 || K <= 0 || N % kTile || K % kTile) return PATCH_ERR_SHAPE;
     const int64_t T = (N / kTile) * (K / kTile);
-    int64_t nd = 0, ns = 0;
+    int64_t n[4] = {0, 0, 0, 0};
     for (int64_t t = 0; t < T; ++t) {
-        if (flags[t] == PATCH_TILE_DENSE) ++nd;
-        else if (flags[t] == PATCH_TILE_SPARSE_2_4) ++ns;
-        else return PATCH_ERR_FLAG;
+        if (flags[t] > PATCH_TILE_SPARSE_2_4_Q4) return PATCH_ERR_FLAG;
+        ++n[flags[t]];
     }
     patch_layout_t L;
     std::memset(&L, 0, sizeof L);
     L.magic = kMagic; L.version = kVersion;
     L.N = N; L.K = K; L.tile_n = kTile; L.tile_k = kTile;
-    L.n_dense = nd; L.n_sparse = ns;
+    L.n_dense = n[PATCH_TILE_DENSE]; L.n_sparse = n[PATCH_TILE_SPARSE_2_4];
+    L.n_dense_q4 = n[PATCH_TILE_DENSE_Q4]; L.n_sparse_q4 = n[PATCH_TILE_SPARSE_2_4_Q4];
     L.table_off = kHeaderBytes;
     L.payload_off = (kHeaderBytes + 16 * uint64_t(T) + 1023) / 1024 * 1024;
-    L.payload_bytes = uint64_t(kDenseBytes) * nd + uint64_t(kSparseBytes) * ns;
+    L.payload_bytes = 0;
+    for (uint32_t k = 0; k < 4; ++k) L.payload_bytes += uint64_t(tile_payload_bytes(k)) * uint64_t(n[k]);
     L.total_bytes = L.payload_off + L.payload_bytes;
     if (L.total_bytes / 16 > 0xFFFFFFF0ull) return PATCH_ERR_SHAPE;
     *out = L;
@@ -314,17 +433,25 @@ static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const
     std::memcpy(head.data(), L, sizeof *L);
     TileDesc* table = reinterpret_cast<TileDesc*>(head.data() + L->table_off);
     uint64_t off = L->payload_off;
-    int64_t nd = 0, ns = 0;
+    int64_t n[4] = {0, 0, 0, 0};
     for (int64_t t = 0; t < T; ++t) {
-        if (flags[t] == PATCH_TILE_DENSE) {
-            table[t] = TileDesc{PATCH_TILE_DENSE, uint32_t(off / 16), 0xFFFFFFFFu, 0};
-            off += kDenseBytes; ++nd;
-        } else if (flags[t] == PATCH_TILE_SPARSE_2_4) {
-            table[t] = TileDesc{PATCH_TILE_SPARSE_2_4, uint32_t(off / 16), uint32_t((off + kAtomBytes) / 16), 0};
-            off += kSparseBytes; ++ns;
-        } else return PATCH_ERR_FLAG;
+        const uint32_t kind = flags[t];
+        if (kind > PATCH_TILE_SPARSE_2_4_Q4 || (patterns_dev && kind > PATCH_TILE_SPARSE_2_4)) return PATCH_ERR_FLAG;
+        TileDesc d = TileDesc{kind, uint32_t(off / 16), 0xFFFFFFFFu, 0};
+        if (kind == PATCH_TILE_SPARSE_2_4) {
+            d.meta_off16 = uint32_t((off + kAtomBytes) / 16);
+        } else if (kind == PATCH_TILE_DENSE_Q4) {
+            d.scales_off16 = uint32_t((off + kDenseQ4CodeBytes) / 16);
+        } else if (kind == PATCH_TILE_SPARSE_2_4_Q4) {
+            d.meta_off16 = uint32_t((off + kSparseQ4CodeBytes) / 16);
+            d.scales_off16 = uint32_t((off + kSparseQ4CodeBytes + kMetaBytes) / 16);
+        }
+        table[t] = d;
+        off += tile_payload_bytes(kind);
+        ++n[kind];
     }
-    if (nd != L->n_dense || ns != L->n_sparse) return PATCH_ERR_FORMAT;  // flags do not match the layout
+    if (n[0] != L->n_dense || n[1] != L->n_sparse || n[2] != L->n_dense_q4 || n[3] != L->n_sparse_q4)
+        return PATCH_ERR_FORMAT;  // flags do not match the layout
     rc = check_device();
     if (rc) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -340,6 +467,9 @@ static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const
         pack_kernel<false, false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
                                                               static_cast<uint8_t*>(packed_dev), L->table_off, nullptr,
                                                               nullptr, none);
+    if (has_q4_tiles(L))
+        pack_q4_kernel<<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                   static_cast<uint8_t*>(packed_dev), L->table_off);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

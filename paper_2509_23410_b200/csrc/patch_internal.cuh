@@ -16,13 +16,22 @@ constexpr uint32_t kSparseBytes = 18432u;   // one 16 KB atom + 2 KB metadata
 constexpr uint32_t kAtomBytes = 16384u;
 constexpr uint32_t kMetaBytes = 2048u;
 constexpr uint32_t kHeaderBytes = 256u;
+// 4-bit kinds: codes (8192 / 4096 B) [+ metadata 2048 B] + 128 bf16 scales
+constexpr uint32_t kScaleBytes = 256u;
+constexpr uint32_t kDenseQ4CodeBytes = 8192u, kSparseQ4CodeBytes = 4096u;
+constexpr uint32_t kDenseQ4Bytes = kDenseQ4CodeBytes + kScaleBytes;                    // 8 448
+constexpr uint32_t kSparseQ4Bytes = kSparseQ4CodeBytes + kMetaBytes + kScaleBytes;     // 6 400
+__host__ __device__ constexpr uint32_t tile_payload_bytes(uint32_t kind) {
+    return kind == PATCH_TILE_DENSE ? kDenseBytes : kind == PATCH_TILE_SPARSE_2_4 ? kSparseBytes
+         : kind == PATCH_TILE_DENSE_Q4 ? kDenseQ4Bytes : kSparseQ4Bytes;
+}
 
 // One entry of the tile table inside the packed blob.
 struct TileDesc {
     uint32_t kind;          // PATCH_TILE_DENSE / PATCH_TILE_SPARSE_2_4
     uint32_t payload_off16; // byte offset / 16 from the start of the blob
     uint32_t meta_off16;    // byte offset / 16 of the metadata block, 0xFFFFFFFF if dense
-    uint32_t reserved;
+    uint32_t scales_off16;  // byte offset / 16 of the scales of a 4-bit kind, 0 otherwise
 };
 static_assert(sizeof(TileDesc) == 16, "tile table entry is 16 bytes");
 
@@ -110,5 +119,9 @@ int launch_decode_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const pa
                         const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev,
                         cudaStream_t stream, bool wstatic, bool xstatic);
 size_t decode_gated_workspace_bytes(const patch_layout_t* L, int64_t M);   // 0 if the gated decode schedule does not apply
+// M <= 16 on a weight whose tiles are all of a 4-bit kind (gemm_decode_q4_sm100.cu)
+int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
+                     __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic);
+inline bool has_q4_tiles(const patch_layout_t* L) { return L->n_dense_q4 != 0 || L->n_sparse_q4 != 0; }
 
 }  // namespace patch

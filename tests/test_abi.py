@@ -3,6 +3,7 @@ header declares, and rejects bad arguments before touching a device."""
 import ctypes
 import os
 import re
+import subprocess
 
 import numpy as np
 import pytest
@@ -33,9 +34,19 @@ def test_every_declared_symbol_is_exported(binding):
     assert sorted(binding.EXPORTS) == names
 
 
-def test_layout_struct_matches_header(binding):
-    assert ctypes.sizeof(binding.Layout) == 80
+def test_layout_struct_matches_header(binding, tmp_path):
+    assert ctypes.sizeof(binding.Layout) == 96
     assert binding.patch_version() == 1
+    # size and field offsets as a C compiler lays the header's struct out
+    src = tmp_path / "layout.c"
+    fields = [f for f, _ in binding.Layout._fields_]
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "patch.h"\nint main(void) {\n'
+                   '  printf("%zu", sizeof(patch_layout_t));\n' +
+                   "".join(f'  printf(" %zu", offsetof(patch_layout_t, {f}));\n' for f in fields) + "  return 0; }\n")
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    got = [int(v) for v in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    assert got == [ctypes.sizeof(binding.Layout)] + [getattr(binding.Layout, f).offset for f in fields]
 
 
 def test_packed_size_and_validation(binding, oracle):
@@ -45,8 +56,15 @@ def test_packed_size_and_validation(binding, oracle):
     for f, _ in binding.Layout._fields_:
         assert getattr(L, f) == getattr(Lo, f), f
     assert L.payload_bytes == 3 * 32768 + 3 * 18432
+    # all four kinds
+    flags4 = np.array([[0, 3, 2], [1, 2, 3]], np.uint8)
+    L = binding.patch_packed_size(256, 384, flags4)
+    Lo = oracle.packed_size(256, 384, flags4)
+    for f, _ in binding.Layout._fields_:
+        assert getattr(L, f) == getattr(Lo, f), f
+    assert L.payload_bytes == 32768 + 18432 + 2 * 8448 + 2 * 6400
     with pytest.raises(binding.PatchError) as e:
-        binding.patch_packed_size(256, 384, np.full((2, 3), 2, np.uint8))
+        binding.patch_packed_size(256, 384, np.full((2, 3), 4, np.uint8))
     assert e.value.status == binding.ERR_FLAG
     with pytest.raises(binding.PatchError) as e:
         binding.patch_packed_size(250, 384, flags)

@@ -1,0 +1,201 @@
+"""GPU parity of the 4-bit tile kinds (2: dense, 3: 2:4, stored values as 4-bit codes with one bf16 scale per tile
+row) against the CPU oracle: the packed blob bit for bit, the dequantised matrix bit for bit, and the small-M matmul
+on a weight made of such tiles."""
+import numpy as np
+import pytest
+
+from paper_2509_23410_b200 import inputs
+from test_gpu_parity import check_parity, f32, gpu, run_gemm, to_bits, to_dev  # noqa: F401  (gpu is a fixture)
+
+pytestmark = pytest.mark.gpu
+
+
+def _flags4(N, K, p, seed_tag, q4="all"):
+    """Tile kinds: bit 0 drawn with probability p; bit 1 set everywhere ("all") or on a random half ("half")."""
+    flags = inputs.tile_flags(N, K, p, inputs.MASTER_SEED, "q4", seed_tag)
+    if q4 == "all":
+        return flags | 2
+    g = inputs.generator(inputs.MASTER_SEED, "q4-bit1", seed_tag, N, K)
+    return flags | (2 * (g.random(flags.shape) < 0.5)).astype(np.uint8)
+
+
+@pytest.mark.parametrize("q4", ["all", "half"])
+@pytest.mark.parametrize("p", [0.0, 1.0, 0.45])
+@pytest.mark.parametrize("N,K", [(128, 128), (384, 640), (1024, 512)])
+def test_pack_bit_exact_and_unpack(gpu, oracle, N, K, p, q4):
+    torch, B = gpu
+    W = inputs.weight(N, K, 31, "q4-pack", N, K)
+    W[::13, ::7] = 0                      # exact zeros and ties in the 2:4 selection
+    W[5, :] = 0                           # a row of zeros: scale 0, every code 8
+    W[7, 128 * (K // 128 - 1):] = inputs.f32_to_bf16_bits(np.float32(0.0371))   # a constant row: every |q| = 7
+    flags = _flags4(N, K, p, (N, K, p), q4)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    blob_o, L_o = oracle.pack(W, flags)
+    for f, _ in B.Layout._fields_:
+        assert getattr(L, f) == getattr(L_o, f), f
+    image = oracle.device_image(blob_o)
+    got = packed.cpu().numpy()
+    assert got.shape == image.shape
+    bad = np.flatnonzero(got != image)
+    assert bad.size == 0, f"{bad.size} bytes differ, first at {bad[:8]}"
+    # the dequantised matrix: what the layer multiplies by
+    What = to_bits(B.patch_unpack(L, packed))
+    assert (What == oracle.prune(W, flags)).all()
+    assert (What == oracle.unpack(blob_o)).all()
+
+
+def test_pack_with_row_pitch_and_extreme_values(gpu, oracle):
+    """Row pitch > K; magnitudes spanning many binades, so that scales and quotients take many exponents."""
+    torch, B = gpu
+    N, K, ld = 256, 384, 448
+    g = inputs.generator(32, "q4-extreme")
+    vals = (g.standard_normal((N, K)) * np.exp2(g.integers(-20, 20, (N, 1)))).astype(np.float32)
+    W = inputs.f32_to_bf16_bits(vals)
+    flags = _flags4(N, K, 0.5, "pitch")
+    Wd = torch.zeros((N, ld), dtype=torch.bfloat16, device="cuda")
+    Wd[:, :K] = to_dev(torch, W)
+    packed, L = B.patch_pack(Wd[:, :K], flags)
+    image = oracle.device_image(oracle.pack(W, flags)[0])
+    assert (packed.cpu().numpy() == image).all()
+    out = torch.full((N, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    B.patch_unpack(L, packed, out=out[:, :K])
+    assert (to_bits(out[:, :K]) == oracle.prune(W, flags)).all()
+    assert (out[:, K:] == 7.0).all()
+
+
+@pytest.mark.parametrize("M", [1, 5, 16])
+@pytest.mark.parametrize("p", [0.0, 1.0, 0.4])
+@pytest.mark.parametrize("N,K", [(128, 128), (256, 1152), (640, 384), (4096, 1024), (512, 8192)])
+def test_gemm_parity(gpu, oracle, N, K, M, p):
+    """Whole output against the oracle's matmul on the dequantised matrix; all three launch forms agree bit for
+    bit with themselves on a second launch (deterministic) and with each other (same summation order)."""
+    torch, B = gpu
+    W = inputs.weight(N, K, 33, "q4-gemm", N, K)
+    X = inputs.activation(M, K, 33, "q4-gemm", N, K, M)
+    flags = _flags4(N, K, p, ("gemm", N, K, p))
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    assert B.patch_gemm_workspace_size(L, M) == 0
+    Y32, Y16 = oracle.gemm_f64(X, What)
+    outs = []
+    for promise in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC):
+        Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | promise)
+        check_parity(oracle, Y, Y32, f"q4 N={N} K={K} M={M} p={p} promise={promise:#x}")
+        assert (Y == Y16).mean() >= 0.99
+        outs.append(Y)
+    assert (outs[0] == outs[1]).all() and (outs[0] == outs[2]).all()
+    assert (run_gemm(gpu, X, L, packed, B.VARIANT_MMA) == outs[0]).all()
+
+
+@pytest.mark.parametrize("p", [0.0, 1.0, 0.5])
+def test_gemm_one_hot_probe(gpu, oracle, p):
+    """Token m is the unit vector e_k(m): every output is one product with 1, so row m of Y must equal column k(m)
+    of the dequantised matrix exactly.  A wrong nibble order, scale row or metadata order shows as exact
+    mismatches.  Sixteen columns per launch, chosen to cover every position of a group of eight and several tiles."""
+    torch, B = gpu
+    N, K = 384, 512
+    W = inputs.weight(N, K, 34, "q4-onehot")
+    flags = _flags4(N, K, p, ("onehot", p))
+    What = f32(oracle.prune(W, flags))
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    for base in (0, 8, 120, 250, 496):
+        cols = [(base + 9 * i) % K for i in range(16)]
+        X = np.zeros((16, K), np.float32)
+        X[np.arange(16), cols] = 1.0
+        Y = run_gemm(gpu, inputs.f32_to_bf16_bits(X), L, packed, B.VARIANT_AUTO)
+        assert (f32(Y) == What[:, cols].T).all(), base
+
+
+def test_gemm_back_to_back_and_chain(gpu, oracle):
+    """Launches in a row on one stream with and without promises, each into its own output; then a chain in which
+    the output of one call is the input of the next (square weight)."""
+    torch, B = gpu
+    M = 16
+    cases = []
+    for i, (N, K) in enumerate([(1024, 512), (640, 768)]):
+        W = inputs.weight(N, K, 35, "q4-b2b", i)
+        X = inputs.activation(M, K, 35, "q4-b2b", i)
+        flags = _flags4(N, K, 0.5, ("b2b", i))
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        cases.append((oracle.prune(W, flags), packed, L, X, to_dev(torch, X)))
+    torch.cuda.synchronize()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    outs = []
+    for i in range(12):
+        What, packed, L, X, Xd = cases[i % 2]
+        promise = (B.WEIGHTS_STATIC | B.INPUT_STATIC) if i % 2 else 0
+        outs.append(B.patch_gemm(Xd, L, packed, status=status, variant=B.VARIANT_AUTO | promise))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    refs = [oracle.gemm_f64(c[3], c[0])[0] for c in cases]
+    for i, Y in enumerate(outs):
+        check_parity(oracle, to_bits(Y), refs[i % 2], f"launch {i}")
+    N = K = 512
+    W = inputs.f32_to_bf16_bits(f32(inputs.weight(N, K, 35, "q4-chain")) * 2.0)
+    X = inputs.activation(M, K, 35, "q4-chain")
+    flags = _flags4(N, K, 0.5, "chain")
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    bufs = [to_dev(torch, X)] + [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(6)]
+    for i in range(6):
+        B.patch_gemm(bufs[i], L, packed, Y=bufs[i + 1], status=status,
+                     variant=B.VARIANT_AUTO | (B.WEIGHTS_STATIC if i % 2 else 0))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = X
+    for i in range(6):
+        Y32, _ = oracle.gemm_f64(ref, What)
+        got = to_bits(bufs[i + 1])
+        check_parity(oracle, got, Y32, f"chain step {i}")
+        ref = got
+
+
+def test_unsupported_combinations_are_refused(gpu):
+    torch, B = gpu
+    N, K = 256, 256
+    W = to_dev(torch, inputs.weight(N, K, 36, "q4-err"))
+    all_q4 = np.array([[2, 3], [3, 2]], np.uint8)
+    mixed = np.array([[2, 0], [3, 1]], np.uint8)
+    packed, L = B.patch_pack(W, all_q4)
+    packed_m, L_m = B.patch_pack(W, mixed)             # packing and unpacking serve any mixture
+    assert (L_m.n_dense, L_m.n_sparse, L_m.n_dense_q4, L_m.n_sparse_q4) == (1, 1, 1, 1)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    X17 = torch.zeros((17, K), dtype=torch.bfloat16, device="cuda")
+    X4 = torch.zeros((4, K), dtype=torch.bfloat16, device="cuda")
+
+    def refused(fn):
+        with pytest.raises(B.PatchError) as e:
+            fn()
+        return e.value.status
+
+    assert refused(lambda: B.patch_gemm(X17, L, packed, workspace=ws)) == B.ERR_SHAPE          # M > 16
+    assert refused(lambda: B.patch_gemm(X4, L_m, packed_m, workspace=ws)) == B.ERR_SHAPE       # bf16 and 4-bit tiles
+    assert refused(lambda: B.patch_gemm(X4, L, packed, workspace=ws, variant=B.VARIANT_GEMV)) == B.ERR_SHAPE
+    assert refused(lambda: B.patch_gemm_gated(X4, L, packed, workspace=ws)) == B.ERR_SHAPE
+    assert refused(lambda: B.patch_gemm_noalloc(X4, L, packed, torch.empty((4, N), dtype=torch.bfloat16, device="cuda"))) == B.ERR_SHAPE
+    flags_dev = torch.from_numpy(all_q4.reshape(-1)).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.patch_pack_dev(W, flags_dev, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_FLAG
+
+
+def test_bad_table_entries_are_reported(gpu, oracle):
+    """A table entry whose kind is not a 4-bit kind, or whose payload lies outside the blob: the launch completes,
+    the status word says PATCH_ERR_FORMAT, nothing is read out of range."""
+    torch, B = gpu
+    N, K, M = 256, 512, 8
+    W = inputs.weight(N, K, 37, "q4-bad")
+    X = inputs.activation(M, K, 37, "q4-bad")
+    flags = _flags4(N, K, 0.5, "bad")
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    good = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO)
+    for word, value in ((0, 1), (0, 9), (1, int(L.total_bytes // 16) - 3), (1, 2)):
+        blob = packed.clone()
+        entry = blob[int(L.table_off) + 16 * 3:int(L.table_off) + 16 * 4].view(torch.int32)
+        entry[word] = value
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.patch_gemm(to_dev(torch, X), L, blob, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == B.ERR_FORMAT, (word, value)
+    assert (run_gemm(gpu, X, L, packed, B.VARIANT_AUTO) == good).all()
