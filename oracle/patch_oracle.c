@@ -479,22 +479,24 @@ int oracle_device_image(const uint8_t* canon, uint64_t blob_bytes, uint8_t* imag
         uint64_t off = (uint64_t)table[4 * t + 1] * 16;
         if (table[4 * t + 0] == KIND_DENSE_Q4 || table[4 * t + 0] == KIND_SPARSE_Q4) {
             /* 4-bit kinds: scales are stored as they are; the metadata of the 2:4 kind takes the same order as
-             * below; the codes keep their 32-bit word (stored values 8w .. 8w+7 of a row in word w of the row)
-             * but inside the word the even values take nibbles 0..3 and the odd ones nibbles 4..7:
-             * value 8w + i sits in nibble (i % 2) * 4 + i / 2.  (A choice of byte order only: the paper fixes none
-             * for 4-bit payloads; with this one (word >> 4j) & 0x000F000F is the pair of neighbours 2j, 2j+1.) */
+             * below.  Codes: the row's stored values (128, or the 64 kept ones) in order, eight to a 32-bit word,
+             * inside a word the even values in nibbles 0..3 and the odd ones in nibbles 4..7 (value 8w + i in nibble
+             * (i % 2) * 4 + i / 2 of word w); four words make a 16-byte unit, and unit j of tile row r lives at byte
+             * (128 j + r) * 16.  (A choice of byte order only: the paper fixes none for 4-bit payloads.) */
             uint64_t size = kind_bytes(table[4 * t + 0], 128, 128);
             memcpy(image + off, canon + off, (size_t)size);
-            uint64_t n_words = (table[4 * t + 0] == KIND_SPARSE_Q4 ? 4096u : 8192u) / 4;
-            for (uint64_t w = 0; w < n_words; ++w) {
-                uint32_t word = 0;
-                for (int i = 0; i < 8; ++i) {
-                    uint8_t byte = canon[off + 4 * w + (uint64_t)(i / 2)];
-                    uint32_t nib = (i % 2) ? (uint32_t)(byte >> 4) : (uint32_t)(byte & 0xF);
-                    word |= nib << (4 * ((i % 2) * 4 + i / 2));
+            int vals = table[4 * t + 0] == KIND_SPARSE_Q4 ? 64 : 128;
+            for (int r = 0; r < 128; ++r)
+                for (int w = 0; w < vals / 8; ++w) {
+                    uint32_t word = 0;
+                    for (int i = 0; i < 8; ++i) {
+                        int c = 8 * w + i;                                   /* stored value c of row r */
+                        uint8_t byte = canon[off + (uint64_t)r * (vals / 2) + (uint64_t)(c / 2)];
+                        uint32_t nib = (c % 2) ? (uint32_t)(byte >> 4) : (uint32_t)(byte & 0xF);
+                        word |= nib << (4 * ((i % 2) * 4 + i / 2));
+                    }
+                    memcpy(image + off + ((uint64_t)(w / 4) * 128 + r) * 16 + (uint64_t)(w % 4) * 4, &word, 4);
                 }
-                memcpy(image + off + 4 * w, &word, 4);
-            }
             if (table[4 * t + 0] == KIND_SPARSE_Q4) {
                 uint64_t moff = (uint64_t)table[4 * t + 2] * 16;
                 const uint32_t* cm = (const uint32_t*)(canon + moff);

@@ -1,48 +1,61 @@
 // Small-M matmul on a weight whose tiles are stored with 4-bit values (tile kinds 2 and 3: the 4-bit weight-only
 // quantisation table of the paper's section on combining the method with other compression).
 //
-// The layer multiplies by the DEQUANTISED weight v^ = bf16(q * s) (public header), so the kernel turns every tile
-// back into the bf16 operand image the tensor core reads -- two swizzled K-major atoms for a dense tile, one atom
-// plus the 2 KB metadata block for a 2:4 tile -- in shared memory, and runs the same tcgen05.mma / .mma.sp as the
-// bf16 kinds on it.  HBM only ever sees 0.52 B (dense) or 0.39 B (2:4) per weight element.
+// The layer multiplies by the DEQUANTISED weight v^ = bf16(q * s) (public header).  The kernel rebuilds each tile's
+// bf16 A operand in TENSOR MEMORY -- tcgen05.mma / .mma.sp take A from there -- so a weight value crosses shared
+// memory once, as half a byte on its way in: HBM sees 0.52 B (dense) or 0.39 B (2:4) per weight element, and shared
+// memory sees the same.  (Rebuilding the operand image in shared memory instead costs 32 KB of stores and 32 KB of
+// tensor-core reads per dense tile, ~700 cycles of the shared-memory port against ~170 cycles of HBM time: that
+// version ran at 1.5 TB/s.)
 //
-//   warp 0       producer: cp.async.bulk of the tile's payload (8 448 / 6 400 B: codes [, metadata], scales) into a
-//                ring of kRaw slots, and the two activation atoms of the tile's K range into the slot's X buffer
-//   warps 6..13  dequantise: slot -> operand stage.  A thread owns one 32-bit word of codes at a time = eight
-//                consecutive stored values of one row = one 16-byte chunk of the atom: the word's nibbles are
-//                ordered (pack.cu) so that (w >> 4j) & 0x000F000F | 0x43004300 is the bf16 pair (128 + n, 128 + n'),
-//                then (x - 136) * s in two bf16x2 instructions, both exact or correctly rounded:
-//                128 + n and n - 8 are integers below 256, and bf16(q * s) is one rounding of the exact product.
-//   warp 1       MMA issuer: operand stage x X buffer -> TMEM accumulator [128 rows x 16 tokens]
-//   warps 2..5   epilogue: accumulator -> shared memory; then, as in the bf16 row-block schedule, the S CTAs of a
-//                cluster (split-K) sum their partials through distributed shared memory in K order and write Y.
+//   warp 0        producer: cp.async.bulk of the tile's payload (8 448 / 6 400 B: codes [, metadata], scales) into
+//                 a ring of kRaw slots, and the two activation atoms of the tile's K range into the slot's X buffer
+//   warps 5..     kGroups groups of four warps; group g takes tiles g, g + kGroups, ... and owns 64 TMEM columns (its
+//                 operand stage) and an accumulator [128 rows x 16 tokens] of its own.
+//                 Dequantise: thread = tile row = TMEM lane.  It reads its row's codes 16 bytes at a time (the image
+//                 stores them so that the 32 threads of a warp read 512 consecutive bytes), turns each 32-bit word
+//                 into eight bf16 -- the nibbles are ordered (pack.cu) so that (w >> 4j) & 0x000F000F | 0x43004300
+//                 is the bf16 pair (128 + n, 128 + n'), then (x - 136) * s in two bf16x2 instructions, exact:
+//                 128 + n and n - 8 are small integers and bf16(q * s) is one rounding of the exact product -- and
+//                 writes 16 columns (32 values) per tcgen05.st.
+//                 Multiply: one thread of the group's first warp issues the tile's MMAs (A = the group's TMEM columns,
+//                 B = the slot's X buffer in shared memory; the metadata of a 2:4 tile goes from the payload slot to
+//                 TMEM with tcgen05.cp).  Issuing from one thread for all tiles took ~1 100 cycles per tile next
+//                 to the dequantising warps it shares issue slots with, and bounded the kernel at 1.7 TB/s.
+//   warps 1..4    epilogue: sum of the groups' accumulators (ascending group) -> shared memory; then, as in the bf16
+//                 row-block schedule, the S CTAs of a cluster (split-K) sum their partials through distributed
+//                 shared memory in K order and write Y.
 //
-// What bounds it: with ~2.2 instructions per value the dequantisation of a dense tile keeps the SM's four issue
-// ports busy for ~350 cycles, about what its 8 448 bytes take to arrive at this SM's share of the HBM bandwidth,
-// so the kernel sits where the ALU and the HBM roofs meet (2:4 tiles: 64 values per row, memory-bound).
+// What bounds it: ~2 instructions per dequantised value, i.e. ~260 issue cycles per dense tile and SM against the
+// ~170 cycles its 8 448 bytes take at this SM's share of the HBM bandwidth: the dense kind is bound by the ALUs,
+// the 2:4 kind (half the values per byte of metadata-carrying payload) sits closer to the memory roof.
 //
+// One CTA per SM by construction: the CTA allocates all 512 TMEM columns, and two CTAs of different clusters on one
+// SM could each hold the columns the other's cluster peer waits for; the rings are sized so that two CTAs do not fit.
 // Same bounded waits, table checks, launch flags and determinism as the other decode kernels; M <= 16.
 #include "sm100_ptx.cuh"
 
 namespace patch {
 
 namespace dq {
-constexpr int kRaw = 8;                                   // payload ring
-constexpr int kOps = 3;                                   // operand ring
-constexpr int kDequantWarps = 8;
-constexpr int kThreads = 192 + 32 * kDequantWarps;
+constexpr int kRaw = 16;                                  // payload ring
+constexpr int kBatch = 4;                                 // tiles requested per producer round
+constexpr int kGroups = 6;                                // dequantising groups = operand stages in TMEM
+constexpr int kThreads = 160 + 128 * kGroups;
 constexpr uint32_t kRawBytes = kDenseQ4Bytes;             // slot size: the larger of the two payloads
 constexpr uint32_t kXAtomBytes = 16 * 128, kXBytes = 2 * kXAtomBytes;
-constexpr uint32_t kOpBytes = kDenseBytes;                // two atoms, or one atom + metadata
-constexpr uint32_t kXOffset = kOps * kOpBytes;
+constexpr uint32_t kPartialBytes = 128 * 16 * 4;          // fp32 partial [128 rows][16 tokens]
+constexpr uint32_t kXOffset = kPartialBytes;
 constexpr uint32_t kRawOffset = kXOffset + kRaw * kXBytes;
 constexpr uint32_t kBarrierOffset = kRawOffset + kRaw * kRawBytes;
-constexpr uint32_t kSmemBytes = kBarrierOffset + 256 + 1024;
-constexpr uint32_t kTmemCols = 32;                        // 16 accumulator columns + 4 metadata columns per operand stage
+constexpr uint32_t kSmemBytes = kBarrierOffset + 512 + 1024;
+constexpr uint32_t kTmemCols = 512;                       // accumulator 16g, metadata 96 + 4g, operand stage 128 + 64g
 constexpr uint32_t kPartialRowBytes = 16 * 4;
-static_assert(16 + 4 * kOps <= kTmemCols, "TMEM columns");
+static_assert(128 + 64 * kGroups <= kTmemCols && 16 * kGroups <= 96 && 96 + 4 * kGroups <= 128, "TMEM columns");
 static_assert(kRawBytes % 128 == 0 && kSparseQ4Bytes <= kRawBytes, "payload slots");
-static_assert(kSmemBytes <= 227 * 1024, "shared memory");
+static_assert(kSmemBytes <= 227 * 1024 && 2 * kSmemBytes > 228 * 1024, "one CTA per SM, see above");
+static_assert(kRaw <= 16 && kGroups <= 8 && kThreads <= 1024, "barrier block, CTA size");
+static_assert(32 % kBatch == 0 && kRaw % kBatch == 0 && kRaw / kBatch <= 8, "producer rounds");
 
 __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -54,8 +67,37 @@ __device__ __forceinline__ float4 ld_peer_f4(uint32_t saddr, uint32_t rank) {
     asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
     return v;
 }
-// generic-proxy writes to shared memory become visible to the async proxy (tcgen05.mma, tcgen05.cp)
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// 16 registers per thread -> 32 lanes x 16 consecutive 32-bit columns (thread = lane)
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem]: lane = row of A, a 32-bit column holds two consecutive K elements
+__device__ __forceinline__ void mma_dense_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_sparse_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t e_tmem,
+                                              uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], [%1], %2, [%3], %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// true in one lane of the (converged) warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+// hardware barrier `id` over the 128 threads of a group
+__device__ __forceinline__ void group_barrier(int id) { asm volatile("barrier.cta.sync %0, 128;" ::"r"(id) : "memory"); }
 
 // A table entry of a 4-bit weight, checked before a byte of it is requested: the kind must be one of the two
 // 4-bit kinds and the payload must lie inside the blob; otherwise the status word says so and the blob's first
@@ -69,24 +111,32 @@ __device__ __forceinline__ void sanitize_q4_tile(uint32_t& kind, uint32_t& off16
     }
 }
 
-// Eight codes -> eight bf16 values (one 16-byte chunk of an atom).  s2 = the row's scale in both halves.
-__device__ __forceinline__ uint4 dequant_word(uint32_t w, __nv_bfloat162 s2) {
+// Eight codes -> eight bf16 values in four registers.  s2 = the row's scale in both halves.
+__device__ __forceinline__ void dequant_word(uint32_t w, __nv_bfloat162 s2, uint32_t* out) {
     const uint32_t kMagic = 0x43004300u;                         // bf16 128.0 twice: 128 + n in the low mantissa bits
     const uint32_t kBias = 0x43084308u;                          // bf16 136.0 twice
     const __nv_bfloat162 bias = *reinterpret_cast<const __nv_bfloat162*>(&kBias);
-    uint32_t out[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        const uint32_t p = ((w >> (4 * j)) & 0x000F000Fu) | kMagic;
+        uint32_t p;                                              // ((w >> 4j) & 0x000F000F) | magic in one instruction
+        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(p) : "r"(w >> (4 * j)), "r"(0x000F000Fu), "r"(kMagic));
         const __nv_bfloat162 v = __hmul2(__hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p), bias), s2);
         out[j] = *reinterpret_cast<const uint32_t*>(&v);
     }
-    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+// 32 codes (16 bytes) -> 16 columns of this thread's TMEM lane
+__device__ __forceinline__ void dequant_store16(uint4 cw, __nv_bfloat162 s2, uint32_t taddr) {
+    uint32_t v[16];
+    dequant_word(cw.x, s2, v);
+    dequant_word(cw.y, s2, v + 4);
+    dequant_word(cw.z, s2, v + 8);
+    dequant_word(cw.w, s2, v + 12);
+    tmem_st16(taddr, v);
 }
 }  // namespace dq
 
 template <bool WSTATIC, bool XSTATIC>
-__global__ void __launch_bounds__(dq::kThreads)
+__global__ void __launch_bounds__(dq::kThreads, 1)
 decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                  uint32_t pay0_16, uint32_t end16, int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy,
                  int* status_dev) {
@@ -95,15 +145,15 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
 
-    const uint32_t bar_raw_full = smem_base + kBarrierOffset;     // kRaw x 8 B
-    const uint32_t bar_raw_empty = bar_raw_full + 64;             // kRaw x 8 B
-    const uint32_t bar_op_full = bar_raw_empty + 64;              // kOps x 8 B (4 reserved)
-    const uint32_t bar_op_empty = bar_op_full + 32;
-    const uint32_t bar_acc_full = bar_op_empty + 32;
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kBarrierOffset + 200);
+    const uint32_t bar_raw_full = smem_base + kBarrierOffset;     // 16 x 8 B reserved for each array
+    const uint32_t bar_raw_empty = bar_raw_full + 128;
+    const uint32_t bar_x_full = bar_raw_empty + 128;              // kRaw / kBatch x 8 B (8 reserved)
+    const uint32_t bar_op_empty = bar_x_full + 64;                // 8 x 8 B reserved
+    const uint32_t bar_acc_full = bar_op_empty + 64;
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kBarrierOffset + 392);
     uint32_t* tmem_slot = misc;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 1);
-    volatile uint32_t* slot_kind = misc + 4;                      // [kRaw]
+    volatile uint32_t* slot_kind = misc + 2;                      // [kRaw] (392 + 8 + 64 <= 512)
 
     grid_launch_dependents();
 
@@ -111,31 +161,33 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     const uint32_t s = cluster_ctarank();
     const int tn = blockIdx.x / S;
     const int k0 = int(int64_t(s) * TK / S), k1 = int(int64_t(s + 1) * TK / S), n_tiles = k1 - k0;
+    const int n_groups = n_tiles < kGroups ? n_tiles : kGroups;   // groups that get a tile: their accumulators count
     const TileDesc* table = reinterpret_cast<const TileDesc*>(blob + table_off) + int64_t(tn) * TK + k0;
 
-    if (threadIdx.x == 64) {
+    if (threadIdx.x == 32) {
         for (int i = 0; i < kRaw; ++i) {
             mbar_init(bar_raw_full + 8 * i, 1);
-            mbar_init(bar_raw_empty + 8 * i, kDequantWarps + 1);   // the dequantising warps (codes) + the MMAs (X)
+            mbar_init(bar_raw_empty + 8 * i, 1);                   // the tile's MMAs (they follow the group's reads)
         }
-        for (int i = 0; i < kOps; ++i) {
-            mbar_init(bar_op_full + 8 * i, kDequantWarps);
-            mbar_init(bar_op_empty + 8 * i, 1);
-        }
-        mbar_init(bar_acc_full, 1);
+        for (int i = 0; i < kRaw / kBatch; ++i) mbar_init(bar_x_full + 8 * i, 1);
+        for (int i = 0; i < kGroups; ++i) mbar_init(bar_op_empty + 8 * i, 1);
+        mbar_init(bar_acc_full, n_groups > 0 ? n_groups : 1);
         *abort_flag = 0;
         mbar_init_fence();
         tma_prefetch_map(&tmap_x);
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_meta = tmem_base + 16;
+    const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
 
     if (warp == 0) {
         // ---------------- producer ----------------
+        // Lanes 0 .. kBatch-1 each request one tile per round: the round's waits, barrier updates and copy
+        // instructions are issued once for all of them (one lane per tile took ~1 000 cycles a tile, four times
+        // what the tile's bytes take to arrive).  A round goes out when its last slot is free, so between
+        // kRaw - kBatch and kRaw tiles are in flight.
         if constexpr (!WSTATIC) grid_dependency_wait();
         const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
         TileDesc mine = TileDesc{0, 0, 0, 0};
@@ -144,137 +196,148 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
         // payloads of the first kRaw tiles may be requested before the grid dependency is resolved (WSTATIC);
         // their activations follow once it is (unless XSTATIC)
         const int n_early = (WSTATIC && !XSTATIC) ? (n_tiles < kRaw ? n_tiles : kRaw) : 0;
-        for (int i = 0; i < n_tiles && ok; ++i) {
-            if ((i & 31) == 0 && i + lane < n_tiles) mine = table[i + lane];
-            uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, i & 31);
-            uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, i & 31);
-            if (lane == 0) {
+        for (int base = 0; base < n_tiles && ok; base += kBatch) {
+            if ((base & 31) == 0 && base + lane < n_tiles) mine = table[base + lane];
+            const int i = base + lane, src = i & 31;               // kBatch divides 32: the round's entries sit in one load
+            uint32_t kind = __shfl_sync(0xFFFFFFFFu, mine.kind, src);
+            uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.payload_off16, src);
+            bool mine_ok = true;
+            if (lane < kBatch) {
                 const int slot = i % kRaw;
-                sanitize_q4_tile(kind, off16, pay0_16, end16, status_dev);
-                const uint32_t wbytes = kind == PATCH_TILE_DENSE_Q4 ? kDenseQ4Bytes : kSparseQ4Bytes;
-                const uint32_t full = bar_raw_full + 8 * slot;
-                if (i >= kRaw) ok = mbar_wait(bar_raw_empty + 8 * slot, (uint32_t(i / kRaw) & 1u) ^ 1u, abort_flag, status_dev);
-                if (ok) {
+                // the slot's previous tile (also where this round has no tile for it: its X buffer is overwritten)
+                if (i >= kRaw) mine_ok = mbar_wait_suspended(bar_raw_empty + 8 * slot, (uint32_t(i / kRaw) & 1u) ^ 1u, abort_flag, status_dev);
+                if (mine_ok && i < n_tiles) {
+                    sanitize_q4_tile(kind, off16, pay0_16, end16, status_dev);
+                    const uint32_t wbytes = kind == PATCH_TILE_DENSE_Q4 ? kDenseQ4Bytes : kSparseQ4Bytes;
+                    const uint32_t full = bar_raw_full + 8 * slot;
                     slot_kind[slot] = kind;
-                    mbar_expect_tx(full, wbytes + kXBytes);
+                    mbar_expect_tx(full, wbytes);
                     tma_bulk_load(smem_base + kRawOffset + slot * kRawBytes, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
-                    if (i < n_early) {
-                        if (i + 1 == n_early) {
-                            grid_dependency_wait();
-                            for (int j = 0; j < n_early; ++j) {
-                                const uint32_t sX = smem_base + kXOffset + j * kXBytes;
-                                tma_tile_load(sX, &tmap_x, (k0 + j) * kTile, 0, bar_raw_full + 8 * j, pol_x);
-                                tma_tile_load(sX + kXAtomBytes, &tmap_x, (k0 + j) * kTile + 64, 0, bar_raw_full + 8 * j, pol_x);
-                            }
-                        }
-                    } else {
-                        const uint32_t sX = smem_base + kXOffset + slot * kXBytes;
-                        tma_tile_load(sX, &tmap_x, (k0 + i) * kTile, 0, full, pol_x);
-                        tma_tile_load(sX + kXAtomBytes, &tmap_x, (k0 + i) * kTile + 64, 0, full, pol_x);
-                    }
-                    issued = i + 1;
                 }
             }
-            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            ok = __all_sync(0xFFFFFFFFu, mine_ok);
+            if (ok) issued = base + kBatch < n_tiles ? base + kBatch : n_tiles;
+            // the round's activations: one copy of 2 kBatch atoms into the X buffers of its kBatch slots
+            if (ok && lane == 0 && base >= n_early) {
+                const uint32_t xb = bar_x_full + 8 * ((base / kBatch) % (kRaw / kBatch));
+                mbar_expect_tx(xb, kBatch * kXBytes);
+                tma_tile_load_3d(smem_base + kXOffset + (base % kRaw) * kXBytes, &tmap_x, 0, 0, (k0 + base) * 2, xb, pol_x);
+            }
+            if (ok && base < n_early && base + kBatch >= n_early) {
+                // the last early payload is on its way: now the activations of all early rounds
+                grid_dependency_wait();
+                if (lane * kBatch < n_early) {
+                    const uint32_t xb = bar_x_full + 8 * lane;
+                    mbar_expect_tx(xb, kBatch * kXBytes);
+                    tma_tile_load_3d(smem_base + kXOffset + lane * kBatch * kXBytes, &tmap_x, 0, 0, (k0 + lane * kBatch) * 2, xb, pol_x);
+                }
+            }
         }
         if (lane == 0 && *abort_flag) {
-            // drain: wait (bounded) until the copies this thread started have landed
+            // drain: wait (bounded) until the copies this warp started have landed
             const uint64_t tstart = global_timer_ns();
             for (int j = issued > kRaw ? issued - kRaw : 0; j < issued; ++j) {
                 const uint32_t bar = bar_raw_full + 8 * (j % kRaw), parity = uint32_t(j / kRaw) & 1u;
                 while (!mbar_try_wait(bar, parity) && global_timer_ns() - tstart < kDrainLimitNs) {}
+                const uint32_t xb = bar_x_full + 8 * ((j / kBatch) % (kRaw / kBatch));
+                while (!mbar_try_wait(xb, parity) && global_timer_ns() - tstart < kDrainLimitNs) {}
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            bool ok = true;
-            for (int i = 0; i < n_tiles && ok; ++i) {
-                const int slot = i % kRaw, op = i % kOps;
-                ok = mbar_wait(bar_op_full + 8 * op, uint32_t(i / kOps) & 1u, abort_flag, status_dev);
-                // the slot's activations arrived with its payload, which the dequantising warps have consumed: this
-                // wait returns at once, and makes the async-proxy writes of X visible to this thread's MMAs
-                if (ok) ok = mbar_wait(bar_raw_full + 8 * slot, uint32_t(i / kRaw) & 1u, abort_flag, status_dev);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t sW = smem_base + op * kOpBytes, sX = smem_base + kXOffset + slot * kXBytes;
-                issue_tile_mma<16>(slot_kind[slot] & 1u, sW, sX, kXAtomBytes, tmem_base, tmem_meta + 4 * op, i == 0);
-                mma_commit(bar_op_empty + 8 * op);
-                mma_commit(bar_raw_empty + 8 * slot);
+    } else if (warp >= 5) {
+        // ---------------- group g: dequantise tile i into its operand stage, then multiply ----------------
+        const int g = (warp - 5) >> 2;
+        const bool issuer = ((warp - 5) & 3) == (g & 3);           // one warp of the group also issues its MMAs (the groups' issuers sit on different schedulers)
+        const uint32_t quarter = warp & 3u, r = quarter * 32u + lane;         // tile row = TMEM lane
+        const uint32_t a_tmem = tmem_base + 128u + 64u * uint32_t(g);
+        const uint32_t a_lane = a_tmem + ((quarter * 32u) << 16);
+        const uint32_t acc_tmem = tmem_base + 16u * uint32_t(g), e_tmem = tmem_base + 96u + 4u * uint32_t(g);
+        constexpr uint32_t idesc_d = instr_desc(16, false), idesc_s = instr_desc(16, true);
+        for (int i = g, n = 0; i < n_tiles; i += kGroups, ++n) {
+            const int slot = i % kRaw;
+            // One thread of the group waits for the tile's payload and for the MMAs that read the operand stage; the
+            // other 127 wait on a hardware barrier, which costs no issue slots (24 polling warps did: a third of
+            // all instructions).  The barrier also tells everyone if the wait was given up.
+            bool failed = false;
+            if (issuer && lane == 0) {
+                failed = !mbar_wait_suspended(bar_raw_full + 8 * slot, uint32_t(i / kRaw) & 1u, abort_flag, status_dev);
+                if (!failed)
+                    failed = !mbar_wait_suspended(bar_x_full + 8 * ((i / kBatch) % (kRaw / kBatch)), uint32_t(i / kRaw) & 1u,
+                                                  abort_flag, status_dev);
+                if (!failed && n > 0)
+                    failed = !mbar_wait_suspended(bar_op_empty + 8 * g, (uint32_t(n) & 1u) ^ 1u, abort_flag, status_dev);
             }
-            if (ok && n_tiles > 0) mma_commit(bar_acc_full);
-        }
-        __syncwarp();
-    } else if (warp >= 6) {
-        // ---------------- dequantisation: payload slot -> operand stage ----------------
-        const uint32_t dt = threadIdx.x - 192;                    // 0 .. 32 * kDequantWarps - 1
-        constexpr uint32_t kDt = 32 * kDequantWarps;
-        bool ok = true;
-        for (int i = 0; i < n_tiles && ok; ++i) {
-            const int slot = i % kRaw, op = i % kOps;
-            if (lane == 0) {
-                ok = mbar_wait(bar_raw_full + 8 * slot, uint32_t(i / kRaw) & 1u, abort_flag, status_dev);
-                if (ok && i >= kOps)
-                    ok = mbar_wait(bar_op_empty + 8 * op, (uint32_t(i / kOps) & 1u) ^ 1u, abort_flag, status_dev);
-            }
-            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-            if (!ok) break;
+            if (barrier_any(failed, 1 + g, 128)) break;
+            tc_fence_after();                                      // the MMAs that read this stage have completed
+            const uint32_t sRaw = smem_base + kRawOffset + slot * kRawBytes;
             const uint8_t* raw = smem + kRawOffset + slot * kRawBytes;
-            uint8_t* dst = smem + op * kOpBytes;
-            const uint32_t* words = reinterpret_cast<const uint32_t*>(raw);
-            if (slot_kind[slot] == PATCH_TILE_DENSE_Q4) {
-                const uint16_t* scales = reinterpret_cast<const uint16_t*>(raw + kDenseQ4CodeBytes);
+            const uint4* codes = reinterpret_cast<const uint4*>(raw) + r;      // unit j of the row at codes[128 j]
+            const bool dense = slot_kind[slot] == PATCH_TILE_DENSE_Q4;
+            if (dense) {
+                const uint32_t sb = reinterpret_cast<const uint16_t*>(raw + kDenseQ4CodeBytes)[r] * 0x00010001u;
+                const __nv_bfloat162 s2 = *reinterpret_cast<const __nv_bfloat162*>(&sb);
 #pragma unroll
-                for (uint32_t it = 0; it < 2048 / kDt; ++it) {
-                    const uint32_t idx = it * kDt + dt, r = idx >> 4, c = idx & 15u;
-                    const uint32_t sb = scales[r] * 0x00010001u;
-                    const uint4 v = dequant_word(words[idx], *reinterpret_cast<const __nv_bfloat162*>(&sb));
-                    *reinterpret_cast<uint4*>(dst + (c >> 3) * kAtomBytes + atom_chunk_offset(r, c & 7u)) = v;
-                }
+                for (int j = 0; j < 4; ++j) dequant_store16(codes[128 * j], s2, a_lane + 16u * j);
             } else {
-                const uint16_t* scales = reinterpret_cast<const uint16_t*>(raw + kSparseQ4CodeBytes + kMetaBytes);
+                const uint32_t sb = reinterpret_cast<const uint16_t*>(raw + kSparseQ4CodeBytes + kMetaBytes)[r] * 0x00010001u;
+                const __nv_bfloat162 s2 = *reinterpret_cast<const __nv_bfloat162*>(&sb);
 #pragma unroll
-                for (uint32_t it = 0; it < 1024 / kDt; ++it) {
-                    const uint32_t idx = it * kDt + dt, r = idx >> 3, c = idx & 7u;
-                    const uint32_t sb = scales[r] * 0x00010001u;
-                    const uint4 v = dequant_word(words[idx], *reinterpret_cast<const __nv_bfloat162*>(&sb));
-                    *reinterpret_cast<uint4*>(dst + atom_chunk_offset(r, c)) = v;
-                }
-                // the metadata block follows the atom, as in a bf16 2:4 payload
-                if (dt < kMetaBytes / 16)
-                    reinterpret_cast<uint4*>(dst + kAtomBytes)[dt] = reinterpret_cast<const uint4*>(raw + kSparseQ4CodeBytes)[dt];
+                for (int j = 0; j < 2; ++j) dequant_store16(codes[128 * j], s2, a_lane + 16u * j);
             }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar_op_full + 8 * op);
-                mbar_arrive(bar_raw_empty + 8 * slot);
+            tmem_st_wait();
+            tc_fence_before();
+            group_barrier(8 + g);                                  // all four warps have written their rows
+            if (issuer) {
+                tc_fence_after();
+                if (elect_one()) {
+                    {
+                        const uint64_t dB = desc_kmajor_sw128(smem_base + kXOffset + slot * kXBytes);
+                        if (dense) {
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks) {       // K = 16 per MMA: 8 columns of A, 32 B of every X row
+                                const uint64_t b = dB + uint64_t(((ks >> 2) * kXAtomBytes + (ks & 3) * 32) >> 4);
+                                mma_dense_ta(acc_tmem, a_tmem + 8u * ks, b, idesc_d, !(n == 0 && ks == 0));
+                            }
+                        } else {
+                            tmem_copy_128x128b(e_tmem, desc_rows16(sRaw + kSparseQ4CodeBytes));
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {       // K = 32 per MMA: 16 kept values = 8 columns of A
+                                const uint64_t b = dB + uint64_t(((ks >> 1) * kXAtomBytes + (ks & 1) * 64) >> 4);
+                                mma_sparse_ta(acc_tmem, a_tmem + 8u * ks, b, e_tmem + (ks & 2), idesc_s | uint32_t(ks & 1),
+                                              !(n == 0 && ks == 0));
+                            }
+                        }
+                        mma_commit(bar_op_empty + 8 * g);
+                        mma_commit(bar_raw_empty + 8 * slot);
+                        if (i + kGroups >= n_tiles) mma_commit(bar_acc_full);    // the group's last tile
+                    }
+                }
+                __syncwarp();
             }
         }
     } else {
-        // ---------------- epilogue warps 2..5: own partial -> own shared memory ----------------
-        // The operand ring is free once the accumulator is complete; the partial [128 rows][16 tokens] fp32
-        // takes the first 8 KB of it.
+        // ---------------- epilogue warps 1..4: sum of the groups' accumulators -> own shared memory ----------------
         const uint32_t quad = warp & 3u, row = quad * 32 + lane;
         bool ok = true;
         if (n_tiles > 0) {
-            if (lane == 0) ok = mbar_wait_relaxed(bar_acc_full, 0, abort_flag, status_dev);
+            if (lane == 0) ok = mbar_wait_suspended(bar_acc_full, 0, abort_flag, status_dev);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             tc_fence_after();
         }
-        float4* dst = reinterpret_cast<float4*>(smem + row * kPartialRowBytes);
-        uint32_t v[16];
-        if (n_tiles > 0 && ok) {
-            tmem_ld16(tmem_base + ((quad * 32u) << 16), v);
-            tmem_ld_wait();
-        } else {
+        float acc[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = 0u;
+        for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
+        if (ok) {
+            for (int gq = 0; gq < n_groups; ++gq) {                // ascending group: a fixed summation order
+                uint32_t v[16];
+                tmem_ld16(tmem_base + ((quad * 32u) << 16) + 16u * uint32_t(gq), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] = gq == 0 ? __uint_as_float(v[j]) : acc[j] + __uint_as_float(v[j]);
+            }
         }
+        float4* dst = reinterpret_cast<float4*>(smem + row * kPartialRowBytes);
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]),
-                                 __uint_as_float(v[4 * q + 3]));
+        for (int q = 0; q < 4; ++q) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
         tc_fence_before();
     }
 
@@ -282,9 +345,9 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     __syncthreads();
     dq::cluster_barrier();
 
-    if (warp >= 2 && warp < 6) {
+    if (warp >= 1 && warp < 5) {
         // ---------------- reduction: this CTA finishes rows [128 s / S, 128 (s + 1) / S) ----------------
-        const int e = threadIdx.x - 64;                            // 0..127
+        const int e = threadIdx.x - 32;                            // 0..127
         const int rows = kTile / S;                                // S in {1, 2, 4, 8}
         const int n_out = rows * 4;                                // groups of four tokens
         grid_dependency_wait();                                    // Y may be in use by the preceding kernel
@@ -312,7 +375,7 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     tc_fence_before();
     __syncthreads();
     dq::cluster_barrier();
-    if (warp == 1) tmem_dealloc(tmem_base, dq::kTmemCols);
+    if (warp == 0) tmem_dealloc(tmem_base, dq::kTmemCols);
 }
 
 template <bool WSTATIC, bool XSTATIC>
@@ -344,7 +407,7 @@ static int launch_q4_t(const CUtensorMap& map, const patch_layout_t* L, const ui
 int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                      __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic) {
     CUtensorMap map;
-    int rc = make_x_tensor_map(&map, X, ldx, M, L->K, 16);
+    int rc = make_x_chunk_tensor_map(&map, X, ldx, M, L->K, 16, 2 * dq::kBatch);
     if (rc) return rc;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     // The smallest power-of-two split of K that makes at least 128 CTAs, at most 8 and at most TK.

@@ -217,6 +217,21 @@ int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int
     return r == CUDA_SUCCESS ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
+// X as a 3-D tensor (column inside a 64-column chunk, token row, chunk): a box of `chunks` chunks lands in shared
+// memory as `chunks` consecutive [n_tok x 128 B] swizzled atoms -- the activations of chunks / 2 weight tiles in one copy.
+int make_x_chunk_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok, int chunks) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return PATCH_ERR_CUDA;
+    const cuuint64_t dims[3] = {64, cuuint64_t(M), cuuint64_t(K / 64)};
+    const cuuint64_t strides[2] = {cuuint64_t(ldx) * 2, 128};
+    const cuuint32_t box[3] = {64, cuuint32_t(n_tok), cuuint32_t(chunks)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(X), dims, strides, box,
+                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PATCH_OK : PATCH_ERR_CUDA;
+}
+
 int make_blob_tensor_map(CUtensorMap* map, const uint8_t* blob, uint64_t total_bytes, int box_rows) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return PATCH_ERR_CUDA;

@@ -237,9 +237,11 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
 // 4-bit kinds.  One warp per tile row, lane g holds the row's g-th group of four consecutive elements.
 //   scale  s = bf16(max|v| / 7) over the row's stored values (all 128, or the 64 the 2:4 selection keeps)
 //   code   q + 8 with q = clamp(rint(v / s), -7, 7), 0 where s = 0; fp32 arithmetic, IEEE division
-// Codes are stored eight to a 32-bit word, values 8w .. 8w + 7 of the row's stored values in word w: the even
-// ones in nibbles 0..3, the odd ones in nibbles 4..7, so that (word >> 4j) & 0x000F000F is the pair (2j, 2j + 1)
-// in the two halves of a register -- what the dequantising GEMM kernel turns into two bf16 with one instruction.
+// Codes are stored eight to a 32-bit word, in the row's order of stored values: the even ones of a word in nibbles
+// 0..3, the odd ones in nibbles 4..7, so that (word >> 4j) & 0x000F000F is the pair (2j, 2j + 1) in the two halves
+// of a register -- what the dequantising GEMM kernel turns into two bf16 with one instruction.  Four words (32
+// values) make a 16-byte unit; unit j of tile row r lives at byte (128 j + r) * 16, so the 32 threads of a warp
+// that each own a row read 512 consecutive bytes.
 
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
 __device__ __forceinline__ uint32_t q4_nibble(float v, float s) {
@@ -291,7 +293,7 @@ pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __r
             for (int i = 0; i < 2; ++i) word |= q4_nibble(v[i], s) << (4 * q4_nibble_slot(2 * lane + i));
             word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
             word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-            if ((lane & 3u) == 0) reinterpret_cast<uint32_t*>(codes)[r * 8 + (lane >> 2)] = word;
+            if ((lane & 3u) == 0) reinterpret_cast<uint32_t*>(codes)[((lane >> 4) * 128 + r) * 4 + ((lane & 15u) >> 2)] = word;
             // position codes of the four groups of a 16-column chunk -> 16 bits of metadata (hardware order)
             uint32_t code = (i0 | (i1 << 2)) << (4 * (lane & 3u));
             code |= __shfl_xor_sync(0xFFFFFFFFu, code, 1);
@@ -303,7 +305,7 @@ pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __r
 #pragma unroll
             for (int i = 0; i < 4; ++i) word |= q4_nibble(v[i], s) << (4 * q4_nibble_slot(4 * lane + i));
             word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-            if ((lane & 1u) == 0) reinterpret_cast<uint32_t*>(codes)[r * 16 + (lane >> 1)] = word;
+            if ((lane & 1u) == 0) reinterpret_cast<uint32_t*>(codes)[((lane >> 3) * 128 + r) * 4 + ((lane & 7u) >> 1)] = word;
         }
     }
 }
@@ -324,7 +326,7 @@ __device__ __forceinline__ void unpack_q4_tile(const TileDesc& d, const uint8_t*
         const float s = bf16_bits_to_f32(scales[r]);
         uint32_t out[4] = {0, 0, 0, 0};
         if (sparse) {
-            const uint32_t word = codes[r * 8 + (lane >> 2)];
+            const uint32_t word = codes[((lane >> 4) * 128 + r) * 4 + ((lane & 15u) >> 2)];
             const uint32_t u = lane >> 2;
             const uint32_t Lr = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
             const uint32_t code = *reinterpret_cast<const uint16_t*>(meta + Lr * 16 + j * 4 + hi * 2);
@@ -334,7 +336,7 @@ __device__ __forceinline__ void unpack_q4_tile(const TileDesc& d, const uint8_t*
 #pragma unroll
             for (uint32_t p = 0; p < 4; ++p) out[p] = p == i0 ? a : p == i1 ? b : 0u;
         } else {
-            const uint32_t word = codes[r * 16 + (lane >> 1)];
+            const uint32_t word = codes[((lane >> 3) * 128 + r) * 4 + ((lane & 7u) >> 1)];
 #pragma unroll
             for (uint32_t p = 0; p < 4; ++p) out[p] = q4_dequant_bits((word >> (4 * q4_nibble_slot(4 * lane + p))) & 0xFu, s);
         }

@@ -29,6 +29,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// The same with a suspend-time hint: the thread may stay suspended in hardware for up to `hint_ns` (it is woken
+// when the phase completes), so a long wait costs few issue slots.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -85,6 +96,24 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
     }
 }
 
+// Bounded wait for warps that share their issue port with busy ones: suspended in hardware between polls.
+__device__ __forceinline__ bool mbar_wait_suspended(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                    int* status_dev) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
+        if ((spin & 3u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (status_dev) atomicCAS(status_dev, PATCH_OK, PATCH_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
 // Hardware barrier `id` over `threads` threads of the CTA that also ORs a predicate (the same decision in all of them).
 __device__ __forceinline__ bool barrier_any(bool pred, int id, int threads) {
     uint32_t out;
@@ -129,6 +158,14 @@ __device__ __forceinline__ void tma_tile_load(uint32_t dst, const CUtensorMap* m
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
         " [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
+}
+// 3-D tiled copy
+__device__ __forceinline__ void tma_tile_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -342,6 +379,9 @@ __device__ __forceinline__ void store_fragment_transposed(const uint32_t (&v)[16
 // Host: tensor map over X [M x ldx] bf16 with a box of 64 columns (128 B) x n_tok rows,
 // 128-byte swizzle, zero fill outside the matrix.
 int make_x_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok);
+// Host: the same matrix as (column in a 64-column chunk, token row, chunk) with a box of `chunks` chunks: one copy
+// brings `chunks` consecutive atoms of n_tok rows x 128 B.
+int make_x_chunk_tensor_map(CUtensorMap* map, const __nv_bfloat16* X, int64_t ldx, int64_t M, int64_t K, int n_tok, int chunks);
 // Host: tensor map over a packed blob seen as rows of 256 bytes, box = `box_rows` whole rows, no swizzle: a
 // tiled copy at row (byte offset / 256) lands in shared memory exactly like a linear copy of box_rows * 256 bytes.
 int make_blob_tensor_map(CUtensorMap* map, const uint8_t* blob, uint64_t total_bytes, int box_rows);

@@ -185,11 +185,16 @@ def test_table_entries_and_device_image_of_the_4bit_kinds(oracle):
     # (by hand below: codes 1..8 of one group, canonical bytes 21 43 65 87 -> the word 0x86427531: the odd values
     # 2,4,6,8 in nibbles 4..7 above the even values 1,3,5,7 in nibbles 0..3)
     # scales as they are; the metadata of a 4-bit 2:4 tile in the order of the bf16 2:4 kind; codes: value i of
-    # each group of eight in nibble (i % 2) * 4 + i // 2 of the group's 32-bit word
-    def image_codes(raw):
+    # each group of eight in nibble (i % 2) * 4 + i // 2 of the group's 32-bit word, and the 16-byte unit j (four
+    # words) of tile row r at byte (128 j + r) * 16
+    def image_codes(raw, vals=None):
         nib = np.stack([raw & 0xF, raw >> 4], axis=1).reshape(-1, 8).astype(np.uint32)     # canonical value order
         slot = np.array([(i % 2) * 4 + i // 2 for i in range(8)], np.uint32)
-        return (nib << (4 * slot)).sum(axis=1, dtype=np.uint32).view(np.uint8)
+        words = (nib << (4 * slot)).sum(axis=1, dtype=np.uint32)
+        if vals is None:
+            return words.view(np.uint8)
+        units = words.reshape(128, vals // 32, 4)                    # [row][unit][word]
+        return np.ascontiguousarray(units.transpose(1, 0, 2)).view(np.uint8).reshape(-1)
     assert image_codes(np.array([0x21, 0x43, 0x65, 0x87], np.uint8)).view(np.uint32)[0] == 0x86427531
     plain_img = oracle.device_image(oracle.pack(W, flags & 1)[0])
     plain_L = oracle.packed_size(N, K, flags & 1)
@@ -197,10 +202,10 @@ def test_table_entries_and_device_image_of_the_4bit_kinds(oracle):
     for t, kind in enumerate(flags.reshape(-1)):
         o = int(table[t, 1]) * 16
         if kind == 2:
-            assert (image[o:o + 8192] == image_codes(blob[o:o + 8192])).all()
+            assert (image[o:o + 8192] == image_codes(blob[o:o + 8192], 128)).all()
             assert (image[o + 8192:o + 8448] == blob[o + 8192:o + 8448]).all()
         elif kind == 3:
-            assert (image[o:o + 4096] == image_codes(blob[o:o + 4096])).all()
+            assert (image[o:o + 4096] == image_codes(blob[o:o + 4096], 64)).all()
             assert (image[o + 6144:o + 6400] == blob[o + 6144:o + 6400]).all()
             pm = int(ptable[t, 2]) * 16
             assert (image[o + 4096:o + 6144] == plain_img[pm:pm + 2048]).all()
