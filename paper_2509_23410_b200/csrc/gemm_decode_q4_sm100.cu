@@ -410,9 +410,20 @@ int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch
     int rc = make_x_chunk_tensor_map(&map, X, ldx, M, L->K, 16, 2 * dq::kBatch);
     if (rc) return rc;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
-    // The smallest power-of-two split of K that makes at least 128 CTAs, at most 8 and at most TK.
-    int S = 1;
-    while (S < 8 && TN * S < 128 && 2 * S <= TK) S *= 2;
+    // Split of K, as for the bf16 row-block schedule: few CTAs per GEMM (several GEMMs resident at once) when the
+    // caller declared the GEMM independent of its predecessor, at least 128 CTAs when it streams alone.
+    int S = decode_cluster_split(TN, TK);
+    if (!xstatic) {
+        // alone on the GPU, one CTA per SM: waves of CTAs x (tiles per CTA x ~0.23 us + ~4 us of set-up, pipeline
+        // fill and reduction), over the power-of-two splits
+        const int sms = sm_count();
+        double best = 1e300;
+        for (int s2 = 1; s2 <= 8 && s2 <= TK; s2 *= 2) {
+            const int waves = (TN * s2 + sms - 1) / sms;
+            const double t = waves * (double((TK + s2 - 1) / s2) * 0.23 + 4.0);
+            if (t < best) { best = t; S = s2; }
+        }
+    }
     if (wstatic && xstatic) return launch_q4_t<true, true>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);
     if (wstatic) return launch_q4_t<true, false>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);
     return launch_q4_t<false, false>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);

@@ -67,8 +67,8 @@ def test_pack_with_row_pitch_and_extreme_values(gpu, oracle):
 @pytest.mark.parametrize("p", [0.0, 1.0, 0.4])
 @pytest.mark.parametrize("N,K", [(128, 128), (256, 1152), (640, 384), (4096, 1024), (512, 8192)])
 def test_gemm_parity(gpu, oracle, N, K, M, p):
-    """Whole output against the oracle's matmul on the dequantised matrix; all three launch forms agree bit for
-    bit with themselves on a second launch (deterministic) and with each other (same summation order)."""
+    """Whole output against the oracle's matmul on the dequantised matrix, for all three launch forms (they may split
+    K differently, so they agree to the last bit only where the split is the same); each form repeats bit for bit."""
     torch, B = gpu
     W = inputs.weight(N, K, 33, "q4-gemm", N, K)
     X = inputs.activation(M, K, 33, "q4-gemm", N, K, M)
@@ -82,8 +82,9 @@ def test_gemm_parity(gpu, oracle, N, K, M, p):
         Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | promise)
         check_parity(oracle, Y, Y32, f"q4 N={N} K={K} M={M} p={p} promise={promise:#x}")
         assert (Y == Y16).mean() >= 0.99
+        assert (run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | promise) == Y).all()
         outs.append(Y)
-    assert (outs[0] == outs[1]).all() and (outs[0] == outs[2]).all()
+    assert (outs[0] == outs[1]).all()              # no promise / weights only: the same split of K
     assert (run_gemm(gpu, X, L, packed, B.VARIANT_MMA) == outs[0]).all()
 
 
