@@ -48,6 +48,8 @@ def workload_cases(name: str, stack_m: int = 1):
         cases = inputs.decode_cases()
         # all M=1 GEMMs first, then all M=16: a matrix is re-read only after ~0.66 GB of other weights
         return sorted(cases, key=lambda c: c["M"])
+    if name == "decode-q4":
+        return sorted(inputs.decode_q4_cases(), key=lambda c: c["M"])
     if name == "prefill":
         return sorted(inputs.prefill_cases(), key=lambda c: c["M"])
     if name == "13b":
@@ -68,8 +70,8 @@ def case_costs(case, layout):
     M, N, K = case["M"], case["N"], case["K"]
     T = (N // 128) * (K // 128)
     nbytes = layout.payload_bytes + 16 * T + M * K * 2 + M * N * 2
-    f_dense = 2.0 * M * 16384 * layout.n_dense
-    f_sparse = 2.0 * M * 16384 * layout.n_sparse
+    f_dense = 2.0 * M * 16384 * (layout.n_dense + layout.n_dense_q4)
+    f_sparse = 2.0 * M * 16384 * (layout.n_sparse + layout.n_sparse_q4)
     return dict(bytes=float(nbytes), flops=f_dense + f_sparse, f_dense=f_dense, f_sparse=f_sparse)
 
 
@@ -263,7 +265,8 @@ def per_case_table(torch, B, jobs, mode, peaks, variant=0):
         table.append(dict(name=j["case"]["name"], us=round(t * 1e6, 2),
                           eff_tflops=round(j["cost"]["flops"] / t / 1e12, 2), bound=b,
                           frac_spec=round(rs / t, 3), frac_measured=round(rm / t, 3),
-                          f_sparse=round(j["layout"].n_sparse / (j["layout"].n_sparse + j["layout"].n_dense), 3)))
+                          f_sparse=round((j["layout"].n_sparse + j["layout"].n_sparse_q4) /
+                                         ((j["layout"].N // 128) * (j["layout"].K // 128)), 3)))
         del copies, js, g
     return table
 
@@ -439,16 +442,21 @@ def run_ours(args):
         pack_secs += e0.elapsed_time(e1) * 1e-3
         pack_bytes += c["N"] * c["K"] * 2 + layout.total_bytes
         # the same with the tile flags already on the device: no host work, header and table built by a kernel
-        flags_dev = torch.from_numpy(np.ascontiguousarray(flags, dtype=np.uint8).reshape(-1)).to(dev)
-        packed2 = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
-        B.patch_pack_dev(W, flags_dev, out=packed2)                # warm
-        e0.record()
-        B.patch_pack_dev(W, flags_dev, out=packed2)
-        e1.record()
-        torch.cuda.synchronize()
-        pack_dev_secs += e0.elapsed_time(e1) * 1e-3
-        if not torch.equal(packed, packed2):
-            raise SystemExit("patch_pack_dev and patch_pack disagree")
+        # (bf16 kinds only; a 4-bit weight is packed from host flags)
+        packed2 = None
+        if c.get("q4"):
+            pack_dev_secs += e0.elapsed_time(e1) * 1e-3
+        else:
+            flags_dev = torch.from_numpy(np.ascontiguousarray(flags, dtype=np.uint8).reshape(-1)).to(dev)
+            packed2 = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
+            B.patch_pack_dev(W, flags_dev, out=packed2)                # warm
+            e0.record()
+            B.patch_pack_dev(W, flags_dev, out=packed2)
+            e1.record()
+            torch.cuda.synchronize()
+            pack_dev_secs += e0.elapsed_time(e1) * 1e-3
+            if not torch.equal(packed, packed2):
+                raise SystemExit("patch_pack_dev and patch_pack disagree")
         keep_w = args.check != "none" and not args.workload.startswith("stack")
         mats[key] = (layout, packed, flags, inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]) if keep_w else None)
         del W, packed2
@@ -548,7 +556,7 @@ def run_ours(args):
         if dom is None or t > dom[1]:
             dom = (M, t, js)
     dM, dt, djs = dom
-    kernel_name = B_kernel_name(dM, args.launch)
+    kernel_name = "decode_q4_kernel" if args.workload == "decode-q4" else B_kernel_name(dM, args.launch)
     bound = roofline_seconds(djs[0]["cost"], HBM_SPEC_GBS, DENSE_SPEC_TFLOPS, SPARSE_SPEC_TFLOPS)[1]
     per_launch = dt / len(djs)
     if bound == "hbm":
@@ -567,7 +575,13 @@ def run_ours(args):
                 traffic=load_traffic(kernel_name, alg) if bound == "hbm" else None, kernel=kernel_name, launches_timed=len(djs),
                 us_per_launch=per_launch * 1e6, peak_source=peaks["source"],
                 algorithmic_per_launch=alg)
-    if bound == "hbm":
+    if args.workload == "decode-q4":
+        # HBM is the roof the bytes are counted against; the kernel's own ceiling is lower: every stored value costs
+        # ~2 issue slots to dequantise (half-rate bf16x2 arithmetic among them), see the kernel's header
+        roof["note"] = ("4-bit payloads: algorithmic bytes are 0.52 B (dense) / 0.39 B (2:4) per weight element; the kernel "
+                        "dequantises into tensor memory and is bound by instruction issue before HBM")
+        roof["frac_of_8tbs"] = achieved / HBM_SPEC_GBS
+    elif bound == "hbm":
         roof["note"] = ("the measured peak is a copy (read + write) bandwidth; this kernel only reads, and a read-only "
                         "stream can exceed it (the ceiling is the 8 TB/s of frac_of_roofline_spec); ncu confirms that "
                         "every algorithmic byte is read from DRAM exactly once")
@@ -655,7 +669,8 @@ def run_ours(args):
         # whole calls, one per matrix, read + written bytes: patch_pack_dev (flags on the device, two kernels) and
         # patch_pack (flags on the host: table built on the host and copied from pageable memory, one kernel)
         "pack": {"gbs": pack_bytes / pack_dev_secs / 1e9, "frac_of_measured_hbm": pack_bytes / pack_dev_secs / 1e9 / peaks["hbm_gbs"],
-                 "entry": "patch_pack_dev", "host_flags_entry_gbs": pack_bytes / pack_secs / 1e9},
+                 "entry": "patch_pack" if args.workload == "decode-q4" else "patch_pack_dev",
+                 "host_flags_entry_gbs": pack_bytes / pack_secs / 1e9},
     }
     if cpu is not None:
         out["cpu_baseline"] = cpu
@@ -965,7 +980,8 @@ def run_masks(args):
 def workload_label(args):
     return {"13b": "llama2-13b linears", "stack": f"llama2-7b full linear stack, M={args.stack_m}",
             "stack-fused": f"llama2-7b full linear stack with q/k/v and gate/up stacked, M={args.stack_m}",
-            "single": "single 1024x1024 GEMM"}.get(args.workload, f"llama2-7b {args.workload} linears")
+            "single": "single 1024x1024 GEMM",
+            "decode-q4": "llama2-7b decode linears, every tile stored with 4-bit values"}.get(args.workload, f"llama2-7b {args.workload} linears")
 
 
 def B_kernel_name(M, launch="independent"):
@@ -992,7 +1008,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused", "block", "masks"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "13b", "single", "stack", "stack-fused", "block", "masks", "decode-q4"])
     ap.add_argument("--stack-m", type=int, default=1, help="tokens per GEMM of the 224-GEMM stack workload")
     ap.add_argument("--launch", default="independent", choices=["dependent", "independent"],
                     help="independent (default; true for this workload, whose GEMMs do not feed each other): "

@@ -125,6 +125,12 @@ def decode_cases():
     return out
 
 
+def decode_q4_cases():
+    """The decode linears with every tile stored with 4-bit values (tile kinds 2 and 3): the same shapes, 2:4-tile
+    fractions and seeded streams as decode_cases(), so the two workloads differ only in the payload format."""
+    return [dict(c, name=c["name"] + ".q4", q4=True) for c in decode_cases()]
+
+
 def prefill_cases():
     """7B prefill linears: 3 shapes x M in {512,2048,4096} x p in {0, .5, 1}."""
     out = []
@@ -178,7 +184,8 @@ def case_flags(case: dict, seed: int = MASTER_SEED) -> np.ndarray:
     """Tile flags of a case; a case made of stacked matrices concatenates its parts' flags along N."""
     if "parts" in case:
         return np.concatenate([tile_flags(q["N"], case["K"], q["p"], seed, *q["stream"]) for q in case["parts"]], axis=0)
-    return tile_flags(case["N"], case["K"], case["p"], seed, *case["stream"])
+    flags = tile_flags(case["N"], case["K"], case["p"], seed, *case["stream"])
+    return flags | 2 if case.get("q4") else flags          # bit 1: the tile's stored values are 4-bit codes
 
 
 def make_case_inputs(case: dict, seed: int = MASTER_SEED, M: int | None = None):
