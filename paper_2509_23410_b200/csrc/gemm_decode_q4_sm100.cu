@@ -30,17 +30,20 @@
 // ~170 cycles its 8 448 bytes take at this SM's share of the HBM bandwidth: the dense kind is bound by the ALUs,
 // the 2:4 kind (half the values per byte of metadata-carrying payload) sits closer to the memory roof.
 //
-// One CTA per SM by construction: the CTA allocates all 512 TMEM columns, and two CTAs of different clusters on one
-// SM could each hold the columns the other's cluster peer waits for; the rings are sized so that two CTAs do not fit.
+// Two CTAs per SM: while one is being set up, drains its last tiles or waits for the preceding kernel before it may
+// write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130).
+// A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
+// columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
+// shared memory.
 // Same bounded waits, table checks, launch flags and determinism as the other decode kernels; M <= 16.
 #include "sm100_ptx.cuh"
 
 namespace patch {
 
 namespace dq {
-constexpr int kRaw = 16;                                  // payload ring
+constexpr int kRaw = 8;                                   // payload ring
 constexpr int kBatch = 4;                                 // tiles requested per producer round
-constexpr int kGroups = 6;                                // dequantising groups = operand stages in TMEM
+constexpr int kGroups = 3;                                // dequantising groups = operand stages in TMEM
 constexpr int kThreads = 160 + 128 * kGroups;
 constexpr uint32_t kRawBytes = kDenseQ4Bytes;             // slot size: the larger of the two payloads
 constexpr uint32_t kXAtomBytes = 16 * 128, kXBytes = 2 * kXAtomBytes;
@@ -49,11 +52,11 @@ constexpr uint32_t kXOffset = kPartialBytes;
 constexpr uint32_t kRawOffset = kXOffset + kRaw * kXBytes;
 constexpr uint32_t kBarrierOffset = kRawOffset + kRaw * kRawBytes;
 constexpr uint32_t kSmemBytes = kBarrierOffset + 512 + 1024;
-constexpr uint32_t kTmemCols = 512;                       // accumulator 16g, metadata 96 + 4g, operand stage 128 + 64g
+constexpr uint32_t kTmemCols = 256;                       // accumulator 16g, metadata 48 + 4g, operand stage 64 + 64g
 constexpr uint32_t kPartialRowBytes = 16 * 4;
-static_assert(128 + 64 * kGroups <= kTmemCols && 16 * kGroups <= 96 && 96 + 4 * kGroups <= 128, "TMEM columns");
+static_assert(64 + 64 * kGroups <= kTmemCols && 16 * kGroups <= 48 && 48 + 4 * kGroups <= 64, "TMEM columns");
 static_assert(kRawBytes % 128 == 0 && kSparseQ4Bytes <= kRawBytes, "payload slots");
-static_assert(kSmemBytes <= 227 * 1024 && 2 * kSmemBytes > 228 * 1024, "one CTA per SM, see above");
+static_assert(2 * kSmemBytes <= 227 * 1024 && 3 * kSmemBytes > 228 * 1024 && 2 * kTmemCols <= 512, "two CTAs per SM, see above");
 static_assert(kRaw <= 16 && kGroups <= 8 && kThreads <= 1024, "barrier block, CTA size");
 static_assert(32 % kBatch == 0 && kRaw % kBatch == 0 && kRaw / kBatch <= 8, "producer rounds");
 
@@ -136,7 +139,7 @@ __device__ __forceinline__ void dequant_store16(uint4 cw, __nv_bfloat162 s2, uin
 }  // namespace dq
 
 template <bool WSTATIC, bool XSTATIC>
-__global__ void __launch_bounds__(dq::kThreads, 1)
+__global__ void __launch_bounds__(dq::kThreads, 2)
 decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                  uint32_t pay0_16, uint32_t end16, int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy,
                  int* status_dev) {
@@ -248,9 +251,9 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
         const int g = (warp - 5) >> 2;
         const bool issuer = ((warp - 5) & 3) == (g & 3);           // one warp of the group also issues its MMAs (the groups' issuers sit on different schedulers)
         const uint32_t quarter = warp & 3u, r = quarter * 32u + lane;         // tile row = TMEM lane
-        const uint32_t a_tmem = tmem_base + 128u + 64u * uint32_t(g);
+        const uint32_t a_tmem = tmem_base + 64u + 64u * uint32_t(g);
         const uint32_t a_lane = a_tmem + ((quarter * 32u) << 16);
-        const uint32_t acc_tmem = tmem_base + 16u * uint32_t(g), e_tmem = tmem_base + 96u + 4u * uint32_t(g);
+        const uint32_t acc_tmem = tmem_base + 16u * uint32_t(g), e_tmem = tmem_base + 48u + 4u * uint32_t(g);
         constexpr uint32_t idesc_d = instr_desc(16, false), idesc_s = instr_desc(16, true);
         for (int i = g, n = 0; i < n_tiles; i += kGroups, ++n) {
             const int slot = i % kRaw;
@@ -414,13 +417,13 @@ int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch
     // caller declared the GEMM independent of its predecessor, at least 128 CTAs when it streams alone.
     int S = decode_cluster_split(TN, TK);
     if (!xstatic) {
-        // alone on the GPU, one CTA per SM: waves of CTAs x (tiles per CTA x ~0.23 us + ~4 us of set-up, pipeline
-        // fill and reduction), over the power-of-two splits
+        // alone on the GPU, two CTAs per SM: waves of CTAs x (tiles per CTA x ~0.35 us, 0.46 us where two CTAs share
+        // an SM, + ~4 us of set-up, pipeline fill and reduction), over the power-of-two splits
         const int sms = sm_count();
         double best = 1e300;
         for (int s2 = 1; s2 <= 8 && s2 <= TK; s2 *= 2) {
-            const int waves = (TN * s2 + sms - 1) / sms;
-            const double t = waves * (double((TK + s2 - 1) / s2) * 0.23 + 4.0);
+            const int ctas = TN * s2, waves = (ctas + 2 * sms - 1) / (2 * sms);
+            const double t = waves * (double((TK + s2 - 1) / s2) * (ctas > sms ? 0.46 : 0.35) + 4.0);
             if (t < best) { best = t; S = s2; }
         }
     }
