@@ -994,7 +994,8 @@ def B_kernel_name(M, launch="independent"):
 # summarised in profiles/decode_cluster_kernel_llama7b_decode.md (1.055, 1.018, 1.007) and
 # profiles/decode_kernel_llama7b_decode.md (1.035, 1.029, 1.008).
 # Traffic grows in proportion to the payload, so the ratio scales to any launch of the kernel.
-NCU_TRAFFIC_RATIO = {"decode_kernel": 1.03, "decode_cluster_kernel": 1.03}
+# profiles/decode_q4_kernel_llama7b_decode_q4.md: 1.006, 1.006, 1.007 (reads only; nothing is written to DRAM).
+NCU_TRAFFIC_RATIO = {"decode_kernel": 1.03, "decode_cluster_kernel": 1.03, "decode_q4_kernel": 1.006}
 
 
 def load_traffic(kernel, algorithmic):

@@ -35,6 +35,10 @@
 // A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
 // columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
 // shared memory.
+// Tried on top of this and dropped (24-GEMM decode step, 0.130 ms): splitting the tile into two K-halves with
+// separate completion tracking, so that a group never waits for its own MMAs (0.142 ms: a third barrier and a second
+// issue sequence per tile cost more than the wait); dequantising the next tile's first 32 values before that wait
+// (0.138 ms: every warp polls again, registers spill); six groups in one CTA per SM (0.150 ms, see above).
 // Same bounded waits, table checks, launch flags and determinism as the other decode kernels; M <= 16.
 #include "sm100_ptx.cuh"
 
