@@ -197,8 +197,10 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  * Weights with 4-bit tiles: served for M <= 16 tokens (the decode case, where the bytes of the weight are
  * what the layer costs) and only if every tile is of a 4-bit kind; a dequantising kernel of its own, no
  * workspace.  Other M, and weights that mix bf16 and 4-bit tiles, return PATCH_ERR_SHAPE -- as do
- * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated, patch_gemm_noalloc and the host entry points
- * for such weights; patch_pack_dev / patch_pack_patterns report flags above 1 as PATCH_ERR_FLAG.
+ * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated and patch_gemm_noalloc for such weights (the host
+ * entry points follow patch_gemm); patch_pack_dev / patch_pack_patterns report flags above 1 as PATCH_ERR_FLAG.
+ * The launch promises mean the same as for bf16 tiles; launches with different promises may split K
+ * differently and then differ in the last bit.
  */
 int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
                const patch_layout_t* layout, const void* packed_dev,
