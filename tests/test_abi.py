@@ -103,6 +103,34 @@ def test_gemm_rejects_bad_arguments_on_host(binding):
     assert b"timed out" in lib.patch_strerror(binding.ERR_TIMEOUT)
 
 
+def test_4bit_weights_are_refused_where_no_kernel_serves_them(binding):
+    """Weights with 4-bit tiles: M > 16, mixtures with bf16 tiles, the GEMV variant, the gated product and the
+    no-allocation entry point are refused on the host, before any device is touched."""
+    lib = binding.lib()
+    null = ctypes.c_void_p(0)
+    fake = ctypes.c_void_p(1024 * 1024)   # never dereferenced: validation fails first
+    L4 = binding.patch_packed_size(256, 256, np.array([[2, 3], [3, 2]], np.uint8))
+    Lm = binding.patch_packed_size(256, 256, np.array([[2, 0], [3, 1]], np.uint8))
+    args = lambda M, Lp: (fake, 256, M, ctypes.byref(Lp), fake, fake, 256, null, 0, null, null)
+    assert lib.patch_gemm(*args(17, L4)) == binding.ERR_SHAPE
+    assert lib.patch_gemm(*args(4, Lm)) == binding.ERR_SHAPE
+    assert lib.patch_gemm_ex(*args(4, L4), binding.VARIANT_GEMV) == binding.ERR_SHAPE
+    assert lib.patch_gemm_gated(*args(4, L4), 0) == binding.ERR_SHAPE
+    assert lib.patch_gemm_noalloc(fake, 256, 4, ctypes.byref(L4), fake, fake, 256, null) == binding.ERR_SHAPE
+    assert binding.patch_gemm_workspace_size(L4, 16) == 0
+    # a layout whose counts do not add up to the tile count, or whose bytes do not follow from the counts
+    bad = binding.Layout.from_buffer_copy(bytes(L4))
+    bad.n_dense_q4 -= 1
+    assert lib.patch_gemm(*args(4, bad)) == binding.ERR_FORMAT
+    bad = binding.Layout.from_buffer_copy(bytes(L4))
+    bad.n_dense_q4, bad.n_sparse_q4 = bad.n_sparse_q4 + 1, bad.n_dense_q4 - 1
+    assert lib.patch_gemm(*args(4, bad)) == binding.ERR_FORMAT
+    # patterns are for the bf16 2:4 kind only
+    f = np.array([2, 3, 3, 2], np.uint8)
+    assert lib.patch_pack_patterns(fake, 256, ctypes.c_void_p(f.ctypes.data), fake, ctypes.byref(L4), fake, 1 << 24,
+                                   null, null) == binding.ERR_FLAG
+
+
 def test_product_package_does_not_import_the_oracle():
     pkg = os.path.join(ROOT, "paper_2509_23410_b200")
     for dirpath, _, files in os.walk(pkg):
