@@ -203,6 +203,18 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
         // payloads of the first kRaw tiles may be requested before the grid dependency is resolved (WSTATIC);
         // their activations follow once it is (unless XSTATIC)
         const int n_early = (WSTATIC && !XSTATIC) ? (n_tiles < kRaw ? n_tiles : kRaw) : 0;
+#ifdef PATCH_FAULT_INJECTION
+        // test build: a status word holding kInjectMagic makes CTA 0 announce sixteen bytes more than its first
+        // slot will ever receive, so that a wait of this kernel runs out (see sm100_ptx.cuh)
+        uint32_t inject_bytes = 0u;
+        if (blockIdx.x == 0 && status_dev && *status_dev == kInjectMagic) {
+            inject_bytes = 16u;
+            __syncwarp();
+            if (lane == 0) *status_dev = PATCH_OK;
+        }
+#else
+        constexpr uint32_t inject_bytes = 0u;
+#endif
         for (int base = 0; base < n_tiles && ok; base += kBatch) {
             if ((base & 31) == 0 && base + lane < n_tiles) mine = table[base + lane];
             const int i = base + lane, src = i & 31;               // kBatch divides 32: the round's entries sit in one load
@@ -218,7 +230,7 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
                     const uint32_t wbytes = kind == PATCH_TILE_DENSE_Q4 ? kDenseQ4Bytes : kSparseQ4Bytes;
                     const uint32_t full = bar_raw_full + 8 * slot;
                     slot_kind[slot] = kind;
-                    mbar_expect_tx(full, wbytes);
+                    mbar_expect_tx(full, wbytes + (i == 0 ? inject_bytes : 0u));
                     tma_bulk_load(smem_base + kRawOffset + slot * kRawBytes, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
                 }
             }

@@ -48,8 +48,9 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 
 #ifdef PATCH_FAULT_INJECTION
 // Test build (libpatch_b200_fi.so, see build.py): waits give up after 300 us, and a launch of the stream-K decode
-// kernel whose status word holds kInjectMagic announces, in CTA 0, sixteen bytes more than its first stage will
-// ever receive -- the one way the tests make a bounded wait run out.  Nothing faults, traps or spins for ever.
+// kernel or of the 4-bit decode kernel whose status word holds kInjectMagic announces, in CTA 0, sixteen bytes more
+// than its first stage will ever receive -- the one way the tests make a bounded wait run out.  Nothing faults,
+// traps or spins for ever.
 constexpr uint64_t kWaitLimitNs = 300000ull;
 constexpr int kInjectMagic = 0x7E57;
 #else

@@ -3,7 +3,8 @@
 * A bounded device-side wait that really runs out: the fault-injection build of the library (same sources, waits
   limited to 300 us) lets the test tell the stream-K decode kernel, through its status word, to announce sixteen
   bytes more than its first stage will ever receive.  The MMA warp's wait expires, the CTA raises its abort flag,
-  reports PATCH_ERR_TIMEOUT, drains, frees its tensor memory and returns; the context stays usable.
+  reports PATCH_ERR_TIMEOUT, drains, frees its tensor memory and returns; the context stays usable.  The kernel of
+  the 4-bit tile kinds has the same hook.
 * A tile table that does not belong to the layout: every kernel checks each entry against the blob's extent before
   it requests a byte of the tile, reports PATCH_ERR_FORMAT and reads the first payload instead.  The bad offsets used
   here point inside the test's own over-allocated buffer, so a check that failed to catch them could not fault."""
@@ -61,6 +62,42 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_survivable(gpu, oracle):
     check_parity(oracle, to_bits(Y), oracle.gemm_f64(X, What)[0], "after the timeout")
     # and the injected build again, without injection
     assert call(torch.zeros(1, dtype=torch.int32, device="cuda")) == B.OK
+
+
+def test_a_wait_of_the_4bit_kernel_that_runs_out(gpu, oracle):
+    """The same for the kernel of the 4-bit tile kinds: the group that waits for CTA 0's first payload gives up,
+    the CTA's other roles follow, the launch completes with PATCH_ERR_TIMEOUT and the next launch is correct."""
+    torch, B = gpu
+    from paper_2509_23410_b200 import build
+    fi = B.load(build.build(fault_injection=True))
+    N, K, M = 512, 2048, 16
+    W, flags, X = inputs.make_case_inputs(dict(N=N, K=K, p=0.5, stream=("timeout-q4",)), 73, M)
+    flags = flags | 2
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Xd = to_dev(torch, X)
+    Y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    ref = oracle.gemm_f64(X, What)[0]
+
+    def call(status, variant):
+        rc = fi.patch_gemm_ex(_ptr(Xd), K, M, ctypes.byref(L), _ptr(packed), _ptr(Y), N, ctypes.c_void_p(0), 0, _ptr(status),
+                              stream, variant)
+        assert rc == B.OK
+        torch.cuda.synchronize()
+        return int(status.item())
+
+    for variant in (B.VARIANT_AUTO, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC):
+        assert call(torch.zeros(1, dtype=torch.int32, device="cuda"), variant) == B.OK
+        check_parity(oracle, to_bits(Y), ref, "fault-injection build, no injection")
+        status = torch.full((1,), INJECT_MAGIC, dtype=torch.int32, device="cuda")
+        assert call(status, variant) == B.ERR_TIMEOUT
+        Y.zero_()
+        status.zero_()
+        B.patch_gemm(Xd, L, packed, Y=Y, status=status, variant=variant)
+        torch.cuda.synchronize()
+        assert int(status.item()) == B.OK
+        check_parity(oracle, to_bits(Y), ref, "after the timeout")
 
 
 @pytest.mark.parametrize("M,variant", [(1, "gemv"), (1, "independent"), (16, "independent"), (16, "streamk"), (48, "streamk"),
