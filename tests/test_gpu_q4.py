@@ -200,3 +200,76 @@ def test_bad_table_entries_are_reported(gpu, oracle):
         torch.cuda.synchronize()
         assert int(status.item()) == B.ERR_FORMAT, (word, value)
     assert (run_gemm(gpu, X, L, packed, B.VARIANT_AUTO) == good).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# the decode-q4 workload as bench.py runs it
+
+
+@pytest.fixture(scope="module")
+def decode_q4_workload(gpu, oracle):
+    """The 24 GEMMs of `bench.py --workload decode-q4`: 12 packed matrices (3 LLaMA-2-7B shapes x four 2:4-tile
+    fractions, every tile 4-bit), M = 1 and 16, with the oracle's result for each."""
+    torch, B = gpu
+    cases = sorted(inputs.decode_q4_cases(), key=lambda c: c["M"])
+    mats, jobs = {}, []
+    for c in cases:
+        key = c["stream"]
+        if key not in mats:
+            W = inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"])
+            flags = inputs.case_flags(c)
+            assert ((flags & 2) == 2).all()
+            packed, L = B.patch_pack(to_dev(torch, W), flags)
+            mats[key] = (oracle.prune(W, flags), packed, L)
+        What, packed, L = mats[key]
+        X = inputs.activation(c["M"], c["K"], inputs.MASTER_SEED, *c["stream"], c["M"])
+        Y32, Y16 = oracle.gemm_f64(X, What)
+        jobs.append(dict(case=c, L=L, packed=packed, X=to_dev(torch, X), Y32=Y32, Y16=Y16,
+                         Y=torch.zeros((c["M"], c["N"]), dtype=torch.bfloat16, device="cuda")))
+    torch.cuda.synchronize()
+    return jobs
+
+
+@pytest.mark.parametrize("mode", ["independent", "dependent", "no promise"])
+def test_decode_q4_workload_graph_replay(gpu, oracle, decode_q4_workload, mode):
+    """The regime the decode-q4 number is timed in: two consecutive steps of the 24 GEMMs captured into one CUDA
+    graph (CTAs of consecutive kernels share SMs, ordered only by their device-side waits), replayed twice; then
+    every one of the 24 outputs, whole, against the oracle."""
+    torch, B = gpu
+    jobs = decode_q4_workload
+    flags = {"independent": B.WEIGHTS_STATIC | B.INPUT_STATIC, "dependent": B.WEIGHTS_STATIC, "no promise": 0}[mode]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step():
+        for j in jobs:
+            B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Y"], status=status, variant=B.VARIANT_AUTO | flags)
+    step()                                   # kernel attributes are set outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+        step()
+    for j in jobs:
+        j["Y"].zero_()
+    torch.cuda.synchronize()
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for j in jobs:
+        got = to_bits(j["Y"])
+        check_parity(oracle, got, j["Y32"], f"{j['case']['name']} ({mode}, graph)")
+        assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
+
+
+def test_decode_q4_workload_pack_bit_exact(gpu, oracle):
+    """The largest matrices of the workload, packed image against the oracle's, bit for bit."""
+    torch, B = gpu
+    for c in inputs.decode_q4_cases():
+        if c["M"] != 1 or c["p"] not in (0.35, 1.0) or c["N"] == c["K"]:
+            continue
+        W = inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"])
+        flags = inputs.case_flags(c)
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        assert (packed.cpu().numpy() == oracle.device_image(oracle.pack(W, flags)[0])).all(), c["name"]
+        assert (to_bits(B.patch_unpack(L, packed)) == oracle.prune(W, flags)).all(), c["name"]
