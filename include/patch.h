@@ -194,9 +194,11 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  *           In both cases Y is undefined.  NULL = not reported.
  * M == 0 returns PATCH_OK without launching.  Calls sharing a workspace must be ordered on
  * one stream.
- * Weights with 4-bit tiles: served for M <= 16 tokens (the decode case, where the bytes of the weight are
- * what the layer costs) and only if every tile is of a 4-bit kind; a dequantising kernel of its own, no
- * workspace.  Other M, and weights that mix bf16 and 4-bit tiles, return PATCH_ERR_SHAPE -- as do
+ * Weights with 4-bit tiles: served if every tile is of a 4-bit kind, by a dequantising kernel of its own made
+ * for M <= 16 tokens (the decode case, where the bytes of the weight are what the layer costs); no workspace.
+ * More tokens are multiplied sixteen at a time, one launch after the other: correct, but every launch streams
+ * the weight again (there is no large-M schedule for these kinds).  Weights that mix bf16 and 4-bit tiles
+ * return PATCH_ERR_SHAPE -- as do
  * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated and patch_gemm_noalloc for such weights (the host
  * entry points follow patch_gemm); patch_pack_dev / patch_pack_patterns report flags above 1 as PATCH_ERR_FLAG.
  * The launch promises mean the same as for bf16 tiles; launches with different promises may split K

@@ -48,12 +48,18 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     if (variant == PATCH_VARIANT_PAIR && M <= 64) return PATCH_ERR_SHAPE;
     if (has_q4_tiles(L)) {
         // 4-bit tiles: the dequantising decode kernel, for weights made of such tiles only
-        if (L->n_dense || L->n_sparse || M > 16 || variant == PATCH_VARIANT_GEMV) return PATCH_ERR_SHAPE;
+        if (L->n_dense || L->n_sparse || variant == PATCH_VARIANT_GEMV || variant == PATCH_VARIANT_PAIR) return PATCH_ERR_SHAPE;
         rc = check_device();
         if (rc) return rc;
-        return launch_decode_q4(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, L, static_cast<const uint8_t*>(packed_dev),
-                                static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, static_cast<cudaStream_t>(stream),
-                                wstatic, xstatic);
+        // more than 16 tokens: sixteen at a time, one launch each, under the caller's promises (a later launch
+        // may not assume more than the first: it can start while the kernels before this call still run)
+        for (int64_t m0 = 0; m0 < M; m0 += 16) {
+            rc = launch_decode_q4(static_cast<const __nv_bfloat16*>(X_dev) + m0 * ldx, ldx, M - m0 < 16 ? M - m0 : 16, L,
+                                  static_cast<const uint8_t*>(packed_dev), static_cast<__nv_bfloat16*>(Y_dev) + m0 * ldy, ldy,
+                                  status_dev, static_cast<cudaStream_t>(stream), wstatic, xstatic);
+            if (rc) return rc;
+        }
+        return PATCH_OK;
     }
     const size_t need = decode_workspace_bytes(L, M);
     if (need > 0) {

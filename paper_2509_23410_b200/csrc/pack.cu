@@ -264,9 +264,15 @@ pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __r
     uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;                    // only used if sparse
     uint16_t* scales = reinterpret_cast<uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    // all sixteen rows of the warp are requested before the first is quantised: 4 KB in flight per warp
+    uint2 xs[16];
+#pragma unroll
+    for (uint32_t rr = 0; rr < 16; ++rr)
+        xs[rr] = *reinterpret_cast<const uint2*>(wt + int64_t(rr * 8 + warp) * ldw + lane * 4);
+#pragma unroll
     for (uint32_t rr = 0; rr < 16; ++rr) {
         const uint32_t r = rr * 8 + warp;
-        const uint2 x = *reinterpret_cast<const uint2*>(wt + int64_t(r) * ldw + lane * 4);
+        const uint2 x = xs[rr];
         float v[4] = {bf16_bits_to_f32(x.x & 0xFFFFu), bf16_bits_to_f32(x.x >> 16),
                       bf16_bits_to_f32(x.y & 0xFFFFu), bf16_bits_to_f32(x.y >> 16)};
         uint32_t i0 = 0, i1 = 1;

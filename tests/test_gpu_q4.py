@@ -151,6 +151,29 @@ def test_gemm_back_to_back_and_chain(gpu, oracle):
         ref = got
 
 
+@pytest.mark.parametrize("M", [17, 40, 100])
+def test_gemm_more_than_16_tokens(gpu, oracle, M):
+    """More than sixteen tokens are multiplied sixteen at a time; every promise; Y with a row pitch."""
+    torch, B = gpu
+    N, K = 640, 768
+    W = inputs.weight(N, K, 38, "q4-chunks")
+    X = inputs.activation(M, K, 38, "q4-chunks", M)
+    flags = _flags4(N, K, 0.5, "chunks")
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y32, Y16 = oracle.gemm_f64(X, What)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for promise in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC):
+        Ybuf = torch.full((M, N + 64), 3.0, dtype=torch.bfloat16, device="cuda")
+        B.patch_gemm(to_dev(torch, X), L, packed, Y=Ybuf[:, :N], status=status, variant=B.VARIANT_AUTO | promise)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got = to_bits(Ybuf[:, :N])
+        check_parity(oracle, got, Y32, f"M={M} promise={promise:#x}")
+        assert (got == Y16).mean() >= 0.99
+        assert (Ybuf[:, N:] == 3.0).all()
+
+
 def test_unsupported_combinations_are_refused(gpu):
     torch, B = gpu
     N, K = 256, 256
@@ -161,7 +184,6 @@ def test_unsupported_combinations_are_refused(gpu):
     packed_m, L_m = B.patch_pack(W, mixed)             # packing and unpacking serve any mixture
     assert (L_m.n_dense, L_m.n_sparse, L_m.n_dense_q4, L_m.n_sparse_q4) == (1, 1, 1, 1)
     ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
-    X17 = torch.zeros((17, K), dtype=torch.bfloat16, device="cuda")
     X4 = torch.zeros((4, K), dtype=torch.bfloat16, device="cuda")
 
     def refused(fn):
@@ -169,7 +191,6 @@ def test_unsupported_combinations_are_refused(gpu):
             fn()
         return e.value.status
 
-    assert refused(lambda: B.patch_gemm(X17, L, packed, workspace=ws)) == B.ERR_SHAPE          # M > 16
     assert refused(lambda: B.patch_gemm(X4, L_m, packed_m, workspace=ws)) == B.ERR_SHAPE       # bf16 and 4-bit tiles
     assert refused(lambda: B.patch_gemm(X4, L, packed, workspace=ws, variant=B.VARIANT_GEMV)) == B.ERR_SHAPE
     assert refused(lambda: B.patch_gemm_gated(X4, L, packed, workspace=ws)) == B.ERR_SHAPE
