@@ -78,8 +78,14 @@ enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2, PA
  *   writes X either (e.g. q, k and v projections enqueued one after the other behind the kernel that
  *   produced their common X; not a GEMM whose X is the Y of a GEMM enqueued directly before it).
  *   Activations are then fetched without waiting too.
- * Writes to Y and to the workspace always wait for everything before them, and no kernel completes
- * before its predecessors, so stream order as seen from later operations is unchanged.
+ * PATCH_GEMM_OUTPUT_STATIC (only honoured together with the first two, and for M <= 64): no operation in the
+ *   overlap window reads or writes Y either (q, k and v projections writing three buffers of their own; not two
+ *   calls that write the same Y with only GEMM calls of this library between them).  The CTAs of the kernel
+ *   then store Y and leave as soon as they are done, instead of each holding its SM until the preceding
+ *   kernels have completed; one cluster of every launch still waits.
+ * Without the third promise, writes to Y wait for everything before them; writes to the workspace always do.
+ * With or without it no kernel completes before its predecessors, so stream order as seen from later
+ * operations is unchanged.
  *
  * With BOTH promises a GEMM of M <= 64 tokens runs on a schedule made for streams of independent
  * GEMMs: one CTA per row-block (a small cluster splitting K where row-blocks are few), so that several
@@ -91,6 +97,7 @@ enum { PATCH_VARIANT_AUTO = 0, PATCH_VARIANT_GEMV = 1, PATCH_VARIANT_MMA = 2, PA
  */
 enum { PATCH_GEMM_WEIGHTS_STATIC = 0x100 };
 enum { PATCH_GEMM_INPUT_STATIC = 0x200 };
+enum { PATCH_GEMM_OUTPUT_STATIC = 0x400 };
 
 /*
  * Description of a packed blob.  Plain host struct, caller-owned, filled by patch_packed_size.
@@ -216,7 +223,7 @@ int patch_gemm(const void* X_dev, int64_t ldx, int64_t M,
  *                       picks the pair schedule for weights whose tiles are all of one kind wherever every CTA
  *                       pair gets a tile of a useful width; for weights that mix kinds it is slower than the
  *                       one-CTA schedule and runs only when asked for
- *   | PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC  see above */
+ *   | PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC | PATCH_GEMM_OUTPUT_STATIC  see above */
 int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
                   const patch_layout_t* layout, const void* packed_dev,
                   void* Y_dev, int64_t ldy,

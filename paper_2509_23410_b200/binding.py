@@ -19,6 +19,7 @@ TILE_DENSE, TILE_SPARSE_2_4, TILE_DENSE_Q4, TILE_SPARSE_2_4_Q4 = 0, 1, 2, 3
 VARIANT_AUTO, VARIANT_GEMV, VARIANT_MMA, VARIANT_PAIR = 0, 1, 2, 3
 WEIGHTS_STATIC = 0x100   # OR into `variant`: the packed weight is not produced by the preceding kernel
 INPUT_STATIC = 0x200     # OR into `variant`: X is not produced by the preceding kernel
+OUTPUT_STATIC = 0x400    # OR into `variant` (with the other two): nothing in the overlap window reads or writes Y
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_TILE, ERR_FLAG, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10

@@ -40,7 +40,8 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     if (M == 0) return PATCH_OK;
     const bool wstatic = (variant & PATCH_GEMM_WEIGHTS_STATIC) != 0;
     const bool xstatic = (variant & PATCH_GEMM_INPUT_STATIC) != 0;
-    variant &= ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC);
+    const bool ystatic = wstatic && xstatic && (variant & PATCH_GEMM_OUTPUT_STATIC) != 0;
+    variant &= ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC | PATCH_GEMM_OUTPUT_STATIC);
     if (variant != PATCH_VARIANT_AUTO && variant != PATCH_VARIANT_GEMV && variant != PATCH_VARIANT_MMA &&
         variant != PATCH_VARIANT_PAIR)
         return PATCH_ERR_SHAPE;
@@ -56,7 +57,7 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
         for (int64_t m0 = 0; m0 < M; m0 += 16) {
             rc = launch_decode_q4(static_cast<const __nv_bfloat16*>(X_dev) + m0 * ldx, ldx, M - m0 < 16 ? M - m0 : 16, L,
                                   static_cast<const uint8_t*>(packed_dev), static_cast<__nv_bfloat16*>(Y_dev) + m0 * ldy, ldy,
-                                  status_dev, static_cast<cudaStream_t>(stream), wstatic, xstatic);
+                                  status_dev, static_cast<cudaStream_t>(stream), wstatic, xstatic, ystatic);
             if (rc) return rc;
         }
         return PATCH_OK;
@@ -74,7 +75,7 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(Y_dev);
     const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
     if (variant == PATCH_VARIANT_GEMV) return launch_gemv(X, ldx, int(M), L, packed, Y, ldy, status_dev, s);
-    if (M <= 64) return launch_decode(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s, wstatic, xstatic);
+    if (M <= 64) return launch_decode(X, ldx, M, L, packed, Y, ldy, workspace_dev, status_dev, s, wstatic, xstatic, ystatic);
     return launch_prefill(X, ldx, M, L, packed, Y, ldy, status_dev, s, wstatic && xstatic, variant == PATCH_VARIANT_PAIR);
 }
 
@@ -103,7 +104,7 @@ extern "C" int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M, const
     if (rc) return rc;
     if (L->N % (2 * kTile)) return PATCH_ERR_SHAPE;      // whole (gate, up) pairs of row-blocks
     if (M < 0 || has_q4_tiles(L)) return PATCH_ERR_SHAPE;
-    if (flags & ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC)) return PATCH_ERR_SHAPE;
+    if (flags & ~(PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC | PATCH_GEMM_OUTPUT_STATIC)) return PATCH_ERR_SHAPE;
     if (M == 0) return PATCH_OK;
     if (!X_dev || !packed_dev || !Y_dev) return PATCH_ERR_NULL;
     if (ldx < L->K || ldy < L->N / 2 || ldx % 8 || ldy % 8) return PATCH_ERR_SHAPE;

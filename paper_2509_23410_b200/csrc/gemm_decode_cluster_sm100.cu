@@ -64,7 +64,10 @@ __device__ __forceinline__ float4 ld_peer_f4(uint32_t saddr, uint32_t rank) {
 // GATED: the weight stacks a gate and an up projection with their row-blocks interleaved (2j: gate, 2j + 1: up);
 // a cluster owns the pair j, streams the gate tiles of its K-slice into one accumulator and the up tiles into a
 // second one, and writes silu(gate) * up for out-feature block j of Y [M x N / 2].
-template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
+// YSTATIC: the caller also promised that nothing in the overlap window touches Y: only the launch's first cluster
+// waits for the preceding kernel (so that launches still complete in order); every other CTA stores Y and leaves
+// as soon as it is done instead of holding its shared memory until then.
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false, bool YSTATIC = false>
 __global__ void __launch_bounds__(192)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                       uint32_t pay0_16, uint32_t end16, int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy,
@@ -228,7 +231,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
         const int rows = kTile / S;                                // S in {1, 2, 4, 8}
         constexpr int kGroups = N_TOK / 4;                         // groups of four tokens per row
         const int n_out = rows * kGroups;
-        grid_dependency_wait();                                    // Y may be in use by the preceding kernel
+        if (!YSTATIC || int(blockIdx.x) < S) grid_dependency_wait();   // Y may be in use by the preceding kernel
         for (int o = e; o < n_out; o += 128) {
             // consecutive threads take consecutive rows of one token group: their stores are neighbours in Y
             const int r = int(s) * rows + (o % rows), tg = o / rows;
@@ -257,7 +260,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
             }
         }
     } else {
-        grid_dependency_wait();     // every thread passes the dependency before the CTA exits
+        if (!YSTATIC || int(blockIdx.x) < S) grid_dependency_wait();   // every thread passes the dependency before the CTA exits
     }
 
     // nobody leaves while a peer may still read its shared memory
@@ -267,11 +270,11 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t*
     if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
 }
 
-template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false>
+template <int N_TOK, int STAGES, bool WSTATIC, bool XSTATIC, bool GATED = false, bool YSTATIC = false>
 static int launch_dc_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int S,
                        __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
     using C = dc::Cfg<N_TOK, STAGES, GATED>;
-    auto kern = decode_cluster_kernel<N_TOK, STAGES, WSTATIC, XSTATIC, GATED>;
+    auto kern = decode_cluster_kernel<N_TOK, STAGES, WSTATIC, XSTATIC, GATED, YSTATIC>;
     static std::atomic<uint64_t> configured{0};
     if (int rc = allow_dynamic_smem(kern, C::kSmemBytes, configured)) return rc;
     const int TN = int(L->N / kTile) / (GATED ? 2 : 1), TK = int(L->K / kTile);     // gated: pairs of row-blocks
@@ -307,7 +310,10 @@ int decode_cluster_split(int TN, int TK) {
 
 template <int N_TOK, int STAGES>
 static int launch_dc_f(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int S,
-                       __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic) {
+                       __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic,
+                       bool ystatic) {
+    if (wstatic && xstatic && ystatic)
+        return launch_dc_t<N_TOK, STAGES, true, true, false, true>(map, L, packed, M, S, Y, ldy, status_dev, stream);
     if (wstatic && xstatic) return launch_dc_t<N_TOK, STAGES, true, true>(map, L, packed, M, S, Y, ldy, status_dev, stream);
     if (wstatic) return launch_dc_t<N_TOK, STAGES, true, false>(map, L, packed, M, S, Y, ldy, status_dev, stream);
     return launch_dc_t<N_TOK, STAGES, false, false>(map, L, packed, M, S, Y, ldy, status_dev, stream);
@@ -315,7 +321,7 @@ static int launch_dc_f(const CUtensorMap& map, const patch_layout_t* L, const ui
 
 int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int n_tok,
                           __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic,
-                          bool xstatic) {
+                          bool xstatic, bool ystatic) {
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
     int S = decode_cluster_split(TN, TK);
     if (!xstatic) {
@@ -327,9 +333,9 @@ int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const
         while (S < 8 && TN * S < 128 && 2 * S <= TK) S *= 2;
     }
     switch (n_tok) {
-        case 16: return launch_dc_f<16, 3>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
-        case 32: return launch_dc_f<32, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
-        default: return launch_dc_f<64, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic);
+        case 16: return launch_dc_f<16, 3>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic, ystatic);
+        case 32: return launch_dc_f<32, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic, ystatic);
+        default: return launch_dc_f<64, 2>(map, L, packed, M, S, Y, ldy, status_dev, stream, wstatic, xstatic, ystatic);
     }
 }
 

@@ -142,7 +142,9 @@ __device__ __forceinline__ void dequant_store16(uint4 cw, __nv_bfloat162 s2, uin
 }
 }  // namespace dq
 
-template <bool WSTATIC, bool XSTATIC>
+// YSTATIC: nothing in the overlap window touches Y (third launch promise): only the launch's first cluster waits for
+// the preceding kernel, so that launches still complete in order; every other CTA stores Y and leaves when it is done.
+template <bool WSTATIC, bool XSTATIC, bool YSTATIC>
 __global__ void __launch_bounds__(dq::kThreads, 2)
 decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ blob, uint64_t table_off,
                  uint32_t pay0_16, uint32_t end16, int TK, int S, int M, __nv_bfloat16* __restrict__ Y, int64_t ldy,
@@ -369,7 +371,7 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
         const int e = threadIdx.x - 32;                            // 0..127
         const int rows = kTile / S;                                // S in {1, 2, 4, 8}
         const int n_out = rows * 4;                                // groups of four tokens
-        grid_dependency_wait();                                    // Y may be in use by the preceding kernel
+        if (!YSTATIC || int(blockIdx.x) < S) grid_dependency_wait();   // Y may be in use by the preceding kernel
         for (int o = e; o < n_out; o += 128) {
             const int r = int(s) * rows + (o % rows), tg = o / rows;
             const uint32_t addr = smem_base + uint32_t(r) * kPartialRowBytes + uint32_t(tg) * 16u;
@@ -387,7 +389,7 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
             }
         }
     } else {
-        grid_dependency_wait();     // every thread passes the dependency before the CTA exits
+        if (!YSTATIC || int(blockIdx.x) < S) grid_dependency_wait();   // every thread passes the dependency before the CTA exits
     }
 
     // nobody leaves while a peer may still read its shared memory
@@ -397,10 +399,10 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     if (warp == 0) tmem_dealloc(tmem_base, dq::kTmemCols);
 }
 
-template <bool WSTATIC, bool XSTATIC>
+template <bool WSTATIC, bool XSTATIC, bool YSTATIC = false>
 static int launch_q4_t(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int S,
                        __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
-    auto kern = decode_q4_kernel<WSTATIC, XSTATIC>;
+    auto kern = decode_q4_kernel<WSTATIC, XSTATIC, YSTATIC>;
     static std::atomic<uint64_t> configured{0};
     if (int rc = allow_dynamic_smem(kern, dq::kSmemBytes, configured)) return rc;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
@@ -424,7 +426,8 @@ static int launch_q4_t(const CUtensorMap& map, const patch_layout_t* L, const ui
 }
 
 int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                     __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic) {
+                     __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic,
+                     bool ystatic) {
     CUtensorMap map;
     int rc = make_x_chunk_tensor_map(&map, X, ldx, M, L->K, 16, 2 * dq::kBatch);
     if (rc) return rc;
@@ -443,6 +446,7 @@ int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch
             if (t < best) { best = t; S = s2; }
         }
     }
+    if (wstatic && xstatic && ystatic) return launch_q4_t<true, true, true>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);
     if (wstatic && xstatic) return launch_q4_t<true, true>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);
     if (wstatic) return launch_q4_t<true, false>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);
     return launch_q4_t<false, false>(map, L, packed, int(M), S, Y, ldy, status_dev, stream);

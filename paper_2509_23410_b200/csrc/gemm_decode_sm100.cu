@@ -682,13 +682,13 @@ static bool use_rowblock_schedule(bool wstatic, bool xstatic) { (void)xstatic; r
 
 int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                   __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev, cudaStream_t stream,
-                  bool wstatic, bool xstatic) {
+                  bool wstatic, bool xstatic, bool ystatic) {
     const int n_tok = decode_n_tok(M);
     CUtensorMap map;
     int rc = make_x_tensor_map(&map, X, ldx, M, L->K, n_tok);
     if (rc) return rc;
     if (use_rowblock_schedule(wstatic, xstatic))
-        return launch_decode_cluster(map, L, packed, int(M), n_tok, Y, ldy, status_dev, stream, wstatic, xstatic);
+        return launch_decode_cluster(map, L, packed, int(M), n_tok, Y, ldy, status_dev, stream, wstatic, xstatic, ystatic);
     switch (n_tok) {
         case 16:
             if (wstatic && xstatic)

@@ -104,7 +104,7 @@ int launch_gemv(const __nv_bfloat16* X, int64_t ldx, int M, const patch_layout_t
                 cudaStream_t stream);
 int launch_decode(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L,
                   const uint8_t* packed, __nv_bfloat16* Y, int64_t ldy, void* workspace, int* status_dev,
-                  cudaStream_t stream, bool wstatic, bool xstatic);
+                  cudaStream_t stream, bool wstatic, bool xstatic, bool ystatic = false);
 // `independent`: the caller declared the GEMM independent of its predecessor (weights and X static): only its
 // Y stores wait for the preceding kernel.
 // `force_pair`: only the CTA-pair schedule will do (PATCH_ERR_SHAPE if the weight mixes tile kinds).
@@ -121,7 +121,8 @@ int launch_decode_gated(const __nv_bfloat16* X, int64_t ldx, int64_t M, const pa
 size_t decode_gated_workspace_bytes(const patch_layout_t* L, int64_t M);   // 0 if the gated decode schedule does not apply
 // M <= 16 on a weight whose tiles are all of a 4-bit kind (gemm_decode_q4_sm100.cu)
 int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
-                     __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic);
+                     __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic,
+                     bool ystatic = false);
 inline bool has_q4_tiles(const patch_layout_t* L) { return L->n_dense_q4 != 0 || L->n_sparse_q4 != 0; }
 
 }  // namespace patch

@@ -391,7 +391,7 @@ int make_blob_tensor_map(CUtensorMap* map, const uint8_t* blob, uint64_t total_b
 // declared independent of their predecessor (`map`: X tensor map with a box of `n_tok` token rows).
 int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M, int n_tok,
                           __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic,
-                          bool xstatic);
+                          bool xstatic, bool ystatic = false);
 int decode_cluster_split(int TN, int TK);     // cluster size of the row-block schedule for independent GEMMs
 int launch_decode_cluster_gated(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
                                 __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);

@@ -393,7 +393,7 @@ def test_decode_workload_all_cases_bench_flags(gpu, oracle, decode_workload):
         assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
 
 
-@pytest.mark.parametrize("mode", ["independent", "dependent"])
+@pytest.mark.parametrize("mode", ["independent", "independent+output", "dependent"])
 def test_decode_workload_graph_replay(gpu, oracle, decode_workload, mode):
     """The regime the headline number is timed in: two consecutive steps of the 24 GEMMs captured into one CUDA
     graph (several kernels resident at once, ordered only by their device-side waits), replayed twice; then
@@ -401,29 +401,35 @@ def test_decode_workload_graph_replay(gpu, oracle, decode_workload, mode):
     promise only (every GEMM waits for its predecessor before reading X)."""
     torch, B = gpu
     jobs, ws = decode_workload
-    flags = B.WEIGHTS_STATIC | (B.INPUT_STATIC if mode == "independent" else 0)
+    flags = B.WEIGHTS_STATIC | {"independent": B.INPUT_STATIC, "independent+output": B.INPUT_STATIC | B.OUTPUT_STATIC,
+                                "dependent": 0}[mode]
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # with the output promise every launch between two drains writes a buffer of its own (bench.py does the
+    # same): the second step of the graph gets a second set of outputs
+    first = [j["Y"] for j in jobs]
+    second = [torch.zeros_like(j["Y"]) for j in jobs]
 
-    def step():
-        for j in jobs:
-            B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Y"], workspace=ws, status=status, variant=B.VARIANT_AUTO | flags)
-    step()                                   # kernel attributes are set outside the capture
+    def step(outs):
+        for j, Y in zip(jobs, outs):
+            B.patch_gemm(j["X"], j["L"], j["packed"], Y=Y, workspace=ws, status=status, variant=B.VARIANT_AUTO | flags)
+    step(first)                              # kernel attributes are set outside the capture
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
-        step()
-        step()
-    for j in jobs:
-        j["Y"].zero_()
+        step(first)
+        step(second)
+    for Y in first + second:
+        Y.zero_()
     torch.cuda.synchronize()
     g.replay()
     g.replay()
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    for j in jobs:
-        got = to_bits(j["Y"])
-        check_parity(oracle, got, j["Y32"], f"{j['case']['name']} ({mode}, graph)")
-        assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
+    for outs in (first, second):
+        for j, Y in zip(jobs, outs):
+            got = to_bits(Y)
+            check_parity(oracle, got, j["Y32"], f"{j['case']['name']} ({mode}, graph)")
+            assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
 
 
 _PREFILL = [(s, p) for s in inputs.LLAMA2_7B_SHAPES for p in (0.0, 0.5, 1.0)]

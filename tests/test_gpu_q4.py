@@ -78,7 +78,8 @@ def test_gemm_parity(gpu, oracle, N, K, M, p):
     assert B.patch_gemm_workspace_size(L, M) == 0
     Y32, Y16 = oracle.gemm_f64(X, What)
     outs = []
-    for promise in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC):
+    for promise in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC,
+                    B.WEIGHTS_STATIC | B.INPUT_STATIC | B.OUTPUT_STATIC):
         Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | promise)
         check_parity(oracle, Y, Y32, f"q4 N={N} K={K} M={M} p={p} promise={promise:#x}")
         assert (Y == Y16).mean() >= 0.99
@@ -124,7 +125,8 @@ def test_gemm_back_to_back_and_chain(gpu, oracle):
     outs = []
     for i in range(12):
         What, packed, L, X, Xd = cases[i % 2]
-        promise = (B.WEIGHTS_STATIC | B.INPUT_STATIC) if i % 2 else 0
+        # every launch writes a buffer of its own, so the odd ones may also carry the output promise
+        promise = (B.WEIGHTS_STATIC | B.INPUT_STATIC | (B.OUTPUT_STATIC if i % 4 == 1 else 0)) if i % 2 else 0
         outs.append(B.patch_gemm(Xd, L, packed, status=status, variant=B.VARIANT_AUTO | promise))
     torch.cuda.synchronize()
     assert int(status.item()) == 0
@@ -251,36 +253,43 @@ def decode_q4_workload(gpu, oracle):
     return jobs
 
 
-@pytest.mark.parametrize("mode", ["independent", "dependent", "no promise"])
+@pytest.mark.parametrize("mode", ["independent", "independent+output", "dependent", "no promise"])
 def test_decode_q4_workload_graph_replay(gpu, oracle, decode_q4_workload, mode):
     """The regime the decode-q4 number is timed in: two consecutive steps of the 24 GEMMs captured into one CUDA
     graph (CTAs of consecutive kernels share SMs, ordered only by their device-side waits), replayed twice; then
     every one of the 24 outputs, whole, against the oracle."""
     torch, B = gpu
     jobs = decode_q4_workload
-    flags = {"independent": B.WEIGHTS_STATIC | B.INPUT_STATIC, "dependent": B.WEIGHTS_STATIC, "no promise": 0}[mode]
+    flags = {"independent": B.WEIGHTS_STATIC | B.INPUT_STATIC,
+             "independent+output": B.WEIGHTS_STATIC | B.INPUT_STATIC | B.OUTPUT_STATIC,
+             "dependent": B.WEIGHTS_STATIC, "no promise": 0}[mode]
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # the output promise: every launch between two drains writes a buffer of its own (the second step of the
+    # graph gets a second set), as bench.py does
+    second = [torch.zeros_like(j["Y"]) for j in jobs]
 
-    def step():
-        for j in jobs:
-            B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Y"], status=status, variant=B.VARIANT_AUTO | flags)
-    step()                                   # kernel attributes are set outside the capture
+    def step(outs):
+        for j, Y in zip(jobs, outs):
+            B.patch_gemm(j["X"], j["L"], j["packed"], Y=Y, status=status, variant=B.VARIANT_AUTO | flags)
+    first = [j["Y"] for j in jobs]
+    step(first)                              # kernel attributes are set outside the capture
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
-        step()
-        step()
-    for j in jobs:
-        j["Y"].zero_()
+        step(first)
+        step(second)
+    for Y in first + second:
+        Y.zero_()
     torch.cuda.synchronize()
     g.replay()
     g.replay()
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    for j in jobs:
-        got = to_bits(j["Y"])
-        check_parity(oracle, got, j["Y32"], f"{j['case']['name']} ({mode}, graph)")
-        assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
+    for outs in (first, second):
+        for j, Y in zip(jobs, outs):
+            got = to_bits(Y)
+            check_parity(oracle, got, j["Y32"], f"{j['case']['name']} ({mode}, graph)")
+            assert (got == j["Y16"]).mean() >= 0.99, j["case"]["name"]
 
 
 def test_decode_q4_workload_pack_bit_exact(gpu, oracle):
