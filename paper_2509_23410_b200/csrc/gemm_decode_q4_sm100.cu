@@ -31,11 +31,12 @@
 // the 2:4 kind (half the values per byte of metadata-carrying payload) sits closer to the memory roof.
 //
 // Two CTAs per SM: while one is being set up, drains its last tiles or waits for the preceding kernel before it may
-// write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130).
+// write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130;
+// with the output promise, under which finished CTAs do not wait at all: 0.110).
 // A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
 // columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
 // shared memory.
-// Tried on top of this and dropped (24-GEMM decode step, 0.130 ms): splitting the tile into two K-halves with
+// Tried on top of this and dropped (24-GEMM decode step without the output promise, 0.130 ms): splitting the tile into two K-halves with
 // separate completion tracking, so that a group never waits for its own MMAs (0.142 ms: a third barrier and a second
 // issue sequence per tile cost more than the wait); dequantising the next tile's first 32 values before that wait
 // (0.138 ms: every warp polls again, registers spill); six groups in one CTA per SM (0.150 ms, see above).
