@@ -32,7 +32,7 @@
 //
 // Two CTAs per SM: while one is being set up, drains its last tiles or waits for the preceding kernel before it may
 // write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130;
-// with the output promise, under which finished CTAs do not wait at all: 0.110).
+// with the output promise, under which finished CTAs do not wait at all: 0.110, and 0.107 with no split of K).
 // A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
 // columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
 // shared memory.
@@ -433,9 +433,13 @@ int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch
     int rc = make_x_chunk_tensor_map(&map, X, ldx, M, L->K, 16, 2 * dq::kBatch);
     if (rc) return rc;
     const int TN = int(L->N / kTile), TK = int(L->K / kTile);
-    // Split of K, as for the bf16 row-block schedule: few CTAs per GEMM (several GEMMs resident at once) when the
-    // caller declared the GEMM independent of its predecessor, at least 128 CTAs when it streams alone.
-    int S = decode_cluster_split(TN, TK);
+    // Split of K.  Independent of its predecessor (several GEMMs resident at once): as few, long CTAs as possible --
+    // a CTA's set-up and drain cost about as much as a dozen tiles -- but at least 32 CTAs and at most 96 tiles each
+    // (measured on the 24-GEMM step: 48 tiles 0.110 ms, 96 tiles 0.107 ms, 24 tiles 0.142 ms).
+    int S = 1;
+    while (S < 8 && (TN * S < 32 || TK > 96 * S)) S *= 2;
+    while (S > 1 && S > TK) S /= 2;
+    // Streaming alone once its predecessor is done: see below.
     if (!xstatic) {
         // alone on the GPU, two CTAs per SM: waves of CTAs x (tiles per CTA x ~0.35 us, 0.46 us where two CTAs share
         // an SM, + ~4 us of set-up, pipeline fill and reduction), over the power-of-two splits
