@@ -337,34 +337,6 @@ int patch_gemm_noalloc(const void* X_dev, int64_t ldx, int64_t M,
                        const patch_layout_t* layout, const void* packed_dev,
                        void* Y_dev, int64_t ldy, void* stream);
 
-/*
- * A chain of small-M matmuls in one launch: Y_i = X_i * What_i^T for i = 0 .. n_jobs - 1, in order, where job
- * i + 1 may read -- as its X -- anything jobs 0 .. i wrote (the linear layers of consecutive decoder sub-blocks
- * during generation, Appendix A's memory-bound case).  The same results as n_jobs calls of patch_gemm; what the
- * single launch buys is that the weights of job i + 1 are already streaming into shared memory while the
- * device waits for job i to be complete everywhere, so HBM does not idle at the hand-over between dependent GEMMs.
- * (Launched one by one, a GEMM that must wait for its predecessor restarts its weight stream from nothing.)
- *   jobs             host array; every pointer inside is a device pointer except `layout` (host).  X bf16
- *                    [M x ldx], Y bf16 [M x ldy], as for patch_gemm; the same M for all jobs, 1 <= M <= 16.
- *                    Weights made of bf16 tiles only (no 4-bit kinds).  A Y may alias an earlier job's X or Y.
- *   workspace_dev    patch_gemm_chain_workspace_size bytes, 256-byte aligned; no initialisation needed (the call
- *                    clears the part that must start from zero); calls sharing it must be ordered on one stream
- *   status_dev       as for patch_gemm: first error of a device-side wait given up (PATCH_ERR_TIMEOUT) or of a
- *                    tile table that does not fit its blob (PATCH_ERR_FORMAT); NULL = not reported
- * The launch is cooperative (one CTA per SM, all resident): it does not overlap with the kernels before or after
- * it, and the weights are assumed static in the sense of PATCH_GEMM_WEIGHTS_STATIC for the duration of the call
- * only.  Deterministic.  More than 16 jobs are issued as consecutive launches of up to 16.
- * Returns PATCH_ERR_SHAPE for M outside 1..16 or weights with 4-bit tiles, PATCH_ERR_SIZE for a short workspace.
- */
-typedef struct patch_chain_job_t {
-    const void* X_dev; int64_t ldx;
-    const patch_layout_t* layout; const void* packed_dev;
-    void* Y_dev; int64_t ldy;
-} patch_chain_job_t;
-int patch_gemm_chain_workspace_size(const patch_chain_job_t* jobs, int n_jobs, size_t* bytes_out);
-int patch_gemm_chain(const patch_chain_job_t* jobs, int n_jobs, int64_t M, void* workspace_dev,
-                     size_t workspace_bytes, int* status_dev, void* stream);
-
 /* =========================================================================================
  * Mask learning (the training side of Algorithm 1): soft masks, regulariser sums, hard masks.
  *

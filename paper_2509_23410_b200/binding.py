@@ -26,7 +26,7 @@ ERR_SIZE, ERR_FORMAT, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
 
 EXPORTS = ["patch_packed_size", "patch_pack", "patch_unpack", "patch_gemm_workspace_size",
            "patch_workspace_init", "patch_gemm", "patch_gemm_ex", "patch_gemm_gated", "patch_gemm_gated_workspace_size", "patch_gemm_host", "patch_gemm_host_batch", "patch_gemm_host_batch_pipelined",
-           "patch_gemm_noalloc", "patch_gemm_chain", "patch_gemm_chain_workspace_size",
+           "patch_gemm_noalloc",
            "patch_hard_mask", "patch_pack_patterns", "patch_pack_dev", "patch_read_layout", "patch_soft_mask_workspace_size", "patch_soft_mask",
            "patch_mask_regularizers", "patch_mask_regularizer_coefficients", "patch_soft_mask_backward",
            "patch_strerror", "patch_version"]
@@ -262,33 +262,6 @@ def patch_gemm_host_batch_pipelined(batch, copy_in_stream, copy_out_stream, n_ch
     _check(lib().patch_gemm_host_batch_pipelined(batch, len(batch), 1 if weights_static else 0, int(n_chunks),
                                                  _stream(stream), _stream(copy_in_stream), _stream(copy_out_stream)),
            "patch_gemm_host_batch_pipelined")
-
-
-class ChainJob(ctypes.Structure):
-    """Mirror of ``patch_chain_job_t``."""
-    _fields_ = [("X_dev", ctypes.c_void_p), ("ldx", ctypes.c_int64), ("layout", ctypes.POINTER(Layout)),
-                ("packed_dev", ctypes.c_void_p), ("Y_dev", ctypes.c_void_p), ("ldy", ctypes.c_int64)]
-
-
-def make_chain(jobs):
-    """Marshal a list of dicts (X, layout, packed, Y) once; the tensors and layouts must outlive the result."""
-    arr = (ChainJob * len(jobs))()
-    for a, j in zip(arr, jobs):
-        a.X_dev, a.ldx, a.layout = j["X"].data_ptr(), j["X"].stride(0), ctypes.pointer(j["layout"])
-        a.packed_dev, a.Y_dev, a.ldy = j["packed"].data_ptr(), j["Y"].data_ptr(), j["Y"].stride(0)
-    return arr
-
-
-def patch_gemm_chain_workspace_size(chain) -> int:
-    n = ctypes.c_size_t(0)
-    _check(lib().patch_gemm_chain_workspace_size(chain, len(chain), ctypes.byref(n)), "patch_gemm_chain_workspace_size")
-    return int(n.value)
-
-
-def patch_gemm_chain(chain, M: int, workspace, status=None, stream=None):
-    """Y_i = X_i @ What_i^T for the jobs of ``chain`` in order, in one launch; job i + 1 may read what job i wrote."""
-    _check(lib().patch_gemm_chain(chain, len(chain), int(M), _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream)),
-           "patch_gemm_chain")
 
 
 def patch_gemm_noalloc(X, layout: Layout, packed, Y, stream=None):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatch_b200.so")
 LIB_FI = os.path.join(HERE, "libpatch_b200_fi.so")
-SOURCES = ["pack.cu", "masks.cu", "gemv.cu", "gemm_decode_sm100.cu", "gemm_decode_cluster_sm100.cu", "gemm_prefill_sm100.cu", "gemm_prefill2_sm100.cu", "gemm_prefill_pair_sm100.cu", "gemm_prefill_pair_mixed_sm100.cu", "gemm_decode_q4_sm100.cu", "gemm_chain_sm100.cu", "api.cu"]
+SOURCES = ["pack.cu", "masks.cu", "gemv.cu", "gemm_decode_sm100.cu", "gemm_decode_cluster_sm100.cu", "gemm_prefill_sm100.cu", "gemm_prefill2_sm100.cu", "gemm_prefill_pair_sm100.cu", "gemm_prefill_pair_mixed_sm100.cu", "gemm_decode_q4_sm100.cu", "api.cu"]
 
 
 def _stale(lib: str = LIB) -> bool:

@@ -287,47 +287,3 @@ extern "C" const char* patch_strerror(int status) {
 }
 
 extern "C" int patch_version(void) { return 1; }
-
-// ---------------------------------------------------------------------------------------------
-// chain of small-M matmuls in one launch
-
-static int check_chain_jobs(const patch_chain_job_t* jobs, int n_jobs) {
-    if (n_jobs < 0) return PATCH_ERR_SHAPE;
-    if (n_jobs == 0) return PATCH_OK;
-    if (!jobs) return PATCH_ERR_NULL;
-    for (int i = 0; i < n_jobs; ++i) {
-        if (!jobs[i].layout) return PATCH_ERR_NULL;
-        int rc = validate_layout(jobs[i].layout);
-        if (rc) return rc;
-        if (has_q4_tiles(jobs[i].layout)) return PATCH_ERR_SHAPE;
-    }
-    return PATCH_OK;
-}
-
-extern "C" int patch_gemm_chain_workspace_size(const patch_chain_job_t* jobs, int n_jobs, size_t* bytes_out) {
-    if (!bytes_out) return PATCH_ERR_NULL;
-    int rc = check_chain_jobs(jobs, n_jobs);
-    if (rc) return rc;
-    *bytes_out = chain_workspace_bytes(jobs, n_jobs);
-    return PATCH_OK;
-}
-
-extern "C" int patch_gemm_chain(const patch_chain_job_t* jobs, int n_jobs, int64_t M, void* workspace_dev,
-                                size_t workspace_bytes, int* status_dev, void* stream) {
-    int rc = check_chain_jobs(jobs, n_jobs);
-    if (rc) return rc;
-    if (M < 1 || M > 16) return PATCH_ERR_SHAPE;
-    if (n_jobs == 0) return PATCH_OK;
-    for (int i = 0; i < n_jobs; ++i) {
-        const patch_chain_job_t& j = jobs[i];
-        if (!j.X_dev || !j.packed_dev || !j.Y_dev) return PATCH_ERR_NULL;
-        if (j.ldx < j.layout->K || j.ldy < j.layout->N || j.ldx % 8 || j.ldy % 8) return PATCH_ERR_SHAPE;
-        if (!aligned16(j.X_dev) || !aligned16(j.Y_dev) || !aligned16(j.packed_dev)) return PATCH_ERR_ALIGN;
-    }
-    if (!workspace_dev) return PATCH_ERR_NULL;
-    if (workspace_bytes < chain_workspace_bytes(jobs, n_jobs)) return PATCH_ERR_SIZE;
-    if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return PATCH_ERR_ALIGN;
-    rc = check_device();
-    if (rc) return rc;
-    return launch_chain(jobs, n_jobs, M, workspace_dev, status_dev, static_cast<cudaStream_t>(stream));
-}

@@ -123,9 +123,6 @@ size_t decode_gated_workspace_bytes(const patch_layout_t* L, int64_t M);   // 0 
 int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch_layout_t* L, const uint8_t* packed,
                      __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool wstatic, bool xstatic,
                      bool ystatic = false);
-// chain of small-M matmuls in one persistent launch (gemm_chain_sm100.cu)
-size_t chain_workspace_bytes(const patch_chain_job_t* jobs, int n_jobs);
-int launch_chain(const patch_chain_job_t* jobs, int n_jobs, int64_t M, void* workspace, int* status_dev, cudaStream_t stream);
 inline bool has_q4_tiles(const patch_layout_t* L) { return L->n_dense_q4 != 0 || L->n_sparse_q4 != 0; }
 
 }  // namespace patch

@@ -130,31 +130,6 @@ def test_4bit_weights_are_refused_where_no_kernel_serves_them(binding):
                                    null, null) == binding.ERR_FLAG
 
 
-def test_chain_arguments_are_checked_on_the_host(binding):
-    lib = binding.lib()
-    fake = 1024 * 1024
-    L = binding.patch_packed_size(256, 256, np.zeros((2, 2), np.uint8))
-    L4 = binding.patch_packed_size(256, 256, np.full((2, 2), 3, np.uint8))
-    job = binding.ChainJob(fake, 256, ctypes.pointer(L), fake, fake, 256)
-    arr = (binding.ChainJob * 1)(job)
-    n = ctypes.c_size_t(0)
-    assert lib.patch_gemm_chain_workspace_size(arr, 1, ctypes.byref(n)) == binding.OK and n.value > 0
-    ws = ctypes.c_void_p(fake)
-    null = ctypes.c_void_p(0)
-    assert lib.patch_gemm_chain(arr, 1, 0, ws, n.value, null, null) == binding.ERR_SHAPE
-    assert lib.patch_gemm_chain(arr, 1, 17, ws, n.value, null, null) == binding.ERR_SHAPE
-    assert lib.patch_gemm_chain(arr, 1, 4, ws, 16, null, null) == binding.ERR_SIZE
-    assert lib.patch_gemm_chain(arr, 1, 4, null, n.value, null, null) == binding.ERR_NULL
-    assert lib.patch_gemm_chain(arr, 1, 4, ctypes.c_void_p(fake + 16), n.value, null, null) == binding.ERR_ALIGN
-    assert lib.patch_gemm_chain(arr, 0, 4, null, 0, null, null) == binding.OK            # nothing to do
-    arr[0].ldx = 100
-    assert lib.patch_gemm_chain(arr, 1, 4, ws, n.value, null, null) == binding.ERR_SHAPE
-    arr[0].ldx = 256
-    arr[0].layout = ctypes.pointer(L4)
-    assert lib.patch_gemm_chain(arr, 1, 4, ws, n.value, null, null) == binding.ERR_SHAPE  # 4-bit tiles
-    assert lib.patch_gemm_chain_workspace_size(arr, 1, ctypes.byref(n)) == binding.ERR_SHAPE
-
-
 def test_product_package_does_not_import_the_oracle():
     pkg = os.path.join(ROOT, "paper_2509_23410_b200")
     for dirpath, _, files in os.walk(pkg):
