@@ -248,8 +248,10 @@ int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M,
  *           fp32 values, the finisher of the matching up row-block multiplies.  Otherwise (or for
  *           larger M) the large-M schedule runs, whose CTA holds both accumulators.
  *   flags   0 or PATCH_GEMM_WEIGHTS_STATIC [| PATCH_GEMM_INPUT_STATIC], as for patch_gemm_ex.
- *           With both flags and M <= 16 the call needs no workspace at all: a cluster of CTAs owns a
- *           (gate, up) pair of row-blocks, holds both accumulators and applies the product itself.
+ *           With the weights promise and M <= 16 the call needs no workspace at all: a cluster of CTAs owns a
+ *           (gate, up) pair of row-blocks, holds both accumulators and applies the product itself -- few CTAs
+ *           per launch with both promises, at least 128 with the weights promise alone (the gated product of
+ *           a decoder block reads what the projection before it wrote).
  * Other arguments and error behaviour as patch_gemm.
  */
 int patch_gemm_gated_workspace_size(const patch_layout_t* layout, int64_t M, size_t* bytes_out);

@@ -115,12 +115,13 @@ extern "C" int patch_gemm_gated(const void* X_dev, int64_t ldx, int64_t M, const
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(Y_dev);
     const uint8_t* packed = static_cast<const uint8_t*>(packed_dev);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // small M declared independent of its predecessor: one cluster per (gate, up) pair of row-blocks, no workspace
-    if (M <= 16 && (flags & PATCH_GEMM_WEIGHTS_STATIC) && (flags & PATCH_GEMM_INPUT_STATIC)) {
+    // small M on static weights: one cluster per (gate, up) pair of row-blocks, no workspace -- few CTAs if the launch
+    // was also declared independent of its predecessor, at least 128 if it has to wait for it
+    if (M <= 16 && (flags & PATCH_GEMM_WEIGHTS_STATIC)) {
         CUtensorMap map;
         rc = make_x_tensor_map(&map, X, ldx, M, L->K, 16);
         if (rc) return rc;
-        return launch_decode_cluster_gated(map, L, packed, int(M), Y, ldy, status_dev, s);
+        return launch_decode_cluster_gated(map, L, packed, int(M), Y, ldy, status_dev, s, (flags & PATCH_GEMM_INPUT_STATIC) != 0);
     }
     // small M with a workspace: the stream-K schedule; otherwise the two-row-block schedule, which needs none
     const size_t need = decode_gated_workspace_bytes(L, M);

@@ -339,13 +339,20 @@ int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const
     }
 }
 
-// silu(gate) * up on a stacked gate/up weight (row-blocks interleaved), M <= 16, independent launches.
+// silu(gate) * up on a stacked gate/up weight (row-blocks interleaved), M <= 16, weights static: independent launches
+// (few CTAs, several GEMMs resident) or, with `xstatic` false, a launch that streams alone once its predecessor is
+// done (at least 128 CTAs) -- the gated product of a decoder block reads the output of the projection before it.
 int launch_decode_cluster_gated(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
-                                __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream) {
-    const int TK = int(L->K / kTile);
-    int S = decode_cluster_split(int(L->N / kTile) / 2, 2 * TK);      // a CTA streams the slices of two row-blocks
+                                __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool xstatic) {
+    const int TN = int(L->N / kTile) / 2, TK = int(L->K / kTile);
+    int S = decode_cluster_split(TN, 2 * TK);                         // a CTA streams the slices of two row-blocks
+    if (!xstatic) {
+        S = 1;
+        while (S < 8 && TN * S < 128 && 2 * S <= TK) S *= 2;
+    }
     while (S > 1 && S > TK) S /= 2;
-    return launch_dc_t<16, 3, true, true, true>(map, L, packed, M, S, Y, ldy, status_dev, stream);
+    if (xstatic) return launch_dc_t<16, 3, true, true, true>(map, L, packed, M, S, Y, ldy, status_dev, stream);
+    return launch_dc_t<16, 3, true, false, true>(map, L, packed, M, S, Y, ldy, status_dev, stream);
 }
 
 }  // namespace patch

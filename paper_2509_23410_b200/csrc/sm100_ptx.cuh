@@ -394,7 +394,7 @@ int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const
                           bool xstatic, bool ystatic = false);
 int decode_cluster_split(int TN, int TK);     // cluster size of the row-block schedule for independent GEMMs
 int launch_decode_cluster_gated(const CUtensorMap& map, const patch_layout_t* L, const uint8_t* packed, int M,
-                                __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream);
+                                __nv_bfloat16* Y, int64_t ldy, int* status_dev, cudaStream_t stream, bool xstatic = true);
 
 
 }  // namespace patch

@@ -609,13 +609,15 @@ def test_gated_product_rejects_bad_shapes(gpu):
 @pytest.mark.parametrize("M", [1, 5, 16])
 @pytest.mark.parametrize("shape", [(1024, 768), (1408, 4096), (11008, 4096)])
 def test_gated_product_small_m_schedule(gpu, oracle, M, shape):
-    """M <= 16 with a workspace: the stream-K schedule, where the gate and up row-blocks of a pair are
-    usually finished by different CTAs; every launch-flag combination."""
+    """M <= 16: without a promise and with a workspace the stream-K schedule, where the gate and up row-blocks of a
+    pair are usually finished by different CTAs; with the weights promise a cluster per (gate, up) pair of
+    row-blocks (workspace ignored or absent); every launch-flag combination."""
     torch, B = gpu
     Nh, K = shape
     for flags_arg in (0, B.WEIGHTS_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC):
         _gated_case(gpu, oracle, Nh, K, M, 0.3, 0.8, ws="own", flags_arg=flags_arg)
-    # declared independent of its predecessor: a cluster per (gate, up) pair of row-blocks, no workspace needed
+    # weights static: a cluster per (gate, up) pair of row-blocks, no workspace needed
+    _gated_case(gpu, oracle, Nh, K, M, 0.3, 0.8, ws=None, flags_arg=B.WEIGHTS_STATIC)
     _gated_case(gpu, oracle, Nh, K, M, 0.3, 0.8, ws=None, flags_arg=B.WEIGHTS_STATIC | B.INPUT_STATIC)
     _gated_case(gpu, oracle, Nh, K, M, 1.0, 0.0, ws=None, flags_arg=B.WEIGHTS_STATIC | B.INPUT_STATIC)
 
