@@ -5,11 +5,13 @@
 // bf16 A operand in TENSOR MEMORY -- tcgen05.mma / .mma.sp take A from there -- so a weight value crosses shared
 // memory once, as half a byte on its way in: HBM sees 0.52 B (dense) or 0.39 B (2:4) per weight element, and shared
 // memory sees the same.  (Rebuilding the operand image in shared memory instead costs 32 KB of stores and 32 KB of
-// tensor-core reads per dense tile, ~700 cycles of the shared-memory port against ~170 cycles of HBM time: that
+// tensor-core reads per dense tile, ~700 cycles of the shared-memory port against ~310 cycles of HBM time: that
 // version ran at 1.5 TB/s.)
 //
-//   warp 0        producer: cp.async.bulk of the tile's payload (8 448 / 6 400 B: codes [, metadata], scales) into
-//                 a ring of kRaw slots, and the two activation atoms of the tile's K range into the slot's X buffer
+//   warp 0        producer, in rounds of kBatch tiles: lane i requests tile i of the round -- one cp.async.bulk of its
+//                 payload (8 448 / 6 400 B: codes [, metadata], scales) into a ring of kRaw slots -- and lane 0 the
+//                 round's activations, 2 kBatch atoms in one 3-D tiled copy into the slots' X buffers (one lane
+//                 per tile and three copies each took ~1 000 cycles a tile, three times the tile's HBM time)
 //   warps 5..     kGroups groups of four warps; group g takes tiles g, g + kGroups, ... and owns 64 TMEM columns (its
 //                 operand stage) and an accumulator [128 rows x 16 tokens] of its own.
 //                 Dequantise: thread = tile row = TMEM lane.  It reads its row's codes 16 bytes at a time (the image
@@ -18,17 +20,20 @@
 //                 is the bf16 pair (128 + n, 128 + n'), then (x - 136) * s in two bf16x2 instructions, exact:
 //                 128 + n and n - 8 are small integers and bf16(q * s) is one rounding of the exact product -- and
 //                 writes 16 columns (32 values) per tcgen05.st.
-//                 Multiply: one thread of the group's first warp issues the tile's MMAs (A = the group's TMEM columns,
-//                 B = the slot's X buffer in shared memory; the metadata of a 2:4 tile goes from the payload slot to
-//                 TMEM with tcgen05.cp).  Issuing from one thread for all tiles took ~1 100 cycles per tile next
-//                 to the dequantising warps it shares issue slots with, and bounded the kernel at 1.7 TB/s.
+//                 Multiply: one thread of the group (of a different warp in each group, so that the issuers sit on
+//                 different schedulers) issues the tile's MMAs: A = the group's TMEM columns, B = the slot's X
+//                 buffer in shared memory; the metadata of a 2:4 tile goes from the payload slot to TMEM with
+//                 tcgen05.cp.  Issuing from one thread for all tiles took ~1 100 cycles per tile next to the
+//                 dequantising warps it shares issue slots with, and bounded the kernel at 1.7 TB/s.
+//                 Inside a group one thread waits on the mbarriers; the other 127 wait on a hardware barrier.
 //   warps 1..4    epilogue: sum of the groups' accumulators (ascending group) -> shared memory; then, as in the bf16
 //                 row-block schedule, the S CTAs of a cluster (split-K) sum their partials through distributed
 //                 shared memory in K order and write Y.
 //
-// What bounds it: ~2 instructions per dequantised value, i.e. ~260 issue cycles per dense tile and SM against the
-// ~170 cycles its 8 448 bytes take at this SM's share of the HBM bandwidth: the dense kind is bound by the ALUs,
-// the 2:4 kind (half the values per byte of metadata-carrying payload) sits closer to the memory roof.
+// What bounds it: instruction issue.  A dense tile costs ~1 750 warp instructions (~2 per dequantised value: mask,
+// shift, subtract, multiply, the last two at half rate, plus synchronisation), i.e. ~440 cycles of the SM's four
+// schedulers, against the ~310 cycles its 8 448 bytes take at this SM's share of 8 TB/s; measured in steady state:
+// 425-460 cycles per tile.  A 2:4 tile has half the values but the same fixed work per tile.
 //
 // Two CTAs per SM: while one is being set up, drains its last tiles or waits for the preceding kernel before it may
 // write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130;
@@ -36,8 +41,8 @@
 // A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
 // columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
 // shared memory.
-// Tried on top of this and dropped (24-GEMM decode step without the output promise, 0.130 ms): splitting the tile into two K-halves with
-// separate completion tracking, so that a group never waits for its own MMAs (0.142 ms: a third barrier and a second
+// Tried on top of this and dropped (24-GEMM decode step without the output promise, 0.130 ms): splitting the tile
+// into two K-halves with separate completion tracking, so that a group never waits for its own MMAs (0.142 ms: a third barrier and a second
 // issue sequence per tile cost more than the wait); dequantising the next tile's first 32 values before that wait
 // (0.138 ms: every warp polls again, registers spill); six groups in one CTA per SM (0.150 ms, see above).
 // Same bounded waits, table checks, launch flags and determinism as the other decode kernels; M <= 16.
