@@ -207,7 +207,8 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  * the weight again (there is no large-M schedule for these kinds).  Weights that mix bf16 and 4-bit tiles
  * return PATCH_ERR_SHAPE -- as do
  * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated and patch_gemm_noalloc for such weights (the host
- * entry points follow patch_gemm); patch_pack_dev / patch_pack_patterns report flags above 1 as PATCH_ERR_FLAG.
+ * entry points follow patch_gemm); patch_pack_dev reports flags above 1 as PATCH_ERR_FLAG (patch_pack_patterns
+ * serves the 4-bit kinds: the given 2:4 mask is applied first, then the kept values are quantised).
  * The launch promises mean the same as for bf16 tiles; launches with different promises may split K
  * differently and then differ in the last bit.
  */
@@ -370,6 +371,8 @@ int patch_hard_mask(const float* P_tile_dev, const float* P24_dev, int64_t N, in
  * patch_pack with the 2:4 mask given instead of chosen by magnitude (the deployment input of
  * a learned or otherwise precomputed mask): in every 2:4 tile, group (n, g) keeps the two
  * positions of candidate patterns_dev[n*(K/4) + g]; groups inside dense tiles ignore theirs.
+ * In a 2:4 tile of the 4-bit kind the kept values are then quantised (the "PATCH + 4-bit" combination of
+ * the paper's quantisation table with PATCH's own, learned masks).
  *   patterns_dev  u8 [N x K/4] device, 4-byte aligned, values 0..5
  *   status_dev    optional device int (caller zeroes it): set to PATCH_ERR_FLAG if a 2:4 tile
  *                 holds an index above 5 (that group is then packed as candidate 0)

@@ -252,8 +252,12 @@ __device__ __forceinline__ uint32_t q4_nibble(float v, float s) {
 // nibble index inside its 32-bit word of stored value c (c & 7 decides)
 __device__ __forceinline__ uint32_t q4_nibble_slot(uint32_t c) { return ((c & 1u) << 2) | ((c & 7u) >> 1); }
 
+// GIVEN: the 2:4 mask of a 2:4 tile comes from `patterns` (one candidate index per group of four, as for
+// pack_kernel) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
+template <bool GIVEN>
 __global__ void __launch_bounds__(256)
-pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob, uint64_t table_off) {
+pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob, uint64_t table_off,
+               const uint8_t* __restrict__ patterns, int* status) {
     const int t = blockIdx.x;
     const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
     if (d.kind < PATCH_TILE_DENSE_Q4) return;
@@ -278,7 +282,15 @@ pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __r
         uint32_t i0 = 0, i1 = 1;
         float m;
         if (sparse) {
-            top2_positions(x.x, x.y, i0, i1);
+            if (GIVEN) {
+                uint32_t c = patterns[(int64_t(tn) * kTile + r) * (int64_t(TK) * 32) + tk * 32 + lane];
+                if (c > 5u) { if (status) *status = PATCH_ERR_FLAG; c = 0; }
+                const uint32_t nib = (kCandidateCodes >> (4 * c)) & 0xFu;
+                i0 = nib & 3u;
+                i1 = nib >> 2;
+            } else {
+                top2_positions(x.x, x.y, i0, i1);
+            }
             const uint32_t kept = gather_pair(x.x, x.y, i0, i1);
             v[0] = bf16_bits_to_f32(kept & 0xFFFFu);
             v[1] = bf16_bits_to_f32(kept >> 16);
@@ -444,7 +456,7 @@ static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const
     int64_t n[4] = {0, 0, 0, 0};
     for (int64_t t = 0; t < T; ++t) {
         const uint32_t kind = flags[t];
-        if (kind > PATCH_TILE_SPARSE_2_4_Q4 || (patterns_dev && kind > PATCH_TILE_SPARSE_2_4)) return PATCH_ERR_FLAG;
+        if (kind > PATCH_TILE_SPARSE_2_4_Q4) return PATCH_ERR_FLAG;
         TileDesc d = TileDesc{kind, uint32_t(off / 16), 0xFFFFFFFFu, 0};
         if (kind == PATCH_TILE_SPARSE_2_4) {
             d.meta_off16 = uint32_t((off + kAtomBytes) / 16);
@@ -475,9 +487,14 @@ static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const
         pack_kernel<false, false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
                                                               static_cast<uint8_t*>(packed_dev), L->table_off, nullptr,
                                                               nullptr, none);
-    if (has_q4_tiles(L))
-        pack_q4_kernel<<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
-                                                   static_cast<uint8_t*>(packed_dev), L->table_off);
+    if (has_q4_tiles(L)) {
+        if (patterns_dev)
+            pack_q4_kernel<true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                             static_cast<uint8_t*>(packed_dev), L->table_off, patterns_dev, status_dev);
+        else
+            pack_q4_kernel<false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
+                                                              static_cast<uint8_t*>(packed_dev), L->table_off, nullptr, nullptr);
+    }
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

@@ -124,10 +124,6 @@ def test_4bit_weights_are_refused_where_no_kernel_serves_them(binding):
     bad = binding.Layout.from_buffer_copy(bytes(L4))
     bad.n_dense_q4, bad.n_sparse_q4 = bad.n_sparse_q4 + 1, bad.n_dense_q4 - 1
     assert lib.patch_gemm(*args(4, bad)) == binding.ERR_FORMAT
-    # patterns are for the bf16 2:4 kind only
-    f = np.array([2, 3, 3, 2], np.uint8)
-    assert lib.patch_pack_patterns(fake, 256, ctypes.c_void_p(f.ctypes.data), fake, ctypes.byref(L4), fake, 1 << 24,
-                                   null, null) == binding.ERR_FLAG
 
 
 def test_product_package_does_not_import_the_oracle():

@@ -153,6 +153,31 @@ def test_gemm_back_to_back_and_chain(gpu, oracle):
         ref = got
 
 
+def test_pack_with_given_patterns_bit_exact(gpu, oracle):
+    """patch_pack_patterns on 4-bit kinds: the learned 2:4 mask first, then the quantiser; blob and dequantised
+    matrix bit for bit; a candidate index above 5 inside a 2:4 tile is reported."""
+    torch, B = gpu
+    N, K = 512, 384
+    W = inputs.weight(N, K, 39, "q4-patterns")
+    g = inputs.generator(39, "q4-patterns-c")
+    patterns = g.integers(0, 6, (N, K // 4)).astype(np.uint8)
+    flags = _flags4(N, K, 0.6, "patterns", "half")
+    pd = torch.from_numpy(patterns.reshape(-1)).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    packed, L = B.patch_pack_patterns(to_dev(torch, W), flags, pd, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    blob_o, _ = oracle.pack_patterns(W, flags, patterns)
+    assert (packed.cpu().numpy() == oracle.device_image(blob_o)).all()
+    assert (to_bits(B.patch_unpack(L, packed)) == oracle.unpack(blob_o)).all()
+    bad = patterns.copy()
+    tn, tk = np.argwhere(flags == 3)[0]
+    bad[tn * 128 + 3, tk * 32 + 5] = 6
+    B.patch_pack_patterns(to_dev(torch, W), flags, torch.from_numpy(bad.reshape(-1)).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_FLAG
+
+
 @pytest.mark.parametrize("M", [17, 40, 100])
 def test_gemm_more_than_16_tokens(gpu, oracle, M):
     """More than sixteen tokens are multiplied sixteen at a time; every promise; Y with a row pitch."""

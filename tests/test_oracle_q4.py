@@ -230,3 +230,34 @@ def test_gemm_on_quantised_weights_is_the_gemm_of_the_dequantised_matrix(oracle)
     step = np.abs(f32(Wp)).reshape(N, K // 128, 128).max(-1) / 7.0
     err = np.abs(f32(Wq) - f32(Wp)).reshape(N, K // 128, 128).max(-1)
     assert (err <= 0.52 * step).all()          # 0.5 s + 7 s 2^-9 with s within 2^-9 of max|v| / 7
+
+
+def test_given_patterns_with_4bit_tiles(oracle):
+    """The learned 2:4 mask (one candidate per group) is applied first, then the kept values are quantised: the
+    dequantised matrix is the quantisation, row by row, of exactly the values the candidates keep."""
+    N, K = 256, 256
+    W = inputs.weight(N, K, 10, "q4-patterns")
+    rng = inputs.generator(10, "q4-patterns-c")
+    patterns = rng.integers(0, 6, (N, K // 4)).astype(np.uint8)
+    flags = np.array([[3, 2], [1, 3]], np.uint8)
+    blob, L = oracle.pack_patterns(W, flags, patterns)
+    What = oracle.unpack(blob)
+    S = np.array([[1, 1, 0, 0], [1, 0, 1, 0], [1, 0, 0, 1], [0, 1, 1, 0], [0, 1, 0, 1], [0, 0, 1, 1]], bool)   # typed by hand
+    keep = S[patterns].reshape(N, K)
+    for tn in range(2):
+        for tk in range(2):
+            kind = flags[tn, tk]
+            rows, cols = slice(tn * 128, tn * 128 + 128), slice(tk * 128, tk * 128 + 128)
+            Wt, Kt, got = W[rows, cols], keep[rows, cols], What[rows, cols]
+            for r in range(0, 128, 17):
+                if kind == 1:
+                    assert (got[r] == np.where(Kt[r], Wt[r], 0)).all()
+                elif kind == 2:
+                    assert (got[r] == oracle.q4_group(Wt[r])[2]).all()
+                else:
+                    deq = oracle.q4_group(Wt[r][Kt[r]])[2]
+                    expect = np.zeros(128, np.uint16)
+                    expect[Kt[r]] = deq
+                    assert (got[r] == expect).all()
+    # and it differs from the magnitude rule's result wherever the candidates do
+    assert (oracle.unpack(oracle.pack(W, flags)[0]) != What).any()
