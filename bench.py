@@ -453,21 +453,16 @@ def run_ours(args):
         pack_secs += e0.elapsed_time(e1) * 1e-3
         pack_bytes += c["N"] * c["K"] * 2 + layout.total_bytes
         # the same with the tile flags already on the device: no host work, header and table built by a kernel
-        # (bf16 kinds only; a 4-bit weight is packed from host flags)
-        packed2 = None
-        if c.get("q4"):
-            pack_dev_secs += e0.elapsed_time(e1) * 1e-3
-        else:
-            flags_dev = torch.from_numpy(np.ascontiguousarray(flags, dtype=np.uint8).reshape(-1)).to(dev)
-            packed2 = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
-            B.patch_pack_dev(W, flags_dev, out=packed2)                # warm
-            e0.record()
-            B.patch_pack_dev(W, flags_dev, out=packed2)
-            e1.record()
-            torch.cuda.synchronize()
-            pack_dev_secs += e0.elapsed_time(e1) * 1e-3
-            if not torch.equal(packed, packed2):
-                raise SystemExit("patch_pack_dev and patch_pack disagree")
+        flags_dev = torch.from_numpy(np.ascontiguousarray(flags, dtype=np.uint8).reshape(-1)).to(dev)
+        packed2 = torch.empty(layout.total_bytes, dtype=torch.uint8, device=dev)
+        B.patch_pack_dev(W, flags_dev, out=packed2)                # warm
+        e0.record()
+        B.patch_pack_dev(W, flags_dev, out=packed2)
+        e1.record()
+        torch.cuda.synchronize()
+        pack_dev_secs += e0.elapsed_time(e1) * 1e-3
+        if not torch.equal(packed, packed2):
+            raise SystemExit("patch_pack_dev and patch_pack disagree")
         keep_w = args.check != "none" and not args.workload.startswith("stack")
         mats[key] = (layout, packed, flags, inputs.weight(c["N"], c["K"], inputs.MASTER_SEED, *c["stream"]) if keep_w else None)
         del W, packed2
@@ -683,7 +678,7 @@ def run_ours(args):
         # whole calls, one per matrix, read + written bytes: patch_pack_dev (flags on the device, two kernels) and
         # patch_pack (flags on the host: table built on the host and copied from pageable memory, one kernel)
         "pack": {"gbs": pack_bytes / pack_dev_secs / 1e9, "frac_of_measured_hbm": pack_bytes / pack_dev_secs / 1e9 / peaks["hbm_gbs"],
-                 "entry": "patch_pack" if args.workload == "decode-q4" else "patch_pack_dev",
+                 "entry": "patch_pack_dev",
                  "host_flags_entry_gbs": pack_bytes / pack_secs / 1e9},
     }
     if cpu is not None:

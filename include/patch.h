@@ -207,8 +207,8 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  * the weight again (there is no large-M schedule for these kinds).  Weights that mix bf16 and 4-bit tiles
  * return PATCH_ERR_SHAPE -- as do
  * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated and patch_gemm_noalloc for such weights (the host
- * entry points follow patch_gemm); patch_pack_dev reports flags above 1 as PATCH_ERR_FLAG (patch_pack_patterns
- * serves the 4-bit kinds: the given 2:4 mask is applied first, then the kept values are quantised).
+ * entry points follow patch_gemm).  All pack entry points serve the four kinds (with a given 2:4 mask, the mask
+ * is applied first, then the kept values are quantised).
  * The launch promises mean the same as for bf16 tiles; launches with different promises may split K
  * differently and then differ in the last bit.
  */
@@ -390,13 +390,14 @@ int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t* tile_flag
  *   tile_flags_dev  u8 [N/128 x K/128] device
  *   patterns_dev    NULL (magnitude top-2, as patch_pack) or u8 [N x K/4] device (as patch_pack_patterns)
  *   packed_capacity must hold the blob the flags imply; N/128 * K/128 * 32768 + table always does.
- *                   The host checks only the smallest possible size (all tiles 2:4).
+ *                   The host checks only the smallest possible size (all tiles 2:4 with 4-bit values).
  *   status_dev      optional device int (caller zeroes it): PATCH_ERR_SIZE if the blob did not fit
  *                   (then nothing but a header without magic number is written), PATCH_ERR_FLAG for
- *                   a flag other than 0 / 1 (packed as dense) or a candidate index above 5.
+ *                   a flag above 3 (packed as dense) or a candidate index above 5.
  * Every CTA reads the whole flag array (one byte per tile, from L2), so the extra work grows with the
  * square of the tile count: negligible for the tens of thousands of tiles of an LLM weight.
- * Enqueues one kernel; no copy, no synchronisation.  The host-side layout that patch_gemm
+ * Enqueues two kernels (the second writes the tiles of the 4-bit kinds and returns at once where there are
+ * none); no copy, no synchronisation.  The host-side layout that patch_gemm
  * needs comes from patch_packed_size when the flags are also known on the host, else from
  * patch_read_layout.
  */

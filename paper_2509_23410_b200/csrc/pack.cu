@@ -89,47 +89,54 @@ struct DeviceFlags {
 // writes the header and the padding behind the table; every CTA writes its own table entry.
 // Returns false if the blob does not fit `capacity` (then only a header without magic number is written).
 __device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int t, uint8_t* blob, int* status, TileDesc& d) {
-    __shared__ unsigned long long s_part[8][2];
+    // per warp: tiles before t and in total whose flag has bit 0 (2:4), bit 1 (4-bit values), both
+    __shared__ unsigned long long s_part[8][6];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // count the 2:4 flags before tile t and in total; four flags per load where the array is word aligned
-    unsigned long long sparse_before = 0, sparse_total = 0;
+    unsigned long long cnt[6] = {0, 0, 0, 0, 0, 0};          // {bit0, bit1, both} before t, then in total
     bool bad = false;
+    // four flags per load where the array is word aligned
     const int64_t words = (reinterpret_cast<uintptr_t>(F.flags) & 3u) == 0 ? F.T / 4 : 0;
     for (int64_t i = tid; i < words; i += 256) {
-        const uint32_t w = reinterpret_cast<const uint32_t*>(F.flags)[i];
-        uint32_t ones = w & 0x01010101u;
-        if (w & 0xFEFEFEFEu) {          // a byte that is neither 0 nor 1: an error, packed as dense
+        uint32_t w = reinterpret_cast<const uint32_t*>(F.flags)[i];
+        if (w & 0xFCFCFCFCu) {          // a byte above 3: an error, packed as dense
             bad = true;
-            ones = 0;
+            uint32_t clean = 0;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) ones |= ((w >> (8 * q)) & 0xFFu) == 1u ? 1u << (8 * q) : 0u;
+            for (int q = 0; q < 4; ++q) { const uint32_t b = (w >> (8 * q)) & 0xFFu; clean |= (b <= 3u ? b : 0u) << (8 * q); }
+            w = clean;
         }
+        const uint32_t b0 = w & 0x01010101u, b1 = (w >> 1) & 0x01010101u, bb = b0 & b1;
         const int64_t first = 4 * i;                      // flags first .. first + 3; those below t count as "before"
         const uint32_t below = first + 4 <= t ? 0xFFFFFFFFu : first >= t ? 0u : (1u << (8 * uint32_t(t - first))) - 1u;
-        sparse_total += __popc(ones);
-        sparse_before += __popc(ones & below);
+        cnt[0] += __popc(b0 & below); cnt[1] += __popc(b1 & below); cnt[2] += __popc(bb & below);
+        cnt[3] += __popc(b0); cnt[4] += __popc(b1); cnt[5] += __popc(bb);
     }
     for (int64_t i = 4 * words + tid; i < F.T; i += 256) {
-        const uint8_t f = F.flags[i];
-        bad |= f > 1;
-        sparse_total += f == PATCH_TILE_SPARSE_2_4;
-        sparse_before += (f == PATCH_TILE_SPARSE_2_4) && i < t;
+        uint32_t f = F.flags[i];
+        if (f > 3u) { bad = true; f = 0; }
+        const uint32_t b0 = f & 1u, b1 = f >> 1, bb = b0 & b1, before = i < t ? 1u : 0u;
+        cnt[0] += b0 & before; cnt[1] += b1 & before; cnt[2] += bb & before;
+        cnt[3] += b0; cnt[4] += b1; cnt[5] += bb;
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        sparse_total += __shfl_xor_sync(0xFFFFFFFFu, sparse_total, off);
-        sparse_before += __shfl_xor_sync(0xFFFFFFFFu, sparse_before, off);
+    for (int q = 0; q < 6; ++q) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) cnt[q] += __shfl_xor_sync(0xFFFFFFFFu, cnt[q], off);
+        if (lane == 0) s_part[warp][q] = cnt[q];
     }
-    if (lane == 0) { s_part[warp][0] = sparse_total; s_part[warp][1] = sparse_before; }
     bad = __syncthreads_or(bad) != 0;
-    sparse_total = sparse_before = 0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) { sparse_total += s_part[w][0]; sparse_before += s_part[w][1]; }
-    // as payload bytes: every tile a dense one, minus the saving of each 2:4 tile
-    constexpr unsigned long long kSaving = kDenseBytes - kSparseBytes;
-    const unsigned long long before = (unsigned long long)t * kDenseBytes - sparse_before * kSaving;
-    const unsigned long long total = (unsigned long long)F.T * kDenseBytes - sparse_total * kSaving;
-    const unsigned long long dense = (unsigned long long)F.T - sparse_total;
+    for (int q = 0; q < 6; ++q) {
+        cnt[q] = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) cnt[q] += s_part[w][q];
+    }
+    // tiles of each kind before t and in total: {dense, 2:4, dense 4-bit, 2:4 4-bit}
+    const unsigned long long nb[4] = {(unsigned long long)t - cnt[0] - cnt[1] + cnt[2], cnt[0] - cnt[2], cnt[1] - cnt[2], cnt[2]};
+    const unsigned long long nt[4] = {(unsigned long long)F.T - cnt[3] - cnt[4] + cnt[5], cnt[3] - cnt[5], cnt[4] - cnt[5], cnt[5]};
+    unsigned long long before = 0, total = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < 4; ++k) { before += nb[k] * tile_payload_bytes(k); total += nt[k] * tile_payload_bytes(k); }
     const uint64_t payload_off = (kHeaderBytes + 16 * uint64_t(F.T) + 1023) / 1024 * 1024;
     const uint64_t size = payload_off + total;
     const bool fits = size <= F.capacity && size / 16 <= 0xFFFFFFF0ull;
@@ -140,8 +147,8 @@ __device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int 
             patch_layout_t L;
             L.magic = fits ? kMagic : 0u; L.version = kVersion;
             L.N = F.N; L.K = F.K; L.tile_n = kTile; L.tile_k = kTile;
-            L.n_dense = int64_t(dense); L.n_sparse = F.T - int64_t(dense);
-            L.n_dense_q4 = 0; L.n_sparse_q4 = 0;
+            L.n_dense = int64_t(nt[0]); L.n_sparse = int64_t(nt[1]);
+            L.n_dense_q4 = int64_t(nt[2]); L.n_sparse_q4 = int64_t(nt[3]);
             L.table_off = kHeaderBytes; L.payload_off = payload_off; L.payload_bytes = total; L.total_bytes = size;
             uint32_t* h = reinterpret_cast<uint32_t*>(blob);
             const uint32_t* src = reinterpret_cast<const uint32_t*>(&L);
@@ -154,8 +161,17 @@ __device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int 
     }
     if (!fits) return false;
     const uint64_t off = payload_off + before;
-    if (F.flags[t] == PATCH_TILE_SPARSE_2_4) d = TileDesc{PATCH_TILE_SPARSE_2_4, uint32_t(off / 16), uint32_t((off + kAtomBytes) / 16), 0};
-    else d = TileDesc{PATCH_TILE_DENSE, uint32_t(off / 16), 0xFFFFFFFFu, 0};
+    uint32_t kind = F.flags[t];
+    if (kind > PATCH_TILE_SPARSE_2_4_Q4) kind = PATCH_TILE_DENSE;
+    d = TileDesc{kind, uint32_t(off / 16), 0xFFFFFFFFu, 0};
+    if (kind == PATCH_TILE_SPARSE_2_4) {
+        d.meta_off16 = uint32_t((off + kAtomBytes) / 16);
+    } else if (kind == PATCH_TILE_DENSE_Q4) {
+        d.scales_off16 = uint32_t((off + kDenseQ4CodeBytes) / 16);
+    } else if (kind == PATCH_TILE_SPARSE_2_4_Q4) {
+        d.meta_off16 = uint32_t((off + kSparseQ4CodeBytes) / 16);
+        d.scales_off16 = uint32_t((off + kSparseQ4CodeBytes + kMetaBytes) / 16);
+    }
     if (tid == 0) reinterpret_cast<TileDesc*>(blob + kHeaderBytes)[t] = d;
     return true;
 }
@@ -175,8 +191,8 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
         if (!descriptor_from_flags(F, t, blob, status, d)) return;
     } else {
         d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
-        if (d.kind > PATCH_TILE_SPARSE_2_4) return;      // a 4-bit kind: pack_q4_kernel writes it
     }
+    if (d.kind > PATCH_TILE_SPARSE_2_4) return;          // a 4-bit kind: pack_q4_kernel writes it
     const int tn = t / TK, tk = t - tn * TK;
     const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
     uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
@@ -254,11 +270,13 @@ __device__ __forceinline__ uint32_t q4_nibble_slot(uint32_t c) { return ((c & 1u
 
 // GIVEN: the 2:4 mask of a 2:4 tile comes from `patterns` (one candidate index per group of four, as for
 // pack_kernel) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
-template <bool GIVEN>
+template <bool GIVEN, bool CHECK_HEADER = false>
 __global__ void __launch_bounds__(256)
 pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob, uint64_t table_off,
                const uint8_t* __restrict__ patterns, int* status) {
     const int t = blockIdx.x;
+    // behind the kernel that derives the table from flags in device memory: no table if the blob did not fit
+    if (CHECK_HEADER && *reinterpret_cast<const uint32_t*>(blob) != kMagic) return;
     const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
     if (d.kind < PATCH_TILE_DENSE_Q4) return;
     const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
@@ -523,7 +541,7 @@ extern "C" int patch_pack_dev(const void* W_dev, int64_t ldw, const uint8_t* fla
     if (!aligned16(W_dev) || !aligned16(packed_dev) || (patterns_dev && (reinterpret_cast<uintptr_t>(patterns_dev) & 3u)))
         return PATCH_ERR_ALIGN;
     const uint64_t payload_off = (kHeaderBytes + 16 * uint64_t(T) + 1023) / 1024 * 1024;
-    if (capacity < payload_off + uint64_t(T) * kSparseBytes) return PATCH_ERR_SIZE;   // below the smallest possible blob
+    if (capacity < payload_off + uint64_t(T) * kSparseQ4Bytes) return PATCH_ERR_SIZE;   // below the smallest possible blob
     int rc = check_device();
     if (rc) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -535,6 +553,13 @@ extern "C" int patch_pack_dev(const void* W_dev, int64_t ldw, const uint8_t* fla
     else
         pack_kernel<false, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
                                                              kHeaderBytes, nullptr, status_dev, F);
+    // tiles of the 4-bit kinds, if the flags hold any (the host cannot know): a second pass over the table just written
+    if (patterns_dev)
+        pack_q4_kernel<true, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
+                                                               kHeaderBytes, patterns_dev, status_dev);
+    else
+        pack_q4_kernel<false, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
+                                                                kHeaderBytes, nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

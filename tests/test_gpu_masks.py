@@ -360,7 +360,7 @@ def test_pack_dev_reports_size_and_flag_errors(gpu):
         B.patch_read_layout(small)
     assert e.value.status == B.ERR_FORMAT
     with pytest.raises(B.PatchError) as e:                      # below the smallest possible blob: refused on the host
-        B.patch_pack_dev(W, fd, out=torch.empty(16 * 18432, dtype=torch.uint8, device="cuda"))
+        B.patch_pack_dev(W, fd, out=torch.empty(16 * 6000, dtype=torch.uint8, device="cuda"))
     assert e.value.status == B.ERR_SIZE
     status.zero_()
     bad = flags.copy()

@@ -178,6 +178,48 @@ def test_pack_with_given_patterns_bit_exact(gpu, oracle):
     assert int(status.item()) == B.ERR_FLAG
 
 
+@pytest.mark.parametrize("with_patterns", [False, True])
+def test_pack_with_flags_in_device_memory(gpu, oracle, with_patterns):
+    """patch_pack_dev on all four kinds: header, table and payloads equal to patch_pack's from host flags (which
+    equal the oracle's), the layout read back from the blob, a flag above 3 reported and packed as dense."""
+    torch, B = gpu
+    N, K = 640, 1152
+    W = inputs.weight(N, K, 40, "q4-dev")
+    flags = _flags4(N, K, 0.5, "dev", "half")
+    assert set(np.unique(flags)) == {0, 1, 2, 3}
+    Wd = to_dev(torch, W)
+    g = inputs.generator(40, "q4-dev-c")
+    patterns = g.integers(0, 6, (N, K // 4)).astype(np.uint8)
+    pd = torch.from_numpy(patterns.reshape(-1)).cuda() if with_patterns else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.patch_pack_dev(Wd, torch.from_numpy(flags.reshape(-1)).cuda(), patterns=pd, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    L = B.patch_read_layout(out)
+    blob_o, L_o = oracle.pack_patterns(W, flags, patterns) if with_patterns else oracle.pack(W, flags)
+    for f, _ in B.Layout._fields_:
+        assert getattr(L, f) == getattr(L_o, f), f
+    assert (out[:L.total_bytes].cpu().numpy() == oracle.device_image(blob_o)).all()
+    # the packed weight is usable as it is: all-4-bit part of the flags through the matmul
+    flags4 = flags | 2
+    out4 = B.patch_pack_dev(Wd, torch.from_numpy(flags4.reshape(-1)).cuda(), patterns=pd, status=status)
+    L4 = B.patch_read_layout(out4)
+    X = inputs.activation(8, K, 40, "q4-dev-x")
+    Y = run_gemm(gpu, X, L4, out4[:L4.total_bytes], B.VARIANT_AUTO)
+    blob4 = oracle.pack_patterns(W, flags4, patterns)[0] if with_patterns else oracle.pack(W, flags4)[0]
+    check_parity(oracle, Y, oracle.gemm_f64(X, oracle.unpack(blob4))[0], "matmul on a blob packed from device flags")
+    bad = flags.reshape(-1).copy()
+    bad[5] = 9
+    out_b = B.patch_pack_dev(Wd, torch.from_numpy(bad).cuda(), patterns=pd, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_FLAG
+    good = bad.copy()
+    good[5] = 0                                  # the bad flag was packed as dense
+    ref = B.patch_pack_dev(Wd, torch.from_numpy(good).cuda(), patterns=pd)
+    Lb = B.patch_read_layout(ref)
+    assert torch.equal(out_b[:Lb.total_bytes], ref[:Lb.total_bytes])
+
+
 @pytest.mark.parametrize("M", [17, 40, 100])
 def test_gemm_more_than_16_tokens(gpu, oracle, M):
     """More than sixteen tokens are multiplied sixteen at a time; every promise; Y with a row pitch."""
@@ -222,11 +264,6 @@ def test_unsupported_combinations_are_refused(gpu):
     assert refused(lambda: B.patch_gemm(X4, L, packed, workspace=ws, variant=B.VARIANT_GEMV)) == B.ERR_SHAPE
     assert refused(lambda: B.patch_gemm_gated(X4, L, packed, workspace=ws)) == B.ERR_SHAPE
     assert refused(lambda: B.patch_gemm_noalloc(X4, L, packed, torch.empty((4, N), dtype=torch.bfloat16, device="cuda"))) == B.ERR_SHAPE
-    flags_dev = torch.from_numpy(all_q4.reshape(-1)).cuda()
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    B.patch_pack_dev(W, flags_dev, status=status)
-    torch.cuda.synchronize()
-    assert int(status.item()) == B.ERR_FLAG
 
 
 def test_bad_table_entries_are_reported(gpu, oracle):
