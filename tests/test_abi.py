@@ -262,7 +262,7 @@ def test_pack_dev_validates_on_the_host():
     assert lib.patch_pack_dev(p, 120, p, None, 128, 128, 128, 128, p, 1 << 20, None, None) == B.ERR_SHAPE
     assert lib.patch_pack_dev(p, 128, p, None, 128, 128, 128, 64, p, 1 << 20, None, None) == B.ERR_TILE
     assert lib.patch_pack_dev(p, 128, p, p + 2, 128, 128, 128, 128, p, 1 << 20, None, None) == B.ERR_ALIGN
-    assert lib.patch_pack_dev(p, 128, p, None, 128, 128, 128, 128, p, 1024 + 18431, None, None) == B.ERR_SIZE
+    assert lib.patch_pack_dev(p, 128, p, None, 128, 128, 128, 128, p, 1024 + 6399, None, None) == B.ERR_SIZE
     assert lib.patch_read_layout(None, None, None) == B.ERR_NULL
 
 
