@@ -389,3 +389,24 @@ def test_device_only_deployment_chain(gpu, oracle):
     Y32, _ = oracle.gemm_f64(X, oracle.unpack(oracle.pack_patterns(W, rf, rp)[0]))
     relF, maxrel = oracle.parity_metrics(f32(Y), Y32)
     assert relF <= 2e-3 and maxrel <= 1e-2, (relF, maxrel)
+
+
+def test_device_only_deployment_chain_with_4bit_tiles(gpu, oracle):
+    """The same chain for the 4-bit combination: learned flags and candidates stay on the device, bit 1 is set on the
+    device, the blob is the oracle's for the same masks, and the matmul multiplies by its dequantised matrix."""
+    torch, B = gpu
+    N, K, M = 768, 512, 5
+    W = inputs.weight(N, K, 54, "chain4")
+    X = inputs.activation(M, K, 54, "chain4", M)
+    PT, P6 = logits(N, K, 0.5, 54, "chain4")
+    flags_d, patterns_d = B.patch_hard_mask(torch.from_numpy(PT).cuda(), torch.from_numpy(P6).cuda(), N, K)
+    packed = B.patch_pack_dev(to_dev(torch, W), flags_d | 2, patterns=patterns_d)
+    L = B.patch_read_layout(packed)
+    rf, rp = oracle.hard_mask(PT, P6, N, K)
+    assert (L.n_dense, L.n_sparse, L.n_dense_q4, L.n_sparse_q4) == (0, 0, int((rf == 0).sum()), int((rf == 1).sum()))
+    blob_o, _ = oracle.pack_patterns(W, rf | 2, rp)
+    assert (packed[:L.total_bytes].cpu().numpy() == oracle.device_image(blob_o)).all()
+    Y = to_bits(B.patch_gemm(to_dev(torch, X), L, packed[:L.total_bytes]))
+    Y32, _ = oracle.gemm_f64(X, oracle.unpack(blob_o))
+    relF, maxrel = oracle.parity_metrics(f32(Y), Y32)
+    assert relF <= 2e-3 and maxrel <= 1e-2, (relF, maxrel)
