@@ -21,7 +21,17 @@ extern "C" int patch_gemm_workspace_size(const patch_layout_t* L, int64_t M, siz
     int rc = validate_layout(L);
     if (rc) return rc;
     if (M < 0) return PATCH_ERR_SHAPE;
-    *bytes_out = has_q4_tiles(L) ? 0 : decode_workspace_bytes(L, M);    // the 4-bit schedule needs none
+    if (has_q4_tiles(L)) {
+        // 4-bit tiles: nothing for the decode kernel; beyond 64 tokens, room for the weight's bf16 image
+        *bytes_out = 0;
+        if (M > 64 && !L->n_dense && !L->n_sparse) {
+            patch_layout_t E;
+            q4_expanded_layout(L, &E);
+            *bytes_out = size_t(E.total_bytes);
+        }
+        return PATCH_OK;
+    }
+    *bytes_out = decode_workspace_bytes(L, M);
     return PATCH_OK;
 }
 
@@ -52,7 +62,22 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
         if (L->n_dense || L->n_sparse || variant == PATCH_VARIANT_GEMV || variant == PATCH_VARIANT_PAIR) return PATCH_ERR_SHAPE;
         rc = check_device();
         if (rc) return rc;
-        // more than 16 tokens: sixteen at a time, one launch each, under the caller's promises (a later launch
+        if (M > 64) {
+            // many tokens: the weight is rewritten once as the bf16 blob of its dequantised values (in the
+            // workspace), and the large-M schedule multiplies by that -- the same values, so the same result as
+            // the decode kernel's definition; the blob was just written, so no promise is passed on
+            patch_layout_t E;
+            q4_expanded_layout(L, &E);
+            if (!workspace_dev) return PATCH_ERR_NULL;
+            if (workspace_bytes < E.total_bytes) return PATCH_ERR_SIZE;
+            if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return PATCH_ERR_ALIGN;
+            cudaStream_t s4 = static_cast<cudaStream_t>(stream);
+            rc = launch_expand_q4(L, static_cast<const uint8_t*>(packed_dev), &E, static_cast<uint8_t*>(workspace_dev), s4);
+            if (rc) return rc;
+            return launch_prefill(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, &E, static_cast<const uint8_t*>(workspace_dev),
+                                  static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, s4, false, false);
+        }
+        // 17 .. 64 tokens: sixteen at a time, one launch each, under the caller's promises (a later launch
         // may not assume more than the first: it can start while the kernels before this call still run)
         for (int64_t m0 = 0; m0 < M; m0 += 16) {
             rc = launch_decode_q4(static_cast<const __nv_bfloat16*>(X_dev) + m0 * ldx, ldx, M - m0 < 16 ? M - m0 : 16, L,

@@ -380,6 +380,59 @@ __device__ __forceinline__ void unpack_q4_tile(const TileDesc& d, const uint8_t*
     }
 }
 
+// A weight of 4-bit tiles rewritten as the blob of bf16 tiles with the same dequantised values: what the large-M
+// kernels multiply by when the layer has many tokens (the dequantisation of a tile is then paid once per call
+// instead of once per token tile).  One CTA per tile, one warp per tile row as above; the output offset of tile t
+// follows from its 4-bit offset (the payloads of both blobs are laid out in tile order, so the number of dense
+// tiles before t is (off4 - 6400 t) / 2048 in units of the two payload sizes' difference).
+__global__ void __launch_bounds__(256)
+expand_q4_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, uint32_t pay0, int64_t T, uint8_t* __restrict__ out,
+                 patch_layout_t out_layout) {
+    const int t = blockIdx.x;
+    const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
+    const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
+    const uint64_t off4 = uint64_t(d.payload_off16) * 16 - pay0;
+    const uint64_t n_dense_before = (off4 - uint64_t(kSparseQ4Bytes) * uint64_t(t)) / (kDenseQ4Bytes - kSparseQ4Bytes);
+    const uint64_t off = pay0 + n_dense_before * kDenseBytes + (uint64_t(t) - n_dense_before) * kSparseBytes;
+    if (threadIdx.x == 0) {
+        reinterpret_cast<TileDesc*>(out + table_off)[t] =
+            TileDesc{sparse ? uint32_t(PATCH_TILE_SPARSE_2_4) : uint32_t(PATCH_TILE_DENSE), uint32_t(off / 16),
+                     sparse ? uint32_t((off + kAtomBytes) / 16) : 0xFFFFFFFFu, 0};
+        if (t == 0) {
+            uint32_t* h = reinterpret_cast<uint32_t*>(out);
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(&out_layout);
+            for (uint32_t i = 0; i < kHeaderBytes / 4; ++i) h[i] = i < sizeof(out_layout) / 4 ? src[i] : 0u;
+        }
+    }
+    const uint32_t* codes = reinterpret_cast<const uint32_t*>(blob + uint64_t(d.payload_off16) * 16);
+    const uint16_t* scales = reinterpret_cast<const uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
+    uint8_t* pay = out + off;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    if (sparse)   // the metadata block is already in hardware order
+        reinterpret_cast<uint2*>(pay + kAtomBytes)[threadIdx.x] =
+            reinterpret_cast<const uint2*>(blob + uint64_t(d.meta_off16) * 16)[threadIdx.x];
+    for (uint32_t rr = 0; rr < 16; ++rr) {
+        const uint32_t r = rr * 8 + warp;
+        const float s = bf16_bits_to_f32(scales[r]);
+        if (sparse) {
+            // kept values 2 lane, 2 lane + 1 of the row: four bytes of the atom
+            const uint32_t word = codes[((lane >> 4) * 128 + r) * 4 + ((lane & 15u) >> 2)];
+            const uint32_t a = q4_dequant_bits((word >> (4 * q4_nibble_slot(2 * lane))) & 0xFu, s);
+            const uint32_t b = q4_dequant_bits((word >> (4 * q4_nibble_slot(2 * lane + 1))) & 0xFu, s);
+            *reinterpret_cast<uint32_t*>(pay + atom_chunk_offset(r, lane >> 2) + (lane & 3u) * 4) = a | (b << 16);
+        } else {
+            // columns 4 lane .. 4 lane + 3: eight bytes of atom (column / 64)
+            const uint32_t word = codes[((lane >> 3) * 128 + r) * 4 + ((lane & 7u) >> 1)];
+            uint32_t o[4];
+#pragma unroll
+            for (uint32_t p = 0; p < 4; ++p) o[p] = q4_dequant_bits((word >> (4 * q4_nibble_slot(4 * lane + p))) & 0xFu, s);
+            *reinterpret_cast<uint2*>(pay + (lane >> 4) * kAtomBytes + atom_chunk_offset(r, (lane & 15u) >> 1) + (lane & 1u) * 8) =
+                make_uint2(o[0] | (o[1] << 16), o[2] | (o[3] << 16));
+        }
+    }
+    (void)T;
+}
+
 __global__ void __launch_bounds__(256)
 unpack_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
               uint16_t* __restrict__ What, int64_t ldw) {
@@ -424,6 +477,27 @@ unpack_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, int TK,
             *reinterpret_cast<uint4*>(dst + 8) = make_uint4(out[4], out[5], out[6], out[7]);
         }
     }
+}
+
+// Layout of the bf16 blob that holds the dequantised values of an all-4-bit weight, and the expansion itself.
+void q4_expanded_layout(const patch_layout_t* L, patch_layout_t* out) {
+    *out = *L;
+    out->n_dense = L->n_dense_q4;
+    out->n_sparse = L->n_sparse_q4;
+    out->n_dense_q4 = 0;
+    out->n_sparse_q4 = 0;
+    out->payload_bytes = uint64_t(kDenseBytes) * out->n_dense + uint64_t(kSparseBytes) * out->n_sparse;
+    out->total_bytes = out->payload_off + out->payload_bytes;
+}
+
+int launch_expand_q4(const patch_layout_t* L, const uint8_t* packed, const patch_layout_t* out_layout, uint8_t* out,
+                     cudaStream_t stream) {
+    const int64_t T = (L->N / kTile) * (L->K / kTile);
+    // the padding behind the table (up to the first payload) is part of the blob
+    if (cudaMemsetAsync(out + L->table_off + 16 * T, 0, L->payload_off - L->table_off - 16 * T, stream) != cudaSuccess)
+        return PATCH_ERR_CUDA;
+    expand_q4_kernel<<<unsigned(T), 256, 0, stream>>>(packed, L->table_off, uint32_t(L->payload_off), T, out, *out_layout);
+    return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
 }  // namespace patch

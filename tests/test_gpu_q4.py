@@ -220,9 +220,9 @@ def test_pack_with_flags_in_device_memory(gpu, oracle, with_patterns):
     assert torch.equal(out_b[:Lb.total_bytes], ref[:Lb.total_bytes])
 
 
-@pytest.mark.parametrize("M", [17, 40, 100])
+@pytest.mark.parametrize("M", [17, 40, 64])
 def test_gemm_more_than_16_tokens(gpu, oracle, M):
-    """More than sixteen tokens are multiplied sixteen at a time; every promise; Y with a row pitch."""
+    """17 to 64 tokens are multiplied sixteen at a time (no workspace); every promise; Y with a row pitch."""
     torch, B = gpu
     N, K = 640, 768
     W = inputs.weight(N, K, 38, "q4-chunks")
@@ -241,6 +241,50 @@ def test_gemm_more_than_16_tokens(gpu, oracle, M):
         check_parity(oracle, got, Y32, f"M={M} promise={promise:#x}")
         assert (got == Y16).mean() >= 0.99
         assert (Ybuf[:, N:] == 3.0).all()
+
+
+@pytest.mark.parametrize("p", [0.0, 1.0, 0.5])
+@pytest.mark.parametrize("M", [65, 300, 1000])
+def test_gemm_many_tokens(gpu, oracle, M, p):
+    """Beyond 64 tokens the weight is rewritten as the bf16 blob of its dequantised values (in the workspace) and the
+    large-M schedule multiplies by it: the same matrix, so the same reference."""
+    torch, B = gpu
+    N, K = 640, 768
+    W = inputs.weight(N, K, 44, "q4-many")
+    X = inputs.activation(M, K, 44, "q4-many", M)
+    flags = _flags4(N, K, p, ("many", p))
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    need = B.patch_gemm_workspace_size(L, M)
+    assert need == oracle.packed_size(N, K, flags & 1).total_bytes         # the size of the bf16 blob of the same mask
+    Y32, Y16 = oracle.gemm_f64(X, What)
+    Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO)
+    check_parity(oracle, Y, Y32, f"q4 M={M} p={p}")
+    assert (Y == Y16).mean() >= 0.99
+    assert (run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC) == Y).all()
+    # what was written to the workspace is the bf16 blob of the dequantised matrix: it unpacks to that matrix
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws)
+    torch.cuda.synchronize()
+    E = B.patch_read_layout(ws)
+    assert (E.n_dense, E.n_sparse, E.n_dense_q4, E.n_sparse_q4) == (L.n_dense_q4, L.n_sparse_q4, 0, 0)
+    assert (to_bits(B.patch_unpack(E, ws)) == What).all()
+    with pytest.raises(B.PatchError) as e:
+        B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws[:need - 256])
+    assert e.value.status == B.ERR_SIZE
+
+
+def test_gemm_many_tokens_llama_shape_sampled(gpu, oracle):
+    torch, B = gpu
+    N, K, M = 4096, 4096, 2048
+    W = inputs.weight(N, K, 45, "q4-many-llama")
+    X = inputs.activation(M, K, 45, "q4-many-llama", M)
+    flags = _flags4(N, K, 0.5, "many-llama")
+    What = oracle.prune(W, flags)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO)
+    rows = np.array([0, 1, 127, 128, 239, 240, 1000, 2047])
+    check_parity(oracle, Y[rows], oracle.gemm_f64_rows(X, rows, What), "q4 4096x4096 M=2048, sampled token rows")
 
 
 def test_unsupported_combinations_are_refused(gpu):
