@@ -743,6 +743,9 @@ def test_independent_launch_schedule(gpu, oracle, N, K, M):
     check_parity(oracle, other, Y32, "stream-K")
     again = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC)
     assert (again == got).all()
+    # with the output promise too (only the launch's first cluster waits for its predecessor): the same bits
+    out = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC | B.OUTPUT_STATIC)
+    assert (out == got).all()
 
 
 def test_independent_launches_back_to_back(gpu, oracle):
@@ -768,6 +771,17 @@ def test_independent_launches_back_to_back(gpu, oracle):
     assert int(status.item()) == 0
     for j in jobs:
         check_parity(oracle, to_bits(j["Y"]), j["ref"], "independent stream")
+    # the same stream under the output promise: every launch between two synchronisations writes a buffer of its own
+    outs = [[torch.zeros_like(j["Y"]) for j in jobs] for _ in range(3)]
+    for rep in range(3):
+        for j, Y in zip(jobs, outs[rep]):
+            B.patch_gemm(j["X"], j["L"], j["packed"], Y=Y, workspace=ws, status=status,
+                         variant=B.VARIANT_AUTO | B.WEIGHTS_STATIC | B.INPUT_STATIC | B.OUTPUT_STATIC)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for rep in range(3):
+        for j, Y in zip(jobs, outs[rep]):
+            assert (to_bits(Y) == to_bits(j["Y"])).all()
 
 
 @pytest.mark.parametrize("M", [4, 48, 300])
