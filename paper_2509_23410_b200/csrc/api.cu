@@ -72,7 +72,7 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
             if (workspace_bytes < E.total_bytes) return PATCH_ERR_SIZE;
             if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return PATCH_ERR_ALIGN;
             cudaStream_t s4 = static_cast<cudaStream_t>(stream);
-            rc = launch_expand_q4(L, static_cast<const uint8_t*>(packed_dev), &E, static_cast<uint8_t*>(workspace_dev), s4);
+            rc = launch_expand_q4(L, static_cast<const uint8_t*>(packed_dev), &E, static_cast<uint8_t*>(workspace_dev), status_dev, s4);
             if (rc) return rc;
             return launch_prefill(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, &E, static_cast<const uint8_t*>(workspace_dev),
                                   static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, s4, false, false);

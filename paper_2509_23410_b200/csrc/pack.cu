@@ -386,31 +386,51 @@ __device__ __forceinline__ void unpack_q4_tile(const TileDesc& d, const uint8_t*
 // follows from its 4-bit offset (the payloads of both blobs are laid out in tile order, so the number of dense
 // tiles before t is (off4 - 6400 t) / 2048 in units of the two payload sizes' difference).
 __global__ void __launch_bounds__(256)
-expand_q4_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, uint32_t pay0, int64_t T, uint8_t* __restrict__ out,
-                 patch_layout_t out_layout) {
+expand_q4_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, uint32_t pay0, uint32_t end16, uint8_t* __restrict__ out,
+                 patch_layout_t out_layout, int* status) {
     const int t = blockIdx.x;
     const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
     const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
-    const uint64_t off4 = uint64_t(d.payload_off16) * 16 - pay0;
-    const uint64_t n_dense_before = (off4 - uint64_t(kSparseQ4Bytes) * uint64_t(t)) / (kDenseQ4Bytes - kSparseQ4Bytes);
+    // The entry is checked before a byte of the tile is read: a 4-bit kind, the payload inside the blob and at an
+    // offset that tiles of the two sizes before it can add up to.  Otherwise the status word says so, nothing is
+    // read, and the tile's entry in the new table points at the first payload as a 2:4 tile (its contents are
+    // unspecified, but every later read stays inside the new blob).
+    const uint32_t len16 = (sparse ? kSparseQ4Bytes : kDenseQ4Bytes) / 16, pay0_16 = pay0 / 16;
+    bool bad = d.kind < PATCH_TILE_DENSE_Q4 || d.kind > PATCH_TILE_SPARSE_2_4_Q4 || d.payload_off16 < pay0_16 ||
+               d.payload_off16 > end16 || len16 > end16 - d.payload_off16;
+    const int64_t rest = int64_t(d.payload_off16) * 16 - int64_t(pay0) - int64_t(kSparseQ4Bytes) * t;
+    constexpr int64_t kStep = int64_t(kDenseQ4Bytes) - int64_t(kSparseQ4Bytes);
+    bad = bad || rest < 0 || rest % kStep != 0 || rest / kStep > t;
+    if (bad) {
+        if (threadIdx.x == 0) {
+            if (status) atomicCAS(status, PATCH_OK, PATCH_ERR_FORMAT);
+            reinterpret_cast<TileDesc*>(out + table_off)[t] =
+                TileDesc{uint32_t(PATCH_TILE_SPARSE_2_4), pay0_16, uint32_t((pay0 + kAtomBytes) / 16), 0};
+        }
+        if (t != 0) return;
+    }
+    const uint64_t n_dense_before = bad ? 0 : uint64_t(rest / kStep);
     const uint64_t off = pay0 + n_dense_before * kDenseBytes + (uint64_t(t) - n_dense_before) * kSparseBytes;
     if (threadIdx.x == 0) {
-        reinterpret_cast<TileDesc*>(out + table_off)[t] =
-            TileDesc{sparse ? uint32_t(PATCH_TILE_SPARSE_2_4) : uint32_t(PATCH_TILE_DENSE), uint32_t(off / 16),
-                     sparse ? uint32_t((off + kAtomBytes) / 16) : 0xFFFFFFFFu, 0};
+        if (!bad)
+            reinterpret_cast<TileDesc*>(out + table_off)[t] =
+                TileDesc{sparse ? uint32_t(PATCH_TILE_SPARSE_2_4) : uint32_t(PATCH_TILE_DENSE), uint32_t(off / 16),
+                         sparse ? uint32_t((off + kAtomBytes) / 16) : 0xFFFFFFFFu, 0};
         if (t == 0) {
             uint32_t* h = reinterpret_cast<uint32_t*>(out);
             const uint32_t* src = reinterpret_cast<const uint32_t*>(&out_layout);
             for (uint32_t i = 0; i < kHeaderBytes / 4; ++i) h[i] = i < sizeof(out_layout) / 4 ? src[i] : 0u;
         }
     }
-    const uint32_t* codes = reinterpret_cast<const uint32_t*>(blob + uint64_t(d.payload_off16) * 16);
-    const uint16_t* scales = reinterpret_cast<const uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
+    if (bad) return;
+    // metadata and scales follow the codes (the table's own offsets for them are not used)
+    const uint8_t* src = blob + uint64_t(d.payload_off16) * 16;
+    const uint32_t* codes = reinterpret_cast<const uint32_t*>(src);
+    const uint16_t* scales = reinterpret_cast<const uint16_t*>(src + (sparse ? kSparseQ4CodeBytes + kMetaBytes : kDenseQ4CodeBytes));
     uint8_t* pay = out + off;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
     if (sparse)   // the metadata block is already in hardware order
-        reinterpret_cast<uint2*>(pay + kAtomBytes)[threadIdx.x] =
-            reinterpret_cast<const uint2*>(blob + uint64_t(d.meta_off16) * 16)[threadIdx.x];
+        reinterpret_cast<uint2*>(pay + kAtomBytes)[threadIdx.x] = reinterpret_cast<const uint2*>(src + kSparseQ4CodeBytes)[threadIdx.x];
     for (uint32_t rr = 0; rr < 16; ++rr) {
         const uint32_t r = rr * 8 + warp;
         const float s = bf16_bits_to_f32(scales[r]);
@@ -430,7 +450,6 @@ expand_q4_kernel(const uint8_t* __restrict__ blob, uint64_t table_off, uint32_t 
                 make_uint2(o[0] | (o[1] << 16), o[2] | (o[3] << 16));
         }
     }
-    (void)T;
 }
 
 __global__ void __launch_bounds__(256)
@@ -491,12 +510,13 @@ void q4_expanded_layout(const patch_layout_t* L, patch_layout_t* out) {
 }
 
 int launch_expand_q4(const patch_layout_t* L, const uint8_t* packed, const patch_layout_t* out_layout, uint8_t* out,
-                     cudaStream_t stream) {
+                     int* status_dev, cudaStream_t stream) {
     const int64_t T = (L->N / kTile) * (L->K / kTile);
     // the padding behind the table (up to the first payload) is part of the blob
     if (cudaMemsetAsync(out + L->table_off + 16 * T, 0, L->payload_off - L->table_off - 16 * T, stream) != cudaSuccess)
         return PATCH_ERR_CUDA;
-    expand_q4_kernel<<<unsigned(T), 256, 0, stream>>>(packed, L->table_off, uint32_t(L->payload_off), T, out, *out_layout);
+    expand_q4_kernel<<<unsigned(T), 256, 0, stream>>>(packed, L->table_off, uint32_t(L->payload_off), uint32_t(L->total_bytes / 16),
+                                                      out, *out_layout, status_dev);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

@@ -126,7 +126,7 @@ int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch
 // all-4-bit weight -> bf16 blob of its dequantised values (pack.cu), for the large-M kernels
 void q4_expanded_layout(const patch_layout_t* L, patch_layout_t* out);
 int launch_expand_q4(const patch_layout_t* L, const uint8_t* packed, const patch_layout_t* out_layout, uint8_t* out,
-                     cudaStream_t stream);
+                     int* status_dev, cudaStream_t stream);
 inline bool has_q4_tiles(const patch_layout_t* L) { return L->n_dense_q4 != 0 || L->n_sparse_q4 != 0; }
 
 }  // namespace patch

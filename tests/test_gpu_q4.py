@@ -329,6 +329,20 @@ def test_bad_table_entries_are_reported(gpu, oracle):
         torch.cuda.synchronize()
         assert int(status.item()) == B.ERR_FORMAT, (word, value)
     assert (run_gemm(gpu, X, L, packed, B.VARIANT_AUTO) == good).all()
+    # the same with many tokens, where the blob is first rewritten as bf16 tiles: also an offset inside the blob that
+    # no sequence of tiles before it can add up to
+    Xm = inputs.activation(100, K, 37, "q4-bad-many")
+    ws = torch.zeros(B.patch_gemm_workspace_size(L, 100), dtype=torch.uint8, device="cuda")
+    for word, value in ((0, 1), (0, 9), (1, int(L.total_bytes // 16) - 3), (1, 2), (1, int(L.payload_off // 16) + 1)):
+        blob = packed.clone()
+        entry = blob[int(L.table_off) + 16 * 3:int(L.table_off) + 16 * 4].view(torch.int32)
+        entry[word] = value
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.patch_gemm(to_dev(torch, Xm), L, blob, workspace=ws, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == B.ERR_FORMAT, (word, value)
+    Ym = run_gemm(gpu, Xm, L, packed, B.VARIANT_AUTO)
+    check_parity(oracle, Ym, oracle.gemm_f64(Xm, oracle.prune(W, flags))[0], "after the bad tables")
 
 
 # ---------------------------------------------------------------------------------------------
