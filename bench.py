@@ -675,7 +675,7 @@ def run_ours(args):
         "replay_stats": replay_stats,
         "gpu_launches": args.steps * len(jobs),
         "clocks": clocks,
-        # whole calls, one per matrix, read + written bytes: patch_pack_dev (flags on the device, two kernels) and
+        # whole calls, one per matrix, read + written bytes: patch_pack_dev (flags on the device, one kernel) and
         # patch_pack (flags on the host: table built on the host and copied from pageable memory, one kernel)
         "pack": {"gbs": pack_bytes / pack_dev_secs / 1e9, "frac_of_measured_hbm": pack_bytes / pack_dev_secs / 1e9 / peaks["hbm_gbs"],
                  "entry": "patch_pack_dev",

@@ -398,8 +398,7 @@ int patch_pack_patterns(const void* W_dev, int64_t ldw, const uint8_t* tile_flag
  *                   a flag above 3 (packed as dense) or a candidate index above 5.
  * Every CTA reads the whole flag array (one byte per tile, from L2), so the extra work grows with the
  * square of the tile count: negligible for the tens of thousands of tiles of an LLM weight.
- * Enqueues two kernels (the second writes the tiles of the 4-bit kinds and returns at once where there are
- * none); no copy, no synchronisation.  The host-side layout that patch_gemm
+ * Enqueues one kernel; no copy, no synchronisation.  The host-side layout that patch_gemm
  * needs comes from patch_packed_size when the flags are also known on the host, else from
  * patch_read_layout.
  */

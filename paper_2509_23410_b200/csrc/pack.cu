@@ -176,13 +176,164 @@ __device__ __forceinline__ bool descriptor_from_flags(const DeviceFlags& F, int 
     return true;
 }
 
+// ---------------------------------------------------------------------------------------------
+// 4-bit kinds.  Sixteen lanes per tile row (a warp works on two rows at a time); a lane holds eight consecutive
+// elements of its row: one 32-bit word of codes of a dense tile, half a word of a 2:4 tile.
+//   scale  s = bf16(max|v| / 7) over the row's stored values (all 128, or the 64 the 2:4 selection keeps)
+//   code   q + 8 with q = clamp(rint(v / s), -7, 7), 0 where s = 0; fp32 arithmetic, IEEE division
+// Codes are stored eight to a 32-bit word, in the row's order of stored values: the even ones of a word in nibbles
+// 0..3, the odd ones in nibbles 4..7, so that (word >> 4j) & 0x000F000F is the pair (2j, 2j + 1) in the two halves
+// of a register -- what the dequantising GEMM kernel turns into two bf16 with one instruction.  Four words (32
+// values) make a 16-byte unit; unit j of tile row r lives at byte (128 j + r) * 16, so the 32 threads of a warp
+// that each own a row read 512 consecutive bytes.
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
+// bit position, inside its 32-bit word, of the code of stored value c (c & 7 decides)
+__host__ __device__ constexpr uint32_t q4_code_shift(uint32_t c) { return 4u * (((c & 1u) << 2) | ((c & 7u) >> 1)); }
+// q = clamp(rint(v / s), -7, 7) with the IEEE quotient; 0 where s = 0
+__device__ __forceinline__ int q4_quantise_exact(float v, float s) {
+    if (s == 0.0f) return 0;
+    return int(fminf(fmaxf(rintf(__fdiv_rn(v, s)), -7.0f), 7.0f));
+}
+__host__ __device__ constexpr uint32_t q4_sum_shifted(uint32_t x, uint32_t n) {   // sum of x << shift(i), i < n, modulo 2^32
+    uint32_t acc = 0;
+    for (uint32_t i = 0; i < n; ++i) acc += x << q4_code_shift(i);
+    return acc;
+}
+// Scale of a row whose largest magnitude is m (a bf16 value): bf16(fp32(m / 7)).  m * fp32(1/7) is within two
+// fp32 steps of the quotient, and the quotient a / 7 of an 8-bit significand a stays at least 1 / 1792 (relative)
+// away from every point c / 2^k, c odd with nine bits, where the rounding to bf16 changes (the difference is
+// |2^j a - 7 c| / 1792 with an even and an odd term), so the product rounds to the same bf16 as the quotient; the
+// division is kept for magnitudes near the bottom of the range, where m may be subnormal.
+__device__ __forceinline__ __nv_bfloat16 q4_scale(float m) {
+    return __float2bfloat16_rn(m >= 0x1p-90f ? m * (1.0f / 7.0f) : __fdiv_rn(m, 7.0f));
+}
+// Codes q + 8 of NV stored values of one row (the first NV of a word), each at its bit position, summed.
+// v and s are bf16 values: significands a, b < 256.  The exact quotient v / s is then either a half-integer or at
+// least 1 / 1020 away from the nearest one (|a 2^j - (2k + 1) b| >= 1 over a denominator 2 b 2^i <= 1020 for
+// quotients above 1/4), and s = bf16(max / 7) keeps every quotient of the row below 7.02, so nothing needs
+// clamping.  t = v * (1 / s), with the reciprocal good to 2^-23, is within 1.3e-6 of the exact quotient.  Adding
+// and subtracting 1.5 * 2^13 snaps t to the grid of 2^-10: onto the half-integer exactly if the quotient is one,
+// never onto or across it otherwise.  Adding 1.5 * 2^23 then rounds to the nearest integer, ties to even -- the
+// result of rint on the IEEE quotient -- and leaves q in the low mantissa bits.  Rows whose scale is zero,
+// subnormal or huge (or whose values are not numbers) take the division itself.
+template <uint32_t NV>
+__device__ __forceinline__ uint32_t q4_codes(const float (&v)[NV], float s) {
+    constexpr float kSnap = 12288.0f, kRound = 12582912.0f;
+    constexpr uint32_t kRoundBits = 0x4B400000u;
+    constexpr uint32_t kBias = q4_sum_shifted(8u - kRoundBits, NV);
+    uint32_t word;
+    if (s >= 0x1p-100f && s <= 0x1p100f) {
+        float inv;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(s));
+        word = kBias;
+#pragma unroll
+        for (uint32_t i = 0; i < NV; ++i) {
+            const float t = v[i] * inv;
+            const float snapped = (t + kSnap) - kSnap;
+            word += __float_as_uint(snapped + kRound) << q4_code_shift(i);
+        }
+    } else {
+        word = 0;
+#pragma unroll
+        for (uint32_t i = 0; i < NV; ++i) word += uint32_t(q4_quantise_exact(v[i], s) + 8) << q4_code_shift(i);
+    }
+    return word;
+}
+// nibble index inside its 32-bit word of stored value c
+__device__ __forceinline__ uint32_t q4_nibble_slot(uint32_t c) { return ((c & 1u) << 2) | ((c & 7u) >> 1); }
+
+// One tile of a 4-bit kind, by the 256 threads of a CTA.
+// GIVEN: the 2:4 mask of a 2:4 tile comes from `patterns` (one candidate index per group of four, as for
+// the bf16 kinds) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
+template <bool GIVEN>
+__device__ __forceinline__ void pack_q4_tile(const TileDesc& d, const uint16_t* __restrict__ W, int64_t ldw, int TK, int t,
+                                             uint8_t* __restrict__ blob, const uint8_t* __restrict__ patterns, int* status) {
+    const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
+    const int tn = t / TK, tk = t - tn * TK;
+    const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
+    uint32_t* codes = reinterpret_cast<uint32_t*>(blob + uint64_t(d.payload_off16) * 16);
+    uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;                    // only used if sparse
+    uint16_t* scales = reinterpret_cast<uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, c = lane & 15u;
+    const uint32_t r0 = warp * 2 + (lane >> 4);           // this lane's rows: r0 + 16 it
+    // all eight loads of the lane are issued before the first row is quantised: 4 KB in flight per warp
+    uint4 xs[8];
+    uint32_t given[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+    for (uint32_t it = 0; it < 8; ++it) {
+        const uint32_t r = r0 + 16 * it;
+        xs[it] = ld_stream(wt + int64_t(r) * ldw + c * 8);
+        if (GIVEN && sparse)   // the candidate indices of this lane's two groups: one aligned 2-byte load
+            given[it] = *reinterpret_cast<const uint16_t*>(patterns + (int64_t(tn) * kTile + r) * (int64_t(TK) * 32) + tk * 32 + c * 2);
+    }
+#pragma unroll
+    for (uint32_t it = 0; it < 8; ++it) {
+        const uint32_t r = r0 + 16 * it;
+        const uint32_t in[4] = {xs[it].x, xs[it].y, xs[it].z, xs[it].w};
+        if (!sparse) {
+            float v[8];
+            float m = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                v[2 * i] = __uint_as_float(in[i] << 16);
+                v[2 * i + 1] = __uint_as_float(in[i] & 0xFFFF0000u);
+                m = fmaxf(m, fmaxf(fabsf(v[2 * i]), fabsf(v[2 * i + 1])));
+            }
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+            const __nv_bfloat16 sb = q4_scale(m);
+            if (c == 0) scales[r] = __bfloat16_as_ushort(sb);
+            codes[((c >> 2) * 128 + r) * 4 + (c & 3u)] = q4_codes<8>(v, __bfloat162float(sb));
+        } else {
+            float v[4];
+            uint32_t pos = 0;            // position codes of the lane's two groups, four bits each
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                uint32_t i0, i1;
+                if (GIVEN) {
+                    uint32_t cand = (given[it] >> (8 * g)) & 0xFFu;
+                    if (cand > 5u) { if (status) *status = PATCH_ERR_FLAG; cand = 0; }
+                    const uint32_t nib = (kCandidateCodes >> (4 * cand)) & 0xFu;
+                    i0 = nib & 3u;
+                    i1 = nib >> 2;
+                } else {
+                    top2_positions(in[2 * g], in[2 * g + 1], i0, i1);
+                }
+                const uint32_t kept = gather_pair(in[2 * g], in[2 * g + 1], i0, i1);
+                v[2 * g] = __uint_as_float(kept << 16);
+                v[2 * g + 1] = __uint_as_float(kept & 0xFFFF0000u);
+                pos |= (i0 | (i1 << 2)) << (4 * g);
+            }
+            float m = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+            const __nv_bfloat16 sb = q4_scale(m);
+            if (c == 0) scales[r] = __bfloat16_as_ushort(sb);
+            // stored values 4c .. 4c + 3 of the row: half of word c / 2 (values 0..3 of a word sit in bits 0-7 and
+            // 16-23, values 4..7 eight bits higher); the even lane of a pair stores the word and the metadata
+            uint32_t half = q4_codes<4>(v, __bfloat162float(sb)) << (8 * (c & 1u));
+            pos <<= 8 * (c & 1u);
+            const uint32_t word = half | __shfl_xor_sync(0xFFFFFFFFu, half, 1);
+            const uint32_t code = pos | __shfl_xor_sync(0xFFFFFFFFu, pos, 1);
+            if ((c & 1u) == 0) {
+                const uint32_t w = c >> 1;                     // word of the row (0..7) = 16-column chunk u
+                codes[((w >> 2) * 128 + r) * 4 + (w & 3u)] = word;
+                // metadata row L = 16q + 8h + i, word j, low half for tile rows 16q+i, high for 16q+8+i
+                const uint32_t Lr = (r & ~15u) + 8u * (w & 1u) + (r & 7u), j = w >> 1, hi = (r >> 3) & 1u;
+                *reinterpret_cast<uint16_t*>(meta + Lr * 16 + j * 4 + hi * 2) = uint16_t(code);
+            }
+        }
+    }
+}
+
 // One CTA per tile.  W is read with 16-byte loads, the payload is written with 16-byte stores.
 // GIVEN: the 2:4 mask comes from `patterns` (one candidate index per group of four, [N x K/4]
 // row-major) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
 // DEVFLAGS: the tile's descriptor is computed from tile flags in device memory instead of read
 // from a table the host wrote.
 template <bool GIVEN, bool DEVFLAGS>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob,
             uint64_t table_off, const uint8_t* __restrict__ patterns, int* status, DeviceFlags F) {
     const int t = blockIdx.x;
@@ -192,7 +343,10 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
     } else {
         d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
     }
-    if (d.kind > PATCH_TILE_SPARSE_2_4) return;          // a 4-bit kind: pack_q4_kernel writes it
+    if (d.kind > PATCH_TILE_SPARSE_2_4) {                // a 4-bit kind
+        pack_q4_tile<GIVEN>(d, W, ldw, TK, t, blob, patterns, status);
+        return;
+    }
     const int tn = t / TK, tk = t - tn * TK;
     const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
     uint8_t* pay = blob + uint64_t(d.payload_off16) * 16;
@@ -245,103 +399,6 @@ pack_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __rest
             // metadata row L = 16q + 8h + i, word j, low half for tile rows 16q+i, high for 16q+8+i
             const uint32_t L = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
             *reinterpret_cast<uint16_t*>(meta + L * 16 + j * 4 + hi * 2) = uint16_t(code);
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// 4-bit kinds.  One warp per tile row, lane g holds the row's g-th group of four consecutive elements.
-//   scale  s = bf16(max|v| / 7) over the row's stored values (all 128, or the 64 the 2:4 selection keeps)
-//   code   q + 8 with q = clamp(rint(v / s), -7, 7), 0 where s = 0; fp32 arithmetic, IEEE division
-// Codes are stored eight to a 32-bit word, in the row's order of stored values: the even ones of a word in nibbles
-// 0..3, the odd ones in nibbles 4..7, so that (word >> 4j) & 0x000F000F is the pair (2j, 2j + 1) in the two halves
-// of a register -- what the dequantising GEMM kernel turns into two bf16 with one instruction.  Four words (32
-// values) make a 16-byte unit; unit j of tile row r lives at byte (128 j + r) * 16, so the 32 threads of a warp
-// that each own a row read 512 consecutive bytes.
-
-__device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
-__device__ __forceinline__ uint32_t q4_nibble(float v, float s) {
-    if (s == 0.0f) return 8u;
-    const float r = fminf(fmaxf(rintf(__fdiv_rn(v, s)), -7.0f), 7.0f);
-    return uint32_t(int(r) + 8);
-}
-// nibble index inside its 32-bit word of stored value c (c & 7 decides)
-__device__ __forceinline__ uint32_t q4_nibble_slot(uint32_t c) { return ((c & 1u) << 2) | ((c & 7u) >> 1); }
-
-// GIVEN: the 2:4 mask of a 2:4 tile comes from `patterns` (one candidate index per group of four, as for
-// pack_kernel) instead of the magnitude rule; an index above 5 raises PATCH_ERR_FLAG in *status.
-template <bool GIVEN, bool CHECK_HEADER = false>
-__global__ void __launch_bounds__(256)
-pack_q4_kernel(const uint16_t* __restrict__ W, int64_t ldw, int TK, uint8_t* __restrict__ blob, uint64_t table_off,
-               const uint8_t* __restrict__ patterns, int* status) {
-    const int t = blockIdx.x;
-    // behind the kernel that derives the table from flags in device memory: no table if the blob did not fit
-    if (CHECK_HEADER && *reinterpret_cast<const uint32_t*>(blob) != kMagic) return;
-    const TileDesc d = reinterpret_cast<const TileDesc*>(blob + table_off)[t];
-    if (d.kind < PATCH_TILE_DENSE_Q4) return;
-    const bool sparse = d.kind == PATCH_TILE_SPARSE_2_4_Q4;
-    const int tn = t / TK, tk = t - tn * TK;
-    const uint16_t* wt = W + int64_t(tn) * kTile * ldw + int64_t(tk) * kTile;
-    uint8_t* codes = blob + uint64_t(d.payload_off16) * 16;
-    uint8_t* meta = blob + uint64_t(d.meta_off16) * 16;                    // only used if sparse
-    uint16_t* scales = reinterpret_cast<uint16_t*>(blob + uint64_t(d.scales_off16) * 16);
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    // all sixteen rows of the warp are requested before the first is quantised: 4 KB in flight per warp
-    uint2 xs[16];
-#pragma unroll
-    for (uint32_t rr = 0; rr < 16; ++rr)
-        xs[rr] = *reinterpret_cast<const uint2*>(wt + int64_t(rr * 8 + warp) * ldw + lane * 4);
-#pragma unroll
-    for (uint32_t rr = 0; rr < 16; ++rr) {
-        const uint32_t r = rr * 8 + warp;
-        const uint2 x = xs[rr];
-        float v[4] = {bf16_bits_to_f32(x.x & 0xFFFFu), bf16_bits_to_f32(x.x >> 16),
-                      bf16_bits_to_f32(x.y & 0xFFFFu), bf16_bits_to_f32(x.y >> 16)};
-        uint32_t i0 = 0, i1 = 1;
-        float m;
-        if (sparse) {
-            if (GIVEN) {
-                uint32_t c = patterns[(int64_t(tn) * kTile + r) * (int64_t(TK) * 32) + tk * 32 + lane];
-                if (c > 5u) { if (status) *status = PATCH_ERR_FLAG; c = 0; }
-                const uint32_t nib = (kCandidateCodes >> (4 * c)) & 0xFu;
-                i0 = nib & 3u;
-                i1 = nib >> 2;
-            } else {
-                top2_positions(x.x, x.y, i0, i1);
-            }
-            const uint32_t kept = gather_pair(x.x, x.y, i0, i1);
-            v[0] = bf16_bits_to_f32(kept & 0xFFFFu);
-            v[1] = bf16_bits_to_f32(kept >> 16);
-            m = fmaxf(fabsf(v[0]), fabsf(v[1]));
-        } else {
-            m = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
-        const __nv_bfloat16 sb = __float2bfloat16_rn(__fdiv_rn(m, 7.0f));
-        const float s = __bfloat162float(sb);
-        if (lane == 0) scales[r] = __bfloat16_as_ushort(sb);
-        // this lane's nibbles, each shifted to its slot of the 32-bit word it belongs to; the lanes of a word
-        // (two for a dense row, four for a 2:4 row) combine them with shuffles and the first one stores
-        uint32_t word = 0;
-        if (sparse) {
-#pragma unroll
-            for (int i = 0; i < 2; ++i) word |= q4_nibble(v[i], s) << (4 * q4_nibble_slot(2 * lane + i));
-            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-            if ((lane & 3u) == 0) reinterpret_cast<uint32_t*>(codes)[((lane >> 4) * 128 + r) * 4 + ((lane & 15u) >> 2)] = word;
-            // position codes of the four groups of a 16-column chunk -> 16 bits of metadata (hardware order)
-            uint32_t code = (i0 | (i1 << 2)) << (4 * (lane & 3u));
-            code |= __shfl_xor_sync(0xFFFFFFFFu, code, 1);
-            code |= __shfl_xor_sync(0xFFFFFFFFu, code, 2);
-            const uint32_t u = lane >> 2;
-            const uint32_t Lr = (r & ~15u) + 8u * (u & 1u) + (r & 7u), j = u >> 1, hi = (r >> 3) & 1u;
-            if ((lane & 3u) == 0) *reinterpret_cast<uint16_t*>(meta + Lr * 16 + j * 4 + hi * 2) = uint16_t(code);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) word |= q4_nibble(v[i], s) << (4 * q4_nibble_slot(4 * lane + i));
-            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-            if ((lane & 1u) == 0) reinterpret_cast<uint32_t*>(codes)[((lane >> 3) * 128 + r) * 4 + ((lane & 7u) >> 1)] = word;
         }
     }
 }
@@ -599,14 +656,6 @@ static int pack_impl(const void* W_dev, int64_t ldw, const uint8_t* flags, const
         pack_kernel<false, false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
                                                               static_cast<uint8_t*>(packed_dev), L->table_off, nullptr,
                                                               nullptr, none);
-    if (has_q4_tiles(L)) {
-        if (patterns_dev)
-            pack_q4_kernel<true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
-                                                             static_cast<uint8_t*>(packed_dev), L->table_off, patterns_dev, status_dev);
-        else
-            pack_q4_kernel<false><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK),
-                                                              static_cast<uint8_t*>(packed_dev), L->table_off, nullptr, nullptr);
-    }
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 
@@ -647,13 +696,6 @@ extern "C" int patch_pack_dev(const void* W_dev, int64_t ldw, const uint8_t* fla
     else
         pack_kernel<false, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
                                                              kHeaderBytes, nullptr, status_dev, F);
-    // tiles of the 4-bit kinds, if the flags hold any (the host cannot know): a second pass over the table just written
-    if (patterns_dev)
-        pack_q4_kernel<true, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
-                                                               kHeaderBytes, patterns_dev, status_dev);
-    else
-        pack_q4_kernel<false, true><<<unsigned(T), 256, 0, s>>>(static_cast<const uint16_t*>(W_dev), ldw, int(TK), blob,
-                                                                kHeaderBytes, nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? PATCH_OK : PATCH_ERR_CUDA;
 }
 

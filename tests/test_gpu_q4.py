@@ -63,6 +63,41 @@ def test_pack_with_row_pitch_and_extreme_values(gpu, oracle):
     assert (out[:, K:] == 7.0).all()
 
 
+@pytest.mark.parametrize("kind", [2, 3])
+def test_pack_quantiser_corner_cases(gpu, oracle, kind):
+    """Rows built to sit on the quantiser's decision points: quotients that are exact half-integers (ties go to the
+    even code), quotients one bf16 step to either side of a half-integer, scales that are subnormal, zero or near
+    the top of the range, and a row whose largest magnitude makes max / 7 round up in bf16."""
+    torch, B = gpu
+    N, K = 256, 256
+    g = inputs.generator(35, "q4-corners", kind)
+    vals = np.zeros((N, K), np.float32)
+    halves = np.arange(-7, 7, dtype=np.float32) + 0.5                      # -6.5 .. 6.5
+    for r in range(N):
+        e = [-3, 0, 5, -60, 40, -126, 100][r % 7]
+        s = np.float32(2.0) ** e                                           # a scale that max / 7 hits exactly
+        row = g.choice(halves, K) * s
+        if r % 3 == 1:                                                     # one bf16 step off the tie, either side
+            bits = inputs.f32_to_bf16_bits(row).astype(np.int32) + g.choice([-1, 1], K)
+            row = (bits.astype(np.uint32) << 16).view(np.float32)
+        row[g.integers(0, K, 8)] = 7 * s * g.choice([-1, 1], 8)             # the row maximum, in both tiles
+        row[:4], row[128:132] = 7 * s, -7 * s
+        vals[r] = row
+    W = inputs.f32_to_bf16_bits(vals)
+    W[3, :] = 0                                                            # scale 0
+    W[4, :] = np.tile(np.arange(1, 65, dtype=np.uint16), 4)                # subnormal values, subnormal scale
+    W[5, :] = np.tile(np.arange(0x0080, 0x00C0, dtype=np.uint16), 4)       # smallest normal values
+    W[6, :] = np.tile(np.arange(0x7F00, 0x7F40, dtype=np.uint16), 4)       # near the largest finite bf16
+    W[7, :] = np.tile(np.array([0x3F80, 0x3E12, 0xBE13, 0x3D55], np.uint16), 64)   # max / 7 = 0.142857: rounds in bf16
+    flags = np.full((N // 128) * (K // 128), kind, np.uint8)
+    packed, L = B.patch_pack(to_dev(torch, W), flags)
+    blob_o, _ = oracle.pack(W, flags)
+    image = oracle.device_image(blob_o)
+    bad = np.flatnonzero(packed.cpu().numpy() != image)
+    assert bad.size == 0, f"{bad.size} bytes differ, first at {bad[:8]}"
+    assert (to_bits(B.patch_unpack(L, packed)) == oracle.unpack(blob_o)).all()
+
+
 @pytest.mark.parametrize("M", [1, 5, 16])
 @pytest.mark.parametrize("p", [0.0, 1.0, 0.4])
 @pytest.mark.parametrize("N,K", [(128, 128), (256, 1152), (640, 384), (4096, 1024), (512, 8192)])
