@@ -216,14 +216,14 @@ __device__ __forceinline__ __nv_bfloat16 q4_scale(float m) {
 // and subtracting 1.5 * 2^13 snaps t to the grid of 2^-10: onto the half-integer exactly if the quotient is one,
 // never onto or across it otherwise.  Adding 1.5 * 2^23 then rounds to the nearest integer, ties to even -- the
 // result of rint on the IEEE quotient -- and leaves q in the low mantissa bits.  Rows whose scale is zero,
-// subnormal or huge (or whose values are not numbers) take the division itself.
+// subnormal or huge, and lanes that hold a NaN (`numbers` false), take the division itself.
 template <uint32_t NV>
-__device__ __forceinline__ uint32_t q4_codes(const float (&v)[NV], float s) {
+__device__ __forceinline__ uint32_t q4_codes(const float (&v)[NV], float s, bool numbers) {
     constexpr float kSnap = 12288.0f, kRound = 12582912.0f;
     constexpr uint32_t kRoundBits = 0x4B400000u;
     constexpr uint32_t kBias = q4_sum_shifted(8u - kRoundBits, NV);
     uint32_t word;
-    if (s >= 0x1p-100f && s <= 0x1p100f) {
+    if (numbers && s >= 0x1p-100f && s <= 0x1p100f) {
         float inv;
         asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(s));
         word = kBias;
@@ -271,6 +271,9 @@ __device__ __forceinline__ void pack_q4_tile(const TileDesc& d, const uint16_t* 
     for (uint32_t it = 0; it < 8; ++it) {
         const uint32_t r = r0 + 16 * it;
         const uint32_t in[4] = {xs[it].x, xs[it].y, xs[it].z, xs[it].w};
+        // a bf16 is a NaN iff its magnitude bits exceed 0x7F80: adding 0x7F then carries into bit 15
+        const bool numbers = (((((in[0] & 0x7FFF7FFFu) + 0x007F007Fu) | ((in[1] & 0x7FFF7FFFu) + 0x007F007Fu)) |
+                               (((in[2] & 0x7FFF7FFFu) + 0x007F007Fu) | ((in[3] & 0x7FFF7FFFu) + 0x007F007Fu))) & 0x80008000u) == 0;
         if (!sparse) {
             float v[8];
             float m = 0.0f;
@@ -284,7 +287,7 @@ __device__ __forceinline__ void pack_q4_tile(const TileDesc& d, const uint16_t* 
             for (int off = 8; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
             const __nv_bfloat16 sb = q4_scale(m);
             if (c == 0) scales[r] = __bfloat16_as_ushort(sb);
-            codes[((c >> 2) * 128 + r) * 4 + (c & 3u)] = q4_codes<8>(v, __bfloat162float(sb));
+            codes[((c >> 2) * 128 + r) * 4 + (c & 3u)] = q4_codes<8>(v, __bfloat162float(sb), numbers);
         } else {
             float v[4];
             uint32_t pos = 0;            // position codes of the lane's two groups, four bits each
@@ -312,7 +315,7 @@ __device__ __forceinline__ void pack_q4_tile(const TileDesc& d, const uint16_t* 
             if (c == 0) scales[r] = __bfloat16_as_ushort(sb);
             // stored values 4c .. 4c + 3 of the row: half of word c / 2 (values 0..3 of a word sit in bits 0-7 and
             // 16-23, values 4..7 eight bits higher); the even lane of a pair stores the word and the metadata
-            uint32_t half = q4_codes<4>(v, __bfloat162float(sb)) << (8 * (c & 1u));
+            uint32_t half = q4_codes<4>(v, __bfloat162float(sb), numbers) << (8 * (c & 1u));
             pos <<= 8 * (c & 1u);
             const uint32_t word = half | __shfl_xor_sync(0xFFFFFFFFu, half, 1);
             const uint32_t code = pos | __shfl_xor_sync(0xFFFFFFFFu, pos, 1);
