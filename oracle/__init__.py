@@ -33,7 +33,18 @@ class Layout(ctypes.Structure):
 
 
 def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (plain -O2, OpenMP over outputs, no fast-math)."""
+    """Compile the oracle with gcc (plain -O2, OpenMP over outputs, no fast-math).
+
+    With PATCH_ORACLE_SANITIZE=1 in the environment: a serial build with AddressSanitizer and
+    UndefinedBehaviorSanitizer, every finding fatal (the process must then be started with the
+    sanitizer's runtime preloaded; ``tests/test_oracle_sanitizers.py`` does that)."""
+    if os.environ.get("PATCH_ORACLE_SANITIZE") == "1":
+        out = os.path.join(_HERE, "libpatch_oracle_san.so")
+        if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(_SRC):
+            subprocess.run(["gcc", "-O1", "-g", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra",
+                            "-Wno-unknown-pragmas", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+                            "-fno-omit-frame-pointer", "-o", out, _SRC, "-lm"], check=True)
+        return out
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
                "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
