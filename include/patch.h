@@ -205,8 +205,9 @@ int patch_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stre
  * for M <= 16 tokens (the decode case, where the bytes of the weight are what the layer costs); no workspace.
  * 17 to 64 tokens are multiplied sixteen at a time, one launch after the other.  Beyond 64 tokens the call first
  * rewrites the weight as the bf16 blob of its dequantised values -- into the workspace, which must then hold
- * patch_gemm_workspace_size(layout, M) bytes (the size of that blob; no initialisation needed) -- and runs the
- * large-M schedule on it: the dequantisation is paid once per call.  Weights that mix bf16 and 4-bit tiles
+ * patch_gemm_workspace_size(layout, M) bytes (32 MiB plus the size of that blob; no initialisation needed: the
+ * blob starts 32 MiB into the workspace, past every word that other calls keep zero there, so the workspace may be
+ * shared with them as before) -- and runs the large-M schedule on it: the dequantisation is paid once per call.  Weights that mix bf16 and 4-bit tiles
  * return PATCH_ERR_SHAPE -- as do
  * PATCH_VARIANT_GEMV / PATCH_VARIANT_PAIR, patch_gemm_gated and patch_gemm_noalloc for such weights (the host
  * entry points follow patch_gemm).  All pack entry points serve the four kinds (with a given 2:4 mask, the mask

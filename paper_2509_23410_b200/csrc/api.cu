@@ -27,7 +27,7 @@ extern "C" int patch_gemm_workspace_size(const patch_layout_t* L, int64_t M, siz
         if (M > 64 && !L->n_dense && !L->n_sparse) {
             patch_layout_t E;
             q4_expanded_layout(L, &E);
-            *bytes_out = size_t(E.total_bytes);
+            *bytes_out = kQ4ExpandOffset + size_t(E.total_bytes);
         }
         return PATCH_OK;
     }
@@ -69,12 +69,13 @@ extern "C" int patch_gemm_ex(const void* X_dev, int64_t ldx, int64_t M, const pa
             patch_layout_t E;
             q4_expanded_layout(L, &E);
             if (!workspace_dev) return PATCH_ERR_NULL;
-            if (workspace_bytes < E.total_bytes) return PATCH_ERR_SIZE;
+            if (workspace_bytes < kQ4ExpandOffset + E.total_bytes) return PATCH_ERR_SIZE;
             if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return PATCH_ERR_ALIGN;
             cudaStream_t s4 = static_cast<cudaStream_t>(stream);
-            rc = launch_expand_q4(L, static_cast<const uint8_t*>(packed_dev), &E, static_cast<uint8_t*>(workspace_dev), status_dev, s4);
+            uint8_t* image = static_cast<uint8_t*>(workspace_dev) + kQ4ExpandOffset;     // the words other calls keep zero stay untouched
+            rc = launch_expand_q4(L, static_cast<const uint8_t*>(packed_dev), &E, image, status_dev, s4);
             if (rc) return rc;
-            return launch_prefill(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, &E, static_cast<const uint8_t*>(workspace_dev),
+            return launch_prefill(static_cast<const __nv_bfloat16*>(X_dev), ldx, M, &E, image,
                                   static_cast<__nv_bfloat16*>(Y_dev), ldy, status_dev, s4, false, false);
         }
         // 17 .. 64 tokens: sixteen at a time, one launch each, under the caller's promises (a later launch

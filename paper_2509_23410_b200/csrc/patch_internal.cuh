@@ -127,6 +127,10 @@ int launch_decode_q4(const __nv_bfloat16* X, int64_t ldx, int64_t M, const patch
 void q4_expanded_layout(const patch_layout_t* L, patch_layout_t* out);
 int launch_expand_q4(const patch_layout_t* L, const uint8_t* packed, const patch_layout_t* out_layout, uint8_t* out,
                      int* status_dev, cudaStream_t stream);
+// Where the many-token call on a 4-bit weight puts that weight's bf16 image inside the caller's workspace: past
+// every word that other calls keep zero there (arrival counters, flagged partial sums, the gated product's flag
+// words: under 20 MB for N <= 131072), so that a workspace shared with them stays valid.
+constexpr size_t kQ4ExpandOffset = size_t(32) << 20;
 inline bool has_q4_tiles(const patch_layout_t* L) { return L->n_dense_q4 != 0 || L->n_sparse_q4 != 0; }
 
 }  // namespace patch

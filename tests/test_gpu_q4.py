@@ -291,7 +291,8 @@ def test_gemm_many_tokens(gpu, oracle, M, p):
     What = oracle.prune(W, flags)
     packed, L = B.patch_pack(to_dev(torch, W), flags)
     need = B.patch_gemm_workspace_size(L, M)
-    assert need == oracle.packed_size(N, K, flags & 1).total_bytes         # the size of the bf16 blob of the same mask
+    off = 32 << 20                                                          # the blob's place in the workspace
+    assert need == off + oracle.packed_size(N, K, flags & 1).total_bytes    # ... and the size of the bf16 blob of the same mask
     Y32, Y16 = oracle.gemm_f64(X, What)
     Y = run_gemm(gpu, X, L, packed, B.VARIANT_AUTO)
     check_parity(oracle, Y, Y32, f"q4 M={M} p={p}")
@@ -301,12 +302,40 @@ def test_gemm_many_tokens(gpu, oracle, M, p):
     ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
     B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws)
     torch.cuda.synchronize()
-    E = B.patch_read_layout(ws)
+    assert int(ws[:off].count_nonzero()) == 0                               # the part other calls share stays zero
+    E = B.patch_read_layout(ws[off:])
     assert (E.n_dense, E.n_sparse, E.n_dense_q4, E.n_sparse_q4) == (L.n_dense_q4, L.n_sparse_q4, 0, 0)
-    assert (to_bits(B.patch_unpack(E, ws)) == What).all()
+    assert (to_bits(B.patch_unpack(E, ws[off:])) == What).all()
     with pytest.raises(B.PatchError) as e:
         B.patch_gemm(to_dev(torch, X), L, packed, workspace=ws[:need - 256])
     assert e.value.status == B.ERR_SIZE
+
+
+def test_workspace_shared_between_bf16_and_4bit_calls(gpu, oracle):
+    """One workspace for a bf16 weight's small-M calls (which count on its counters and flag words being zero) and a
+    4-bit weight's many-token call (which writes a whole blob into it): in any order, every result stays right."""
+    torch, B = gpu
+    N, K = 512, 1024
+    W = inputs.weight(N, K, 46, "q4-shared-ws")
+    fb = inputs.tile_flags(N, K, 0.5, inputs.MASTER_SEED, "q4-shared-ws")
+    f4 = fb | 2
+    pb, Lb = B.patch_pack(to_dev(torch, W), fb)
+    p4, L4 = B.patch_pack(to_dev(torch, W), f4)
+    size = max(B.patch_gemm_workspace_size(Lb, 64), B.patch_gemm_workspace_size(L4, 200))
+    ws = torch.zeros(size, dtype=torch.uint8, device="cuda")
+    Xs, Xl = inputs.activation(7, K, 46, "q4-shared-ws", 7), inputs.activation(200, K, 46, "q4-shared-ws", 200)
+    Ys32, _ = oracle.gemm_f64(Xs, oracle.prune(W, fb))
+    Yl32, _ = oracle.gemm_f64(Xl, oracle.prune(W, f4))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for rnd in range(2):
+        Ys = B.patch_gemm(to_dev(torch, Xs), Lb, pb, workspace=ws, status=status, variant=B.VARIANT_MMA)   # the schedule with counters
+        Yl = B.patch_gemm(to_dev(torch, Xl), L4, p4, workspace=ws, status=status)
+        Ys2 = B.patch_gemm(to_dev(torch, Xs), Lb, pb, workspace=ws, status=status, variant=B.VARIANT_MMA)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        check_parity(oracle, to_bits(Ys), Ys32, f"bf16 before, round {rnd}")
+        check_parity(oracle, to_bits(Yl), Yl32, f"4-bit many tokens, round {rnd}")
+        assert (Ys2 == Ys).all()
 
 
 def test_gemm_many_tokens_llama_shape_sampled(gpu, oracle):
