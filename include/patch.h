@@ -152,7 +152,7 @@ int patch_packed_size(int64_t N, int64_t K, int tile_n, int tile_k,
  * In every 2:4 tile, each group of four consecutive elements along K keeps its two largest
  * magnitudes (equal magnitudes: lower index first; magnitude = bit pattern without sign);
  * dense tiles are copied.  A weight that is already 2:4 inside those tiles is packed losslessly.
- * Tiles of the 4-bit kinds are quantised as described at the tile kinds (a second kernel).
+ * Tiles of the 4-bit kinds are quantised as described at the tile kinds (by the same kernel).
  *   W_dev            bf16 [N x ldw], ldw >= K elements, ldw % 8 == 0
  *   tile_flags_host  as for patch_packed_size; must be the flags `layout` was computed from
  *   packed_dev       destination, packed_capacity >= layout->total_bytes, 16-byte aligned

@@ -275,8 +275,9 @@ extern "C" int patch_gemm_host_batch_pipelined(const patch_host_job_t* jobs, int
             cleanup();
             return PATCH_ERR_CUDA;
         }
-    // every X is on the device before the GEMM that reads it (event), and is written by a copy on another stream
-    const int flags = weights_static ? (PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC) : 0;
+    // every X is on the device before the GEMM that reads it (event), and is written by a copy on another stream;
+    // a Y is written by its own GEMM only and read by a copy that waits for the whole run (event)
+    const int flags = weights_static ? (PATCH_GEMM_WEIGHTS_STATIC | PATCH_GEMM_INPUT_STATIC | PATCH_GEMM_OUTPUT_STATIC) : 0;
     rc = PATCH_OK;
     bool ok = true;
     for (int c = 0; c < n_chunks && ok && !rc; ++c) {
