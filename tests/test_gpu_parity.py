@@ -622,8 +622,8 @@ def test_gated_product_small_m_schedule(gpu, oracle, M, shape):
     _gated_case(gpu, oracle, Nh, K, M, 1.0, 0.0, ws=None, flags_arg=B.WEIGHTS_STATIC | B.INPUT_STATIC)
 
 
-@pytest.mark.parametrize("M", [17, 32, 33, 48, 64])
-@pytest.mark.parametrize("shape", [(256, 128), (1024, 768), (1408, 4096), (11008, 4096)])
+@pytest.mark.parametrize("M,shape", [(M, s) for M in (17, 32, 33, 48, 64) for s in ((256, 128), (1024, 768), (1408, 4096))] +
+                         [(33, (11008, 4096))])
 def test_gated_product_17_to_64_tokens(gpu, oracle, M, shape):
     """17 to 64 tokens: the schedule whose CTA holds the gate and the up accumulator of a pair of row-blocks, under
     every combination of launch promises, on weights from one pair of row-blocks to the LLaMA MLP shape."""
