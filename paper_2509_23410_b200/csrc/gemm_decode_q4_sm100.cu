@@ -45,6 +45,14 @@
 // into two K-halves with separate completion tracking, so that a group never waits for its own MMAs (0.142 ms: a third barrier and a second
 // issue sequence per tile cost more than the wait); dequantising the next tile's first 32 values before that wait
 // (0.138 ms: every warp polls again, registers spill); six groups in one CTA per SM (0.150 ms, see above).
+// A slot of the payload ring serves the groups in turn (eight slots, three groups), so the thread that waits for a
+// slot's "full" phase is not the one that waited for its previous phase, and an mbarrier wait names a phase by its
+// parity only.  Without further ordering, a group that ran ahead of the slot's previous user could take that tile's
+// unfinished phase for its own finished one and read the slot before anything had landed: one wrong tile in one
+// row-block, seen about once in 10^5 launches, and only in streams where kernels of other kinds share the SMs and
+// delay single copies (a launch that ended with "unspecified launch failure" in the same runs fits the barrier
+// protocol going wrong after such a read).  Every group now waits first until the slot's previous tile has been
+// consumed -- see the comment at the waits.  The kernels with one consuming thread per ring cannot meet this.
 // Same bounded waits, table checks, launch flags and determinism as the other decode kernels; M <= 16.
 #include "sm100_ptx.cuh"
 
@@ -286,10 +294,19 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
             // all instructions).  The barrier also tells everyone if the wait was given up.
             bool failed = false;
             if (issuer && lane == 0) {
-                failed = !mbar_wait_suspended(bar_raw_full + 8 * slot, uint32_t(i / kRaw) & 1u, abort_flag, status_dev);
+                // A slot's successive tiles belong to DIFFERENT groups (kRaw is not a multiple of kGroups), and a wait
+                // names a phase by its parity only.  A group that ran ahead of the slot's previous user -- whose
+                // payload may still be on its way when later ones have landed and been multiplied -- would take that
+                // tile's unfinished "full" phase for its own finished one and read the slot too early.  So it first
+                // waits until the previous tile of the slot has been consumed (the condition the producer waits for
+                // before it requests this tile; that phase cannot be mistaken: the one before it ended before this
+                // group's last tile was requested, and the next one ends only with this tile's own MMAs).  After it,
+                // the slot's "full" barrier and the round's activation barrier are in this tile's phase.
+                const uint32_t par = uint32_t(i / kRaw) & 1u;
+                if (i >= kRaw) failed = !mbar_wait_suspended(bar_raw_empty + 8 * slot, par ^ 1u, abort_flag, status_dev);
+                if (!failed) failed = !mbar_wait_suspended(bar_raw_full + 8 * slot, par, abort_flag, status_dev);
                 if (!failed)
-                    failed = !mbar_wait_suspended(bar_x_full + 8 * ((i / kBatch) % (kRaw / kBatch)), uint32_t(i / kRaw) & 1u,
-                                                  abort_flag, status_dev);
+                    failed = !mbar_wait_suspended(bar_x_full + 8 * ((i / kBatch) % (kRaw / kBatch)), par, abort_flag, status_dev);
                 if (!failed && n > 0)
                     failed = !mbar_wait_suspended(bar_op_empty + 8 * g, (uint32_t(n) & 1u) ^ 1u, abort_flag, status_dev);
             }

@@ -338,6 +338,52 @@ def test_workspace_shared_between_bf16_and_4bit_calls(gpu, oracle):
         assert (Ys2 == Ys).all()
 
 
+def test_mixed_stream_of_4bit_and_bf16_launches(gpu, oracle):
+    """A long stream in which 4-bit GEMMs share the GPU with bf16 GEMMs of other shapes, token counts and launch
+    promises (several kernels resident at once, copies completing out of order).  Every job is checked once against
+    the oracle; after that every launch must repeat, bit for bit, the first result of its launch form -- the kernels
+    are deterministic, so one tile read too early or too late in any launch shows."""
+    torch, B = gpu
+    g = inputs.generator(47, "mixed-stream")
+    jobs = []
+    ws = torch.zeros(8192 + 3145728 + 2 * 192 * 64 * 128 * 4, dtype=torch.uint8, device="cuda")
+    for it in range(20):
+        TN, TK = int(g.integers(8, 60)), int(g.integers(8, 60))
+        N, K = 128 * TN, 128 * TK
+        q4 = it % 2 == 0
+        M = int(g.choice([1, 2, 5, 16] if q4 else [1, 3, 8, 16, 17, 40, 64]))
+        flags = inputs.tile_flags(N, K, float(g.choice([0.0, 1.0, 0.5])), 47, "mixed-stream", it) | (2 if q4 else 0)
+        W = inputs.weight(N, K, 47, "mixed-stream", it)
+        X = inputs.activation(M, K, 47, "mixed-stream", it)
+        packed, L = B.patch_pack(to_dev(torch, W), flags)
+        rows = np.unique(g.integers(0, M, 2))
+        ref_rows = oracle.gemm_f64_rows(X, rows, oracle.prune(W, flags))
+        jobs.append(dict(X=to_dev(torch, X), L=L, packed=packed, rows=rows, ref_rows=ref_rows, first={},
+                         Ys=[torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(4)], n=0, form=[None] * 4))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    forms = [B.WEIGHTS_STATIC | B.INPUT_STATIC | B.OUTPUT_STATIC, B.WEIGHTS_STATIC | B.INPUT_STATIC, B.WEIGHTS_STATIC, 0]
+    for rnd in range(12):
+        order = g.permutation(len(jobs))
+        for rep in range(25):
+            for i in order:
+                j = jobs[i]
+                k = j["n"] % 4
+                j["n"] += 1
+                j["form"][k] = forms[int(g.integers(0, 4))]
+                B.patch_gemm(j["X"], j["L"], j["packed"], Y=j["Ys"][k], workspace=ws, status=status,
+                             variant=B.VARIANT_AUTO | j["form"][k])
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for j in jobs:
+            for k, Y in enumerate(j["Ys"]):
+                form = j["form"][k]
+                if form not in j["first"]:
+                    check_parity(oracle, to_bits(Y)[j["rows"]], j["ref_rows"], f"first result of launch form {form:#x}")
+                    j["first"][form] = Y.clone()
+                assert torch.equal(Y, j["first"][form]), f"round {rnd}: launch form {form:#x} did not repeat its result"
+                Y.zero_()
+
+
 def test_gemm_many_tokens_llama_shape_sampled(gpu, oracle):
     torch, B = gpu
     N, K, M = 4096, 4096, 2048
