@@ -37,7 +37,8 @@
 //
 // Two CTAs per SM: while one is being set up, drains its last tiles or waits for the preceding kernel before it may
 // write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130;
-// with the output promise, under which finished CTAs do not wait at all: 0.110, and 0.107 with no split of K).
+// with the output promise, under which finished CTAs do not wait at all: 0.110, and 0.107 with no split of K;
+// 0.111 with the ordering wait described below).
 // A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
 // columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
 // shared memory.
