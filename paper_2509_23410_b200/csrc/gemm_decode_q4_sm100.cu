@@ -38,7 +38,8 @@
 // Two CTAs per SM: while one is being set up, drains its last tiles or waits for the preceding kernel before it may
 // write Y, the other streams (one CTA with twice the groups and ring: 0.150 ms on the 24-GEMM decode step, two: 0.130;
 // with the output promise, under which finished CTAs do not wait at all: 0.110, and 0.107 with no split of K;
-// 0.111 with the ordering wait described below).
+// 0.111 when every group first waited for the consumption of its slot's previous tile, the first fix of the
+// ordering described below).
 // A CTA allocates 256 TMEM columns, so the two allocations always fit -- an allocation that had to wait for the
 // columns of a CTA whose cluster peer waits for this cluster's would never return -- and a third CTA never fits in
 // shared memory.
@@ -52,8 +53,8 @@
 // unfinished phase for its own finished one and read the slot before anything had landed: one wrong tile in one
 // row-block, seen about once in 10^5 launches, and only in streams where kernels of other kinds share the SMs and
 // delay single copies (a launch that ended with "unspecified launch failure" in the same runs fits the barrier
-// protocol going wrong after such a read).  Every group now waits first until the slot's previous tile has been
-// consumed -- see the comment at the waits.  The kernels with one consuming thread per ring cannot meet this.
+// protocol going wrong after such a read).  A slot now alternates between two "full" barriers -- see the comment
+// at the waits.  The kernels with one consuming thread per ring cannot meet this.
 // Same bounded waits, table checks, launch flags and determinism as the other decode kernels; M <= 16.
 #include "sm100_ptx.cuh"
 
@@ -76,8 +77,8 @@ constexpr uint32_t kPartialRowBytes = 16 * 4;
 static_assert(64 + 64 * kGroups <= kTmemCols && 16 * kGroups <= 48 && 48 + 4 * kGroups <= 64, "TMEM columns");
 static_assert(kRawBytes % 128 == 0 && kSparseQ4Bytes <= kRawBytes, "payload slots");
 static_assert(2 * kSmemBytes <= 227 * 1024 && 3 * kSmemBytes > 228 * 1024 && 2 * kTmemCols <= 512, "two CTAs per SM, see above");
-static_assert(kRaw <= 16 && kGroups <= 8 && kThreads <= 1024, "barrier block, CTA size");
-static_assert(32 % kBatch == 0 && kRaw % kBatch == 0 && kRaw / kBatch <= 8, "producer rounds");
+static_assert(2 * kRaw <= 16 && kGroups <= 8 && kThreads <= 1024, "barrier block, CTA size");
+static_assert(32 % kBatch == 0 && kRaw % kBatch == 0 && 2 * kRaw / kBatch <= 8, "producer rounds");
 
 __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -169,9 +170,10 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
 
-    const uint32_t bar_raw_full = smem_base + kBarrierOffset;     // 16 x 8 B reserved for each array
-    const uint32_t bar_raw_empty = bar_raw_full + 128;
-    const uint32_t bar_x_full = bar_raw_empty + 128;              // kRaw / kBatch x 8 B (8 reserved)
+    // "Full" barriers come in two sets that a slot (a round) uses alternately -- see the consumers' waits for why.
+    const uint32_t bar_raw_full = smem_base + kBarrierOffset;     // 2 kRaw x 8 B (16 reserved)
+    const uint32_t bar_raw_empty = bar_raw_full + 128;            // kRaw x 8 B (16 reserved)
+    const uint32_t bar_x_full = bar_raw_empty + 128;              // 2 kRaw / kBatch x 8 B (8 reserved)
     const uint32_t bar_op_empty = bar_x_full + 64;                // 8 x 8 B reserved
     const uint32_t bar_acc_full = bar_op_empty + 64;
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kBarrierOffset + 392);
@@ -191,9 +193,10 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
     if (threadIdx.x == 32) {
         for (int i = 0; i < kRaw; ++i) {
             mbar_init(bar_raw_full + 8 * i, 1);
+            mbar_init(bar_raw_full + 8 * (kRaw + i), 1);
             mbar_init(bar_raw_empty + 8 * i, 1);                   // the tile's MMAs (they follow the group's reads)
         }
-        for (int i = 0; i < kRaw / kBatch; ++i) mbar_init(bar_x_full + 8 * i, 1);
+        for (int i = 0; i < 2 * kRaw / kBatch; ++i) mbar_init(bar_x_full + 8 * i, 1);
         for (int i = 0; i < kGroups; ++i) mbar_init(bar_op_empty + 8 * i, 1);
         mbar_init(bar_acc_full, n_groups > 0 ? n_groups : 1);
         *abort_flag = 0;
@@ -245,7 +248,7 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
                 if (mine_ok && i < n_tiles) {
                     sanitize_q4_tile(kind, off16, pay0_16, end16, status_dev);
                     const uint32_t wbytes = kind == PATCH_TILE_DENSE_Q4 ? kDenseQ4Bytes : kSparseQ4Bytes;
-                    const uint32_t full = bar_raw_full + 8 * slot;
+                    const uint32_t full = bar_raw_full + 8 * (i % (2 * kRaw));
                     slot_kind[slot] = kind;
                     mbar_expect_tx(full, wbytes + (i == 0 ? inject_bytes : 0u));
                     tma_bulk_load(smem_base + kRawOffset + slot * kRawBytes, blob + uint64_t(off16) * 16, wbytes, full, pol_w);
@@ -255,7 +258,7 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
             if (ok) issued = base + kBatch < n_tiles ? base + kBatch : n_tiles;
             // the round's activations: one copy of 2 kBatch atoms into the X buffers of its kBatch slots
             if (ok && lane == 0 && base >= n_early) {
-                const uint32_t xb = bar_x_full + 8 * ((base / kBatch) % (kRaw / kBatch));
+                const uint32_t xb = bar_x_full + 8 * ((base / kBatch) % (2 * kRaw / kBatch));
                 mbar_expect_tx(xb, kBatch * kXBytes);
                 tma_tile_load_3d(smem_base + kXOffset + (base % kRaw) * kXBytes, &tmap_x, 0, 0, (k0 + base) * 2, xb, pol_x);
             }
@@ -273,9 +276,9 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
             // drain: wait (bounded) until the copies this warp started have landed
             const uint64_t tstart = global_timer_ns();
             for (int j = issued > kRaw ? issued - kRaw : 0; j < issued; ++j) {
-                const uint32_t bar = bar_raw_full + 8 * (j % kRaw), parity = uint32_t(j / kRaw) & 1u;
+                const uint32_t bar = bar_raw_full + 8 * (j % (2 * kRaw)), parity = uint32_t(j / (2 * kRaw)) & 1u;
                 while (!mbar_try_wait(bar, parity) && global_timer_ns() - tstart < kDrainLimitNs) {}
-                const uint32_t xb = bar_x_full + 8 * ((j / kBatch) % (kRaw / kBatch));
+                const uint32_t xb = bar_x_full + 8 * ((j / kBatch) % (2 * kRaw / kBatch));
                 while (!mbar_try_wait(xb, parity) && global_timer_ns() - tstart < kDrainLimitNs) {}
             }
         }
@@ -296,18 +299,16 @@ decode_q4_kernel(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __re
             bool failed = false;
             if (issuer && lane == 0) {
                 // A slot's successive tiles belong to DIFFERENT groups (kRaw is not a multiple of kGroups), and a wait
-                // names a phase by its parity only.  A group that ran ahead of the slot's previous user -- whose
-                // payload may still be on its way when later ones have landed and been multiplied -- would take that
-                // tile's unfinished "full" phase for its own finished one and read the slot too early.  So it first
-                // waits until the previous tile of the slot has been consumed (the condition the producer waits for
-                // before it requests this tile; that phase cannot be mistaken: the one before it ended before this
-                // group's last tile was requested, and the next one ends only with this tile's own MMAs).  After it,
-                // the slot's "full" barrier and the round's activation barrier are in this tile's phase.
-                const uint32_t par = uint32_t(i / kRaw) & 1u;
-                if (i >= kRaw) failed = !mbar_wait_suspended(bar_raw_empty + 8 * slot, par ^ 1u, abort_flag, status_dev);
-                if (!failed) failed = !mbar_wait_suspended(bar_raw_full + 8 * slot, par, abort_flag, status_dev);
+                // names a phase by its parity only.  With one "full" barrier per slot, a group that ran ahead of the
+                // slot's previous user -- whose payload may still be on its way when later ones have landed and been
+                // multiplied -- took that tile's unfinished phase for its own finished one and read the slot too
+                // early.  Hence two barriers per slot, used alternately: the phase before this tile's on ITS barrier is
+                // the slot's tile before last, which was consumed before the previous one was even requested, and
+                // that request precedes the request of this group's last tile.  The same for the rounds' activations.
+                const uint32_t par = uint32_t(i / (2 * kRaw)) & 1u;
+                failed = !mbar_wait_suspended(bar_raw_full + 8 * (i % (2 * kRaw)), par, abort_flag, status_dev);
                 if (!failed)
-                    failed = !mbar_wait_suspended(bar_x_full + 8 * ((i / kBatch) % (kRaw / kBatch)), par, abort_flag, status_dev);
+                    failed = !mbar_wait_suspended(bar_x_full + 8 * ((i / kBatch) % (2 * kRaw / kBatch)), par, abort_flag, status_dev);
                 if (!failed && n > 0)
                     failed = !mbar_wait_suspended(bar_op_empty + 8 * g, (uint32_t(n) & 1u) ^ 1u, abort_flag, status_dev);
             }
