@@ -683,7 +683,7 @@ double oracle_regularizers(const double* sums, int n, double rho, double lambda1
 }
 
 /* Hard masks from the logits (Algorithm 1): tile t is dense iff P_tile[t] > 0 (flag 0), else 2:4 (flag 1);
- * every group takes the candidate with the largest logit ("select best 2:4 mask"), the first of equals. */
+ * every group takes the candidate with the largest logit (the algorithm's best-mask selection), the first of equals. */
 int oracle_hard_mask(const float* P_tile, const float* P24, int64_t N, int64_t K, int tile_n, int tile_k,
                      uint8_t* flags, uint8_t* patterns) {
     int rc = check_shape(N, K, tile_n, tile_k);
