@@ -329,6 +329,9 @@ int launch_decode_cluster(const CUtensorMap& map, const patch_layout_t* L, const
         // can keep HBM busy (the independent schedule wants few CTAs per GEMM and several GEMMs resident instead).
         // Tried on top of this and dropped: asking L2 for the rest of the CTA's weight tiles before the wait
         // (0.332 against 0.322 ms on the 24-GEMM step) -- a three-stage ring drains L2 hardly faster than HBM.
+        // Also tried: at least one CTA per SM instead of 128 (the 4096-row weights then split K eight ways, 256 CTAs):
+        // 0.303 ms on that step, but the decoder-block chain, where independent launches of the next block already
+        // hold SM slots, goes from 1.99 to 2.20 ms -- the chain is the case that matters, so 128 stays.
         S = 1;
         while (S < 8 && TN * S < 128 && 2 * S <= TK) S *= 2;
     }
